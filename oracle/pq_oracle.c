@@ -1,0 +1,287 @@
+/*
+ * pq_oracle.c -- plain CPU oracle for the quantized linear layer (W8A8 / W4A8).
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, obviously-correct statement of
+ * what the quantized linear layer computes, written from the paper's equations.  It
+ * shares no code, header, table or constant with the CUDA library; only tests, the
+ * smoke check and the benchmark's CPU-baseline leg may call it.  The product path
+ * never routes through it.
+ *
+ * What it follows:
+ *   - Eq. 1 (integer code = round(X / s)) and Eq. 2 (s = 2*max|X| / (2^n - 1),
+ *     clamp to [-2^(n-1), 2^(n-1)-1], round-to-nearest) of the paper's
+ *     "Preliminary" section, with n = 8 for activations and W8 weights and n = 4
+ *     for W4 weights.
+ *   - The granularities named in the same section: one scale per token for
+ *     activations, one per output channel for W8 weights, one per fixed-size
+ *     group along K for W4 weights.
+ *   - Symmetric quantization (no zero point), as the experimental set-up states.
+ *   - The "Unified low-bit inference framework" section: integer matrix product of
+ *     the codes followed by dequantization back to FP16.
+ *
+ * Readings taken where the paper is silent (also listed in the design notes):
+ *   - ties in the rounding go to even;
+ *   - the quotient X/s of Eq. 1 is evaluated in IEEE binary32 as X * (c / max|X|)
+ *     for activations (c = (2^n-1)/2), and as a binary32 division X / s for the
+ *     offline weight packers;
+ *   - an all-zero row or group has scale 0 and codes 0;
+ *   - W4 codes are chosen against the FP16-rounded group scale that is stored;
+ *   - dequantization is evaluated in binary64 and rounded once to FP16.
+ *
+ * Arithmetic notes: integer dot products accumulate in int64 and are checked to
+ * fit int32.  All binary32 steps are single IEEE operations (compile with
+ * -ffp-contract=off, no fast-math).  FP16 is handled with the bit-level
+ * conversions below; no hardware half type is used.
+ *
+ * Parity pins live in tests/test_oracle_pins.py (closed forms with power-of-two
+ * scales, exact-rational cross-check, brute force, identity / one-hot weights,
+ * error bound, overflow bound, exhaustive FP16 round trip).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define PQO_OK 0
+#define PQO_ERR_OVERFLOW 1 /* an integer accumulator left the int32 range */
+#define PQO_ERR_ARG 2
+
+/* ------------------------------------------------------------------ FP16 */
+
+/* FP16 bit pattern -> binary32 value (exact). */
+float pqo_half_to_float(uint16_t h) {
+  int sign = (h >> 15) & 1;
+  int e = (h >> 10) & 0x1f;
+  int m = h & 0x3ff;
+  double v;
+  if (e == 0) {
+    v = ldexp((double)m, -24); /* zero and subnormals: m * 2^-24 */
+  } else if (e == 31) {
+    v = m ? NAN : INFINITY;
+  } else {
+    v = ldexp((double)(1024 + m), e - 25); /* (1 + m/1024) * 2^(e-15) */
+  }
+  return (float)(sign ? -v : v);
+}
+
+/* binary64 value -> FP16 bit pattern, one rounding, round-to-nearest-even,
+ * overflow to infinity, subnormals kept. */
+uint16_t pqo_double_to_half_rne(double d) {
+  uint16_t sign = signbit(d) ? 0x8000u : 0u;
+  double a = fabs(d);
+  if (isnan(d)) return (uint16_t)(sign | 0x7e00u);
+  if (a >= 65520.0) return (uint16_t)(sign | 0x7c00u); /* >= midpoint(65504, 65536) */
+  if (a < ldexp(1.0, -14)) {
+    /* subnormal range: spacing 2^-24 */
+    double r = nearbyint(ldexp(a, 24)); /* 0 .. 1024; 1024 encodes the smallest normal */
+    return (uint16_t)(sign | (uint16_t)r);
+  }
+  int e2;
+  (void)frexp(a, &e2); /* a = f * 2^e2 with f in [0.5, 1) */
+  int e = e2 - 1;      /* a in [2^e, 2^(e+1)) */
+  double r = nearbyint(ldexp(a, 10 - e)); /* in [1024, 2048] */
+  if (r >= 2048.0) {
+    r = 1024.0;
+    e += 1;
+  }
+  if (e > 15) return (uint16_t)(sign | 0x7c00u);
+  return (uint16_t)(sign | (uint16_t)((e + 15) << 10) | ((uint16_t)r - 1024u));
+}
+
+uint16_t pqo_float_to_half_rne(float f) { return pqo_double_to_half_rne((double)f); }
+
+/* ------------------------------------------------------------ quantizers */
+
+static float clampf(float v, float lo, float hi) { return v < lo ? lo : (v > hi ? hi : v); }
+
+/*
+ * Per-token activation quantization, Eq. 1-2 with n = 8.
+ *   a = max_k |X[m,k]|;  s_tok[m] = a / 127.5  (= 2a / 255)
+ *   Q[m,k] = clamp(rne(X[m,k] * (127.5 / a)), -128, 127)
+ * x: FP16 bit patterns [M,K] row-major.  q: [M,K].  s_tok: [M].
+ */
+int pqo_quantize_act(const uint16_t* x, int64_t M, int64_t K, int8_t* q, float* s_tok) {
+  if (M < 0 || K <= 0) return PQO_ERR_ARG;
+#pragma omp parallel for schedule(static)
+  for (int64_t m = 0; m < M; ++m) {
+    const uint16_t* xr = x + m * K;
+    float a = 0.0f;
+    for (int64_t k = 0; k < K; ++k) {
+      float v = fabsf(pqo_half_to_float(xr[k]));
+      if (v > a) a = v;
+    }
+    if (a == 0.0f) {
+      s_tok[m] = 0.0f;
+      for (int64_t k = 0; k < K; ++k) q[m * K + k] = 0;
+      continue;
+    }
+    float s = a / 127.5f;
+    float inv = 127.5f / a;
+    s_tok[m] = s;
+    for (int64_t k = 0; k < K; ++k) {
+      float t = pqo_half_to_float(xr[k]) * inv;
+      float r = nearbyintf(t); /* ties to even */
+      q[m * K + k] = (int8_t)clampf(r, -128.0f, 127.0f);
+    }
+  }
+  return PQO_OK;
+}
+
+/*
+ * Per-output-channel INT8 weight quantization, Eq. 2 with n = 8.
+ *   a = max_k |W[n,k]|;  s_ch[n] = a / 127.5;  Wq = clamp(rne(W / s_ch[n]), -128, 127)
+ * w: FP16 bit patterns [N,K] (one output channel per row).
+ */
+int pqo_pack_w8(const uint16_t* w, int64_t N, int64_t K, int8_t* wq, float* s_ch) {
+  if (N < 0 || K <= 0) return PQO_ERR_ARG;
+#pragma omp parallel for schedule(static)
+  for (int64_t n = 0; n < N; ++n) {
+    const uint16_t* wr = w + n * K;
+    float a = 0.0f;
+    for (int64_t k = 0; k < K; ++k) {
+      float v = fabsf(pqo_half_to_float(wr[k]));
+      if (v > a) a = v;
+    }
+    if (a == 0.0f) {
+      s_ch[n] = 0.0f;
+      for (int64_t k = 0; k < K; ++k) wq[n * K + k] = 0;
+      continue;
+    }
+    float s = a / 127.5f;
+    s_ch[n] = s;
+    for (int64_t k = 0; k < K; ++k) {
+      float r = nearbyintf(pqo_half_to_float(wr[k]) / s);
+      wq[n * K + k] = (int8_t)clampf(r, -128.0f, 127.0f);
+    }
+  }
+  return PQO_OK;
+}
+
+/*
+ * Group-wise INT4 weight quantization, Eq. 2 with n = 4, one scale per
+ * (output channel, group of `group` consecutive k).
+ *   a = max_{k in g} |W[n,k]|;  s_grp[n,g] = fp16(a / 7.5)
+ *   code = clamp(rne(W / float(s_grp[n,g])), -8, 7)      (against the stored scale)
+ * codes: int8 [N,K] holding values in [-8,7].  s_grp: FP16 bit patterns [N, K/group].
+ */
+int pqo_pack_w4(const uint16_t* w, int64_t N, int64_t K, int64_t group, int8_t* codes,
+                uint16_t* s_grp) {
+  if (N < 0 || K <= 0 || group <= 0 || K % group) return PQO_ERR_ARG;
+  int64_t G = K / group;
+#pragma omp parallel for schedule(static)
+  for (int64_t n = 0; n < N; ++n) {
+    for (int64_t g = 0; g < G; ++g) {
+      const uint16_t* wr = w + n * K + g * group;
+      float a = 0.0f;
+      for (int64_t k = 0; k < group; ++k) {
+        float v = fabsf(pqo_half_to_float(wr[k]));
+        if (v > a) a = v;
+      }
+      uint16_t s16 = pqo_float_to_half_rne(a / 7.5f);
+      float sf = pqo_half_to_float(s16);
+      s_grp[n * G + g] = s16;
+      for (int64_t k = 0; k < group; ++k) {
+        int8_t c = 0;
+        if (sf != 0.0f) {
+          float r = nearbyintf(pqo_half_to_float(wr[k]) / sf);
+          c = (int8_t)clampf(r, -8.0f, 7.0f);
+        }
+        codes[n * K + g * group + k] = c;
+      }
+    }
+  }
+  return PQO_OK;
+}
+
+/* Interchange form of INT4 codes: byte j of a row holds k = 2j in bits 0-3 and
+ * k = 2j+1 in bits 4-7, two's complement. */
+int pqo_nibble_pack(const int8_t* codes, int64_t N, int64_t K, uint8_t* bytes) {
+  if (K % 2) return PQO_ERR_ARG;
+  for (int64_t n = 0; n < N; ++n)
+    for (int64_t j = 0; j < K / 2; ++j) {
+      uint8_t lo = (uint8_t)codes[n * K + 2 * j] & 0xf;
+      uint8_t hi = (uint8_t)codes[n * K + 2 * j + 1] & 0xf;
+      bytes[n * (K / 2) + j] = (uint8_t)(lo | (hi << 4));
+    }
+  return PQO_OK;
+}
+
+int pqo_nibble_unpack(const uint8_t* bytes, int64_t N, int64_t K, int8_t* codes) {
+  if (K % 2) return PQO_ERR_ARG;
+  for (int64_t n = 0; n < N; ++n)
+    for (int64_t j = 0; j < K / 2; ++j) {
+      uint8_t b = bytes[n * (K / 2) + j];
+      int lo = b & 0xf, hi = b >> 4;
+      codes[n * K + 2 * j] = (int8_t)(lo >= 8 ? lo - 16 : lo);
+      codes[n * K + 2 * j + 1] = (int8_t)(hi >= 8 ? hi - 16 : hi);
+    }
+  return PQO_OK;
+}
+
+/* ------------------------------------------------------------------ GEMMs */
+
+/*
+ * W8A8 linear: ACC[m,n] = sum_k Q[m,k] * Wq[n,k] (exact integer),
+ *              Y[m,n]  = fp16( ACC[m,n] * s_tok[m] * s_ch[n] ).
+ * acc (int32 [M,N]) and y (FP16 bits [M,N]) may each be NULL to skip that output.
+ */
+int pqo_gemm_w8a8(const int8_t* q, const float* s_tok, const int8_t* wq, const float* s_ch,
+                  int64_t M, int64_t N, int64_t K, int32_t* acc, uint16_t* y) {
+  if (M < 0 || N < 0 || K <= 0) return PQO_ERR_ARG;
+  int overflow = 0;
+#pragma omp parallel for schedule(static) reduction(| : overflow)
+  for (int64_t m = 0; m < M; ++m) {
+    for (int64_t n = 0; n < N; ++n) {
+      int64_t s = 0;
+      for (int64_t k = 0; k < K; ++k) s += (int64_t)q[m * K + k] * (int64_t)wq[n * K + k];
+      if (s > INT32_MAX || s < INT32_MIN) overflow |= 1;
+      if (acc) acc[m * N + n] = (int32_t)s;
+      if (y) {
+        double v = (double)s * (double)s_tok[m] * (double)s_ch[n];
+        y[m * N + n] = pqo_double_to_half_rne(v);
+      }
+    }
+  }
+  return overflow ? PQO_ERR_OVERFLOW : PQO_OK;
+}
+
+/*
+ * W4A8 linear with per-group dequantization:
+ *   ACC_g[m,n] = sum_{k in group g} Q[m,k] * C[n,k]          (exact integer)
+ *   R[m,n]     = sum_g ACC_g[m,n] * float(s_grp[n,g])        (g ascending)
+ *   Y[m,n]     = fp16( R[m,n] * s_tok[m] )
+ * codes: int8 [N,K] with values in [-8,7].  acc_g (int32 [M,N,G]) and y may be NULL.
+ */
+int pqo_gemm_w4a8(const int8_t* q, const float* s_tok, const int8_t* codes,
+                  const uint16_t* s_grp, int64_t group, int64_t M, int64_t N, int64_t K,
+                  int32_t* acc_g, uint16_t* y) {
+  if (M < 0 || N < 0 || K <= 0 || group <= 0 || K % group) return PQO_ERR_ARG;
+  int64_t G = K / group;
+  int overflow = 0;
+#pragma omp parallel for schedule(static) reduction(| : overflow)
+  for (int64_t m = 0; m < M; ++m) {
+    for (int64_t n = 0; n < N; ++n) {
+      double R = 0.0;
+      for (int64_t g = 0; g < G; ++g) {
+        int64_t s = 0;
+        for (int64_t k = g * group; k < (g + 1) * group; ++k)
+          s += (int64_t)q[m * K + k] * (int64_t)codes[n * K + k];
+        if (s > INT32_MAX || s < INT32_MIN) overflow |= 1;
+        if (acc_g) acc_g[(m * N + n) * G + g] = (int32_t)s;
+        R += (double)s * (double)pqo_half_to_float(s_grp[n * G + g]);
+      }
+      if (y) y[m * N + n] = pqo_double_to_half_rne(R * (double)s_tok[m]);
+    }
+  }
+  return overflow ? PQO_ERR_OVERFLOW : PQO_OK;
+}
+
+int pqo_num_threads(void) {
+#ifdef _OPENMP
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}

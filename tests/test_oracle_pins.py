@@ -1,0 +1,371 @@
+"""Pins for the CPU oracle: every check here is something the paper's equations or plain
+mathematics fix, evaluated by a route that does not go through the oracle's own code
+(hand-worked closed forms, exact rational arithmetic, numpy int64 products, brute-force
+Python loops, numpy's own FP16 conversion)."""
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+
+import oracle
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+# ----------------------------------------------------------------------------- FP16
+
+def test_half_to_float_matches_numpy_exhaustively():
+    bits = np.arange(65536, dtype=np.uint16)
+    ref = bits.view(np.float16).astype(np.float32)
+    got = np.array([oracle.half_to_float(int(b)) for b in bits], dtype=np.float32)
+    nan = np.isnan(ref)
+    assert np.array_equal(np.isnan(got), nan)
+    assert np.array_equal(got[~nan].view(np.uint32), ref[~nan].view(np.uint32))
+
+
+def test_half_round_trip_is_identity_for_all_patterns():
+    for b in range(65536):
+        e, m = (b >> 10) & 31, b & 1023
+        if e == 31 and m:  # NaN payloads are not preserved
+            continue
+        assert oracle.float_to_half_bits(oracle.half_to_float(b)) == b
+
+
+def test_double_to_half_ties_between_adjacent_halves():
+    # midpoint of two adjacent finite halves rounds to the one with an even last bit
+    for b in list(range(0, 0x7BFF, 37)) + [0, 1, 0x3FF, 0x400, 0x7BFE]:
+        lo = float(np.uint16(b).view(np.float16))
+        hi = float(np.uint16(b + 1).view(np.float16))
+        mid = (lo + hi) / 2  # exact in binary64
+        want = b if b % 2 == 0 else b + 1
+        assert oracle.double_to_half_bits(mid) == want
+        assert oracle.double_to_half_bits(-mid) == (want | 0x8000)
+        assert oracle.double_to_half_bits(np.nextafter(mid, np.inf)) == b + 1
+        assert oracle.double_to_half_bits(np.nextafter(mid, -np.inf)) == b
+
+
+def test_double_to_half_overflow_and_random_against_numpy():
+    assert oracle.double_to_half_bits(65504.0) == 0x7BFF
+    assert oracle.double_to_half_bits(65519.99) == 0x7BFF
+    assert oracle.double_to_half_bits(65520.0) == 0x7C00  # tie goes to even = infinity
+    assert oracle.double_to_half_bits(-1e9) == 0xFC00
+    assert oracle.double_to_half_bits(0.0) == 0 and oracle.double_to_half_bits(-0.0) == 0x8000
+    rng = np.random.default_rng(1)
+    vals = np.concatenate([rng.standard_normal(4000) * 10.0 ** rng.integers(-9, 5, 4000),
+                           rng.uniform(-2 ** -14, 2 ** -14, 2000)])
+    with np.errstate(over="ignore"):
+        ref = vals.astype(np.float16).view(np.uint16)
+    got = np.array([oracle.double_to_half_bits(v) for v in vals], dtype=np.uint16)
+    assert np.array_equal(got, ref)
+
+
+# ------------------------------------------------------------------------ quantizers
+
+def _golden_rows(bits):
+    rows = []
+    with open(os.path.join(GOLDEN, "quantizer_closed_form.txt")) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            n, x, c = line.split()
+            if int(n) == bits:
+                rows.append((float(x), int(c)))
+    return rows
+
+
+@pytest.mark.parametrize("e", [0, -3, 4])
+def test_quantize_act_closed_form_power_of_two_scale(e):
+    rows = _golden_rows(8)
+    x = np.array([[v for v, _ in rows]], dtype=np.float64) * 2.0 ** e
+    x16 = x.astype(np.float16)
+    assert np.array_equal(x16.astype(np.float64), x)  # the fixture is FP16-exact
+    q, s = oracle.quantize_act(x16)
+    assert s[0] == np.float32(2.0 ** e)
+    assert q[0].tolist() == [c for _, c in rows]
+
+
+@pytest.mark.parametrize("e", [0, -5, 2])
+def test_pack_w8_and_w4_closed_form_power_of_two_scale(e):
+    rows = _golden_rows(8)
+    w = (np.array([[v for v, _ in rows]]) * 2.0 ** e).astype(np.float16)
+    wq, s = oracle.pack_w8(w)
+    assert s[0] == np.float32(2.0 ** e) and wq[0].tolist() == [c for _, c in rows]
+    rows4 = _golden_rows(4)
+    vals = [v for v, _ in rows4]
+    group = 32
+    vals = vals + [0.0] * (group - len(vals))
+    # second group: all zeros -> scale 0, codes 0
+    w4 = (np.array([vals + [0.0] * group]) * 2.0 ** e).astype(np.float16)
+    codes, sg = oracle.pack_w4(w4, group=group)
+    assert sg.dtype == np.float16 and sg.shape == (1, 2)
+    assert float(sg[0, 0]) == 2.0 ** e and float(sg[0, 1]) == 0.0
+    assert codes[0, :len(rows4)].tolist() == [c for _, c in rows4]
+    assert not codes[0, group:].any()
+
+
+def _exact_code(x: float, a: float, bits: int) -> tuple[int, bool]:
+    """Eq. 2 in exact rational arithmetic: clamp(rne((2^n-1) x / (2 a))); also says if it was a tie."""
+    t = Fraction(x) * (2 ** bits - 1) / (2 * Fraction(a))
+    fl = t.numerator // t.denominator
+    frac = t - fl
+    tie = frac == Fraction(1, 2)
+    if frac > Fraction(1, 2) or (tie and fl % 2 == 1):
+        r = fl + 1
+    else:
+        r = fl
+    lo, hi = -(2 ** (bits - 1)), 2 ** (bits - 1) - 1
+    return max(lo, min(hi, r)), tie
+
+
+def test_quantize_act_agrees_with_exact_rational_rule_away_from_ties():
+    rng = np.random.default_rng(7)
+    x = (rng.standard_normal((24, 160)) * 10.0 ** rng.integers(-3, 3, (24, 1))).astype(np.float16)
+    x[:, 5] *= 50
+    # plant exact ties: x = a * (2j+1)/255 is rarely FP16-exact, so use x = -a (t = -127.5) and a/3-like values
+    x[3, 7] = -np.abs(x[3]).max()
+    q, s = oracle.quantize_act(x)
+    n_tie = 0
+    for m in range(x.shape[0]):
+        a = float(np.abs(x[m]).max())
+        assert s[m] == np.float32(a) / np.float32(127.5)
+        for k in range(x.shape[1]):
+            want, tie = _exact_code(float(x[m, k]), a, 8)
+            if tie:
+                n_tie += 1
+                assert abs(int(q[m, k]) - want) <= 1
+            else:
+                assert int(q[m, k]) == want, (m, k, float(x[m, k]), a)
+    assert n_tie >= 1
+
+
+def test_pack_w8_agrees_with_exact_rational_rule_away_from_ties():
+    rng = np.random.default_rng(8)
+    w = (rng.standard_normal((12, 96)) * 0.02).astype(np.float16)
+    wq, s = oracle.pack_w8(w)
+    for n in range(w.shape[0]):
+        a = float(np.abs(w[n]).max())
+        for k in range(w.shape[1]):
+            want, tie = _exact_code(float(w[n, k]), a, 8)
+            # dividing by the binary32-rounded scale can move a value across a rounding
+            # boundary only when it sits within 2^-22 (relative) of that boundary
+            t = Fraction(float(w[n, k])) * 255 / (2 * Fraction(a))
+            near = abs((t - Fraction(1, 2)) - round(t - Fraction(1, 2))) < Fraction(1, 2 ** 14)
+            if not (tie or near):
+                assert int(wq[n, k]) == want
+
+
+def test_quantizer_invariants():
+    rng = np.random.default_rng(3)
+    x = rng.standard_normal((32, 256)).astype(np.float16)
+    x[:, [3, 77, 130, 200]] *= 50
+    x[5] = 0  # all-zero row
+    x[6, 10] = 0
+    q, s = oracle.quantize_act(x)
+    xf = x.astype(np.float64)
+    # quantize -> dequantize error bound |x - q s| <= s/2 (small slack for the binary32 scale)
+    err = np.abs(xf - q.astype(np.float64) * s[:, None].astype(np.float64))
+    assert (err <= s[:, None] * (0.5 + 2.0 ** -14)).all()
+    assert s[5] == 0 and not q[5].any()
+    assert q[6, 10] == 0
+    nz = [m for m in range(32) if m != 5]
+    assert (np.abs(q[nz].astype(np.int32)).max(axis=1) >= 127).all()  # the range is used
+    assert q.min() >= -128 and q.max() <= 127
+    # codes are monotone in x within a row
+    for m in nz[:8]:
+        order = np.argsort(xf[m], kind="stable")
+        assert (np.diff(q[m][order].astype(np.int32)) >= 0).all()
+    # scaling a row by a power of two scales s and leaves the codes unchanged
+    q2, s2 = oracle.quantize_act((xf * 0.25).astype(np.float16))
+    assert np.array_equal(q2, q) and np.array_equal(s2, s * np.float32(0.25))
+    # symmetric: negating the input negates the codes except where the clamp acts
+    qn, sn = oracle.quantize_act((-xf).astype(np.float16))
+    assert np.array_equal(sn, s)
+    inner = (np.abs(q.astype(np.int32)) < 127) & (np.abs(qn.astype(np.int32)) < 127)
+    assert np.array_equal(qn[inner], -q[inner])
+    # the row maximum maps to +127 (clamped from 127.5 -> 128) and its negative to -128
+    m = 0
+    k = int(np.argmax(np.abs(xf[m])))
+    assert int(q[m, k]) == (127 if xf[m, k] > 0 else -128)
+    assert int(qn[m, k]) == (-128 if xf[m, k] > 0 else 127)
+
+
+def test_pack_w4_invariants_and_stored_scale():
+    rng = np.random.default_rng(4)
+    w = (rng.standard_normal((16, 512)) * 0.02).astype(np.float16)
+    w[2, 128:256] = 0
+    codes, sg = oracle.pack_w4(w, 128)
+    assert codes.min() >= -8 and codes.max() <= 7
+    assert sg.shape == (16, 4) and float(sg[2, 1]) == 0.0 and not codes[2, 128:256].any()
+    wf = w.astype(np.float64).reshape(16, 4, 128)
+    a = np.abs(wf).max(axis=2)
+    want_s = (a.astype(np.float32) / np.float32(7.5)).astype(np.float16)
+    assert np.array_equal(sg, want_s)
+    sf = sg.astype(np.float64)[:, :, None]
+    err = np.abs(wf - codes.reshape(16, 4, 128) * sf)
+    # codes are chosen against the stored FP16 scale: half a step everywhere, except the
+    # element clamped from +8 to +7, whose error is a - 7 s with a <= 7.5 s (1 + 2^-11)
+    assert (err <= sf * (0.5 + 7.5 * 2.0 ** -11 + 1e-6)).all()
+    # exact rational rule against the stored scale, away from ties
+    for n in range(3):
+        for k in range(512):
+            s = float(sg[n, k // 128])
+            if s == 0:
+                continue
+            t = Fraction(float(w[n, k])) / Fraction(s)
+            dist = abs((t - Fraction(1, 2)) - round(t - Fraction(1, 2)))
+            if dist > Fraction(1, 2 ** 16):
+                assert int(codes[n, k]) == max(-8, min(7, round(t)))
+
+
+def test_nibble_pack_round_trips_all_byte_values():
+    allb = np.arange(256, dtype=np.uint8).reshape(2, 128)
+    codes = oracle.nibble_unpack(allb)
+    assert codes.min() == -8 and codes.max() == 7
+    # byte j holds k = 2j in its low nibble and k = 2j+1 in its high nibble, two's complement
+    for j, b in enumerate(allb[0][:40]):
+        lo, hi = int(b) & 15, int(b) >> 4
+        assert codes[0, 2 * j] == (lo - 16 if lo >= 8 else lo)
+        assert codes[0, 2 * j + 1] == (hi - 16 if hi >= 8 else hi)
+    assert np.array_equal(oracle.nibble_pack(codes), allb)
+
+
+# ----------------------------------------------------------------------------- GEMMs
+
+def _ones(n):
+    return np.ones((n,), np.float32)
+
+
+def test_gemm_w8a8_brute_force_tiny_with_extremes():
+    rng = np.random.default_rng(11)
+    M, N, K = 5, 7, 9
+    q = rng.integers(-128, 128, (M, K)).astype(np.int8)
+    wq = rng.integers(-128, 128, (N, K)).astype(np.int8)
+    q[0, :] = -128
+    wq[0, :] = -128
+    q[1, :] = 127
+    wq[1, :] = -128
+    acc, _ = oracle.gemm_w8a8(q, _ones(M), wq, _ones(N), want_y=False)
+    for m in range(M):
+        for n in range(N):
+            want = sum(int(q[m, k]) * int(wq[n, k]) for k in range(K))
+            assert int(acc[m, n]) == want
+    assert int(acc[0, 0]) == K * 16384 and int(acc[1, 0]) == -K * 127 * 128
+
+
+def test_gemm_w8a8_matches_numpy_int64_product_and_is_not_transposed():
+    rng = np.random.default_rng(12)
+    M, N, K = 33, 40, 300
+    q = rng.integers(-128, 128, (M, K)).astype(np.int8)
+    wq = rng.integers(-128, 128, (N, K)).astype(np.int8)
+    acc, _ = oracle.gemm_w8a8(q, _ones(M), wq, _ones(N), want_y=False)
+    assert np.array_equal(acc.astype(np.int64), q.astype(np.int64) @ wq.astype(np.int64).T)
+
+
+def test_gemm_w8a8_identity_and_one_hot_weights():
+    rng = np.random.default_rng(13)
+    K = 64
+    x = rng.standard_normal((8, K)).astype(np.float16)
+    q, s_tok = oracle.quantize_act(x)
+    eye = (np.eye(K) * 0.75).astype(np.float16)
+    wq, s_ch = oracle.pack_w8(eye)           # +a -> 127.5 -> 128 -> clamped to 127
+    assert np.array_equal(wq, (np.eye(K) * 127).astype(np.int8))
+    acc, _ = oracle.gemm_w8a8(q, s_tok, wq, s_ch, want_y=False)
+    assert np.array_equal(acc, 127 * q.astype(np.int32))
+    wqn, _ = oracle.pack_w8((-eye).astype(np.float16))  # -a -> -127.5 -> -128 (tie to even)
+    assert np.array_equal(wqn, (np.eye(K) * -128).astype(np.int8))
+    accn, _ = oracle.gemm_w8a8(q, s_tok, wqn, s_ch, want_y=False)
+    assert np.array_equal(accn, -128 * q.astype(np.int32))
+    onehot = np.zeros((3, K), np.int8)
+    onehot[0, 5], onehot[1, 63], onehot[2, 0] = 9, -128, 1
+    acc1, _ = oracle.gemm_w8a8(q, s_tok, onehot, _ones(3), want_y=False)
+    assert np.array_equal(acc1[:, 0], 9 * q[:, 5].astype(np.int32))
+    assert np.array_equal(acc1[:, 1], -128 * q[:, 63].astype(np.int32))
+    assert np.array_equal(acc1[:, 2], q[:, 0].astype(np.int32))
+
+
+def test_int32_no_overflow_bound():
+    # K * 128 * 128 < 2^31  <=>  K < 131072; the largest K of the workloads is 11008
+    K = 11008
+    q = np.full((1, K), -128, np.int8)
+    w = np.full((1, K), -128, np.int8)
+    acc, _ = oracle.gemm_w8a8(q, _ones(1), w, _ones(1), want_y=False)
+    assert int(acc[0, 0]) == K * 16384 < 2 ** 31
+    assert K * 127 * 127 < 2 ** 31
+    K = 131072
+    q = np.full((1, K), -128, np.int8)
+    w = np.full((1, K), -128, np.int8)
+    with pytest.raises(OverflowError):
+        oracle.gemm_w8a8(q, _ones(1), w, _ones(1))
+    w[0, 0] = 127  # one step inside the range again
+    acc, _ = oracle.gemm_w8a8(q, _ones(1), w, _ones(1), want_y=False)
+    assert int(acc[0, 0]) == (K - 1) * 16384 - 128 * 127
+
+
+def test_dequant_power_of_two_scales_is_exact():
+    rng = np.random.default_rng(14)
+    M, N, K = 6, 10, 16
+    q = rng.integers(-20, 21, (M, K)).astype(np.int8)
+    wq = rng.integers(-20, 21, (N, K)).astype(np.int8)
+    s_tok = (2.0 ** rng.integers(-6, 1, M)).astype(np.float32)
+    s_ch = (2.0 ** rng.integers(-6, 1, N)).astype(np.float32)
+    acc, y = oracle.gemm_w8a8(q, s_tok, wq, s_ch)
+    # |acc| <= 6400 needs 13 bits > FP16's 11, so compare with numpy's own double -> half rounding
+    want = (acc.astype(np.float64) * s_tok[:, None].astype(np.float64) * s_ch[None, :].astype(np.float64))
+    assert np.array_equal(y.view(np.uint16), want.astype(np.float16).view(np.uint16))
+    small = np.abs(acc) <= 2048
+    assert small.any() and np.array_equal(y[small].astype(np.float64), want[small])  # exact there
+    # zero scale gives an exact +0
+    s_tok[0] = 0
+    _, y0 = oracle.gemm_w8a8(q, s_tok, wq, s_ch)
+    assert (y0[0].view(np.uint16) & 0x7FFF == 0).all()
+
+
+def test_gemm_w4a8_group_accumulators_and_reduction_to_w8a8():
+    rng = np.random.default_rng(15)
+    M, N, K, G = 9, 12, 512, 4
+    q = rng.integers(-128, 128, (M, K)).astype(np.int8)
+    codes = rng.integers(-8, 8, (N, K)).astype(np.int8)
+    codes[3, 128:256] = 0  # an all-zero group contributes exactly 0
+    s_tok = (2.0 ** rng.integers(-4, 1, M)).astype(np.float32)
+    sg_equal = np.full((N, G), 0.125, np.float16)
+    acc_g, y = oracle.gemm_w4a8(q, s_tok, codes, sg_equal, 128)
+    q64, c64 = q.astype(np.int64), codes.astype(np.int64)
+    for g in range(G):
+        sl = slice(128 * g, 128 * (g + 1))
+        assert np.array_equal(acc_g[:, :, g].astype(np.int64), q64[:, sl] @ c64[:, sl].T)
+    assert not acc_g[:, 3, 1].any()
+    full = q64 @ c64.T
+    assert np.array_equal(acc_g.astype(np.int64).sum(axis=2), full)
+    # with all group scales equal to one power of two it reduces to the per-channel formula
+    _, y8 = oracle.gemm_w8a8(q, s_tok, codes, np.full((N,), 0.125, np.float32))
+    assert np.array_equal(y.view(np.uint16), y8.view(np.uint16))
+    # distinct group scales: compare with the definition written out in numpy binary64
+    sg = (rng.uniform(0.5, 2.0, (N, G)) * 2.0 ** -8).astype(np.float16)
+    acc_g2, y2 = oracle.gemm_w4a8(q, s_tok, codes, sg, 128)
+    R = (acc_g2.astype(np.float64) * sg.astype(np.float64)[None]).sum(axis=2)
+    want = (R * s_tok[:, None].astype(np.float64)).astype(np.float16)
+    diff = np.abs(y2.astype(np.float64) - want.astype(np.float64))
+    assert (diff <= 2.0 ** -10 * np.abs(want.astype(np.float64))).all()  # summation order only
+    # extremes: -128 x -8 over one group
+    qe = np.full((1, 128), -128, np.int8)
+    ce = np.full((1, 128), -8, np.int8)
+    ae, _ = oracle.gemm_w4a8(qe, _ones(1), ce, np.ones((1, 1), np.float16), 128, want_y=False)
+    assert int(ae[0, 0, 0]) == 128 * 128 * 8 == 2 ** 17
+
+
+def test_end_to_end_error_is_consistent_with_half_step_noise():
+    from paper_2512_23367_b200 import synth
+    x = synth.activations(64, 1024, seed=5)
+    w = synth.weights(96, 1024, seed=5)
+    q, s_tok = oracle.quantize_act(x)
+    exact = x.astype(np.float64) @ w.astype(np.float64).T
+    wq, s_ch = oracle.pack_w8(w)
+    _, y8 = oracle.gemm_w8a8(q, s_tok, wq, s_ch)
+    rel8 = np.linalg.norm(y8.astype(np.float64) - exact) / np.linalg.norm(exact)
+    codes, sg = oracle.pack_w4(w, 128)
+    _, y4 = oracle.gemm_w4a8(q, s_tok, codes, sg, 128)
+    rel4 = np.linalg.norm(y4.astype(np.float64) - exact) / np.linalg.norm(exact)
+    # activation half-step noise against outlier-dominated signal gives a few percent for W8A8;
+    # 4-bit weights add roughly (1/sqrt(12)) * s/sigma ~ 10 %.
+    assert rel8 < 0.10 and rel8 < rel4 < 0.25
