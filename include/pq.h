@@ -1,0 +1,145 @@
+/*
+ * pq.h -- C ABI of the B200 (sm_100a) quantized linear layer: W8A8 and W4A8.
+ *
+ * The library implements the quantized linear operator of a decoder LLM as the
+ * paper's "Unified low-bit inference framework" section states it: activations are
+ * quantized per token to INT8, multiplied with INT8 (or packed INT4) weights in
+ * integer arithmetic, and the INT32 result is dequantized to FP16.  The quantizer is
+ * the paper's Eq. 1-2 with symmetric scaling (no zero point).
+ *
+ * Conventions for every call
+ *   - All data pointers are DEVICE pointers owned by the caller, 16-byte aligned.
+ *     The library allocates and frees no device memory.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *     Calls are asynchronous and stream-ordered; none synchronizes the device.
+ *   - Matrices are dense row-major: X/Q/Y have one token per row, W has one output
+ *     channel per row (K contiguous).
+ *   - The return value is a pq_status.  Argument errors are detected before anything
+ *     is launched.  Nothing aborts, throws or traps; non-finite inputs are memory
+ *     safe with unspecified results.
+ *   - Every wait inside a kernel is bounded; if one expires the kernel records
+ *     PQ_ERR_TIMEOUT in a device status word, drains and returns.  pq_device_status()
+ *     reads that word.
+ *   - Requires compute capability 10.0; anything else returns PQ_ERR_ARCH (there is
+ *     no fallback path).
+ */
+#ifndef PQ_H_
+#define PQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define PQ_API __attribute__((visibility("default")))
+#else
+#define PQ_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  PQ_OK = 0,
+  PQ_ERR_NULL = 1,    /* a required pointer is NULL */
+  PQ_ERR_SHAPE = 2,   /* a size is non-positive or violates a divisibility rule */
+  PQ_ERR_ALIGN = 3,   /* a pointer is not 16-byte aligned */
+  PQ_ERR_ARCH = 4,    /* the current device is not compute capability 10.0 */
+  PQ_ERR_CUDA = 5,    /* a CUDA runtime/driver call or a launch failed */
+  PQ_ERR_TIMEOUT = 6, /* a bounded wait inside a kernel expired (device status word) */
+  PQ_ERR_LIMIT = 7    /* a size exceeds a stated maximum of the entry point */
+} pq_status;
+
+/* Static string for a status code. */
+PQ_API const char* pq_status_str(int status);
+
+/* Shape rules shared by the calls below (else PQ_ERR_SHAPE):
+ *   M >= 1, N >= 8 with N % 8 == 0, K >= 16 with K % 16 == 0, K < 131072 (so that
+ *   K * 128 * 128 fits INT32); W4 additionally needs group == 128 and K % 128 == 0. */
+
+/*
+ * Per-token symmetric INT8 activation quantization (Eq. 1-2 with n = 8; one scale
+ * per token over the feature dimension).  For each row m:
+ *   a = max_k |X[m,k]|,  s_tok[m] = a / 127.5 (= 2a/255),
+ *   Q[m,k] = clamp(rne(X[m,k] * (127.5 / a)), -128, 127),
+ * evaluated in IEEE binary32 with round-half-to-even; an all-zero row gives scale 0
+ * and codes 0.
+ *   x_f16 [M,K] FP16 in;  q [M,K] INT8 out;  s_tok [M] FP32 out.
+ */
+PQ_API int pq_quantize_act(const void* x_f16, int64_t M, int64_t K, int8_t* q, float* s_tok,
+                    void* stream);
+
+/*
+ * Offline per-output-channel INT8 weight quantization (Eq. 2 with n = 8, one scale
+ * per output channel) into the layout the W8A8 GEMM reads.
+ *   s_ch[n] = max_k |W[n,k]| / 127.5,  code = clamp(rne(W[n,k] / s_ch[n]), -128, 127).
+ *   w_f16 [N,K] FP16 in;  wq: pq_packed_w8_bytes(N,K) bytes out (opaque);
+ *   s_ch [N] FP32 out.
+ */
+PQ_API int pq_pack_w8(const void* w_f16, int64_t N, int64_t K, void* wq, float* s_ch, void* stream);
+
+/*
+ * Offline group-wise INT4 weight quantization (Eq. 2 with n = 4, one scale per output
+ * channel and group of `group` consecutive k) into the packed layout the W4A8 GEMM
+ * reads (two codes per byte along K).
+ *   s = fp16(max_{k in g} |W[n,k]| / 7.5),  code = clamp(rne(W[n,k] / float(s)), -8, 7).
+ *   w_f16 [N,K] FP16 in;  wp: pq_packed_w4_bytes(N,K) bytes out (opaque);
+ *   s_grp_f16 [K/group, N] FP16 out (the scales of one K-group are contiguous over n).
+ */
+PQ_API int pq_pack_w4(const void* w_f16, int64_t N, int64_t K, int32_t group, void* wp,
+               void* s_grp_f16, void* stream);
+
+PQ_API size_t pq_packed_w8_bytes(int64_t N, int64_t K);
+PQ_API size_t pq_packed_w4_bytes(int64_t N, int64_t K);
+
+/* Recover the integer codes from the opaque layouts as row-major INT8 [N,K]
+ * (W4 codes lie in [-8,7]).  For checking and interchange; not on the hot path. */
+PQ_API int pq_unpack_w8(const void* wq, int64_t N, int64_t K, int8_t* codes, void* stream);
+PQ_API int pq_unpack_w4(const void* wp, int64_t N, int64_t K, int8_t* codes, void* stream);
+
+/*
+ * W8A8 linear ("weight layout, dequantization logic and matrix multiplication" of the
+ * framework section; weight-activation quantization runs the product itself in
+ * integers):
+ *   ACC[m,n] = sum_k Q[m,k] * Wq[n,k]                      exact, INT32
+ *   Y[m,n]   = fp16( float(ACC[m,n]) * s_tok[m] * s_ch[n] )
+ *   q [M,K] INT8, s_tok [M] FP32 (from pq_quantize_act);  wq, s_ch [N] (from pq_pack_w8);
+ *   y_f16 [M,N] FP16 out.
+ * Any M is accepted; small M (decode shapes) is routed to a weight-streaming schedule
+ * that computes the same result.
+ */
+PQ_API int pq_gemm_w8a8(const int8_t* q, const float* s_tok, const void* wq, const float* s_ch,
+                 int64_t M, int64_t N, int64_t K, void* y_f16, void* stream);
+
+/*
+ * W4A8 linear: INT4 codes are widened to INT8 inside the kernel, multiplied in
+ * integers per K-group and dequantized per group into an FP32 running sum:
+ *   ACC_g[m,n] = sum_{k in group g} Q[m,k] * C[n,k]        exact, INT32
+ *   R[m,n]     = sum_g float(ACC_g[m,n]) * float(s_grp[g,n])   (FP32, g ascending)
+ *   Y[m,n]     = fp16( R[m,n] * s_tok[m] )
+ *   wp, s_grp_f16 [K/group, N] from pq_pack_w4;  group must be 128.
+ */
+PQ_API int pq_gemm_w4a8(const int8_t* q, const float* s_tok, const void* wp, const void* s_grp_f16,
+                 int32_t group, int64_t M, int64_t N, int64_t K, void* y_f16, void* stream);
+
+/*
+ * The exact INT32 accumulators of the two linears, computed by the same tensor-core
+ * main loops as the calls above and written out instead of the FP16 result (for
+ * parity checking).   acc [M,N];   acc_g [K/group, M, N] (group-major).
+ */
+PQ_API int pq_acc_w8a8(const int8_t* q, const void* wq, int64_t M, int64_t N, int64_t K, int32_t* acc,
+                void* stream);
+PQ_API int pq_acc_w4a8(const int8_t* q, const void* wp, int32_t group, int64_t M, int64_t N, int64_t K,
+                int32_t* acc_g, void* stream);
+
+/*
+ * Reads the device status word of the current device into *host_status (PQ_OK or
+ * PQ_ERR_TIMEOUT) and clears it.  Synchronizes the device; call it outside timed
+ * regions.
+ */
+PQ_API int pq_device_status(int* host_status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PQ_H_ */

@@ -1,0 +1,23 @@
+"""B200 (sm_100a) quantized linear layer: per-token INT8 activations times INT8 / packed-INT4
+weights on the tcgen05 tensor cores, dequantized to FP16.
+
+The compute lives in ``libpq.so`` (CUDA, C ABI declared in ``include/pq.h``); this package is
+the argument-marshalling binding with the same call names.  ``synth`` holds the seeded input
+generators.  Importing the package does not load the CUDA library; the first call does, and
+raises if it cannot be loaded -- there is no CPU or library fallback.
+"""
+from . import synth  # noqa: F401
+from .binding import (  # noqa: F401
+    PQError,
+    lib,
+    pq_acc_w4a8,
+    pq_acc_w8a8,
+    pq_device_status,
+    pq_gemm_w4a8,
+    pq_gemm_w8a8,
+    pq_pack_w4,
+    pq_pack_w8,
+    pq_quantize_act,
+    pq_unpack_w4,
+    pq_unpack_w8,
+)

@@ -1,0 +1,174 @@
+"""ctypes binding of libpq.so.  Marshals torch CUDA tensors (device pointers, sizes, the current
+stream) into the C calls of ``include/pq.h``; every step of the computation runs in the library's
+kernels.  torch is used for device memory and streams only."""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+from . import build as _build
+
+GROUP = 128
+
+_lib = None
+
+_i64, _i32, _vp = ctypes.c_int64, ctypes.c_int32, ctypes.c_void_p
+
+# name -> (restype, argtypes); mirrors include/pq.h
+SIGNATURES = {
+    "pq_status_str": (ctypes.c_char_p, [ctypes.c_int]),
+    "pq_packed_w8_bytes": (ctypes.c_size_t, [_i64, _i64]),
+    "pq_packed_w4_bytes": (ctypes.c_size_t, [_i64, _i64]),
+    "pq_quantize_act": (ctypes.c_int, [_vp, _i64, _i64, _vp, _vp, _vp]),
+    "pq_pack_w8": (ctypes.c_int, [_vp, _i64, _i64, _vp, _vp, _vp]),
+    "pq_pack_w4": (ctypes.c_int, [_vp, _i64, _i64, _i32, _vp, _vp, _vp]),
+    "pq_unpack_w8": (ctypes.c_int, [_vp, _i64, _i64, _vp, _vp]),
+    "pq_unpack_w4": (ctypes.c_int, [_vp, _i64, _i64, _vp, _vp]),
+    "pq_gemm_w8a8": (ctypes.c_int, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _vp, _vp]),
+    "pq_gemm_w4a8": (ctypes.c_int, [_vp, _vp, _vp, _vp, _i32, _i64, _i64, _i64, _vp, _vp]),
+    "pq_acc_w8a8": (ctypes.c_int, [_vp, _vp, _i64, _i64, _i64, _vp, _vp]),
+    "pq_acc_w4a8": (ctypes.c_int, [_vp, _vp, _i32, _i64, _i64, _i64, _vp, _vp]),
+    "pq_device_status": (ctypes.c_int, [ctypes.POINTER(ctypes.c_int)]),
+}
+
+
+class PQError(RuntimeError):
+    def __init__(self, call: str, status: int):
+        self.status = status
+        msg = lib().pq_status_str(status).decode() if _lib is not None else "?"
+        super().__init__(f"{call} failed: status {status} ({msg})")
+
+
+def lib() -> ctypes.CDLL:
+    """Load (building first if missing or stale) libpq.so.  Raises if that is impossible."""
+    global _lib
+    if _lib is None:
+        path = _build.LIB
+        if _build.stale():
+            path = _build.build()
+        if not os.path.exists(path):
+            raise RuntimeError(f"CUDA library {path} is missing and could not be built")
+        handle = ctypes.CDLL(path)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(handle, name)  # AttributeError if the library lacks a declared symbol
+            fn.restype, fn.argtypes = res, args
+        _lib = handle
+    return _lib
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _dev(t: torch.Tensor, dtype: torch.dtype, what: str) -> torch.Tensor:
+    if not t.is_cuda:
+        raise ValueError(f"{what}: expected a CUDA tensor (this library has no CPU path)")
+    if t.dtype != dtype:
+        raise TypeError(f"{what}: expected {dtype}, got {t.dtype}")
+    if not t.is_contiguous():
+        raise ValueError(f"{what}: expected a contiguous tensor")
+    return t
+
+
+def _check(call: str, status: int) -> None:
+    if status != 0:
+        raise PQError(call, status)
+
+
+def pq_quantize_act(x: torch.Tensor, q: torch.Tensor | None = None, s_tok: torch.Tensor | None = None):
+    """x f16 [M,K] -> (q int8 [M,K], s_tok f32 [M])."""
+    x = _dev(x, torch.float16, "x")
+    M, K = x.shape
+    if q is None:
+        q = torch.empty((M, K), dtype=torch.int8, device=x.device)
+    if s_tok is None:
+        s_tok = torch.empty((M,), dtype=torch.float32, device=x.device)
+    _check("pq_quantize_act", lib().pq_quantize_act(x.data_ptr(), M, K, q.data_ptr(), s_tok.data_ptr(), _stream()))
+    return q, s_tok
+
+
+def pq_pack_w8(w: torch.Tensor):
+    """w f16 [N,K] -> (wq opaque uint8 buffer, s_ch f32 [N])."""
+    w = _dev(w, torch.float16, "w")
+    N, K = w.shape
+    wq = torch.empty((lib().pq_packed_w8_bytes(N, K),), dtype=torch.uint8, device=w.device)
+    s_ch = torch.empty((N,), dtype=torch.float32, device=w.device)
+    _check("pq_pack_w8", lib().pq_pack_w8(w.data_ptr(), N, K, wq.data_ptr(), s_ch.data_ptr(), _stream()))
+    return wq, s_ch
+
+
+def pq_pack_w4(w: torch.Tensor, group: int = GROUP):
+    """w f16 [N,K] -> (wp opaque uint8 buffer, s_grp f16 [K/group, N])."""
+    w = _dev(w, torch.float16, "w")
+    N, K = w.shape
+    wp = torch.empty((lib().pq_packed_w4_bytes(N, K),), dtype=torch.uint8, device=w.device)
+    s_grp = torch.empty((max(K // max(group, 1), 1), N), dtype=torch.float16, device=w.device)
+    _check("pq_pack_w4", lib().pq_pack_w4(w.data_ptr(), N, K, group, wp.data_ptr(), s_grp.data_ptr(), _stream()))
+    return wp, s_grp
+
+
+def pq_unpack_w8(wq: torch.Tensor, N: int, K: int) -> torch.Tensor:
+    wq = _dev(wq, torch.uint8, "wq")
+    codes = torch.empty((N, K), dtype=torch.int8, device=wq.device)
+    _check("pq_unpack_w8", lib().pq_unpack_w8(wq.data_ptr(), N, K, codes.data_ptr(), _stream()))
+    return codes
+
+
+def pq_unpack_w4(wp: torch.Tensor, N: int, K: int) -> torch.Tensor:
+    wp = _dev(wp, torch.uint8, "wp")
+    codes = torch.empty((N, K), dtype=torch.int8, device=wp.device)
+    _check("pq_unpack_w4", lib().pq_unpack_w4(wp.data_ptr(), N, K, codes.data_ptr(), _stream()))
+    return codes
+
+
+def pq_gemm_w8a8(q, s_tok, wq, s_ch, N: int, y: torch.Tensor | None = None) -> torch.Tensor:
+    """q int8 [M,K], s_tok f32 [M], wq/s_ch from pq_pack_w8 -> y f16 [M,N]."""
+    q = _dev(q, torch.int8, "q")
+    M, K = q.shape
+    _dev(s_tok, torch.float32, "s_tok"), _dev(wq, torch.uint8, "wq"), _dev(s_ch, torch.float32, "s_ch")
+    if y is None:
+        y = torch.empty((M, N), dtype=torch.float16, device=q.device)
+    _check("pq_gemm_w8a8", lib().pq_gemm_w8a8(q.data_ptr(), s_tok.data_ptr(), wq.data_ptr(), s_ch.data_ptr(),
+                                              M, N, K, y.data_ptr(), _stream()))
+    return y
+
+
+def pq_gemm_w4a8(q, s_tok, wp, s_grp, N: int, group: int = GROUP, y: torch.Tensor | None = None) -> torch.Tensor:
+    """q int8 [M,K], s_tok f32 [M], wp/s_grp from pq_pack_w4 -> y f16 [M,N]."""
+    q = _dev(q, torch.int8, "q")
+    M, K = q.shape
+    _dev(s_tok, torch.float32, "s_tok"), _dev(wp, torch.uint8, "wp"), _dev(s_grp, torch.float16, "s_grp")
+    if y is None:
+        y = torch.empty((M, N), dtype=torch.float16, device=q.device)
+    _check("pq_gemm_w4a8", lib().pq_gemm_w4a8(q.data_ptr(), s_tok.data_ptr(), wp.data_ptr(), s_grp.data_ptr(),
+                                              group, M, N, K, y.data_ptr(), _stream()))
+    return y
+
+
+def pq_acc_w8a8(q, wq, N: int) -> torch.Tensor:
+    """Exact INT32 accumulators [M,N] of the W8A8 product."""
+    q = _dev(q, torch.int8, "q")
+    M, K = q.shape
+    _dev(wq, torch.uint8, "wq")
+    acc = torch.empty((M, N), dtype=torch.int32, device=q.device)
+    _check("pq_acc_w8a8", lib().pq_acc_w8a8(q.data_ptr(), wq.data_ptr(), M, N, K, acc.data_ptr(), _stream()))
+    return acc
+
+
+def pq_acc_w4a8(q, wp, N: int, group: int = GROUP) -> torch.Tensor:
+    """Exact INT32 per-group accumulators [K/group, M, N] of the W4A8 product."""
+    q = _dev(q, torch.int8, "q")
+    M, K = q.shape
+    _dev(wp, torch.uint8, "wp")
+    acc = torch.empty((K // group, M, N), dtype=torch.int32, device=q.device)
+    _check("pq_acc_w4a8", lib().pq_acc_w4a8(q.data_ptr(), wp.data_ptr(), group, M, N, K, acc.data_ptr(), _stream()))
+    return acc
+
+
+def pq_device_status() -> int:
+    """Synchronizes; returns and clears the device status word (0 = ok, 6 = a bounded wait expired)."""
+    v = ctypes.c_int(0)
+    _check("pq_device_status", lib().pq_device_status(ctypes.byref(v)))
+    return int(v.value)

@@ -1,0 +1,249 @@
+// C-ABI entry points of libpq: argument validation, device checks, dispatch.
+// See include/pq.h for the contract of every call.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include "pq_internal.h"
+
+namespace pq {
+
+__device__ int g_status_word = 0;
+
+namespace {
+
+constexpr int kMaxDevices = 64;
+constexpr int64_t kSmallM = 64;  // M at or below this takes the weight-streaming schedule
+
+struct DeviceInfo {
+  bool probed = false;
+  bool ok = false;
+  int sms = 0;
+  int* status = nullptr;
+};
+DeviceInfo g_dev[kMaxDevices];
+
+DeviceInfo* current_device() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  DeviceInfo& d = g_dev[dev];
+  if (!d.probed) {
+    int major = 0, minor = 0, sms = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return nullptr;
+    if (cudaDeviceGetAttribute(&minor, cudaDevAttrComputeCapabilityMinor, dev) != cudaSuccess) return nullptr;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return nullptr;
+    d.sms = sms;
+    d.ok = (major == 10 && minor == 0);
+    if (d.ok) {
+      void* p = nullptr;
+      if (cudaGetSymbolAddress(&p, g_status_word) != cudaSuccess) return nullptr;
+      d.status = static_cast<int*>(p);
+    }
+    d.probed = true;
+  }
+  return &d;
+}
+
+int check_arch() {
+  DeviceInfo* d = current_device();
+  if (d == nullptr) {
+    cudaGetLastError();
+    return PQ_ERR_CUDA;
+  }
+  return d->ok ? PQ_OK : PQ_ERR_ARCH;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_rows(int64_t rows, int64_t K) {
+  if (rows < 1 || rows > 0x7fffffff) return PQ_ERR_SHAPE;
+  if (K < 16 || K % 16 != 0 || K >= 131072) return PQ_ERR_SHAPE;
+  return PQ_OK;
+}
+
+int check_gemm(int64_t M, int64_t N, int64_t K) {
+  int rc = check_rows(M, K);
+  if (rc != PQ_OK) return rc;
+  if (N < 8 || N % 8 != 0 || N > 0x7fffffff) return PQ_ERR_SHAPE;
+  if (M * N > (int64_t(1) << 40)) return PQ_ERR_SHAPE;
+  return PQ_OK;
+}
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                   CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+
+}  // namespace
+
+int* device_status_ptr() {
+  DeviceInfo* d = current_device();
+  return d ? d->status : nullptr;
+}
+
+int sm_count() {
+  DeviceInfo* d = current_device();
+  return d ? d->sms : 1;
+}
+
+int make_tmap_2d(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows,
+                 uint32_t box_cols, uint32_t elem_bytes, bool swizzle128) {
+  if (g_encode == nullptr) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess || fn == nullptr) {
+      cudaGetLastError();
+      return PQ_ERR_CUDA;
+    }
+    g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+  }
+  CUtensorMapDataType dt = elem_bytes == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8
+                           : elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_UINT16
+                                             : CU_TENSOR_MAP_DATA_TYPE_UINT32;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * elem_bytes};
+  cuuint32_t box[2] = {box_cols, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = g_encode(out, dt, 2, const_cast<void*>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? PQ_OK : PQ_ERR_CUDA;
+}
+
+}  // namespace pq
+
+using namespace pq;
+
+extern "C" {
+
+const char* pq_status_str(int status) {
+  switch (status) {
+    case PQ_OK: return "ok";
+    case PQ_ERR_NULL: return "null pointer argument";
+    case PQ_ERR_SHAPE: return "invalid shape";
+    case PQ_ERR_ALIGN: return "pointer not 16-byte aligned";
+    case PQ_ERR_ARCH: return "device is not compute capability 10.0";
+    case PQ_ERR_CUDA: return "CUDA call or launch failed";
+    case PQ_ERR_TIMEOUT: return "bounded wait inside a kernel expired";
+    case PQ_ERR_LIMIT: return "size exceeds the entry point's maximum";
+    default: return "unknown status";
+  }
+}
+
+size_t pq_packed_w8_bytes(int64_t N, int64_t K) {
+  return (N > 0 && K > 0) ? static_cast<size_t>(N) * static_cast<size_t>(K) : 0;
+}
+size_t pq_packed_w4_bytes(int64_t N, int64_t K) {
+  return (N > 0 && K > 0) ? static_cast<size_t>(N) * static_cast<size_t>(K) / 2 : 0;
+}
+
+int pq_quantize_act(const void* x_f16, int64_t M, int64_t K, int8_t* q, float* s_tok, void* stream) {
+  if (!x_f16 || !q || !s_tok) return PQ_ERR_NULL;
+  int rc = check_rows(M, K);
+  if (rc != PQ_OK) return rc;
+  if (!aligned16(x_f16) || !aligned16(q)) return PQ_ERR_ALIGN;
+  if ((rc = check_arch()) != PQ_OK) return rc;
+  return launch_quantize_act(x_f16, M, K, q, s_tok, false, static_cast<cudaStream_t>(stream));
+}
+
+int pq_pack_w8(const void* w_f16, int64_t N, int64_t K, void* wq, float* s_ch, void* stream) {
+  if (!w_f16 || !wq || !s_ch) return PQ_ERR_NULL;
+  int rc = check_gemm(1, N, K);
+  if (rc != PQ_OK) return rc;
+  if (!aligned16(w_f16) || !aligned16(wq)) return PQ_ERR_ALIGN;
+  if ((rc = check_arch()) != PQ_OK) return rc;
+  // The W8 layout the GEMM reads is the row-major code matrix itself (K contiguous per channel).
+  return launch_quantize_act(w_f16, N, K, static_cast<int8_t*>(wq), s_ch, true, static_cast<cudaStream_t>(stream));
+}
+
+int pq_pack_w4(const void* w_f16, int64_t N, int64_t K, int32_t group, void* wp, void* s_grp_f16, void* stream) {
+  if (!w_f16 || !wp || !s_grp_f16) return PQ_ERR_NULL;
+  int rc = check_gemm(1, N, K);
+  if (rc != PQ_OK) return rc;
+  if (group != 128 || K % 128 != 0) return PQ_ERR_SHAPE;
+  if (!aligned16(w_f16) || !aligned16(wp) || !aligned16(s_grp_f16)) return PQ_ERR_ALIGN;
+  if ((rc = check_arch()) != PQ_OK) return rc;
+  return launch_pack_w4(w_f16, N, K, wp, s_grp_f16, static_cast<cudaStream_t>(stream));
+}
+
+int pq_unpack_w8(const void* wq, int64_t N, int64_t K, int8_t* codes, void* stream) {
+  if (!wq || !codes) return PQ_ERR_NULL;
+  int rc = check_gemm(1, N, K);
+  if (rc != PQ_OK) return rc;
+  if ((rc = check_arch()) != PQ_OK) return rc;
+  return cuda_status(cudaMemcpyAsync(codes, wq, static_cast<size_t>(N) * K, cudaMemcpyDeviceToDevice,
+                                     static_cast<cudaStream_t>(stream)));
+}
+
+int pq_unpack_w4(const void* wp, int64_t N, int64_t K, int8_t* codes, void* stream) {
+  if (!wp || !codes) return PQ_ERR_NULL;
+  int rc = check_gemm(1, N, K);
+  if (rc != PQ_OK) return rc;
+  if (K % 128 != 0) return PQ_ERR_SHAPE;
+  if ((rc = check_arch()) != PQ_OK) return rc;
+  return launch_unpack_w4(wp, N, K, codes, static_cast<cudaStream_t>(stream));
+}
+
+static int gemm_w8a8_common(const int8_t* q, const float* s_tok, const void* wq, const float* s_ch, int64_t M,
+                            int64_t N, int64_t K, void* y, int32_t* acc, void* stream) {
+  int rc = check_gemm(M, N, K);
+  if (rc != PQ_OK) return rc;
+  if (!aligned16(q) || !aligned16(wq) || !aligned16(y) || !aligned16(acc)) return PQ_ERR_ALIGN;
+  if ((rc = check_arch()) != PQ_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (M <= kSmallM) return launch_smallm_w8a8(q, s_tok, wq, s_ch, M, N, K, y, acc, st);
+  return launch_gemm_w8a8(q, s_tok, wq, s_ch, M, N, K, y, acc, st);
+}
+
+int pq_gemm_w8a8(const int8_t* q, const float* s_tok, const void* wq, const float* s_ch, int64_t M, int64_t N,
+                 int64_t K, void* y_f16, void* stream) {
+  if (!q || !s_tok || !wq || !s_ch || !y_f16) return PQ_ERR_NULL;
+  return gemm_w8a8_common(q, s_tok, wq, s_ch, M, N, K, y_f16, nullptr, stream);
+}
+
+int pq_acc_w8a8(const int8_t* q, const void* wq, int64_t M, int64_t N, int64_t K, int32_t* acc, void* stream) {
+  if (!q || !wq || !acc) return PQ_ERR_NULL;
+  return gemm_w8a8_common(q, nullptr, wq, nullptr, M, N, K, nullptr, acc, stream);
+}
+
+static int gemm_w4a8_common(const int8_t* q, const float* s_tok, const void* wp, const void* s_grp, int32_t group,
+                            int64_t M, int64_t N, int64_t K, void* y, int32_t* acc_g, void* stream) {
+  int rc = check_gemm(M, N, K);
+  if (rc != PQ_OK) return rc;
+  if (group != 128 || K % 128 != 0) return PQ_ERR_SHAPE;
+  if (!aligned16(q) || !aligned16(wp) || !aligned16(s_grp) || !aligned16(y) || !aligned16(acc_g)) return PQ_ERR_ALIGN;
+  if ((rc = check_arch()) != PQ_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (M <= kSmallM) return launch_smallm_w4a8(q, s_tok, wp, s_grp, M, N, K, y, acc_g, st);
+  return launch_gemm_w4a8(q, s_tok, wp, s_grp, M, N, K, y, acc_g, st);
+}
+
+int pq_gemm_w4a8(const int8_t* q, const float* s_tok, const void* wp, const void* s_grp_f16, int32_t group,
+                 int64_t M, int64_t N, int64_t K, void* y_f16, void* stream) {
+  if (!q || !s_tok || !wp || !s_grp_f16 || !y_f16) return PQ_ERR_NULL;
+  return gemm_w4a8_common(q, s_tok, wp, s_grp_f16, group, M, N, K, y_f16, nullptr, stream);
+}
+
+int pq_acc_w4a8(const int8_t* q, const void* wp, int32_t group, int64_t M, int64_t N, int64_t K, int32_t* acc_g,
+                void* stream) {
+  if (!q || !wp || !acc_g) return PQ_ERR_NULL;
+  return gemm_w4a8_common(q, nullptr, wp, nullptr, group, M, N, K, nullptr, acc_g, stream);
+}
+
+int pq_device_status(int* host_status) {
+  if (!host_status) return PQ_ERR_NULL;
+  int rc = check_arch();
+  if (rc != PQ_OK) return rc;
+  int* p = device_status_ptr();
+  if (!p) return PQ_ERR_CUDA;
+  if (cudaDeviceSynchronize() != cudaSuccess) return PQ_ERR_CUDA;
+  int v = 0;
+  if (cudaMemcpy(&v, p, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return PQ_ERR_CUDA;
+  if (v != 0 && cudaMemset(p, 0, sizeof(int)) != cudaSuccess) return PQ_ERR_CUDA;
+  *host_status = v;
+  return PQ_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,43 @@
+// Internal declarations shared by the translation units of libpq (not part of the ABI).
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/pq.h"
+
+namespace pq {
+
+// Device status word (one per device that loaded the library): PQ_OK or PQ_ERR_TIMEOUT.
+int* device_status_ptr();  // device address of the status word of the current device, or nullptr
+
+// Number of SMs of the current device (cached per device).
+int sm_count();
+
+// cuTensorMapEncodeTiled obtained through the runtime (no link-time dependency on libcuda).
+// Encodes a 2-D row-major tensor [rows, cols] of `elem_bytes`-sized elements with a
+// box of [box_rows, box_cols]; swizzle128 selects the 128-byte shared-memory swizzle.
+int make_tmap_2d(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows,
+                 uint32_t box_cols, uint32_t elem_bytes, bool swizzle128);
+
+// ---- launchers (each returns a pq_status; all are asynchronous on `stream`) ----
+int launch_quantize_act(const void* x, int64_t M, int64_t K, int8_t* q, float* s, bool divide_by_scale,
+                        cudaStream_t stream);
+int launch_pack_w4(const void* w, int64_t N, int64_t K, void* wp, void* s_grp, cudaStream_t stream);
+int launch_unpack_w4(const void* wp, int64_t N, int64_t K, int8_t* codes, cudaStream_t stream);
+
+// Prefill-shaped W8A8 GEMM (tcgen05 kind::i8).  Exactly one of y / acc is non-null.
+int launch_gemm_w8a8(const int8_t* q, const float* s_tok, const void* wq, const float* s_ch, int64_t M,
+                     int64_t N, int64_t K, void* y, int32_t* acc, cudaStream_t stream);
+// Prefill-shaped W4A8 GEMM.  Exactly one of y / acc_g is non-null.
+int launch_gemm_w4a8(const int8_t* q, const float* s_tok, const void* wp, const void* s_grp, int64_t M,
+                     int64_t N, int64_t K, void* y, int32_t* acc_g, cudaStream_t stream);
+// Small-M (decode-shaped) weight-streaming variants; same results as the calls above.
+int launch_smallm_w8a8(const int8_t* q, const float* s_tok, const void* wq, const float* s_ch, int64_t M,
+                       int64_t N, int64_t K, void* y, int32_t* acc, cudaStream_t stream);
+int launch_smallm_w4a8(const int8_t* q, const float* s_tok, const void* wp, const void* s_grp, int64_t M,
+                       int64_t N, int64_t K, void* y, int32_t* acc_g, cudaStream_t stream);
+
+inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? PQ_OK : PQ_ERR_CUDA; }
+
+}  // namespace pq

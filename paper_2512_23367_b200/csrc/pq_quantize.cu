@@ -1,0 +1,198 @@
+// Row-wise symmetric quantizers (Eq. 1-2 of the paper):
+//   - per-token INT8 activation quantization (hot path, HBM bound: 2 B read + 1 B written
+//     per element),
+//   - per-output-channel INT8 weight quantization (offline),
+//   - group-wise INT4 weight quantization + nibble packing (offline), and its inverse.
+#include <cuda_fp16.h>
+
+#include "pq_internal.h"
+
+namespace pq {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kCached = 8;  // 16-byte chunks of a row that one thread keeps in registers
+
+__device__ __forceinline__ float absmax8(const uint4& v) {
+  const __half2* h = reinterpret_cast<const __half2*>(&v);
+  __half2 m = __hmax2(__hmax2(__habs2(h[0]), __habs2(h[1])), __hmax2(__habs2(h[2]), __habs2(h[3])));
+  return fmaxf(__low2float(m), __high2float(m));
+}
+
+// Eq. 1 for one value: round-half-to-even of the scaled value, clamped to [-128, 127].
+template <bool kDivide>
+__device__ __forceinline__ int code8(__half x, float f) {
+  float t = kDivide ? __fdiv_rn(__half2float(x), f) : __fmul_rn(__half2float(x), f);
+  int r = __float2int_rn(t);
+  return max(-128, min(127, r));
+}
+
+template <bool kDivide>
+__device__ __forceinline__ uint2 quantize8(const uint4& v, float f) {
+  const __half* h = reinterpret_cast<const __half*>(&v);
+  uint32_t lo = 0, hi = 0;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    lo |= static_cast<uint32_t>(code8<kDivide>(h[i], f) & 0xff) << (8 * i);
+    hi |= static_cast<uint32_t>(code8<kDivide>(h[4 + i], f) & 0xff) << (8 * i);
+  }
+  return make_uint2(lo, hi);
+}
+
+// T threads cooperate on one row; a block of 256 threads handles 256/T rows.
+//   kDivide = false: activations, code = rne(x * (127.5 / a))
+//   kDivide = true : weights,     code = rne(x / (a / 127.5))
+template <int T, bool kDivide>
+__global__ void __launch_bounds__(kThreads) quantize_rows_kernel(const uint4* __restrict__ x, int64_t M,
+                                                                 int K8, uint2* __restrict__ q,
+                                                                 float* __restrict__ scale) {
+  constexpr int kRowsPerBlock = kThreads / T;
+  constexpr int kWarpsPerRow = T / 32;
+  __shared__ float red[kThreads / 32];
+
+  const int tid = threadIdx.x;
+  const int t = tid % T;
+  const int64_t row = static_cast<int64_t>(blockIdx.x) * kRowsPerBlock + tid / T;
+  const bool live = row < M;
+  const uint4* xr = x + row * K8;
+
+  uint4 cache[kCached];
+  float a = 0.0f;
+  if (live) {
+#pragma unroll
+    for (int i = 0; i < kCached; ++i) {
+      int c = t + i * T;
+      if (c < K8) {
+        cache[i] = __ldg(xr + c);
+        a = fmaxf(a, absmax8(cache[i]));
+      }
+    }
+    for (int c = t + kCached * T; c < K8; c += T) a = fmaxf(a, absmax8(__ldg(xr + c)));
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
+  if constexpr (kWarpsPerRow > 1) {
+    if ((tid & 31) == 0) red[tid >> 5] = a;
+    __syncthreads();
+    const int w0 = (tid / T) * kWarpsPerRow;
+#pragma unroll
+    for (int w = 0; w < kWarpsPerRow; ++w) a = fmaxf(a, red[w0 + w]);
+  }
+  if (!live) return;
+
+  const float s = __fdiv_rn(a, 127.5f);
+  float f;
+  if (kDivide) {
+    f = (a == 0.0f) ? 1.0f : s;  // x / 1 = 0 for the all-zero row
+  } else {
+    f = (a == 0.0f) ? 0.0f : __fdiv_rn(127.5f, a);
+  }
+  if (t == 0) scale[row] = s;
+
+  uint2* qr = q + row * K8;
+#pragma unroll
+  for (int i = 0; i < kCached; ++i) {
+    int c = t + i * T;
+    if (c < K8) qr[c] = quantize8<kDivide>(cache[i], f);
+  }
+  for (int c = t + kCached * T; c < K8; c += T) qr[c] = quantize8<kDivide>(__ldg(xr + c), f);
+}
+
+template <bool kDivide>
+int launch_rows(const void* x, int64_t M, int64_t K, int8_t* q, float* s, cudaStream_t stream) {
+  const int K8 = static_cast<int>(K / 8);
+  const uint4* xp = static_cast<const uint4*>(x);
+  uint2* qp = reinterpret_cast<uint2*>(q);
+  // Pick the narrowest row team that still keeps the whole row in registers.
+  if (K8 <= 32 * kCached) {
+    quantize_rows_kernel<32, kDivide><<<static_cast<unsigned>((M + 7) / 8), kThreads, 0, stream>>>(xp, M, K8, qp, s);
+  } else if (K8 <= 64 * kCached) {
+    quantize_rows_kernel<64, kDivide><<<static_cast<unsigned>((M + 3) / 4), kThreads, 0, stream>>>(xp, M, K8, qp, s);
+  } else if (K8 <= 128 * kCached) {
+    quantize_rows_kernel<128, kDivide><<<static_cast<unsigned>((M + 1) / 2), kThreads, 0, stream>>>(xp, M, K8, qp, s);
+  } else {
+    quantize_rows_kernel<256, kDivide><<<static_cast<unsigned>(M), kThreads, 0, stream>>>(xp, M, K8, qp, s);
+  }
+  return cuda_status(cudaGetLastError());
+}
+
+// ---------------------------------------------------------------------------- INT4
+// Packed layout of one weight row: K/2 bytes; inside every run of 32 consecutive k
+// (16 bytes) byte b holds code(k0 + b) in bits 0-3 and code(k0 + 16 + b) in bits 4-7,
+// two's complement.  A 32-bit word w of that run then widens with two logic ops into
+// four consecutive INT8 values each:  (w << 4) & 0xF0F0F0F0 -> 16 * code(k0 + 4j .. 4j+3),
+// w & 0xF0F0F0F0 -> 16 * code(k0 + 16 + 4j ..).
+
+// One warp per (output channel n, group g of 128 k).  Lane l owns bytes 2*(l%8), 2*(l%8)+1
+// of 32-k run l/8, i.e. codes k0+b, k0+b+1, k0+16+b, k0+16+b+1.
+__global__ void __launch_bounds__(kThreads) pack_w4_kernel(const __half* __restrict__ w, int64_t N, int K,
+                                                           uint8_t* __restrict__ wp,
+                                                           __half* __restrict__ s_grp) {
+  const int G = K / 128;
+  const int64_t warp = static_cast<int64_t>(blockIdx.x) * (kThreads / 32) + (threadIdx.x >> 5);
+  if (warp >= N * G) return;
+  const int lane = threadIdx.x & 31;
+  const int64_t n = warp / G;
+  const int g = static_cast<int>(warp % G);
+  const int k0 = g * 128 + (lane >> 3) * 32;
+  const int b = (lane & 7) * 2;
+  const __half* wr = w + n * K + k0;
+  const __half2 lo = *reinterpret_cast<const __half2*>(wr + b);
+  const __half2 hi = *reinterpret_cast<const __half2*>(wr + 16 + b);
+  __half2 m2 = __hmax2(__habs2(lo), __habs2(hi));
+  float a = fmaxf(__low2float(m2), __high2float(m2));
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
+  const __half s16 = __float2half_rn(__fdiv_rn(a, 7.5f));
+  const float sf = __half2float(s16);
+  if (lane == 0) s_grp[static_cast<int64_t>(g) * N + n] = s16;
+  auto code4 = [sf](__half x) -> uint32_t {
+    if (sf == 0.0f) return 0u;
+    int r = __float2int_rn(__fdiv_rn(__half2float(x), sf));
+    return static_cast<uint32_t>(max(-8, min(7, r))) & 0xfu;
+  };
+  const uint32_t byte0 = code4(__low2half(lo)) | (code4(__low2half(hi)) << 4);
+  const uint32_t byte1 = code4(__high2half(lo)) | (code4(__high2half(hi)) << 4);
+  uint8_t* out = wp + n * (K / 2) + k0 / 2 + b;
+  *reinterpret_cast<uint16_t*>(out) = static_cast<uint16_t>(byte0 | (byte1 << 8));
+}
+
+// One thread per packed byte -> two row-major INT8 codes in [-8, 7].
+__global__ void __launch_bounds__(kThreads) unpack_w4_kernel(const uint8_t* __restrict__ wp, int64_t N, int K,
+                                                             int8_t* __restrict__ codes) {
+  const int64_t i = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x;
+  const int K2 = K / 2;
+  if (i >= N * K2) return;
+  const int64_t n = i / K2;
+  const int j = static_cast<int>(i % K2);
+  const int k0 = (j / 16) * 32, b = j % 16;
+  const uint8_t v = wp[i];
+  const int lo = static_cast<int8_t>(v << 4) >> 4;
+  const int hi = static_cast<int8_t>(v) >> 4;
+  codes[n * K + k0 + b] = static_cast<int8_t>(lo);
+  codes[n * K + k0 + 16 + b] = static_cast<int8_t>(hi);
+}
+
+}  // namespace
+
+int launch_quantize_act(const void* x, int64_t M, int64_t K, int8_t* q, float* s, bool divide_by_scale,
+                        cudaStream_t stream) {
+  return divide_by_scale ? launch_rows<true>(x, M, K, q, s, stream) : launch_rows<false>(x, M, K, q, s, stream);
+}
+
+int launch_pack_w4(const void* w, int64_t N, int64_t K, void* wp, void* s_grp, cudaStream_t stream) {
+  const int64_t warps = N * (K / 128);
+  const unsigned blocks = static_cast<unsigned>((warps + kThreads / 32 - 1) / (kThreads / 32));
+  pack_w4_kernel<<<blocks, kThreads, 0, stream>>>(static_cast<const __half*>(w), N, static_cast<int>(K),
+                                                  static_cast<uint8_t*>(wp), static_cast<__half*>(s_grp));
+  return cuda_status(cudaGetLastError());
+}
+
+int launch_unpack_w4(const void* wp, int64_t N, int64_t K, int8_t* codes, cudaStream_t stream) {
+  const int64_t n = N * (K / 2);
+  const unsigned blocks = static_cast<unsigned>((n + kThreads - 1) / kThreads);
+  unpack_w4_kernel<<<blocks, kThreads, 0, stream>>>(static_cast<const uint8_t*>(wp), N, static_cast<int>(K), codes);
+  return cuda_status(cudaGetLastError());
+}
+
+}  // namespace pq

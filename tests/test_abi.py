@@ -1,0 +1,40 @@
+"""The C-ABI library loads without a GPU and exports every symbol include/pq.h declares;
+argument errors are reported before anything touches a device."""
+import ctypes
+import os
+import re
+
+import paper_2512_23367_b200 as pq
+from paper_2512_23367_b200 import binding
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "pq.h")).read()
+    return sorted(set(re.findall(r"PQ_API\s+[\w\s\*]+?\b(pq_\w+)\s*\(", text)))
+
+
+def test_header_symbols_are_exported_and_bound():
+    names = _declared()
+    assert {"pq_quantize_act", "pq_pack_w8", "pq_pack_w4", "pq_gemm_w8a8", "pq_gemm_w4a8"} <= set(names)
+    handle = ctypes.CDLL(pq.lib()._name)
+    for n in names:
+        assert hasattr(handle, n), n
+    assert set(names) == set(binding.SIGNATURES), set(names) ^ set(binding.SIGNATURES)
+
+
+def test_argument_errors_come_back_as_status_codes_without_a_device():
+    L = pq.lib()
+    PQ_ERR_NULL, PQ_ERR_SHAPE, PQ_ERR_ALIGN = 1, 2, 3
+    assert L.pq_quantize_act(None, 4, 64, None, None, None) == PQ_ERR_NULL
+    assert L.pq_quantize_act(16, 4, 60, 16, 16, None) == PQ_ERR_SHAPE      # K % 16
+    assert L.pq_quantize_act(16, 0, 64, 16, 16, None) == PQ_ERR_SHAPE      # M < 1
+    assert L.pq_quantize_act(8, 4, 64, 16, 16, None) == PQ_ERR_ALIGN
+    assert L.pq_gemm_w8a8(16, 16, 16, 16, 4, 12, 64, 16, None) == PQ_ERR_SHAPE   # N % 8
+    assert L.pq_gemm_w8a8(16, 16, 16, 16, 4, 16, 131072, 16, None) == PQ_ERR_SHAPE  # INT32 bound
+    assert L.pq_gemm_w4a8(16, 16, 16, 16, 64, 4, 16, 256, 16, None) == PQ_ERR_SHAPE   # group != 128
+    assert L.pq_gemm_w4a8(16, 16, 16, 16, 128, 4, 16, 192, 16, None) == PQ_ERR_SHAPE  # K % 128
+    assert L.pq_pack_w4(16, 16, 256, 128, None, 16, None) == PQ_ERR_NULL
+    assert L.pq_packed_w8_bytes(8, 256) == 2048 and L.pq_packed_w4_bytes(8, 256) == 1024
+    assert L.pq_status_str(0) == b"ok" and b"wait" in L.pq_status_str(6)

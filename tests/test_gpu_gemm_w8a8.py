@@ -1,0 +1,99 @@
+"""GPU parity: W8A8 linear against the CPU oracle.  INT32 accumulators bit-exact, FP16 output
+within 2^-10 relative + 1e-3 absolute."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2512_23367_b200 as pq
+from paper_2512_23367_b200 import synth
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+REL, ABS = 2.0 ** -10, 1e-3
+
+
+def _np(t):
+    return t.cpu().numpy()
+
+
+def assert_y_close(y_gpu, y_ref):
+    g, r = y_gpu.astype(np.float64), y_ref.astype(np.float64)
+    assert np.isfinite(g).all()
+    bad = np.abs(g - r) > REL * np.abs(r) + ABS
+    assert not bad.any(), (int(bad.sum()), np.argwhere(bad)[:5], g[bad][:5], r[bad][:5])
+
+
+def run_case(M, N, K, seed, n_out=None, rows=None):
+    x = synth.activations(M, K, seed, n_out)
+    w = synth.weights(N, K, seed)
+    xd, wd = torch.from_numpy(x).to(DEV), torch.from_numpy(w).to(DEV)
+    q, s_tok = pq.pq_quantize_act(xd)
+    wq, s_ch = pq.pq_pack_w8(wd)
+    acc = pq.pq_acc_w8a8(q, wq, N)
+    y = pq.pq_gemm_w8a8(q, s_tok, wq, s_ch, N)
+    assert pq.pq_device_status() == 0
+    q_ref, s_tok_ref = oracle.quantize_act(x)
+    wq_ref, s_ch_ref = oracle.pack_w8(w)
+    assert np.array_equal(_np(q), q_ref)
+    sel = np.arange(M) if rows is None else rows
+    acc_ref, y_ref = oracle.gemm_w8a8(q_ref[sel], s_tok_ref[sel], wq_ref, s_ch_ref)
+    assert np.array_equal(_np(acc)[sel], acc_ref)
+    assert_y_close(_np(y)[sel], y_ref)
+
+
+def test_config1_tiny_linear_every_element():
+    run_case(16, 256, 256, seed=0, n_out=4)
+
+
+@pytest.mark.parametrize("M,N,K", [
+    (128, 256, 128), (130, 264, 144), (257, 520, 1040), (200, 384, 2048), (65, 8, 16),
+    (300, 1024, 4096), (129, 136, 11008), (512, 256, 256), (96, 4096, 512),
+])
+def test_shapes_spanning_tiles_and_ragged_tails(M, N, K):
+    run_case(M, N, K, seed=M + N + K)
+
+
+def test_extreme_codes_minus128_times_minus128():
+    M, N, K = 130, 264, 11008
+    q = torch.full((M, K), -128, dtype=torch.int8, device=DEV)
+    wq = torch.full((N * K,), 0x80, dtype=torch.uint8, device=DEV)      # code -128 everywhere
+    acc = pq.pq_acc_w8a8(q, wq, N)
+    assert pq.pq_device_status() == 0
+    assert (acc == K * 16384).all()
+    q[1::2] = 127
+    acc = _np(pq.pq_acc_w8a8(q, wq, N))
+    assert (acc[0::2] == K * 16384).all() and (acc[1::2] == -K * 127 * 128).all()
+
+
+def test_identity_weights_return_the_codes():
+    M, K = 140, 256
+    x = synth.activations(M, K, seed=3)
+    q, s_tok = pq.pq_quantize_act(torch.from_numpy(x).to(DEV))
+    eye = torch.eye(K, dtype=torch.float16, device=DEV) * 0.5
+    wq, s_ch = pq.pq_pack_w8(eye)
+    acc = pq.pq_acc_w8a8(q, wq, K)
+    assert torch.equal(acc, 127 * q.to(torch.int32))
+    wqn, _ = pq.pq_pack_w8(-eye)
+    assert torch.equal(pq.pq_acc_w8a8(q, wqn, K), -128 * q.to(torch.int32))
+
+
+def test_output_guard_bands_stay_untouched():
+    M, N, K = 130, 264, 256
+    x = synth.activations(M, K, seed=9)
+    w = synth.weights(N, K, seed=9)
+    q, s_tok = pq.pq_quantize_act(torch.from_numpy(x).to(DEV))
+    wq, s_ch = pq.pq_pack_w8(torch.from_numpy(w).to(DEV))
+    pad = 4096
+    buf = torch.full((pad + M * N + pad,), 7.0, dtype=torch.float16, device=DEV)
+    y = buf[pad:pad + M * N].view(M, N)
+    pq.pq_gemm_w8a8(q, s_tok, wq, s_ch, N, y=y)
+    assert pq.pq_device_status() == 0
+    assert (buf[:pad] == 7.0).all() and (buf[pad + M * N:] == 7.0).all()
+
+
+@pytest.mark.parametrize("M,K,N", [(2048, 2048, 6144), (4096, 4096, 11008), (512, 11008, 4096)])
+def test_full_size_layers_on_sampled_rows(M, K, N):
+    rng = np.random.default_rng(M + K + N)
+    rows = np.unique(np.concatenate([[0, 127, 128, M - 129, M - 1], rng.integers(0, M, 19)]))
+    run_case(M, N, K, seed=2000 + N % 97, rows=rows)
