@@ -70,11 +70,13 @@ def test_identity_weights_return_the_codes():
     M, K = 140, 256
     x = synth.activations(M, K, seed=3)
     q, s_tok = pq.pq_quantize_act(torch.from_numpy(x).to(DEV))
-    eye = torch.eye(K, dtype=torch.float16, device=DEV) * 0.5
+    eye = torch.eye(K, dtype=torch.float16, device=DEV) * 0.75
     wq, s_ch = pq.pq_pack_w8(eye)
+    assert np.array_equal(_np(pq.pq_unpack_w8(wq, K, K)), oracle.pack_w8(_np(eye))[0])
     acc = pq.pq_acc_w8a8(q, wq, K)
-    assert torch.equal(acc, 127 * q.to(torch.int32))
+    assert torch.equal(acc, 127 * q.to(torch.int32))       # +max -> 127.5 -> 128 -> clamped to 127
     wqn, _ = pq.pq_pack_w8(-eye)
+    assert np.array_equal(_np(pq.pq_unpack_w8(wqn, K, K)), oracle.pack_w8(_np(-eye))[0])
     assert torch.equal(pq.pq_acc_w8a8(q, wqn, K), -128 * q.to(torch.int32))
 
 
