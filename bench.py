@@ -191,7 +191,7 @@ class OracleLayer:
 def cpu_baseline(wl: synth.Workload, M: int, budget_s: float = 12.0) -> dict:
     """The oracle as it stands, timed on the host cores on a bounded sample of the workload."""
     import oracle
-    layer = OracleLayer(wl, M, 64)
+    layer = OracleLayer(wl, M, 1024)
     t, ops = layer.run(2)                                  # calibration
     rows = int(max(2, min(layer.max_rows, budget_s * (2 / t))))
     t, ops = layer.run(rows)
@@ -344,8 +344,12 @@ def run_ours(args, wl: synth.Workload, M: int):
 
     # ---- per-kernel durations (same steps, eager launches, CUDA events around every launch)
     timers = {"quantize": [], "gemm": []}
+    # A short device-side delay in front of every instrumented step lets the host queue the
+    # step's launches and event records ahead, so the events bracket back-to-back kernel time
+    # and not the host's launch latency.
     with torch.cuda.stream(stream):
         for i in range(min(args.steps, 4 * n_layers)):
+            torch.cuda._sleep(3_000_000)
             run_layer(layers[i % n_layers], timers)
         torch.cuda.synchronize()
     gemm_ms = [a.elapsed_time(b) for a, b in timers["gemm"]]
@@ -452,8 +456,8 @@ def _timed(torch, fn):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
-    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(synth.WORKLOADS))
     ap.add_argument("--M", type=int, default=None, help="token count (default: the workload's largest)")

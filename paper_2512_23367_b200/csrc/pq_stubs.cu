@@ -5,8 +5,6 @@ int launch_smallm_w8a8(const int8_t* q, const float* s_tok, const void* wq, cons
                        int64_t N, int64_t K, void* y, int32_t* acc, cudaStream_t stream) {
   return launch_gemm_w8a8(q, s_tok, wq, s_ch, M, N, K, y, acc, stream);
 }
-int launch_gemm_w4a8(const int8_t*, const float*, const void*, const void*, int64_t, int64_t, int64_t, void*,
-                     int32_t*, cudaStream_t) { return PQ_ERR_CUDA; }
 int launch_smallm_w4a8(const int8_t*, const float*, const void*, const void*, int64_t, int64_t, int64_t, void*,
                        int32_t*, cudaStream_t) { return PQ_ERR_CUDA; }
 }
