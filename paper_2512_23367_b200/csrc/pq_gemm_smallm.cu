@@ -1,0 +1,465 @@
+// Small-M (decode-shaped, M <= 64) W8A8 / W4A8 linear for sm_100a: a weight-streaming schedule
+// that computes the same result as the prefill kernels.
+//
+// The roles of the two operands are swapped: a tile of 128 WEIGHT rows is the 128-lane operand
+// of tcgen05.mma and the (zero-padded) tokens are the narrow N dimension (16, 32 or 64), so one
+// instruction consumes 4 KB of weights and the tensor pipe stays far below its limit while the
+// weights stream from HBM exactly once.  The K dimension is split over the CTAs of a thread-block
+// cluster (up to 8) so that ~2 CTAs per SM pull weights concurrently; the partial results are
+// reduced through distributed shared memory in a fixed order (exact for the INT32 accumulators
+// of W8A8, deterministic for the FP32 group sums of W4A8) and the cluster's CTAs share the
+// dequantize + FP16 store work.  No global scratch memory is used.
+//
+//   warp 0      TMA producer (weights + token tile per 128-deep K block)
+//   warp 1      MMA issuer
+//   warps 2-3   W4 only: nibble -> INT8 widening into the swizzled operand layout
+//   warps 4-7   TMEM -> registers (W4: per-group promotion with the row's own group scale),
+//               cross-CTA reduction, dequantization, FP16 store
+#include <cuda_fp16.h>
+
+#include "pq_internal.h"
+#include "pq_ptx.cuh"
+
+namespace pq {
+namespace {
+
+constexpr int BW = 128;   // weight rows per tile (TMEM lanes)
+constexpr int BK = 128;   // K per block = one W4 group
+constexpr int UMMA_K = 32;
+constexpr int kNumThreads = 256;
+constexpr int kUnpackThreads = 64;
+constexpr int kMaxSplit = 8;  // portable cluster size
+
+template <int MPAD, bool kW4>
+struct Cfg {
+  static constexpr int kWBytes = kW4 ? BW * BK / 2 : BW * BK;    // weight tile as loaded
+  static constexpr int kQBytes = MPAD * BK;                      // token tile (128-byte swizzle)
+  static constexpr int kSBytes = kW4 ? BW * 2 : 0;               // FP16 group scales of the tile
+  static constexpr int kStageBytes = kWBytes + kQBytes + (kW4 ? 1024 : 0);
+  static constexpr int kTxBytes = kWBytes + kQBytes + kSBytes;
+  static constexpr int STAGES = kW4 ? 4 : (MPAD == 64 ? 4 : 5);
+  static constexpr int A8_SLOTS = kW4 ? 2 : 0;                   // widened weight tiles
+  static constexpr int kA8Bytes = BW * BK;
+  static constexpr int SC_SLOTS = kW4 ? 6 : 0;                   // FP32 scale rows (128 floats)
+  static constexpr int ACC_SLOTS = kW4 ? 4 : 1;
+  static constexpr int kA8Off = STAGES * kStageBytes;
+  static constexpr int kScOff = kA8Off + A8_SLOTS * kA8Bytes;
+  static constexpr int kRingEnd = kScOff + SC_SLOTS * BW * 4;
+  static constexpr int kRedBytes = MPAD * BW * 4;                // aliases the stage ring
+  static constexpr int kBarOff = (kRingEnd > kRedBytes ? kRingEnd : kRedBytes);
+  static constexpr int kNumBars = 2 * STAGES + 2 * A8_SLOTS + 2 * SC_SLOTS + 2 * ACC_SLOTS;
+  static constexpr int kMiscOff = kBarOff + kNumBars * 8;
+  static constexpr int kDynamic = kMiscOff + 16 + 1024;
+  static constexpr uint32_t kTmemCols = (ACC_SLOTS * MPAD) < 32 ? 32 : (ACC_SLOTS * MPAD);
+};
+
+struct SmallArgs {
+  const float* s_tok;
+  const float* s_ch;     // W8
+  __half* y;
+  int32_t* acc;          // export: W8 [M,N]; W4 [G,M,N]
+  int* status;
+  int M, N, K;
+  int k_blocks, splits;
+};
+
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t ld_dsmem_u32(uint32_t local_addr, uint32_t rank) {
+  uint32_t v;
+  asm volatile(
+      "{\n\t.reg .b32 ra;\n\t"
+      "mapa.shared::cluster.u32 ra, %1, %2;\n\t"
+      "ld.shared::cluster.b32 %0, [ra];\n\t}"
+      : "=r"(v)
+      : "r"(local_addr), "r"(rank)
+      : "memory");
+  return v;
+}
+
+template <int MPAD>
+__device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t (&r)[MPAD]) {
+  if constexpr (MPAD == 16) {
+    tmem_ld_32x16(taddr, r);
+  } else if constexpr (MPAD == 32) {
+    tmem_ld_32x32(taddr, r);
+  } else {
+    uint32_t(&lo)[32] = *reinterpret_cast<uint32_t(*)[32]>(&r[0]);
+    uint32_t(&hi)[32] = *reinterpret_cast<uint32_t(*)[32]>(&r[32]);
+    tmem_ld_32x32(taddr, lo);
+    tmem_ld_32x32(taddr + 32, hi);
+  }
+}
+
+template <int MPAD, bool kW4, bool kExportAcc>
+__global__ void __launch_bounds__(kNumThreads, 2)
+smallm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_q,
+              const __grid_constant__ CUtensorMap tm_s, const SmallArgs p) {
+  using C = Cfg<MPAD, kW4>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t smem_base = smem_u32(smem);
+  const uint32_t bar_full = smem_base + C::kBarOff;
+  const uint32_t bar_empty = bar_full + C::STAGES * 8;
+  const uint32_t bar_a8_full = bar_empty + C::STAGES * 8;
+  const uint32_t bar_a8_empty = bar_a8_full + C::A8_SLOTS * 8;
+  const uint32_t bar_sc_full = bar_a8_empty + C::A8_SLOTS * 8;
+  const uint32_t bar_sc_empty = bar_sc_full + C::SC_SLOTS * 8;
+  const uint32_t bar_acc_full = bar_sc_empty + C::SC_SLOTS * 8;
+  const uint32_t bar_acc_empty = bar_acc_full + C::ACC_SLOTS * 8;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + C::kMiscOff);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + C::kMiscOff + 4);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int n0 = blockIdx.x * BW;
+  const int split = blockIdx.y;                       // == rank in the cluster (cluster = all of grid.y)
+  const int kb0 = static_cast<int>(static_cast<int64_t>(p.k_blocks) * split / p.splits);
+  const int kb1 = static_cast<int>(static_cast<int64_t>(p.k_blocks) * (split + 1) / p.splits);
+  const int nkb = kb1 - kb0;
+
+  auto issue_load = [&](int j) {  // j-th K block of this CTA into stage j % STAGES
+    const uint32_t s = static_cast<uint32_t>(j) % C::STAGES;
+    const uint32_t dst = smem_base + s * C::kStageBytes;
+    const int kb = kb0 + j;
+    mbar_arrive_expect_tx(bar_full + s * 8, C::kTxBytes);
+    tma_load_2d(dst, &tm_w, bar_full + s * 8, kW4 ? kb * (BK / 2) : kb * BK, n0);
+    tma_load_2d(dst + C::kWBytes, &tm_q, bar_full + s * 8, kb * BK, 0);
+    if constexpr (kW4) tma_load_2d(dst + C::kWBytes + C::kQBytes, &tm_s, bar_full + s * 8, n0, kb);
+  };
+
+  if (threadIdx.x == 0) {
+    *abort_flag = 0;
+    for (int s = 0; s < C::STAGES; ++s) {
+      mbar_init(bar_full + s * 8, 1);
+      mbar_init(bar_empty + s * 8, kW4 ? 1 + kUnpackThreads / 32 : 1);
+    }
+    for (int s = 0; s < C::A8_SLOTS; ++s) {
+      mbar_init(bar_a8_full + s * 8, kUnpackThreads / 32);
+      mbar_init(bar_a8_empty + s * 8, 1);
+    }
+    for (int s = 0; s < C::SC_SLOTS; ++s) {
+      mbar_init(bar_sc_full + s * 8, kUnpackThreads / 32);
+      mbar_init(bar_sc_empty + s * 8, 4);
+    }
+    for (int s = 0; s < C::ACC_SLOTS; ++s) {
+      mbar_init(bar_acc_full + s * 8, 1);
+      mbar_init(bar_acc_empty + s * 8, 4);
+    }
+    fence_mbar_init();
+    // Start the weight stream at once: the first ring pass needs no wait.
+    const int first = nkb < C::STAGES ? nkb : C::STAGES;
+    for (int j = 0; j < first; ++j) issue_load(j);
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(tmem_slot), C::kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  // Per-thread partial results of the epilogue warps: P[m] for weight row n0 + 32*quad + lane.
+  uint32_t P[MPAD];
+#pragma unroll
+  for (int m = 0; m < MPAD; ++m) P[m] = 0u;
+  bool ok = true;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer (remaining blocks)
+    if (lane == 0) {
+      int j = C::STAGES;
+      for (; j < nkb; ++j) {
+        const uint32_t s = static_cast<uint32_t>(j) % C::STAGES, ph = (static_cast<uint32_t>(j) / C::STAGES) & 1u;
+        if (!mbar_wait(bar_empty + s * 8, ph ^ 1u, abort_flag)) { ok = false; break; }
+        issue_load(j);
+      }
+      if (!ok) {
+        const int first = j >= C::STAGES ? j - C::STAGES : 0;
+        for (int i = first; i < j; ++i) {
+          const uint32_t s = static_cast<uint32_t>(i) % C::STAGES, ph = (static_cast<uint32_t>(i) / C::STAGES) & 1u;
+          for (uint32_t w = 0; w < (1u << 16) && !mbar_try_wait(bar_full + s * 8, ph); ++w) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = umma_idesc_s8(BW, MPAD);
+      for (int j = 0; j < nkb; ++j) {
+        const uint32_t it = static_cast<uint32_t>(j);
+        const uint32_t s = it % C::STAGES, ph = (it / C::STAGES) & 1u;
+        if (!mbar_wait(bar_full + s * 8, ph, abort_flag)) { ok = false; break; }
+        const uint32_t stage = smem_base + s * C::kStageBytes;
+        uint64_t w_desc;
+        uint32_t d_tmem = tmem_base;
+        if constexpr (kW4) {
+          const uint32_t u = it % C::A8_SLOTS, uph = (it / C::A8_SLOTS) & 1u;
+          const uint32_t a = it % C::ACC_SLOTS, aph = (it / C::ACC_SLOTS) & 1u;
+          if (!mbar_wait(bar_a8_full + u * 8, uph, abort_flag) ||
+              !mbar_wait(bar_acc_empty + a * 8, aph ^ 1u, abort_flag)) { ok = false; break; }
+          w_desc = umma_desc_k_sw128(smem_base + C::kA8Off + u * C::kA8Bytes);
+          d_tmem = tmem_base + a * MPAD;
+        } else {
+          w_desc = umma_desc_k_sw128(stage);
+        }
+        tc_fence_after_sync();
+        const uint64_t q_desc = umma_desc_k_sw128(stage + C::kWBytes);
+#pragma unroll
+        for (int k = 0; k < BK / UMMA_K; ++k) {
+          const uint32_t accumulate = kW4 ? (k != 0) : ((j | k) != 0);
+          umma_i8(d_tmem, w_desc + 2 * k, q_desc + 2 * k, idesc, accumulate);
+        }
+        umma_commit(bar_empty + s * 8);
+        if constexpr (kW4) {
+          umma_commit(bar_a8_empty + (it % C::A8_SLOTS) * 8);
+          umma_commit(bar_acc_full + (it % C::ACC_SLOTS) * 8);
+        }
+      }
+      if constexpr (!kW4) {
+        if (ok) umma_commit(bar_acc_full);
+      }
+    }
+  } else if (warp < 4) {
+    // ------------------------------------------------------------ W4: widen nibbles to INT8
+    if constexpr (kW4) {
+      const int ut = threadIdx.x - 64;
+      for (int j = 0; j < nkb; ++j) {
+        const uint32_t it = static_cast<uint32_t>(j);
+        const uint32_t s = it % C::STAGES, ph = (it / C::STAGES) & 1u;
+        const uint32_t u = it % C::A8_SLOTS, uph = (it / C::A8_SLOTS) & 1u;
+        const uint32_t v = it % C::SC_SLOTS, vph = (it / C::SC_SLOTS) & 1u;
+        bool w = mbar_wait(bar_full + s * 8, ph, abort_flag);
+        w = w && mbar_wait(bar_a8_empty + u * 8, uph ^ 1u, abort_flag);
+        w = w && mbar_wait(bar_sc_empty + v * 8, vph ^ 1u, abort_flag);
+        ok = __all_sync(0xffffffffu, w);
+        if (!ok) break;
+        const uint8_t* stage = smem + s * C::kStageBytes;
+        const uint4* packed = reinterpret_cast<const uint4*>(stage);
+        uint8_t* a8 = smem + C::kA8Off + u * C::kA8Bytes;
+#pragma unroll
+        for (int i = 0; i < (BW * 4) / kUnpackThreads; ++i) {
+          const int idx = ut + i * kUnpackThreads;
+          const int r = idx >> 2, c = idx & 3;
+          const uint4 w4 = packed[idx];
+          uint4 lo, hi;
+          lo.x = (w4.x << 4) & 0xF0F0F0F0u; hi.x = w4.x & 0xF0F0F0F0u;
+          lo.y = (w4.y << 4) & 0xF0F0F0F0u; hi.y = w4.y & 0xF0F0F0F0u;
+          lo.z = (w4.z << 4) & 0xF0F0F0F0u; hi.z = w4.z & 0xF0F0F0F0u;
+          lo.w = (w4.w << 4) & 0xF0F0F0F0u; hi.w = w4.w & 0xF0F0F0F0u;
+          uint8_t* row = a8 + r * 128;
+          const int sw = r & 7;
+          *reinterpret_cast<uint4*>(row + (((2 * c) ^ sw) << 4)) = lo;
+          *reinterpret_cast<uint4*>(row + (((2 * c + 1) ^ sw) << 4)) = hi;
+        }
+        const __half* sh = reinterpret_cast<const __half*>(stage + C::kWBytes + C::kQBytes);
+        float* sc = reinterpret_cast<float*>(smem + C::kScOff) + v * BW;
+        for (int c = ut; c < BW; c += kUnpackThreads) sc[c] = __half2float(sh[c]) * 0.0625f;
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive(bar_a8_full + u * 8);
+          mbar_arrive(bar_sc_full + v * 8);
+          mbar_arrive(bar_empty + s * 8);
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ TMEM -> registers
+    const int quad = warp & 3;
+    const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
+    const int n_local = quad * 32 + lane;
+    if constexpr (kW4) {
+      constexpr int CH = MPAD < 32 ? MPAD : 32;  // columns promoted per tcgen05.ld
+      for (int j = 0; j < nkb; ++j) {
+        const uint32_t it = static_cast<uint32_t>(j);
+        const uint32_t a = it % C::ACC_SLOTS, aph = (it / C::ACC_SLOTS) & 1u;
+        const uint32_t v = it % C::SC_SLOTS, vph = (it / C::SC_SLOTS) & 1u;
+        bool w = mbar_wait(bar_acc_full + a * 8, aph, abort_flag);
+        w = w && mbar_wait(bar_sc_full + v * 8, vph, abort_flag);
+        ok = __all_sync(0xffffffffu, w);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const float sg = (reinterpret_cast<const float*>(smem + C::kScOff) + v * BW)[n_local];
+#pragma unroll
+        for (int c0 = 0; c0 < MPAD; c0 += CH) {
+          uint32_t r[CH];
+          tmem_ld_cols<CH>(lane_addr + a * MPAD + c0, r);
+          tmem_ld_wait();
+          if constexpr (kExportAcc) {
+            const int n = n0 + n_local;
+#pragma unroll
+            for (int m = 0; m < CH; ++m) {
+              if (c0 + m < p.M && n < p.N)
+                p.acc[(static_cast<int64_t>(kb0 + j) * p.M + c0 + m) * p.N + n] = static_cast<int32_t>(r[m]) >> 4;
+            }
+          } else {
+#pragma unroll
+            for (int m = 0; m < CH; ++m)
+              P[c0 + m] = __float_as_uint(fmaf(__int2float_rn(static_cast<int32_t>(r[m])), sg, __uint_as_float(P[c0 + m])));
+          }
+        }
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive(bar_acc_empty + a * 8);
+          mbar_arrive(bar_sc_empty + v * 8);
+        }
+      }
+    } else {
+      if (nkb > 0) {
+        ok = __all_sync(0xffffffffu, mbar_wait(bar_acc_full, 0u, abort_flag));
+        if (ok) {
+          tc_fence_after_sync();
+          tmem_ld_cols<MPAD>(lane_addr, P);
+          tmem_ld_wait();
+          tc_fence_before_sync();
+        }
+      }
+    }
+  }
+
+  // ------------------------------------------------------------ cross-CTA reduction + store
+  // All K blocks of this CTA are consumed (the epilogue warps saw the last accumulator), so the
+  // stage ring is free and holds this CTA's partial tile as red[m][n] (32-bit words).
+  uint32_t* red = reinterpret_cast<uint32_t*>(smem);
+  const bool do_reduce = !(kW4 && kExportAcc);
+  if (do_reduce && warp >= 4) {
+    const int n_local = (warp & 3) * 32 + lane;
+#pragma unroll
+    for (int m = 0; m < MPAD; ++m) red[m * BW + n_local] = P[m];
+  }
+  tc_fence_before_sync();
+  __syncwarp();
+  cluster_sync_all();
+  if (do_reduce && warp >= 4) {
+    const int n_local = (warp & 3) * 32 + lane;
+    const int n = n0 + n_local;
+    const uint32_t my_rank = cluster_ctarank();
+    float sc = 0.0f;
+    if (!kW4 && !kExportAcc && n < p.N) sc = __ldg(p.s_ch + n);
+    for (int m = static_cast<int>(my_rank); m < p.M; m += p.splits) {
+      const uint32_t addr = smem_base + static_cast<uint32_t>(m * BW + n_local) * 4u;
+      if constexpr (kW4) {
+        float tot = 0.0f;
+        for (int r = 0; r < p.splits; ++r) tot += __uint_as_float(ld_dsmem_u32(addr, static_cast<uint32_t>(r)));
+        if (n < p.N) p.y[static_cast<int64_t>(m) * p.N + n] = __float2half_rn(tot * __ldg(p.s_tok + m));
+      } else {
+        int32_t tot = 0;
+        for (int r = 0; r < p.splits; ++r) tot += static_cast<int32_t>(ld_dsmem_u32(addr, static_cast<uint32_t>(r)));
+        if (n < p.N) {
+          if constexpr (kExportAcc) {
+            p.acc[static_cast<int64_t>(m) * p.N + n] = tot;
+          } else {
+            const float v = __fmul_rn(__fmul_rn(__int2float_rn(tot), __ldg(p.s_tok + m)), sc);
+            p.y[static_cast<int64_t>(m) * p.N + n] = __float2half_rn(v);
+          }
+        }
+      }
+    }
+  }
+  __syncwarp();
+  cluster_sync_all();  // nobody leaves while a peer may still read its shared memory
+  tc_fence_after_sync();
+  if (warp == 1) {
+    __syncwarp();
+    tmem_dealloc(tmem_base, C::kTmemCols);
+  }
+  if (threadIdx.x == 0 && *abort_flag) atomicExch(p.status, static_cast<int>(PQ_ERR_TIMEOUT));
+}
+
+template <int MPAD, bool kW4, bool kExportAcc>
+int launch_cfg(const CUtensorMap& tw, const CUtensorMap& tq, const CUtensorMap& ts, const SmallArgs& a, int n_tiles,
+               cudaStream_t stream) {
+  using C = Cfg<MPAD, kW4>;
+  auto kern = smallm_kernel<MPAD, kW4, kExportAcc>;
+  static bool configured = false;
+  if (!configured) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kDynamic) != cudaSuccess)
+      return PQ_ERR_CUDA;
+    configured = true;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(n_tiles), static_cast<unsigned>(a.splits), 1);
+  cfg.blockDim = dim3(kNumThreads, 1, 1);
+  cfg.dynamicSmemBytes = C::kDynamic;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 1;
+  attr[0].val.clusterDim.y = static_cast<unsigned>(a.splits);
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cuda_status(cudaLaunchKernelEx(&cfg, kern, tw, tq, ts, a));
+}
+
+template <bool kW4>
+int launch_smallm(const int8_t* q, const float* s_tok, const void* w, const float* s_ch, const void* s_grp,
+                  int64_t M, int64_t N, int64_t K, void* y, int32_t* acc, cudaStream_t stream) {
+  const int mpad = M <= 16 ? 16 : (M <= 32 ? 32 : 64);
+  const int n_tiles = static_cast<int>((N + BW - 1) / BW);
+  const int k_blocks = static_cast<int>((K + BK - 1) / BK);
+  // Aim at two resident CTAs per SM; the split is the cluster size (<= 8) and <= K blocks.
+  int splits = (2 * sm_count()) / n_tiles;
+  splits = splits < 1 ? 1 : (splits > kMaxSplit ? kMaxSplit : splits);
+  if (splits > k_blocks) splits = k_blocks;
+
+  CUtensorMap tw, tq, ts;
+  int rc;
+  if (kW4) {
+    rc = make_tmap_2d(&tw, w, static_cast<uint64_t>(N), static_cast<uint64_t>(K / 2), BW, BK / 2, 1, false);
+  } else {
+    rc = make_tmap_2d(&tw, w, static_cast<uint64_t>(N), static_cast<uint64_t>(K), BW, BK, 1, true);
+  }
+  if (rc != PQ_OK) return rc;
+  rc = make_tmap_2d(&tq, q, static_cast<uint64_t>(M), static_cast<uint64_t>(K), static_cast<uint32_t>(mpad), BK, 1, true);
+  if (rc != PQ_OK) return rc;
+  if (kW4 && s_grp != nullptr) {
+    rc = make_tmap_2d(&ts, s_grp, static_cast<uint64_t>(K / 128), static_cast<uint64_t>(N), 1, BW, 2, false);
+  } else {
+    ts = tq;  // unused by W8; the W4 accumulator export reads (and ignores) token bytes instead of scales
+    if (kW4) rc = make_tmap_2d(&ts, q, static_cast<uint64_t>(M), static_cast<uint64_t>(K / 2), 1, BW, 2, false);
+  }
+  if (rc != PQ_OK) return rc;
+
+  SmallArgs a;
+  a.s_tok = s_tok;
+  a.s_ch = s_ch;
+  a.y = static_cast<__half*>(y);
+  a.acc = acc;
+  a.status = device_status_ptr();
+  if (a.status == nullptr) return PQ_ERR_CUDA;
+  a.M = static_cast<int>(M);
+  a.N = static_cast<int>(N);
+  a.K = static_cast<int>(K);
+  a.k_blocks = k_blocks;
+  a.splits = splits;
+  const bool ex = acc != nullptr;
+  switch (mpad) {
+    case 16: return ex ? launch_cfg<16, kW4, true>(tw, tq, ts, a, n_tiles, stream) : launch_cfg<16, kW4, false>(tw, tq, ts, a, n_tiles, stream);
+    case 32: return ex ? launch_cfg<32, kW4, true>(tw, tq, ts, a, n_tiles, stream) : launch_cfg<32, kW4, false>(tw, tq, ts, a, n_tiles, stream);
+    default: return ex ? launch_cfg<64, kW4, true>(tw, tq, ts, a, n_tiles, stream) : launch_cfg<64, kW4, false>(tw, tq, ts, a, n_tiles, stream);
+  }
+}
+
+}  // namespace
+
+int launch_smallm_w8a8(const int8_t* q, const float* s_tok, const void* wq, const float* s_ch, int64_t M,
+                       int64_t N, int64_t K, void* y, int32_t* acc, cudaStream_t stream) {
+  return launch_smallm<false>(q, s_tok, wq, s_ch, nullptr, M, N, K, y, acc, stream);
+}
+
+int launch_smallm_w4a8(const int8_t* q, const float* s_tok, const void* wp, const void* s_grp, int64_t M,
+                       int64_t N, int64_t K, void* y, int32_t* acc_g, cudaStream_t stream) {
+  return launch_smallm<true>(q, s_tok, wp, nullptr, s_grp, M, N, K, y, acc_g, stream);
+}
+
+}  // namespace pq
