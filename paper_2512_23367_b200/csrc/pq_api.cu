@@ -3,6 +3,8 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <cstdlib>
+
 #include "pq_internal.h"
 
 namespace pq {
@@ -194,6 +196,9 @@ static int gemm_w8a8_common(const int8_t* q, const float* s_tok, const void* wq,
   if ((rc = check_arch()) != PQ_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (M <= kSmallM) return launch_smallm_w8a8(q, s_tok, wq, s_ch, M, N, K, y, acc, st);
+  bool pair = M > 128;  // below that the second CTA of a pair would only hold padding rows
+  if (const char* e = getenv("PQ_W8A8_PAIR")) pair = (e[0] != '0');  // ablation knob
+  if (pair) return launch_gemm_w8a8_pair(q, s_tok, wq, s_ch, M, N, K, y, acc, st);
   return launch_gemm_w8a8(q, s_tok, wq, s_ch, M, N, K, y, acc, st);
 }
 

@@ -10,6 +10,8 @@
 // (which add nothing to an integer dot product) and the epilogue predicates its stores.
 #include <cuda_fp16.h>
 
+#include <cstdlib>
+
 #include "pq_internal.h"
 #include "pq_ptx.cuh"
 
@@ -239,15 +241,18 @@ int launch_cfg(const CUtensorMap& tq, const CUtensorMap& tw, const GemmArgs& a, 
 
 int launch_gemm_w8a8(const int8_t* q, const float* s_tok, const void* wq, const float* s_ch, int64_t M,
                      int64_t N, int64_t K, void* y, int32_t* acc, cudaStream_t stream) {
-  // Tile width: 256 columns unless that leaves many SMs idle and 128 fills them better.
+  // Tile width.  The main loop is bound by the bytes each SM pulls from L2 per multiply-add
+  // (48 KB per 128x256x128 step against 32 KB per 128x128x128 step), so the cost of a
+  // configuration is (waves of tiles over the SMs) x (bytes per tile step).
   const int sms = sm_count();
   const int64_t mb = (M + BM - 1) / BM;
   const int64_t t256 = mb * ((N + 255) / 256), t128 = mb * ((N + 127) / 128);
-  auto waves_eff = [sms](int64_t tiles) {
-    const int64_t waves = (tiles + sms - 1) / sms;
-    return static_cast<double>(tiles) / static_cast<double>(waves * sms);
-  };
-  const bool use128 = (N <= 128) || (waves_eff(t128) > waves_eff(t256) + 0.10);
+  auto waves = [sms](int64_t tiles) { return (tiles + sms - 1) / sms; };
+  bool use128 = (N <= 128) || (waves(t128) * 32 < waves(t256) * 48);
+  if (const char* e = getenv("PQ_W8A8_BN")) {  // ablation knob: force the tile width
+    if (e[0] == '1') use128 = true;
+    if (e[0] == '2') use128 = false;
+  }
   const int BN = use128 ? 128 : 256;
 
   CUtensorMap tq, tw;

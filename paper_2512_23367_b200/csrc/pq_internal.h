@@ -29,6 +29,9 @@ int launch_unpack_w4(const void* wp, int64_t N, int64_t K, int8_t* codes, cudaSt
 // Prefill-shaped W8A8 GEMM (tcgen05 kind::i8).  Exactly one of y / acc is non-null.
 int launch_gemm_w8a8(const int8_t* q, const float* s_tok, const void* wq, const float* s_ch, int64_t M,
                      int64_t N, int64_t K, void* y, int32_t* acc, cudaStream_t stream);
+// Same contract on CTA pairs (cta_group::2, 256-row tiles); preferred when M > 128.
+int launch_gemm_w8a8_pair(const int8_t* q, const float* s_tok, const void* wq, const float* s_ch, int64_t M,
+                          int64_t N, int64_t K, void* y, int32_t* acc, cudaStream_t stream);
 // Prefill-shaped W4A8 GEMM.  Exactly one of y / acc_g is non-null.
 int launch_gemm_w4a8(const int8_t* q, const float* s_tok, const void* wp, const void* s_grp, int64_t M,
                      int64_t N, int64_t K, void* y, int32_t* acc_g, cudaStream_t stream);
