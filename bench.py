@@ -189,15 +189,22 @@ class OracleLayer:
 
 
 def cpu_baseline(wl: synth.Workload, M: int, budget_s: float = 12.0) -> dict:
-    """The oracle as it stands, timed on the host cores on a bounded sample of the workload."""
+    """The oracle as it stands, timed on the host cores on a bounded sample of the workload
+    (about `budget_s` seconds of CPU work: a row sample of one layer, repeated if it is short)."""
     import oracle
-    layer = OracleLayer(wl, M, 1024)
+    layer = OracleLayer(wl, M, M)
     t, ops = layer.run(2)                                  # calibration
     rows = int(max(2, min(layer.max_rows, budget_s * (2 / t))))
-    t, ops = layer.run(rows)
-    return {"value": ops / t / 1e12, "unit": "TOPS", "cores": oracle.num_threads(), "kind": "oracle",
+    t1, ops1 = layer.run(rows)
+    reps = int(max(1, min(50, budget_s / max(t1, 1e-3))))
+    t_sum, ops_sum = t1, ops1
+    for _ in range(reps - 1):
+        t, ops = layer.run(rows)
+        t_sum += t
+        ops_sum += ops
+    return {"value": ops_sum / t_sum / 1e12, "unit": "TOPS", "cores": oracle.num_threads(), "kind": "oracle",
             "sample": f"{rows} of {M} token rows through each of the {len(wl.linears)} linears of one layer "
-                      f"(quantize + GEMM + dequant), {t:.1f} s"}
+                      f"(quantize + GEMM + dequant), {reps} passes, {t_sum:.1f} s"}
 
 
 def run_reference(args, wl: synth.Workload, M: int):
@@ -278,23 +285,19 @@ def run_ours(args, wl: synth.Workload, M: int):
     n_layers = layers_for_rotation(wl, M)
     layers = [LayerBuffers(pq, torch, wl, M, dev, src_x, src_w) for _ in range(n_layers)]
 
-    def run_layer(L: LayerBuffers, timers=None):
+    def run_layer(L: LayerBuffers, only: str | None = None):
         for gi, (K, idxs) in enumerate(L.groups):
-            if timers is not None:
-                timers["quantize"].append(_timed(torch, lambda: pq.pq_quantize_act(L.xs[gi], L.qs[gi], L.s_toks[gi])))
-            else:
+            if only != "gemm":
                 pq.pq_quantize_act(L.xs[gi], L.qs[gi], L.s_toks[gi])
+            if only == "quantize":
+                continue
             for i in idxs:
                 N = wl.linears[i].N
                 a, b = L.packed[i]
                 if wl.w_bits == 8:
-                    fn = lambda: pq.pq_gemm_w8a8(L.qs[gi], L.s_toks[gi], a, b, N, y=L.ys[i])  # noqa: E731
+                    pq.pq_gemm_w8a8(L.qs[gi], L.s_toks[gi], a, b, N, y=L.ys[i])
                 else:
-                    fn = lambda: pq.pq_gemm_w4a8(L.qs[gi], L.s_toks[gi], a, b, N, y=L.ys[i])  # noqa: E731
-                if timers is not None:
-                    timers["gemm"].append(_timed(torch, fn))
-                else:
-                    fn()
+                    pq.pq_gemm_w4a8(L.qs[gi], L.s_toks[gi], a, b, N, y=L.ys[i])
 
     launches_per_step = len(groups) + len(wl.linears)
 
@@ -342,23 +345,45 @@ def run_ours(args, wl: synth.Workload, M: int):
     ops = step_ops(wl, M)
     total_ms, total_ops = aggregate_over_ranks(local_ms, float(ops) * args.steps, world)
 
-    # ---- per-kernel durations (same steps, eager launches, CUDA events around every launch)
-    timers = {"quantize": [], "gemm": []}
-    # A short device-side delay in front of every instrumented step lets the host queue the
-    # step's launches and event records ahead, so the events bracket back-to-back kernel time
-    # and not the host's launch latency.
-    with torch.cuda.stream(stream):
-        for i in range(min(args.steps, 4 * n_layers)):
-            torch.cuda._sleep(3_000_000)
-            run_layer(layers[i % n_layers], timers)
-        torch.cuda.synchronize()
-    gemm_ms = [a.elapsed_time(b) for a, b in timers["gemm"]]
-    quant_ms = [a.elapsed_time(b) for a, b in timers["quantize"]]
-    n_timed_steps = len(gemm_ms) // len(wl.linears)
-    gemm_avg_ms = sum(gemm_ms) / len(gemm_ms)
-    gemm_tops = (ops * n_timed_steps) / (sum(gemm_ms) * 1e-3) / 1e12
+    # ---- per-kernel durations: the same launches on the same buffers, replayed as graphs that hold
+    # only the GEMMs (or only the quantizers) of a layer, timed with CUDA events on the launching
+    # stream.  Event time / launches = average launch duration of that kernel inside a back-to-back
+    # stream of its own kind (launch gaps included, so the figure is conservative).
+    def kind_graphs(which: str):
+        gs = []
+        for L in layers:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                run_layer(L, only=which)
+            gs.append(g)
+        return gs
+
+    def time_kind(gs, launches_per_replay: int, budget_ms: float = 400.0):
+        with torch.cuda.stream(stream):
+            for g in gs:
+                g.replay()
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for g in gs:
+                g.replay()
+            b.record(stream)
+            torch.cuda.synchronize()
+            rounds = int(max(3, min(2000, budget_ms / max(a.elapsed_time(b), 1e-3))))
+            a.record(stream)
+            for _ in range(rounds):
+                for g in gs:
+                    g.replay()
+            b.record(stream)
+            torch.cuda.synchronize()
+        n = rounds * len(gs) * launches_per_replay
+        return a.elapsed_time(b) / n, n
+
+    gemm_avg_ms, gemm_launches = time_kind(kind_graphs("gemm"), len(wl.linears))
+    quant_avg_ms, quant_launches = time_kind(kind_graphs("quantize"), len(groups))
+    gemm_tops = ops / (gemm_avg_ms * len(wl.linears) * 1e-3) / 1e12
     sbytes = step_bytes(wl, M)
-    quant_gbs = sbytes["quantize"] * n_timed_steps / (sum(quant_ms) * 1e-3) / 1e9
+    quant_gbs = sbytes["quantize"] / (quant_avg_ms * len(groups) * 1e-3) / 1e9
 
     # ---- end to end: pinned host inputs -> device -> quantize + GEMMs -> pinned host outputs
     L0 = layers[0]
@@ -402,14 +427,14 @@ def run_ours(args, wl: synth.Workload, M: int):
                     "peak_kind": f"2 x bf16_tflops (burst) of {peak_kind}: INT8 peak = bf16 peak x nominal 4.5/2.25",
                     "frac_of_sustained": gemm_tops / (2.0 * float(peaks["bf16_tflops_sustained"])),
                     "frac_of_datasheet_4500": gemm_tops / DATASHEET_INT8_TOPS,
-                    "avg_launch_us": gemm_avg_ms * 1e3, "launches_timed": len(gemm_ms)}
+                    "avg_launch_us": gemm_avg_ms * 1e3, "launches_timed": gemm_launches}
         else:
-            gbs = sbytes["gemm"] * n_timed_steps / (sum(gemm_ms) * 1e-3) / 1e9
+            gbs = sbytes["gemm"] / (gemm_avg_ms * len(wl.linears) * 1e-3) / 1e9
             peak = float(peaks["hbm_gbs"])
             roof = {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
                     "traffic": load_traffic(f"gemm_w{wl.w_bits}a8:{wl.name}"),
                     "kernel": f"small-M gemm_w{wl.w_bits}a8", "peak_kind": f"hbm_gbs of {peak_kind}",
-                    "avg_launch_us": gemm_avg_ms * 1e3, "launches_timed": len(gemm_ms)}
+                    "avg_launch_us": gemm_avg_ms * 1e3, "launches_timed": gemm_launches}
         decode = M <= 64
         if decode:
             metric, unit = "quantized_linear_gbs", "GB/s"
@@ -432,7 +457,7 @@ def run_ours(args, wl: synth.Workload, M: int):
                        "launch": "cuda_graph_per_layer" if graphs else "eager", "parallelism": "replicas"},
             "roofline": roof,
             "quantize": {"achieved_gbs": quant_gbs, "frac_of_hbm": quant_gbs / float(peaks["hbm_gbs"]),
-                         "avg_launch_us": sum(quant_ms) / len(quant_ms) * 1e3},
+                         "avg_launch_us": quant_avg_ms * 1e3, "launches_timed": quant_launches},
             "e2e": {"value": e2e_value, "unit": unit, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps},
             "gpu_launches": launches_per_step * args.steps,
@@ -445,18 +470,10 @@ def run_ours(args, wl: synth.Workload, M: int):
         dist.destroy_process_group()
 
 
-def _timed(torch, fn):
-    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    a.record()
-    fn()
-    b.record()
-    return a, b
-
-
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--steps", type=int, default=20000)
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(synth.WORKLOADS))

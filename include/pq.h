@@ -12,6 +12,14 @@
  *     The library allocates and frees no device memory.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
  *     Calls are asynchronous and stream-ordered; none synchronizes the device.
+ *   - The kernels are launched with programmatic stream serialization: a call may begin its
+ *     set-up while the kernel before it in the stream drains, and waits for that kernel's
+ *     completion before it reads activations, codes or token scales and before it writes.
+ *     Packed weights and weight scales are treated as constants of the model and may be
+ *     read ahead of that wait: they must be complete before the operation that directly
+ *     precedes the GEMM call in the stream begins.  pq_pack_w8 / pq_pack_w4 guarantee this
+ *     for GEMM calls that follow them; a caller that writes weight buffers by other means
+ *     puts any stream operation (or a synchronization) between that write and the GEMM.
  *   - Matrices are dense row-major: X/Q/Y have one token per row, W has one output
  *     channel per row (K contiguous).
  *   - The return value is a pq_status.  Argument errors are detected before anything

@@ -88,8 +88,16 @@ int sm_count() {
   return d ? d->sms : 1;
 }
 
+bool pdl_enabled() {
+  static const bool on = [] {
+    const char* e = getenv("PQ_PDL");
+    return !(e != nullptr && e[0] == '0');
+  }();
+  return on;
+}
+
 int make_tmap_2d(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows,
-                 uint32_t box_cols, uint32_t elem_bytes, bool swizzle128) {
+                 uint32_t box_cols, uint32_t elem_bytes, int swizzle_bytes) {
   if (g_encode == nullptr) {
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
@@ -107,9 +115,12 @@ int make_tmap_2d(CUtensorMap* out, const void* base, uint64_t rows, uint64_t col
   cuuint64_t strides[1] = {cols * elem_bytes};
   cuuint32_t box[2] = {box_cols, box_rows};
   cuuint32_t estr[2] = {1, 1};
+  const CUtensorMapSwizzle sw = swizzle_bytes == 128  ? CU_TENSOR_MAP_SWIZZLE_128B
+                               : swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
+                               : swizzle_bytes == 32 ? CU_TENSOR_MAP_SWIZZLE_32B
+                                                     : CU_TENSOR_MAP_SWIZZLE_NONE;
   CUresult r = g_encode(out, dt, 2, const_cast<void*>(base), dims, strides, box, estr,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE,
-                        swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? PQ_OK : PQ_ERR_CUDA;
 }
@@ -157,7 +168,8 @@ int pq_pack_w8(const void* w_f16, int64_t N, int64_t K, void* wq, float* s_ch, v
   if (!aligned16(w_f16) || !aligned16(wq)) return PQ_ERR_ALIGN;
   if ((rc = check_arch()) != PQ_OK) return rc;
   // The W8 layout the GEMM reads is the row-major code matrix itself (K contiguous per channel).
-  return launch_quantize_act(w_f16, N, K, static_cast<int8_t*>(wq), s_ch, true, static_cast<cudaStream_t>(stream));
+  rc = launch_quantize_act(w_f16, N, K, static_cast<int8_t*>(wq), s_ch, true, static_cast<cudaStream_t>(stream));
+  return rc != PQ_OK ? rc : launch_pack_fence(static_cast<cudaStream_t>(stream));
 }
 
 int pq_pack_w4(const void* w_f16, int64_t N, int64_t K, int32_t group, void* wp, void* s_grp_f16, void* stream) {
@@ -167,7 +179,8 @@ int pq_pack_w4(const void* w_f16, int64_t N, int64_t K, int32_t group, void* wp,
   if (group != 128 || K % 128 != 0) return PQ_ERR_SHAPE;
   if (!aligned16(w_f16) || !aligned16(wp) || !aligned16(s_grp_f16)) return PQ_ERR_ALIGN;
   if ((rc = check_arch()) != PQ_OK) return rc;
-  return launch_pack_w4(w_f16, N, K, wp, s_grp_f16, static_cast<cudaStream_t>(stream));
+  rc = launch_pack_w4(w_f16, N, K, wp, s_grp_f16, static_cast<cudaStream_t>(stream));
+  return rc != PQ_OK ? rc : launch_pack_fence(static_cast<cudaStream_t>(stream));
 }
 
 int pq_unpack_w8(const void* wq, int64_t N, int64_t K, int8_t* codes, void* stream) {

@@ -407,18 +407,18 @@ int launch_smallm(const int8_t* q, const float* s_tok, const void* w, const floa
   CUtensorMap tw, tq, ts;
   int rc;
   if (kW4) {
-    rc = make_tmap_2d(&tw, w, static_cast<uint64_t>(N), static_cast<uint64_t>(K / 2), BW, BK / 2, 1, false);
+    rc = make_tmap_2d(&tw, w, static_cast<uint64_t>(N), static_cast<uint64_t>(K / 2), BW, BK / 2, 1, 0);
   } else {
-    rc = make_tmap_2d(&tw, w, static_cast<uint64_t>(N), static_cast<uint64_t>(K), BW, BK, 1, true);
+    rc = make_tmap_2d(&tw, w, static_cast<uint64_t>(N), static_cast<uint64_t>(K), BW, BK, 1, 128);
   }
   if (rc != PQ_OK) return rc;
-  rc = make_tmap_2d(&tq, q, static_cast<uint64_t>(M), static_cast<uint64_t>(K), static_cast<uint32_t>(mpad), BK, 1, true);
+  rc = make_tmap_2d(&tq, q, static_cast<uint64_t>(M), static_cast<uint64_t>(K), static_cast<uint32_t>(mpad), BK, 1, 128);
   if (rc != PQ_OK) return rc;
   if (kW4 && s_grp != nullptr) {
-    rc = make_tmap_2d(&ts, s_grp, static_cast<uint64_t>(K / 128), static_cast<uint64_t>(N), 1, BW, 2, false);
+    rc = make_tmap_2d(&ts, s_grp, static_cast<uint64_t>(K / 128), static_cast<uint64_t>(N), 1, BW, 2, 0);
   } else {
     ts = tq;  // unused by W8; the W4 accumulator export reads (and ignores) token bytes instead of scales
-    if (kW4) rc = make_tmap_2d(&ts, q, static_cast<uint64_t>(M), static_cast<uint64_t>(K / 2), 1, BW, 2, false);
+    if (kW4) rc = make_tmap_2d(&ts, q, static_cast<uint64_t>(M), static_cast<uint64_t>(K / 2), 1, BW, 2, 0);
   }
   if (rc != PQ_OK) return rc;
 

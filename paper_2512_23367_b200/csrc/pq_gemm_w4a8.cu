@@ -316,15 +316,15 @@ int launch_w4(const CUtensorMap& tq, const CUtensorMap& tw, const CUtensorMap& t
 int launch_gemm_w4a8(const int8_t* q, const float* s_tok, const void* wp, const void* s_grp, int64_t M,
                      int64_t N, int64_t K, void* y, int32_t* acc_g, cudaStream_t stream) {
   CUtensorMap tq, tw, ts;
-  int rc = make_tmap_2d(&tq, q, static_cast<uint64_t>(M), static_cast<uint64_t>(K), BM, BK, 1, true);
+  int rc = make_tmap_2d(&tq, q, static_cast<uint64_t>(M), static_cast<uint64_t>(K), BM, BK, 1, 128);
   if (rc != PQ_OK) return rc;
-  rc = make_tmap_2d(&tw, wp, static_cast<uint64_t>(N), static_cast<uint64_t>(K / 2), BN, BK / 2, 1, false);
+  rc = make_tmap_2d(&tw, wp, static_cast<uint64_t>(N), static_cast<uint64_t>(K / 2), BN, BK / 2, 1, 0);
   if (rc != PQ_OK) return rc;
   // Group scales [K/128, N] FP16; the accumulator-export variant has none and reads a dummy map of Q.
   if (s_grp != nullptr) {
-    rc = make_tmap_2d(&ts, s_grp, static_cast<uint64_t>(K / 128), static_cast<uint64_t>(N), 1, BN, 2, false);
+    rc = make_tmap_2d(&ts, s_grp, static_cast<uint64_t>(K / 128), static_cast<uint64_t>(N), 1, BN, 2, 0);
   } else {
-    rc = make_tmap_2d(&ts, q, static_cast<uint64_t>(M), static_cast<uint64_t>(K / 2), 1, BN, 2, false);
+    rc = make_tmap_2d(&ts, q, static_cast<uint64_t>(M), static_cast<uint64_t>(K / 2), 1, BN, 2, 0);
   }
   if (rc != PQ_OK) return rc;
   W4Args a;

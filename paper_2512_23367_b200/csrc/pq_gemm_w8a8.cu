@@ -256,9 +256,9 @@ int launch_gemm_w8a8(const int8_t* q, const float* s_tok, const void* wq, const 
   const int BN = use128 ? 128 : 256;
 
   CUtensorMap tq, tw;
-  int rc = make_tmap_2d(&tq, q, static_cast<uint64_t>(M), static_cast<uint64_t>(K), BM, BK, 1, true);
+  int rc = make_tmap_2d(&tq, q, static_cast<uint64_t>(M), static_cast<uint64_t>(K), BM, BK, 1, 128);
   if (rc != PQ_OK) return rc;
-  rc = make_tmap_2d(&tw, wq, static_cast<uint64_t>(N), static_cast<uint64_t>(K), static_cast<uint32_t>(BN), BK, 1, true);
+  rc = make_tmap_2d(&tw, wq, static_cast<uint64_t>(N), static_cast<uint64_t>(K), static_cast<uint32_t>(BN), BK, 1, 128);
   if (rc != PQ_OK) return rc;
 
   GemmArgs a;

@@ -1,16 +1,29 @@
 // W8A8 prefill GEMM on CTA pairs (tcgen05 cta_group::2) for sm_100a.
 //
-// The single-CTA kernel is bound by the bytes every SM pulls from L2 per multiply-add.  Here
-// two CTAs of a cluster share one 256 x BN output tile: each loads its own 128 rows of Q and
+// Two CTAs of a cluster share one 256 x BN output tile: each loads its own 128 rows of Q and
 // only HALF of the weight tile (BN/2 rows); one tcgen05.mma issued by the leader CTA reads both
 // halves from the two CTAs' shared memory and writes each CTA's 128 x BN accumulator into that
-// CTA's tensor memory.  Per 128 x 256 x 128 step a CTA now loads 32 KB instead of 48 KB, and the
-// smaller stages allow a six-deep ring.
+// CTA's tensor memory.  Per 128 x 256 x 128 step a CTA loads 32 KB instead of the 48 KB a lone
+// CTA would need, which keeps the main loop on the tensor-pipe limit instead of the L2 limit.
 //
-// Roles per CTA (192 threads): warp 0 TMA producer (its loads are counted on the LEADER's
-// barrier), warp 1 MMA issuer (leader CTA only; also owns TMEM allocation in both CTAs),
-// warps 2-5 epilogue (tcgen05.ld -> x token scale x channel scale -> FP16 stores) for the CTA's
-// own 128 rows.  Two TMEM accumulators overlap tile i's epilogue with tile i+1's main loop.
+// Roles per CTA:
+//   warp 0      TMA producer (its loads are counted on the LEADER's barrier)
+//   warp 1      MMA issuer (leader CTA only; also owns TMEM allocation in both CTAs)
+//   warps 2..   epilogue for the CTA's own 128 rows: one or two warps per TMEM lane quadrant
+//               (two: each takes half of the tile's columns).  tcgen05.ld of the next 32 columns
+//               is in flight while the current 32 are dequantized (x token scale x channel
+//               scale), converted to FP16 and written to a swizzled staging buffer that a TMA
+//               store drains (full 64-byte row segments; ragged edges are clipped by the tensor
+//               map).  The accumulator is handed back to the MMA issuer as soon as its last
+//               column block is in registers.
+// Two ways to overlap a tile's epilogue with the next tile's main loop are compiled:
+//   "wide":  one CTA per SM, two TMEM accumulators, deep stage ring, eight epilogue warps;
+//   "light": two co-resident CTAs per SM, each with one accumulator, a three-stage ring and four
+//            epilogue warps -- while one CTA drains its accumulator the other one multiplies, and
+//            a successor kernel launched with programmatic stream serialization finds room to
+//            set up and prefetch its weights while this kernel's last tiles finish.
+// The weight tiles of a CTA's first ring pass are requested BEFORE the wait on the preceding
+// kernel (weights are constants of the model); everything else comes after it.
 #include <cuda_fp16.h>
 
 #include <cstdlib>
@@ -25,35 +38,37 @@ constexpr int BM_CTA = 128;       // rows of Q per CTA
 constexpr int BM_PAIR = 256;      // rows of Q per tile
 constexpr int BK = 128;
 constexpr int UMMA_K = 32;
-constexpr int kNumThreads = 192;
+constexpr int kOutBoxBytes = 32 * 32 * 2;   // one staged store: 32 rows x 32 FP16 columns
 
 struct PairArgs {
   const float* s_tok;
   const float* s_ch;
-  __half* y;
   int32_t* acc;
   int* status;
   int M, N, K;
   int m_blocks, n_blocks, k_blocks;
 };
 
-template <int BN, int STAGES>
+template <int BN, int STAGES, int EPI_BUFS, int EPI_WARPS>
 struct PairSmem {
   static constexpr int kABytes = BM_CTA * BK;
   static constexpr int kBBytes = (BN / 2) * BK;
   static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kScaleOff = STAGES * kStageBytes;   // BN floats per epilogue warp
-  static constexpr int kBarOff = kScaleOff + 4 * BN * 4;
+  static constexpr int kOutOff = STAGES * kStageBytes;                     // staging, 2 KB boxes
+  static constexpr int kScaleOff = kOutOff + EPI_WARPS * EPI_BUFS * kOutBoxBytes;
+  static constexpr int kBarOff = kScaleOff + 4 * BN * 4;   // each warp's own copy of its columns' scales
   static constexpr int kNumBars = 2 * STAGES + 4;
   static constexpr int kMiscOff = kBarOff + kNumBars * 8;
   static constexpr int kDynamic = kMiscOff + 16 + 1024;
+  static_assert(kDynamic <= 232448, "exceeds the shared memory of one CTA");
 };
 
-template <int BN, int STAGES, bool kExportAcc>
-__global__ void __launch_bounds__(kNumThreads, 1)
+template <int BN, int STAGES, int EPI_BUFS, int ACC_BUFS, int EPI_WARPS, int MIN_CTAS, bool kExportAcc>
+__global__ void __launch_bounds__(64 + 32 * EPI_WARPS, MIN_CTAS)
 gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_w,
-                      const PairArgs p) {
-  using L = PairSmem<BN, STAGES>;
+                      const __grid_constant__ CUtensorMap tm_y, const PairArgs p) {
+  using L = PairSmem<BN, STAGES, EPI_BUFS, EPI_WARPS>;
+  static_assert(EPI_WARPS == 4 || EPI_WARPS == 8, "one or two epilogue warps per lane quadrant");
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t smem_base = smem_u32(smem);
@@ -61,7 +76,7 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
   const uint32_t bar_full = smem_base + L::kBarOff;     // used in the leader: both CTAs' loads landed
   const uint32_t bar_empty = bar_full + STAGES * 8;     // per CTA: the pair's MMAs released the stage
   const uint32_t bar_tfull = bar_empty + STAGES * 8;    // per CTA: accumulator complete
-  const uint32_t bar_tempty = bar_tfull + 2 * 8;        // used in the leader: both epilogues drained it
+  const uint32_t bar_tempty = bar_tfull + ACC_BUFS * 8;        // used in the leader: both epilogues drained it
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::kMiscOff);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::kMiscOff + 4);
 
@@ -71,7 +86,7 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
   const int pair_id = blockIdx.x >> 1;
   const int num_pairs = gridDim.x >> 1;
   const int num_tiles = p.m_blocks * p.n_blocks;
-  constexpr uint32_t kTmemCols = 2 * BN;
+  constexpr uint32_t kTmemCols = ACC_BUFS * BN;
 
   if (threadIdx.x == 0) {
     *abort_flag = 0;
@@ -79,15 +94,16 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
       mbar_init(bar_full + s * 8, 1);    // the leader's producer posts the byte count of BOTH CTAs
       mbar_init(bar_empty + s * 8, 1);
     }
-    for (int b = 0; b < 2; ++b) {
+    for (int b = 0; b < ACC_BUFS; ++b) {
       mbar_init(bar_tfull + b * 8, 1);
-      mbar_init(bar_tempty + b * 8, 8);  // four epilogue warps in each CTA
+      mbar_init(bar_tempty + b * 8, 2 * EPI_WARPS);  // the epilogue warps of both CTAs
     }
     fence_mbar_init();
   }
   if (warp == 0 && lane == 0) {
     tma_prefetch_desc(&tm_q);
     tma_prefetch_desc(&tm_w);
+    if constexpr (!kExportAcc) tma_prefetch_desc(&tm_y);
   }
   if (warp == 1) {
     tmem_alloc_pair(smem_u32(tmem_slot), kTmemCols);
@@ -99,22 +115,41 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
 
+  // Everything above touched no global data.  The successor kernel may start its own set-up now.
+  grid_dep_launch();
+
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer (both CTAs)
     if (lane == 0) {
       const uint32_t full0 = mapa_u32(bar_full, 0);  // the leader's ring of "stage landed" barriers
-      uint32_t it = 0;
+      // First ring pass of the first tile: weights before the wait on the preceding kernel, the
+      // codes it may have produced after it.  (Only the leader arrives on the barrier -- a plain
+      // CTA-scope arrive; the peer's bytes may land first, the transaction count then runs
+      // negative until the leader's expect_tx, which is allowed.)
+      int pre = 0;
+      if (pair_id < num_tiles) {
+        pre = p.k_blocks < STAGES ? p.k_blocks : STAGES;
+        const int n0 = (pair_id / p.m_blocks) * BN + static_cast<int>(rank) * (BN / 2);
+        for (int kb = 0; kb < pre; ++kb) {
+          if (rank == 0) mbar_arrive_expect_tx(bar_full + kb * 8, 2 * L::kStageBytes);
+          tma_load_2d_pair(smem_base + kb * L::kStageBytes + L::kABytes, &tm_w, full0 + kb * 8, kb * BK, n0);
+        }
+      }
+      grid_dep_wait();
+      if (pair_id < num_tiles) {
+        const int m0 = (pair_id % p.m_blocks) * BM_PAIR + static_cast<int>(rank) * BM_CTA;
+        for (int kb = 0; kb < pre; ++kb)
+          tma_load_2d_pair(smem_base + kb * L::kStageBytes, &tm_q, full0 + kb * 8, kb * BK, m0);
+      }
+      uint32_t it = static_cast<uint32_t>(pre);
       bool ok = true;
       for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs) {
         const int m0 = (tile % p.m_blocks) * BM_PAIR + static_cast<int>(rank) * BM_CTA;
         const int n0 = (tile / p.m_blocks) * BN + static_cast<int>(rank) * (BN / 2);
-        for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+        for (int kb = (tile == pair_id ? pre : 0); kb < p.k_blocks; ++kb, ++it) {
           const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
           if (!mbar_wait(bar_empty + s * 8, ph ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t dst = smem_base + s * L::kStageBytes;
-          // Only the leader arrives (plain CTA-scope arrive; a cluster-scope release per K block
-          // would serialise the ring).  The peer's bytes may land first: the transaction count
-          // then runs negative until the leader's expect_tx, which is allowed.
           if (rank == 0) mbar_arrive_expect_tx(bar_full + s * 8, 2 * L::kStageBytes);
           tma_load_2d_pair(dst, &tm_q, full0 + s * 8, kb * BK, m0);
           tma_load_2d_pair(dst + L::kABytes, &tm_w, full0 + s * 8, kb * BK, n0);
@@ -129,8 +164,8 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
       uint32_t it = 0, t = 0;
       bool ok = true;
       for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs, ++t) {
-        const uint32_t b = t & 1u;
-        if (!mbar_wait(bar_tempty + b * 8, ((t >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+        const uint32_t b = t % ACC_BUFS;
+        if (!mbar_wait(bar_tempty + b * 8, ((t / ACC_BUFS) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + b * BN;
         for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
@@ -149,65 +184,92 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
       }
     }
   } else {
-    // ------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
-    const int quad = warp & 3;
-    float* sc_warp = s_ch_smem + (warp - 2) * BN;
+    // ------------------------------------------------------------ epilogue (warps 2.., both CTAs)
+    grid_dep_wait();                       // token scales come from the preceding kernel; Y is overwritten
+    constexpr int HC = BN / (EPI_WARPS / 4);   // columns per epilogue warp
+    constexpr int NCH = HC / 32;           // 32-column blocks per warp and tile
+    const int e = warp - 2;
+    const int quad = warp & 3;             // TMEM lanes 32*quad .. 32*quad+31 are this warp's
+    const int half = e >> 2;               // which part of the tile's columns
+    float* sc_warp = s_ch_smem + e * HC;
+    uint8_t* out_warp = smem + L::kOutOff + e * (EPI_BUFS * kOutBoxBytes);
+    const uint32_t out_warp_u32 = smem_base + L::kOutOff + e * (EPI_BUFS * kOutBoxBytes);
     const uint32_t tempty0 = mapa_u32(bar_tempty, 0);
-    uint32_t t = 0;
+    const int sw = (lane >> 1) & 3;        // 64-byte swizzle: 16-byte chunk index XOR (row / 2) mod 4
+    uint32_t t = 0, nstore = 0;
     bool ok = true;
     for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs, ++t) {
-      const uint32_t b = t & 1u;
-      const int m0 = (tile % p.m_blocks) * BM_PAIR + static_cast<int>(rank) * BM_CTA;
-      const int n0 = (tile / p.m_blocks) * BN;
-      const int row = m0 + quad * 32 + lane;
+      const uint32_t b = t % ACC_BUFS;
+      const int row0 = (tile % p.m_blocks) * BM_PAIR + static_cast<int>(rank) * BM_CTA + quad * 32;
+      const int n0 = (tile / p.m_blocks) * BN + half * HC;
+      const int row = row0 + lane;
       float st = 0.0f;
       if constexpr (!kExportAcc) {
         __syncwarp();
-        for (int c = lane; c < BN; c += 32) sc_warp[c] = (n0 + c < p.N) ? __ldg(p.s_ch + n0 + c) : 0.0f;
+        for (int c = lane; c < HC; c += 32) sc_warp[c] = (n0 + c < p.N) ? __ldg(p.s_ch + n0 + c) : 0.0f;
         if (row < p.M) st = __ldg(p.s_tok + row);
         __syncwarp();
       }
-      ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + b * 8, (t >> 1) & 1u, abort_flag));
+      ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + b * 8, (t / ACC_BUFS) & 1u, abort_flag));
       if (!ok) break;
       tc_fence_after_sync();
-      const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + b * BN;
-#pragma unroll 1
-      for (int c0 = 0; c0 < BN; c0 += 32) {
-        uint32_t r[32];
-        tmem_ld_32x32(t_addr + c0, r);
+      const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + b * BN + half * HC;
+      uint32_t r[2][32];
+      tmem_ld_32x32(t_addr, r[0]);
+#pragma unroll
+      for (int c = 0; c < NCH; ++c) {
         tmem_ld_wait();
-        if (row < p.M) {
-          if constexpr (kExportAcc) {
-            int32_t* dst = p.acc + static_cast<int64_t>(row) * p.N + n0 + c0;
+        if (c + 1 < NCH) {
+          tmem_ld_32x32(t_addr + (c + 1) * 32, r[(c + 1) & 1]);
+        } else {
+          // The whole slice is in registers: hand the accumulator back before the arithmetic.
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster_addr(tempty0 + b * 8);
+        }
+        const uint32_t(&v)[32] = r[c & 1];
+        const int col0 = n0 + c * 32;
+        if constexpr (kExportAcc) {
+          if (row < p.M) {
+            int32_t* dst = p.acc + static_cast<int64_t>(row) * p.N + col0;
 #pragma unroll
             for (int j = 0; j < 32; j += 4) {
-              if (n0 + c0 + j < p.N)
-                *reinterpret_cast<uint4*>(dst + j) = make_uint4(r[j], r[j + 1], r[j + 2], r[j + 3]);
-            }
-          } else {
-            const float* sc = sc_warp + c0;
-            __half* dst = p.y + static_cast<int64_t>(row) * p.N + n0 + c0;
-#pragma unroll
-            for (int j = 0; j < 32; j += 8) {
-              if (n0 + c0 + j < p.N) {
-                uint32_t o[4];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                  const float2 s2 = *reinterpret_cast<const float2*>(sc + j + 2 * i);
-                  const float v0 = __fmul_rn(__fmul_rn(__int2float_rn(static_cast<int32_t>(r[j + 2 * i])), st), s2.x);
-                  const float v1 = __fmul_rn(__fmul_rn(__int2float_rn(static_cast<int32_t>(r[j + 2 * i + 1])), st), s2.y);
-                  const __half2 h = __floats2half2_rn(v0, v1);
-                  o[i] = *reinterpret_cast<const uint32_t*>(&h);
-                }
-                *reinterpret_cast<uint4*>(dst + j) = make_uint4(o[0], o[1], o[2], o[3]);
-              }
+              if (col0 + j < p.N) *reinterpret_cast<uint4*>(dst + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
             }
           }
+        } else {
+          const uint32_t buf = nstore % EPI_BUFS;
+          if (lane == 0) tma_store_wait_read<EPI_BUFS - 1>();  // the store that last read `buf` is done
+          __syncwarp();
+          const float* sc = sc_warp + c * 32;
+          uint8_t* dst = out_warp + buf * kOutBoxBytes + lane * 64;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            uint32_t o[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const float2 s2 = *reinterpret_cast<const float2*>(sc + 8 * j + 2 * i);
+              const float v0 = __fmul_rn(__fmul_rn(__int2float_rn(static_cast<int32_t>(v[8 * j + 2 * i])), st), s2.x);
+              const float v1 = __fmul_rn(__fmul_rn(__int2float_rn(static_cast<int32_t>(v[8 * j + 2 * i + 1])), st), s2.y);
+              const __half2 h = __floats2half2_rn(v0, v1);
+              o[i] = *reinterpret_cast<const uint32_t*>(&h);
+            }
+            *reinterpret_cast<uint4*>(dst + ((j ^ sw) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+          }
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            if (col0 < p.N && row0 < p.M) tma_store_2d(&tm_y, out_warp_u32 + buf * kOutBoxBytes, col0, row0);
+            tma_store_commit();  // also when nothing was stored: keeps one group per buffer use
+          }
+          ++nstore;
         }
       }
-      tc_fence_before_sync();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_cluster_addr(tempty0 + b * 8);
+    }
+    if constexpr (!kExportAcc) {
+      // The staging buffers must outlive the stores' reads; the writes themselves complete with
+      // the kernel.
+      if (lane == 0) tma_store_wait_read<0>();
     }
   }
 
@@ -224,10 +286,13 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
   if (threadIdx.x == 0 && *abort_flag) atomicExch(p.status, static_cast<int>(PQ_ERR_TIMEOUT));
 }
 
-template <int BN, int STAGES, bool kExportAcc>
-int launch_pair_cfg(const CUtensorMap& tq, const CUtensorMap& tw, const PairArgs& a, cudaStream_t stream) {
-  using L = PairSmem<BN, STAGES>;
-  auto kern = gemm_w8a8_pair_kernel<BN, STAGES, kExportAcc>;
+template <int BN, int STAGES, int EPI_BUFS, int ACC_BUFS, int EPI_WARPS, int MIN_CTAS, bool kExportAcc>
+int launch_pair_cfg(const CUtensorMap& tq, const CUtensorMap& tw, const CUtensorMap& ty, const PairArgs& a,
+                    cudaStream_t stream) {
+  using L = PairSmem<BN, STAGES, EPI_BUFS, EPI_WARPS>;
+  static_assert(MIN_CTAS * (L::kDynamic + 1024) <= 233472, "co-resident CTAs exceed the SM's shared memory");
+  static_assert(MIN_CTAS * ACC_BUFS * BN <= 512, "co-resident CTAs exceed the SM's tensor memory");
+  auto kern = gemm_w8a8_pair_kernel<BN, STAGES, EPI_BUFS, ACC_BUFS, EPI_WARPS, MIN_CTAS, kExportAcc>;
   static bool configured = false;
   if (!configured) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamic) != cudaSuccess)
@@ -235,21 +300,23 @@ int launch_pair_cfg(const CUtensorMap& tq, const CUtensorMap& tw, const PairArgs
     configured = true;
   }
   const int tiles = a.m_blocks * a.n_blocks;
-  const int max_pairs = sm_count() / 2;
+  const int max_pairs = MIN_CTAS * (sm_count() / 2);
   const int pairs = tiles < max_pairs ? tiles : max_pairs;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(static_cast<unsigned>(2 * pairs), 1, 1);
-  cfg.blockDim = dim3(kNumThreads, 1, 1);
+  cfg.blockDim = dim3(64 + 32 * EPI_WARPS, 1, 1);
   cfg.dynamicSmemBytes = L::kDynamic;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  return cuda_status(cudaLaunchKernelEx(&cfg, kern, tq, tw, a));
+  cfg.numAttrs = pdl_enabled() ? 2 : 1;
+  return cuda_status(cudaLaunchKernelEx(&cfg, kern, tq, tw, ty, a));
 }
 
 }  // namespace
@@ -269,16 +336,22 @@ int launch_gemm_w8a8_pair(const int8_t* q, const float* s_tok, const void* wq, c
   }
   const int BN = use128 ? 128 : 256;
 
-  CUtensorMap tq, tw;
-  int rc = make_tmap_2d(&tq, q, static_cast<uint64_t>(M), static_cast<uint64_t>(K), BM_CTA, BK, 1, true);
+  CUtensorMap tq, tw, ty;
+  int rc = make_tmap_2d(&tq, q, static_cast<uint64_t>(M), static_cast<uint64_t>(K), BM_CTA, BK, 1, 128);
   if (rc != PQ_OK) return rc;
-  rc = make_tmap_2d(&tw, wq, static_cast<uint64_t>(N), static_cast<uint64_t>(K), static_cast<uint32_t>(BN / 2), BK, 1, true);
+  rc = make_tmap_2d(&tw, wq, static_cast<uint64_t>(N), static_cast<uint64_t>(K), static_cast<uint32_t>(BN / 2), BK, 1, 128);
   if (rc != PQ_OK) return rc;
+  if (y != nullptr) {
+    // FP16 result [M, N]; stores go out as 32 x 32 boxes staged with the 64-byte swizzle.
+    rc = make_tmap_2d(&ty, y, static_cast<uint64_t>(M), static_cast<uint64_t>(N), 32, 32, 2, 64);
+    if (rc != PQ_OK) return rc;
+  } else {
+    ty = tq;  // the accumulator export stores directly; the map is not used
+  }
 
   PairArgs a;
   a.s_tok = s_tok;
   a.s_ch = s_ch;
-  a.y = static_cast<__half*>(y);
   a.acc = acc;
   a.status = device_status_ptr();
   if (a.status == nullptr) return PQ_ERR_CUDA;
@@ -289,9 +362,14 @@ int launch_gemm_w8a8_pair(const int8_t* q, const float* s_tok, const void* wq, c
   a.n_blocks = static_cast<int>((N + BN - 1) / BN);
   a.k_blocks = static_cast<int>((K + BK - 1) / BK);
   if (acc != nullptr) {
-    return use128 ? launch_pair_cfg<128, 8, true>(tq, tw, a, stream) : launch_pair_cfg<256, 6, true>(tq, tw, a, stream);
+    return use128 ? launch_pair_cfg<128, 7, 2, 2, 8, 1, true>(tq, tw, ty, a, stream)
+                  : launch_pair_cfg<256, 5, 2, 2, 8, 1, true>(tq, tw, ty, a, stream);
   }
-  return use128 ? launch_pair_cfg<128, 8, false>(tq, tw, a, stream) : launch_pair_cfg<256, 6, false>(tq, tw, a, stream);
+  static const int variant = [] { const char* e = getenv("PQ_W8A8_PAIR_CFG"); return e ? atoi(e) : 0; }();
+  if (use128) return launch_pair_cfg<128, 7, 2, 2, 8, 1, false>(tq, tw, ty, a, stream);
+  if (variant == 1) return launch_pair_cfg<256, 6, 1, 2, 8, 1, false>(tq, tw, ty, a, stream);
+  if (variant == 2) return launch_pair_cfg<256, 3, 1, 1, 4, 2, false>(tq, tw, ty, a, stream);
+  return launch_pair_cfg<256, 5, 2, 2, 8, 1, false>(tq, tw, ty, a, stream);
 }
 
 }  // namespace pq

@@ -14,15 +14,20 @@ int* device_status_ptr();  // device address of the status word of the current d
 // Number of SMs of the current device (cached per device).
 int sm_count();
 
+// Whether kernels are launched with the programmatic-stream-serialization attribute (default
+// yes; PQ_PDL=0 in the environment turns it off, for ablations).
+bool pdl_enabled();
+
 // cuTensorMapEncodeTiled obtained through the runtime (no link-time dependency on libcuda).
 // Encodes a 2-D row-major tensor [rows, cols] of `elem_bytes`-sized elements with a
-// box of [box_rows, box_cols]; swizzle128 selects the 128-byte shared-memory swizzle.
+// box of [box_rows, box_cols]; swizzle_bytes (0, 32, 64 or 128) selects the shared-memory swizzle.
 int make_tmap_2d(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows,
-                 uint32_t box_cols, uint32_t elem_bytes, bool swizzle128);
+                 uint32_t box_cols, uint32_t elem_bytes, int swizzle_bytes);
 
 // ---- launchers (each returns a pq_status; all are asynchronous on `stream`) ----
 int launch_quantize_act(const void* x, int64_t M, int64_t K, int8_t* q, float* s, bool divide_by_scale,
                         cudaStream_t stream);
+int launch_pack_fence(cudaStream_t stream);
 int launch_pack_w4(const void* w, int64_t N, int64_t K, void* wp, void* s_grp, cudaStream_t stream);
 int launch_unpack_w4(const void* wp, int64_t N, int64_t K, int8_t* codes, cudaStream_t stream);
 

@@ -6,6 +6,7 @@
 #include <cuda_fp16.h>
 
 #include "pq_internal.h"
+#include "pq_ptx.cuh"
 
 namespace pq {
 namespace {
@@ -56,6 +57,12 @@ __global__ void __launch_bounds__(kThreads) quantize_rows_kernel(const uint4* __
   const bool live = row < M;
   const uint4* xr = x + row * K8;
 
+  // The input may come from the kernel that precedes this one in the stream, and the codes
+  // written below may still be read by it: both wait for its completion.  The offline weight
+  // quantizer never lets its successor start early (a GEMM may prefetch the weights it writes).
+  if constexpr (!kDivide) grid_dep_launch();
+  grid_dep_wait();
+
   uint4 cache[kCached];
   float a = 0.0f;
   if (live) {
@@ -98,22 +105,32 @@ __global__ void __launch_bounds__(kThreads) quantize_rows_kernel(const uint4* __
   for (int c = t + kCached * T; c < K8; c += T) qr[c] = quantize8<kDivide>(__ldg(xr + c), f);
 }
 
+template <int T, bool kDivide>
+int launch_rows_team(const uint4* xp, int64_t M, int K8, uint2* qp, float* s, cudaStream_t stream) {
+  constexpr int kRowsPerBlock = kThreads / T;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>((M + kRowsPerBlock - 1) / kRowsPerBlock), 1, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = (!kDivide && pdl_enabled()) ? 1 : 0;
+  return cuda_status(cudaLaunchKernelEx(&cfg, quantize_rows_kernel<T, kDivide>, xp, M, K8, qp, s));
+}
+
 template <bool kDivide>
 int launch_rows(const void* x, int64_t M, int64_t K, int8_t* q, float* s, cudaStream_t stream) {
   const int K8 = static_cast<int>(K / 8);
   const uint4* xp = static_cast<const uint4*>(x);
   uint2* qp = reinterpret_cast<uint2*>(q);
   // Pick the narrowest row team that still keeps the whole row in registers.
-  if (K8 <= 32 * kCached) {
-    quantize_rows_kernel<32, kDivide><<<static_cast<unsigned>((M + 7) / 8), kThreads, 0, stream>>>(xp, M, K8, qp, s);
-  } else if (K8 <= 64 * kCached) {
-    quantize_rows_kernel<64, kDivide><<<static_cast<unsigned>((M + 3) / 4), kThreads, 0, stream>>>(xp, M, K8, qp, s);
-  } else if (K8 <= 128 * kCached) {
-    quantize_rows_kernel<128, kDivide><<<static_cast<unsigned>((M + 1) / 2), kThreads, 0, stream>>>(xp, M, K8, qp, s);
-  } else {
-    quantize_rows_kernel<256, kDivide><<<static_cast<unsigned>(M), kThreads, 0, stream>>>(xp, M, K8, qp, s);
-  }
-  return cuda_status(cudaGetLastError());
+  if (K8 <= 32 * kCached) return launch_rows_team<32, kDivide>(xp, M, K8, qp, s, stream);
+  if (K8 <= 64 * kCached) return launch_rows_team<64, kDivide>(xp, M, K8, qp, s, stream);
+  if (K8 <= 128 * kCached) return launch_rows_team<128, kDivide>(xp, M, K8, qp, s, stream);
+  return launch_rows_team<256, kDivide>(xp, M, K8, qp, s, stream);
 }
 
 // ---------------------------------------------------------------------------- INT4
@@ -173,7 +190,17 @@ __global__ void __launch_bounds__(kThreads) unpack_w4_kernel(const uint8_t* __re
   codes[n * K + k0 + 16 + b] = static_cast<int8_t>(hi);
 }
 
+// Launched (plainly, stream-ordered) behind the offline weight kernels.  A GEMM that follows in
+// the stream may request weight tiles before its own wait on its predecessor; with this kernel
+// in between, that predecessor starts only after the packed weights are complete and visible.
+__global__ void pack_fence_kernel() {}
+
 }  // namespace
+
+int launch_pack_fence(cudaStream_t stream) {
+  pack_fence_kernel<<<1, 32, 0, stream>>>();
+  return cuda_status(cudaGetLastError());
+}
 
 int launch_quantize_act(const void* x, int64_t M, int64_t K, int8_t* q, float* s, bool divide_by_scale,
                         cudaStream_t stream) {
