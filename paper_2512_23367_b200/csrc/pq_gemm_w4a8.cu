@@ -61,6 +61,7 @@ constexpr int kNumBars = 3 * STAGES + 2 * B8_SLOTS + 2 * SC_SLOTS + 2 * ACC_SLOT
 constexpr int kMiscOff = kBarOff + kNumBars * 8;
 constexpr int kDynamicSmem = kMiscOff + 16 + 1024;
 static_assert(kDynamicSmem <= 232448, "exceeds the shared memory of one CTA");
+static_assert(BK / UMMA_K == 4, "the MMA issuer is unrolled for four steps per group");
 static_assert(128 * kRegsCtl + 128 * kRegsUnpack + 256 * kRegsPromote <= 65536, "register budget");
 
 struct W4Args {
@@ -198,18 +199,23 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
           const uint32_t u = it % B8_SLOTS, uph = (it / B8_SLOTS) & 1u;
           const uint32_t a = it % ACC_SLOTS, aph = (it / ACC_SLOTS) & 1u;
-          if (!mbar_wait_cluster(bar_acc_empty + a * 8, aph ^ 1u, abort_flag) ||
-              !mbar_wait(bar_fullA + s * 8, ph, abort_flag) ||
-              !mbar_wait_cluster(bar_b8_full + u * 8, uph, abort_flag)) { ok = false; break; }
-          tc_fence_after_sync();
+          // This one thread shares its scheduler with three busy warps, so every instruction between
+          // a barrier opening and the MMAs leaving costs tens of cycles: operands are prepared
+          // before the waits, and the wait most likely to open last comes last.
           const uint64_t a_desc = umma_desc_k_sw128(smem_base + s * kStageBytes);
           const uint64_t b_desc = umma_desc_k_sw128(smem_base + kB8Off + u * kB8Bytes);
           const uint32_t d_tmem = tmem_base + a * BN;
-#pragma unroll
-          for (int k = 0; k < BK / UMMA_K; ++k) umma_i8_pair(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, k != 0);
+          if (!mbar_wait(bar_fullA + s * 8, ph, abort_flag) ||
+              !mbar_wait_cluster(bar_b8_full + u * 8, uph, abort_flag) ||
+              !mbar_wait_cluster(bar_acc_empty + a * 8, aph ^ 1u, abort_flag)) { ok = false; break; }
+          tc_fence_after_sync();
+          umma_i8_pair_imm<0>(d_tmem, a_desc, b_desc, idesc);
+          umma_i8_pair_imm<1>(d_tmem, a_desc + 2, b_desc + 2, idesc);
+          umma_i8_pair_imm<1>(d_tmem, a_desc + 4, b_desc + 4, idesc);
+          umma_i8_pair_imm<1>(d_tmem, a_desc + 6, b_desc + 6, idesc);
+          umma_commit_pair_mcast(bar_acc_full + a * 8, 0x3);
           umma_commit_pair_mcast(bar_empty + s * 8, 0x3);
           umma_commit_pair_mcast(bar_b8_empty + u * 8, 0x3);
-          umma_commit_pair_mcast(bar_acc_full + a * 8, 0x3);
         }
       }
     }
