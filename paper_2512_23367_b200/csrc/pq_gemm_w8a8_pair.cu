@@ -223,9 +223,11 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
           tmem_ld_32x32(t_addr + (c + 1) * 32, r[(c + 1) & 1]);
         } else {
           // The whole slice is in registers: hand the accumulator back before the arithmetic.
+          // (Relaxed arrive: the data moved through tensor memory, ordered by the tcgen05 fence; a
+          // release at cluster scope would cost a full memory barrier here.)
           tc_fence_before_sync();
           __syncwarp();
-          if (lane == 0) mbar_arrive_cluster_addr(tempty0 + b * 8);
+          if (lane == 0) mbar_arrive_cluster_addr_relaxed(tempty0 + b * 8);
         }
         const uint32_t(&v)[32] = r[c & 1];
         const int col0 = n0 + c * 32;
