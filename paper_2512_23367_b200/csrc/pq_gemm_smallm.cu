@@ -116,14 +116,20 @@ smallm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   const int kb1 = static_cast<int>(static_cast<int64_t>(p.k_blocks) * (split + 1) / p.splits);
   const int nkb = kb1 - kb0;
 
-  auto issue_load = [&](int j) {  // j-th K block of this CTA into stage j % STAGES
+  // The j-th K block of this CTA goes into stage j % STAGES.  Weights (and W4 group scales) are
+  // constants of the model and may be requested before the wait on the preceding kernel; the
+  // token codes may be its output and are requested after it.
+  auto issue_weights = [&](int j) {
     const uint32_t s = static_cast<uint32_t>(j) % C::STAGES;
     const uint32_t dst = smem_base + s * C::kStageBytes;
     const int kb = kb0 + j;
     mbar_arrive_expect_tx(bar_full + s * 8, C::kTxBytes);
     tma_load_2d(dst, &tm_w, bar_full + s * 8, kW4 ? kb * (BK / 2) : kb * BK, n0);
-    tma_load_2d(dst + C::kWBytes, &tm_q, bar_full + s * 8, kb * BK, 0);
     if constexpr (kW4) tma_load_2d(dst + C::kWBytes + C::kQBytes, &tm_s, bar_full + s * 8, n0, kb);
+  };
+  auto issue_codes = [&](int j) {
+    const uint32_t s = static_cast<uint32_t>(j) % C::STAGES;
+    tma_load_2d(smem_base + s * C::kStageBytes + C::kWBytes, &tm_q, bar_full + s * 8, (kb0 + j) * BK, 0);
   };
 
   if (threadIdx.x == 0) {
@@ -145,10 +151,12 @@ smallm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
       mbar_init(bar_acc_empty + s * 8, 4);
     }
     fence_mbar_init();
-    // Start the weight stream at once: the first ring pass needs no wait.
+    // Start the weight stream at once: the first ring pass needs no wait, neither on a stage
+    // nor on the preceding kernel.
     const int first = nkb < C::STAGES ? nkb : C::STAGES;
-    for (int j = 0; j < first; ++j) issue_load(j);
+    for (int j = 0; j < first; ++j) issue_weights(j);
   }
+  grid_dep_launch();   // the successor may start streaming its own weights
   if (warp == 1) {
     tmem_alloc(smem_u32(tmem_slot), C::kTmemCols);
     tmem_relinquish();
@@ -167,11 +175,15 @@ smallm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer (remaining blocks)
     if (lane == 0) {
+      grid_dep_wait();   // the token codes may come from the preceding kernel
+      const int first = nkb < C::STAGES ? nkb : C::STAGES;
+      for (int j = 0; j < first; ++j) issue_codes(j);
       int j = C::STAGES;
       for (; j < nkb; ++j) {
         const uint32_t s = static_cast<uint32_t>(j) % C::STAGES, ph = (static_cast<uint32_t>(j) / C::STAGES) & 1u;
         if (!mbar_wait(bar_empty + s * 8, ph ^ 1u, abort_flag)) { ok = false; break; }
-        issue_load(j);
+        issue_weights(j);
+        issue_codes(j);
       }
       if (!ok) {
         const int first = j >= C::STAGES ? j - C::STAGES : 0;
@@ -265,6 +277,7 @@ smallm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
     }
   } else {
     // ------------------------------------------------------------ TMEM -> registers
+    grid_dep_wait();   // token scales come from the preceding kernel; outputs are overwritten
     const int quad = warp & 3;
     const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
     const int n_local = quad * 32 + lane;
@@ -383,13 +396,15 @@ int launch_cfg(const CUtensorMap& tw, const CUtensorMap& tq, const CUtensorMap& 
   cfg.blockDim = dim3(kNumThreads, 1, 1);
   cfg.dynamicSmemBytes = C::kDynamic;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 1;
   attr[0].val.clusterDim.y = static_cast<unsigned>(a.splits);
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = pdl_enabled() ? 2 : 1;
   return cuda_status(cudaLaunchKernelEx(&cfg, kern, tw, tq, ts, a));
 }
 
