@@ -37,7 +37,10 @@ struct Cfg {
   static constexpr int kSBytes = kW4 ? BW * 2 : 0;               // FP16 group scales of the tile
   static constexpr int kStageBytes = kWBytes + kQBytes + (kW4 ? 1024 : 0);
   static constexpr int kTxBytes = kWBytes + kQBytes + kSBytes;
-  static constexpr int STAGES = kW4 ? 4 : (MPAD == 64 ? 4 : 5);
+  // Short rings and small footprints: three or four CTAs fit on an SM, so the CTAs of the NEXT
+  // launch become resident (and stream their weights) while this launch reduces and stores.
+  static constexpr int STAGES = MPAD == 64 ? 4 : 3;
+  static constexpr int kMinCtasPerSm = MPAD == 64 ? 2 : (kW4 ? 3 : 4);
   static constexpr int A8_SLOTS = kW4 ? 2 : 0;                   // widened weight tiles
   static constexpr int kA8Bytes = BW * BK;
   static constexpr int SC_SLOTS = kW4 ? 6 : 0;                   // FP32 scale rows (128 floats)
@@ -90,7 +93,7 @@ __device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t (&r)[MPAD]
 }
 
 template <int MPAD, bool kW4, bool kExportAcc>
-__global__ void __launch_bounds__(kNumThreads, 2)
+__global__ void __launch_bounds__(kNumThreads, Cfg<MPAD, kW4>::kMinCtasPerSm)
 smallm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_q,
               const __grid_constant__ CUtensorMap tm_s, const SmallArgs p) {
   using C = Cfg<MPAD, kW4>;
@@ -132,6 +135,11 @@ smallm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
     tma_load_2d(smem_base + s * C::kStageBytes + C::kWBytes, &tm_q, bar_full + s * 8, (kb0 + j) * BK, 0);
   };
 
+  if (threadIdx.x == 64) {
+    tma_prefetch_desc(&tm_w);
+    tma_prefetch_desc(&tm_q);
+    if constexpr (kW4) tma_prefetch_desc(&tm_s);
+  }
   if (threadIdx.x == 0) {
     *abort_flag = 0;
     for (int s = 0; s < C::STAGES; ++s) {
