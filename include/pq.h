@@ -141,6 +141,20 @@ PQ_API int pq_acc_w4a8(const int8_t* q, const void* wp, int32_t group, int64_t M
                 int32_t* acc_g, void* stream);
 
 /*
+ * Optional scratch memory for the current device.  With few output tiles and a long K (e.g. a
+ * 7B-class layer at M = 512) the W8A8 GEMM cuts K into parts that run on different SMs; the parts'
+ * INT32 partial accumulators pass through this scratch and are summed exactly, so results do not
+ * change.  Without registered scratch (or when it is too small for a shape) the GEMM simply does
+ * not split.  (The paper's "matrix multiplication ... within the operator template library" leaves
+ * scheduling to the kernel; this is scheduling only.)
+ *   workspace: device pointer, 256-byte aligned, owned by the caller, at least 64 KB + 1 MB
+ *   (64 MB serves every 7B-class shape); NULL or 0 bytes unregisters.  Its first 64 KB are cleared
+ *   on `stream`; GEMM calls enqueued afterwards on that stream (or after a synchronization) may use
+ *   it.  Calls that overlap on the GPU must not share one workspace.
+ */
+PQ_API int pq_set_workspace(void* workspace, size_t bytes, void* stream);
+
+/*
  * Reads the device status word of the current device into *host_status (PQ_OK or
  * PQ_ERR_TIMEOUT) and clears it.  Synchronizes the device; call it outside timed
  * regions.

@@ -31,6 +31,7 @@ SIGNATURES = {
     "pq_acc_w8a8": (ctypes.c_int, [_vp, _vp, _i64, _i64, _i64, _vp, _vp]),
     "pq_acc_w4a8": (ctypes.c_int, [_vp, _vp, _i32, _i64, _i64, _i64, _vp, _vp]),
     "pq_device_status": (ctypes.c_int, [ctypes.POINTER(ctypes.c_int)]),
+    "pq_set_workspace": (ctypes.c_int, [_vp, ctypes.c_size_t, _vp]),
 }
 
 
@@ -123,9 +124,36 @@ def pq_unpack_w4(wp: torch.Tensor, N: int, K: int) -> torch.Tensor:
     return codes
 
 
+_workspaces: dict[int, torch.Tensor] = {}
+WORKSPACE_BYTES = int(os.environ.get("PQ_WORKSPACE_MB", "64")) << 20
+
+
+def pq_set_workspace(workspace: torch.Tensor | None) -> None:
+    """Registers (or, with None, unregisters) scratch memory for the current device: a uint8 CUDA
+    tensor the caller keeps alive.  The W8A8 GEMM uses it to split K on shapes with few tiles."""
+    if workspace is None:
+        _check("pq_set_workspace", lib().pq_set_workspace(None, 0, _stream()))
+        return
+    workspace = _dev(workspace, torch.uint8, "workspace")
+    _check("pq_set_workspace", lib().pq_set_workspace(workspace.data_ptr(), workspace.numel(), _stream()))
+
+
+def _ensure_workspace(device: torch.device) -> None:
+    """Gives each device one scratch buffer on first use (torch owns the memory; the library never
+    allocates).  PQ_WORKSPACE_MB=0 turns this off."""
+    idx = device.index if device.index is not None else torch.cuda.current_device()
+    if idx in _workspaces or WORKSPACE_BYTES <= 0:
+        return
+    with torch.cuda.device(idx):
+        buf = torch.empty((WORKSPACE_BYTES,), dtype=torch.uint8, device=device)
+        pq_set_workspace(buf)
+    _workspaces[idx] = buf
+
+
 def pq_gemm_w8a8(q, s_tok, wq, s_ch, N: int, y: torch.Tensor | None = None) -> torch.Tensor:
     """q int8 [M,K], s_tok f32 [M], wq/s_ch from pq_pack_w8 -> y f16 [M,N]."""
     q = _dev(q, torch.int8, "q")
+    _ensure_workspace(q.device)
     M, K = q.shape
     _dev(s_tok, torch.float32, "s_tok"), _dev(wq, torch.uint8, "wq"), _dev(s_ch, torch.float32, "s_ch")
     if y is None:

@@ -21,6 +21,7 @@ struct DeviceInfo {
   bool ok = false;
   int sms = 0;
   int* status = nullptr;
+  Scratch scratch;
 };
 DeviceInfo g_dev[kMaxDevices];
 
@@ -81,6 +82,11 @@ EncodeTiledFn g_encode = nullptr;
 int* device_status_ptr() {
   DeviceInfo* d = current_device();
   return d ? d->status : nullptr;
+}
+
+Scratch scratch() {
+  DeviceInfo* d = current_device();
+  return d ? d->scratch : Scratch();
 }
 
 int sm_count() {
@@ -248,6 +254,30 @@ int pq_acc_w4a8(const int8_t* q, const void* wp, int32_t group, int64_t M, int64
                 void* stream) {
   if (!q || !wp || !acc_g) return PQ_ERR_NULL;
   return gemm_w4a8_common(q, nullptr, wp, nullptr, group, M, N, K, nullptr, acc_g, stream);
+}
+
+int pq_set_workspace(void* workspace, size_t bytes, void* stream) {
+  int rc = check_arch();
+  if (rc != PQ_OK) return rc;
+  DeviceInfo* d = current_device();
+  if (d == nullptr) return PQ_ERR_CUDA;
+  if (workspace == nullptr || bytes == 0) {
+    d->scratch = Scratch();
+    return PQ_OK;
+  }
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return PQ_ERR_ALIGN;
+  if (bytes < kScratchHeaderBytes + (size_t(1) << 20)) return PQ_ERR_SHAPE;
+  // the arrival counters must read zero when a GEMM first uses them
+  if (cudaMemsetAsync(workspace, 0, kScratchHeaderBytes, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+    cudaGetLastError();
+    return PQ_ERR_CUDA;
+  }
+  Scratch sc;
+  sc.counters = static_cast<unsigned int*>(workspace);
+  sc.partials = reinterpret_cast<int32_t*>(static_cast<uint8_t*>(workspace) + kScratchHeaderBytes);
+  sc.partial_bytes = bytes - kScratchHeaderBytes;
+  d->scratch = sc;
+  return PQ_OK;
 }
 
 int pq_device_status(int* host_status) {

@@ -24,6 +24,12 @@
 //            set up and prefetch its weights while this kernel's last tiles finish.
 // The weight tiles of a CTA's first ring pass are requested BEFORE the wait on the preceding
 // kernel (weights are constants of the model); everything else comes after it.
+//
+// Split-K (few tiles, long K -- e.g. M = 512): a work unit is (tile, K part).  Every unit writes
+// its INT32 partial accumulator to global scratch, fences, and bumps the tile's arrival counter;
+// the unit that arrives last adds the other parts to its own accumulator (still in tensor memory)
+// and runs the normal dequantizing epilogue.  Nobody waits for anybody, integer addition makes the
+// result independent of the arrival order, and the last unit puts the counter back to zero.
 #include <cuda_fp16.h>
 
 #include <cstdlib>
@@ -45,8 +51,11 @@ struct PairArgs {
   const float* s_ch;
   int32_t* acc;
   int* status;
+  int32_t* ws;              // split-K partial accumulators (global scratch), or nullptr
+  unsigned int* counters;   // split-K arrival counters, one per (tile, CTA of the pair); zero between calls
   int M, N, K;
   int m_blocks, n_blocks, k_blocks;
+  int splits;               // K is cut into this many parts; 1 = no split
 };
 
 template <int BN, int STAGES, int EPI_BUFS, int EPI_WARPS>
@@ -86,6 +95,9 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
   const int pair_id = blockIdx.x >> 1;
   const int num_pairs = gridDim.x >> 1;
   const int num_tiles = p.m_blocks * p.n_blocks;
+  const int num_units = num_tiles * p.splits;     // unit u = (tile u / splits, K part u % splits)
+  auto kb_begin = [&](int unit) { return static_cast<int>(static_cast<int64_t>(p.k_blocks) * (unit % p.splits) / p.splits); };
+  auto kb_end = [&](int unit) { return static_cast<int>(static_cast<int64_t>(p.k_blocks) * (unit % p.splits + 1) / p.splits); };
   constexpr uint32_t kTmemCols = ACC_BUFS * BN;
 
   if (threadIdx.x == 0) {
@@ -127,26 +139,30 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
       // CTA-scope arrive; the peer's bytes may land first, the transaction count then runs
       // negative until the leader's expect_tx, which is allowed.)
       int pre = 0;
-      if (pair_id < num_tiles) {
-        pre = p.k_blocks < STAGES ? p.k_blocks : STAGES;
-        const int n0 = (pair_id / p.m_blocks) * BN + static_cast<int>(rank) * (BN / 2);
-        for (int kb = 0; kb < pre; ++kb) {
-          if (rank == 0) mbar_arrive_expect_tx(bar_full + kb * 8, 2 * L::kStageBytes);
-          tma_load_2d_pair(smem_base + kb * L::kStageBytes + L::kABytes, &tm_w, full0 + kb * 8, kb * BK, n0);
+      if (pair_id < num_units) {
+        const int tile = pair_id / p.splits, kb0 = kb_begin(pair_id), nkb = kb_end(pair_id) - kb0;
+        pre = nkb < STAGES ? nkb : STAGES;
+        const int n0 = (tile / p.m_blocks) * BN + static_cast<int>(rank) * (BN / 2);
+        for (int j = 0; j < pre; ++j) {
+          if (rank == 0) mbar_arrive_expect_tx(bar_full + j * 8, 2 * L::kStageBytes);
+          tma_load_2d_pair(smem_base + j * L::kStageBytes + L::kABytes, &tm_w, full0 + j * 8, (kb0 + j) * BK, n0);
         }
       }
       grid_dep_wait();
-      if (pair_id < num_tiles) {
-        const int m0 = (pair_id % p.m_blocks) * BM_PAIR + static_cast<int>(rank) * BM_CTA;
-        for (int kb = 0; kb < pre; ++kb)
-          tma_load_2d_pair(smem_base + kb * L::kStageBytes, &tm_q, full0 + kb * 8, kb * BK, m0);
+      if (pair_id < num_units) {
+        const int tile = pair_id / p.splits, kb0 = kb_begin(pair_id);
+        const int m0 = (tile % p.m_blocks) * BM_PAIR + static_cast<int>(rank) * BM_CTA;
+        for (int j = 0; j < pre; ++j)
+          tma_load_2d_pair(smem_base + j * L::kStageBytes, &tm_q, full0 + j * 8, (kb0 + j) * BK, m0);
       }
       uint32_t it = static_cast<uint32_t>(pre);
       bool ok = true;
-      for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs) {
+      for (int unit = pair_id; unit < num_units && ok; unit += num_pairs) {
+        const int tile = unit / p.splits;
         const int m0 = (tile % p.m_blocks) * BM_PAIR + static_cast<int>(rank) * BM_CTA;
         const int n0 = (tile / p.m_blocks) * BN + static_cast<int>(rank) * (BN / 2);
-        for (int kb = (tile == pair_id ? pre : 0); kb < p.k_blocks; ++kb, ++it) {
+        const int kb1 = kb_end(unit);
+        for (int kb = kb_begin(unit) + (unit == pair_id ? pre : 0); kb < kb1; ++kb, ++it) {
           const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
           if (!mbar_wait(bar_empty + s * 8, ph ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t dst = smem_base + s * L::kStageBytes;
@@ -163,12 +179,13 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
       constexpr uint32_t idesc = umma_idesc_s8(BM_PAIR, BN);
       uint32_t it = 0, t = 0;
       bool ok = true;
-      for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs, ++t) {
+      for (int unit = pair_id; unit < num_units && ok; unit += num_pairs, ++t) {
         const uint32_t b = t % ACC_BUFS;
         if (!mbar_wait(bar_tempty + b * 8, ((t / ACC_BUFS) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + b * BN;
-        for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+        const int kb0 = kb_begin(unit), kb1 = kb_end(unit);
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
           if (!mbar_wait(bar_full + s * 8, ph, abort_flag)) { ok = false; break; }
           tc_fence_after_sync();
@@ -177,7 +194,7 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
           const uint64_t b_desc = umma_desc_k_sw128(a_addr + L::kABytes);
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k)
-            umma_i8_pair(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0);
+            umma_i8_pair(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb != kb0 || k != 0) ? 1u : 0u);
           umma_commit_pair_mcast(bar_empty + s * 8, 0x3);   // frees the stage in both CTAs
         }
         if (ok) umma_commit_pair_mcast(bar_tfull + b * 8, 0x3);  // accumulator ready in both CTAs
@@ -198,7 +215,9 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     const int sw = (lane >> 1) & 3;        // 64-byte swizzle: 16-byte chunk index XOR (row / 2) mod 4
     uint32_t t = 0, nstore = 0;
     bool ok = true;
-    for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs, ++t) {
+    volatile int* last_flag = reinterpret_cast<volatile int*>(smem + L::kMiscOff + 8);
+    for (int unit = pair_id; unit < num_units && ok; unit += num_pairs, ++t) {
+      const int tile = unit / p.splits;
       const uint32_t b = t % ACC_BUFS;
       const int row0 = (tile % p.m_blocks) * BM_PAIR + static_cast<int>(rank) * BM_CTA + quad * 32;
       const int n0 = (tile / p.m_blocks) * BN + half * HC;
@@ -214,6 +233,47 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
       if (!ok) break;
       tc_fence_after_sync();
       const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + b * BN + half * HC;
+      // Split-K: this CTA's slice of the tile's partials, one slot per K part.  The scratch is
+      // private, so it is laid out for coalescing: [4-column piece][row] of 16-byte words -- a warp's
+      // store of one piece covers 512 contiguous bytes.
+      const int sp = unit % p.splits;
+      const int64_t slot_elems = static_cast<int64_t>(BM_CTA) * BN;
+      uint4* ws_tile = nullptr;
+      if constexpr (!kExportAcc) {
+        if (p.splits > 1) {
+          ws_tile = reinterpret_cast<uint4*>(p.ws + (static_cast<int64_t>(tile) * 2 + rank) * p.splits * slot_elems) +
+                    static_cast<int64_t>(half * (HC / 4)) * BM_CTA + (quad * 32 + lane);
+          uint4* mine = ws_tile + sp * (slot_elems / 4);
+#pragma unroll 1
+          for (int c = 0; c < NCH; ++c) {
+            uint32_t v[32];
+            tmem_ld_32x32(t_addr + c * 32, v);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 32; j += 4)
+              __stcg(mine + (c * 8 + j / 4) * BM_CTA, make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]));
+          }
+          __threadfence();                               // the partial is visible before the arrival
+          named_bar_sync(1, EPI_WARPS * 32);
+          if (warp == 2 && lane == 0) {
+            unsigned int* ctr = p.counters + (tile * 2 + static_cast<int>(rank));
+            const unsigned int old = atomicAdd(ctr, 1u);
+            const int last = (old == static_cast<unsigned int>(p.splits - 1));
+            if (last) *ctr = 0u;                         // nobody else touches it in this call; zero for the next
+            *last_flag = last;
+          }
+          named_bar_sync(1, EPI_WARPS * 32);
+          const bool last = *last_flag != 0;
+          __threadfence();                               // the other parts' partials are read after the arrival count
+          if (!last) {
+            // Not the last part of this tile: the accumulator is saved, hand it back and move on.
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster_addr_relaxed(tempty0 + b * 8);
+            continue;
+          }
+        }
+      }
       uint32_t r[2][32];
       tmem_ld_32x32(t_addr, r[0]);
 #pragma unroll
@@ -229,8 +289,22 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
           __syncwarp();
           if (lane == 0) mbar_arrive_cluster_addr_relaxed(tempty0 + b * 8);
         }
-        const uint32_t(&v)[32] = r[c & 1];
+        uint32_t(&v)[32] = r[c & 1];
         const int col0 = n0 + c * 32;
+        if constexpr (!kExportAcc) {
+          if (p.splits > 1) {
+            // add the other K parts (exact integer sums; read through L2, where they were written)
+            for (int o = 0; o < p.splits; ++o) {
+              if (o == sp) continue;
+              const uint4* theirs = ws_tile + o * (slot_elems / 4) + c * 8 * BM_CTA;
+#pragma unroll
+              for (int j = 0; j < 32; j += 4) {
+                const uint4 w4 = __ldcg(theirs + (j / 4) * BM_CTA);
+                v[j] += w4.x; v[j + 1] += w4.y; v[j + 2] += w4.z; v[j + 3] += w4.w;
+              }
+            }
+          }
+        }
         if constexpr (kExportAcc) {
           if (row < p.M) {
             int32_t* dst = p.acc + static_cast<int64_t>(row) * p.N + col0;
@@ -301,9 +375,9 @@ int launch_pair_cfg(const CUtensorMap& tq, const CUtensorMap& tw, const CUtensor
       return PQ_ERR_CUDA;
     configured = true;
   }
-  const int tiles = a.m_blocks * a.n_blocks;
+  const int units = a.m_blocks * a.n_blocks * a.splits;
   const int max_pairs = MIN_CTAS * (sm_count() / 2);
-  const int pairs = tiles < max_pairs ? tiles : max_pairs;
+  const int pairs = units < max_pairs ? units : max_pairs;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(static_cast<unsigned>(2 * pairs), 1, 1);
   cfg.blockDim = dim3(64 + 32 * EPI_WARPS, 1, 1);
@@ -325,18 +399,44 @@ int launch_pair_cfg(const CUtensorMap& tq, const CUtensorMap& tw, const CUtensor
 
 int launch_gemm_w8a8_pair(const int8_t* q, const float* s_tok, const void* wq, const float* s_ch, int64_t M,
                           int64_t N, int64_t K, void* y, int32_t* acc, cudaStream_t stream) {
-  // Tile width by the same cost model as the single-CTA kernel: waves of pair tiles over the
-  // SM pairs x bytes a CTA loads per K block (16 KB of Q + BN/2 rows of weights).
+  // Plan: tile width (256 or 128 columns) x number of K parts.  Cost of a plan in SM cycles:
+  //   waves of work units over the SM pairs x (K blocks per unit x cycles per K block + fixed cost
+  //   of a unit's epilogue, plus the scratch round trip when K is split: ~9000 cycles measured).
+  // Cycles per K block are measured figures: 512 for a 256-wide tile (the tensor-pipe time), 550
+  // for a 128-wide one (bound by the bytes each SM pulls per multiply-add, not faster per block).
   const int pairs = sm_count() / 2;
   const int64_t mb = (M + BM_PAIR - 1) / BM_PAIR;
-  const int64_t t256 = mb * ((N + 255) / 256), t128 = mb * ((N + 127) / 128);
-  auto waves = [pairs](int64_t tiles) { return (tiles + pairs - 1) / pairs; };
-  bool use128 = (N <= 128) || (waves(t128) * 24 < waves(t256) * 32);
-  if (const char* e = getenv("PQ_W8A8_BN")) {  // ablation knob: force the tile width
-    if (e[0] == '1') use128 = true;
-    if (e[0] == '2') use128 = false;
+  const int64_t kblocks = (K + BK - 1) / BK;
+  const Scratch sc = scratch();
+  auto waves = [pairs](int64_t units) { return (units + pairs - 1) / pairs; };
+  int best_bn = 256, best_splits = 1;
+  int64_t best_cost = -1;
+  const int force_bn = [] { const char* e = getenv("PQ_W8A8_BN"); return e ? (e[0] == '1' ? 128 : (e[0] == '2' ? 256 : 0)) : 0; }();
+  const int force_splits = [] { const char* e = getenv("PQ_W8A8_SPLITS"); return e ? atoi(e) : 0; }();
+  for (int bn = 256; bn >= 128; bn /= 2) {
+    if (force_bn != 0 && bn != force_bn) continue;
+    if (bn == 256 && N <= 128) continue;
+    const int64_t tiles = mb * ((N + bn - 1) / bn);
+    for (int sp = 1; sp <= 4; ++sp) {
+      if (force_splits != 0 && sp != force_splits) continue;
+      if (sp > 1) {
+        if (acc != nullptr || kblocks / sp < 8) break;
+        const size_t need = static_cast<size_t>(tiles) * 2 * sp * BM_CTA * bn * sizeof(int32_t);
+        if (sc.partials == nullptr || need > sc.partial_bytes || tiles * 2 > kScratchCounters) break;
+      }
+      const int64_t per_unit = ((kblocks + sp - 1) / sp) * (bn == 256 ? 512 : 550) + (bn == 256 ? 3000 : 1800) +
+                               (sp > 1 ? 9000 : 0);   // measured: partial save + fence + reload ~ 4.7 us
+      const int64_t cost = waves(tiles * sp) * per_unit;
+      if (best_cost < 0 || cost < best_cost) {
+        best_cost = cost;
+        best_bn = bn;
+        best_splits = sp;
+      }
+    }
   }
-  const int BN = use128 ? 128 : 256;
+  if (best_cost < 0) return PQ_ERR_SHAPE;   // only reachable through contradictory ablation knobs
+  const bool use128 = best_bn == 128;
+  const int BN = best_bn;
 
   CUtensorMap tq, tw, ty;
   int rc = make_tmap_2d(&tq, q, static_cast<uint64_t>(M), static_cast<uint64_t>(K), BM_CTA, BK, 1, 128);
@@ -362,7 +462,10 @@ int launch_gemm_w8a8_pair(const int8_t* q, const float* s_tok, const void* wq, c
   a.K = static_cast<int>(K);
   a.m_blocks = static_cast<int>(mb);
   a.n_blocks = static_cast<int>((N + BN - 1) / BN);
-  a.k_blocks = static_cast<int>((K + BK - 1) / BK);
+  a.k_blocks = static_cast<int>(kblocks);
+  a.splits = best_splits;
+  a.ws = best_splits > 1 ? sc.partials : nullptr;
+  a.counters = best_splits > 1 ? sc.counters : nullptr;
   if (acc != nullptr) {
     return use128 ? launch_pair_cfg<128, 7, 2, 2, 8, 1, true>(tq, tw, ty, a, stream)
                   : launch_pair_cfg<256, 5, 2, 2, 8, 1, true>(tq, tw, ty, a, stream);

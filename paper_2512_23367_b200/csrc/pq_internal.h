@@ -14,6 +14,17 @@ int* device_status_ptr();  // device address of the status word of the current d
 // Number of SMs of the current device (cached per device).
 int sm_count();
 
+// Caller-provided scratch of the current device (pq_set_workspace): arrival counters first, then
+// room for split-K partial accumulators.  All null/zero when none is registered.
+struct Scratch {
+  unsigned int* counters = nullptr;   // kScratchCounters words, zero between calls
+  int32_t* partials = nullptr;
+  size_t partial_bytes = 0;
+};
+constexpr int kScratchCounters = 16384;                       // 64 KB
+constexpr size_t kScratchHeaderBytes = kScratchCounters * 4;
+Scratch scratch();
+
 // Whether kernels are launched with the programmatic-stream-serialization attribute (default
 // yes; PQ_PDL=0 in the environment turns it off, for ablations).
 bool pdl_enabled();

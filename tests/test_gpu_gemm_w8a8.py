@@ -99,3 +99,36 @@ def test_full_size_layers_on_sampled_rows(M, K, N):
     rng = np.random.default_rng(M + K + N)
     rows = np.unique(np.concatenate([[0, 127, 128, M - 129, M - 1], rng.integers(0, M, 19)]))
     run_case(M, N, K, seed=2000 + N % 97, rows=rows)
+
+
+@pytest.mark.parametrize("M,K,N", [(512, 11008, 1024), (300, 11008, 520), (140, 6144, 136), (257, 8192, 264)])
+def test_split_k_through_scratch_matches_the_unsplit_result_bit_for_bit(M, K, N):
+    """Few tiles and a long K: with registered scratch the GEMM cuts K into parts and sums the INT32
+    partials exactly, so the FP16 output must equal the one computed without scratch, twice in a row
+    (the arrival counters go back to zero), and must match the oracle."""
+    x = synth.activations(M, K, seed=77)
+    w = synth.weights(N, K, seed=78)
+    q, s_tok = pq.pq_quantize_act(torch.from_numpy(x).to(DEV))
+    wq, s_ch = pq.pq_pack_w8(torch.from_numpy(w).to(DEV))
+    pad = 2048
+    buf = torch.full((pad + M * N + pad,), 7.0, dtype=torch.float16, device=DEV)
+    y_split = buf[pad:pad + M * N].view(M, N)
+    pq.pq_gemm_w8a8(q, s_tok, wq, s_ch, N, y=y_split)          # scratch registered by the binding
+    y_again = pq.pq_gemm_w8a8(q, s_tok, wq, s_ch, N)
+    torch.cuda.synchronize()
+    pq.pq_set_workspace(None)
+    try:
+        y_plain = pq.pq_gemm_w8a8(q, s_tok, wq, s_ch, N)
+        torch.cuda.synchronize()
+    finally:
+        ws = torch.empty((64 << 20,), dtype=torch.uint8, device=DEV)
+        pq.pq_set_workspace(ws)
+        pq.binding._workspaces[torch.device(DEV).index or 0] = ws
+    assert pq.pq_device_status() == 0
+    assert torch.equal(y_split, y_plain) and torch.equal(y_again, y_plain)
+    assert (buf[:pad] == 7.0).all() and (buf[pad + M * N:] == 7.0).all()
+    q_ref, st_ref = oracle.quantize_act(x)
+    wq_ref, sc_ref = oracle.pack_w8(w)
+    rows = np.unique(np.concatenate([[0, 127, 128, M - 1], np.arange(0, M, 37)]))
+    _, y_ref = oracle.gemm_w8a8(q_ref[rows], st_ref[rows], wq_ref, sc_ref)
+    assert_y_close(_np(y_split)[rows], y_ref)
