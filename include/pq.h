@@ -155,6 +155,29 @@ PQ_API int pq_acc_w4a8(const int8_t* q, const void* wp, int32_t group, int64_t M
 PQ_API int pq_set_workspace(void* workspace, size_t bytes, void* stream);
 
 /*
+ * W8A8 linear for callers that cannot allocate device memory (the paper has no counterpart to
+ * this call; it exists for deployment constraints, not for the method).
+ *
+ * Same arguments, same result as pq_gemm_w8a8.  The difference is where the split-K scratch comes
+ * from: not from a buffer registered with pq_set_workspace -- which somebody had to cudaMalloc --
+ * but from a fixed 32 MiB + 64 KiB array inside the library, held by every GPU that loads the
+ * library until the process exits.  Meant for hosts that hand a plug-in nothing but its inputs and
+ * outputs, for serving loops and capture regions in which cudaMalloc (a synchronizing call) is
+ * off limits, and for programs that fix their whole device-memory budget at start-up.  The call
+ * itself invokes no allocation or free routine of any kind.
+ *   - Limit: M and N each rounded up to a multiple of 256, multiplied, may not exceed 2,097,152
+ *     (e.g. 512 x 4096, 1024 x 2048, 256 x 8192); beyond that the call returns PQ_ERR_LIMIT and
+ *     launches nothing.  M <= 128 needs no scratch and is simply forwarded to pq_gemm_w8a8.
+ *   - The first call on each device looks up the array's device address; make that first call
+ *     outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps whatever the last call left in it
+ *     (the kernel restores the few words that must read zero).  Two calls that overlap on the GPU
+ *     -- different streams, parallel graph branches -- would race on it: keep them ordered.
+ */
+PQ_API int pq_gemm_w8a8_noalloc(const int8_t* q, const float* s_tok, const void* wq, const float* s_ch,
+                                int64_t M, int64_t N, int64_t K, void* y_f16, void* stream);
+
+/*
  * Reads the device status word of the current device into *host_status (PQ_OK or
  * PQ_ERR_TIMEOUT) and clears it.  Synchronizes the device; call it outside timed
  * regions.

@@ -32,6 +32,7 @@ SIGNATURES = {
     "pq_acc_w4a8": (ctypes.c_int, [_vp, _vp, _i32, _i64, _i64, _i64, _vp, _vp]),
     "pq_device_status": (ctypes.c_int, [ctypes.POINTER(ctypes.c_int)]),
     "pq_set_workspace": (ctypes.c_int, [_vp, ctypes.c_size_t, _vp]),
+    "pq_gemm_w8a8_noalloc": (ctypes.c_int, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _vp, _vp]),
 }
 
 
@@ -160,6 +161,20 @@ def pq_gemm_w8a8(q, s_tok, wq, s_ch, N: int, y: torch.Tensor | None = None) -> t
         y = torch.empty((M, N), dtype=torch.float16, device=q.device)
     _check("pq_gemm_w8a8", lib().pq_gemm_w8a8(q.data_ptr(), s_tok.data_ptr(), wq.data_ptr(), s_ch.data_ptr(),
                                               M, N, K, y.data_ptr(), _stream()))
+    return y
+
+
+def pq_gemm_w8a8_noalloc(q, s_tok, wq, s_ch, N: int, y: torch.Tensor) -> torch.Tensor:
+    """Same product as pq_gemm_w8a8, for callers that may not allocate: the output tensor is
+    required (this wrapper creates none) and the library's built-in scratch array is used instead of
+    a registered workspace.  Raises PQError with status 7 when the padded output exceeds 2 Mi
+    elements.  Calls on one device must not overlap on the GPU."""
+    q = _dev(q, torch.int8, "q")
+    M, K = q.shape
+    _dev(s_tok, torch.float32, "s_tok"), _dev(wq, torch.uint8, "wq"), _dev(s_ch, torch.float32, "s_ch")
+    _dev(y, torch.float16, "y")
+    _check("pq_gemm_w8a8_noalloc", lib().pq_gemm_w8a8_noalloc(q.data_ptr(), s_tok.data_ptr(), wq.data_ptr(),
+                                                              s_ch.data_ptr(), M, N, K, y.data_ptr(), _stream()))
     return y
 
 

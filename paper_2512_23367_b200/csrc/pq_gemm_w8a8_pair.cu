@@ -397,8 +397,9 @@ int launch_pair_cfg(const CUtensorMap& tq, const CUtensorMap& tw, const CUtensor
 
 }  // namespace
 
-int launch_gemm_w8a8_pair(const int8_t* q, const float* s_tok, const void* wq, const float* s_ch, int64_t M,
-                          int64_t N, int64_t K, void* y, int32_t* acc, cudaStream_t stream) {
+int launch_gemm_w8a8_pair_with(const Scratch& sc, const int8_t* q, const float* s_tok, const void* wq,
+                               const float* s_ch, int64_t M, int64_t N, int64_t K, void* y, int32_t* acc,
+                               cudaStream_t stream) {
   // Plan: tile width (256 or 128 columns) x number of K parts.  Cost of a plan in SM cycles:
   //   waves of work units over the SM pairs x (K blocks per unit x cycles per K block + fixed cost
   //   of a unit's epilogue, plus the scratch round trip when K is split: ~9000 cycles measured).
@@ -407,7 +408,6 @@ int launch_gemm_w8a8_pair(const int8_t* q, const float* s_tok, const void* wq, c
   const int pairs = sm_count() / 2;
   const int64_t mb = (M + BM_PAIR - 1) / BM_PAIR;
   const int64_t kblocks = (K + BK - 1) / BK;
-  const Scratch sc = scratch();
   auto waves = [pairs](int64_t units) { return (units + pairs - 1) / pairs; };
   int best_bn = 256, best_splits = 1;
   int64_t best_cost = -1;
@@ -475,6 +475,11 @@ int launch_gemm_w8a8_pair(const int8_t* q, const float* s_tok, const void* wq, c
   if (variant == 1) return launch_pair_cfg<256, 6, 1, 2, 8, 1, false>(tq, tw, ty, a, stream);
   if (variant == 2) return launch_pair_cfg<256, 3, 1, 1, 4, 2, false>(tq, tw, ty, a, stream);
   return launch_pair_cfg<256, 5, 2, 2, 8, 1, false>(tq, tw, ty, a, stream);
+}
+
+int launch_gemm_w8a8_pair(const int8_t* q, const float* s_tok, const void* wq, const float* s_ch, int64_t M,
+                          int64_t N, int64_t K, void* y, int32_t* acc, cudaStream_t stream) {
+  return launch_gemm_w8a8_pair_with(scratch(), q, s_tok, wq, s_ch, M, N, K, y, acc, stream);
 }
 
 }  // namespace pq

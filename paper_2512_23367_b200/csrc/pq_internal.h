@@ -48,6 +48,10 @@ int launch_gemm_w8a8(const int8_t* q, const float* s_tok, const void* wq, const 
 // Same contract on CTA pairs (cta_group::2, 256-row tiles); preferred when M > 128.
 int launch_gemm_w8a8_pair(const int8_t* q, const float* s_tok, const void* wq, const float* s_ch, int64_t M,
                           int64_t N, int64_t K, void* y, int32_t* acc, cudaStream_t stream);
+// The same with the split-K scratch given explicitly instead of taken from the device's registry.
+int launch_gemm_w8a8_pair_with(const Scratch& sc, const int8_t* q, const float* s_tok, const void* wq,
+                               const float* s_ch, int64_t M, int64_t N, int64_t K, void* y, int32_t* acc,
+                               cudaStream_t stream);
 // Prefill-shaped W4A8 GEMM.  Exactly one of y / acc_g is non-null.
 int launch_gemm_w4a8(const int8_t* q, const float* s_tok, const void* wp, const void* s_grp, int64_t M,
                      int64_t N, int64_t K, void* y, int32_t* acc_g, cudaStream_t stream);
