@@ -155,6 +155,15 @@ PQ_API int pq_acc_w4a8(const int8_t* q, const void* wp, int32_t group, int64_t M
 PQ_API int pq_set_workspace(void* workspace, size_t bytes, void* stream);
 
 /*
+ * Host-only query (touches no device): the schedule pq_gemm_w8a8 picks for M > 128 on a GPU with
+ * `sms` multiprocessors and a registered workspace of `scratch_bytes` (0 = none): the output tile
+ * width (*tile_n = 256 or 128 columns) and the number of parts K is cut into (*k_parts, 1 = no
+ * split).  For capacity planning and tests; the result has no effect on later calls.
+ */
+PQ_API int pq_plan_w8a8(int64_t M, int64_t N, int64_t K, int32_t sms, size_t scratch_bytes, int32_t* tile_n,
+                        int32_t* k_parts);
+
+/*
  * W8A8 linear for callers that cannot allocate device memory (the paper has no counterpart to
  * this call; it exists for deployment constraints, not for the method).
  *

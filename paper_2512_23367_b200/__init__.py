@@ -18,6 +18,7 @@ from .binding import (  # noqa: F401
     pq_gemm_w8a8_noalloc,
     pq_pack_w4,
     pq_pack_w8,
+    pq_plan_w8a8,
     pq_quantize_act,
     pq_set_workspace,
     pq_unpack_w4,

@@ -32,6 +32,7 @@ SIGNATURES = {
     "pq_acc_w4a8": (ctypes.c_int, [_vp, _vp, _i32, _i64, _i64, _i64, _vp, _vp]),
     "pq_device_status": (ctypes.c_int, [ctypes.POINTER(ctypes.c_int)]),
     "pq_set_workspace": (ctypes.c_int, [_vp, ctypes.c_size_t, _vp]),
+    "pq_plan_w8a8": (ctypes.c_int, [_i64, _i64, _i64, _i32, ctypes.c_size_t, ctypes.POINTER(_i32), ctypes.POINTER(_i32)]),
     "pq_gemm_w8a8_noalloc": (ctypes.c_int, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _vp, _vp]),
 }
 
@@ -123,6 +124,13 @@ def pq_unpack_w4(wp: torch.Tensor, N: int, K: int) -> torch.Tensor:
     codes = torch.empty((N, K), dtype=torch.int8, device=wp.device)
     _check("pq_unpack_w4", lib().pq_unpack_w4(wp.data_ptr(), N, K, codes.data_ptr(), _stream()))
     return codes
+
+
+def pq_plan_w8a8(M: int, N: int, K: int, sms: int = 148, scratch_bytes: int = 0) -> tuple[int, int]:
+    """(tile width, number of K parts) the W8A8 GEMM would choose; host-only, needs no GPU."""
+    bn, sp = _i32(0), _i32(0)
+    _check("pq_plan_w8a8", lib().pq_plan_w8a8(M, N, K, sms, scratch_bytes, ctypes.byref(bn), ctypes.byref(sp)))
+    return int(bn.value), int(sp.value)
 
 
 _workspaces: dict[int, torch.Tensor] = {}

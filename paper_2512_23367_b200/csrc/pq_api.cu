@@ -256,6 +256,20 @@ int pq_acc_w4a8(const int8_t* q, const void* wp, int32_t group, int64_t M, int64
   return gemm_w4a8_common(q, nullptr, wp, nullptr, group, M, N, K, nullptr, acc_g, stream);
 }
 
+int pq_plan_w8a8(int64_t M, int64_t N, int64_t K, int32_t sms, size_t scratch_bytes, int32_t* tile_n,
+                 int32_t* k_parts) {
+  if (!tile_n || !k_parts) return PQ_ERR_NULL;
+  int rc = check_gemm(M, N, K);
+  if (rc != PQ_OK) return rc;
+  if (sms < 2) return PQ_ERR_SHAPE;
+  int bn = 256, sp = 1;
+  const size_t room = scratch_bytes > kScratchHeaderBytes ? scratch_bytes - kScratchHeaderBytes : 0;
+  if (plan_w8a8_pair(M, N, K, sms, room, 0, 0, &bn, &sp) < 0) return PQ_ERR_SHAPE;
+  *tile_n = bn;
+  *k_parts = sp;
+  return PQ_OK;
+}
+
 int pq_set_workspace(void* workspace, size_t bytes, void* stream) {
   int rc = check_arch();
   if (rc != PQ_OK) return rc;

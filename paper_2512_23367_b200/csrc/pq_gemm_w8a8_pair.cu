@@ -397,43 +397,54 @@ int launch_pair_cfg(const CUtensorMap& tq, const CUtensorMap& tw, const CUtensor
 
 }  // namespace
 
-int launch_gemm_w8a8_pair_with(const Scratch& sc, const int8_t* q, const float* s_tok, const void* wq,
-                               const float* s_ch, int64_t M, int64_t N, int64_t K, void* y, int32_t* acc,
-                               cudaStream_t stream) {
-  // Plan: tile width (256 or 128 columns) x number of K parts.  Cost of a plan in SM cycles:
-  //   waves of work units over the SM pairs x (K blocks per unit x cycles per K block + fixed cost
-  //   of a unit's epilogue, plus the scratch round trip when K is split: ~9000 cycles measured).
-  // Cycles per K block are measured figures: 512 for a 256-wide tile (the tensor-pipe time), 550
-  // for a 128-wide one (bound by the bytes each SM pulls per multiply-add, not faster per block).
-  const int pairs = sm_count() / 2;
+// Plan: tile width (256 or 128 columns) x number of K parts.  Cost of a plan in SM cycles:
+//   waves of work units over the SM pairs x (K blocks per unit x cycles per K block + fixed cost
+//   of a unit's epilogue, plus the scratch round trip when K is split: ~9000 cycles measured).
+// Cycles per K block are measured figures: 512 for a 256-wide tile (the tensor-pipe time), 550
+// for a 128-wide one (bound by the bytes each SM pulls per multiply-add, not faster per block).
+// `scratch_bytes` = room for split-K partials (0: never split); force_* = 0 means "free choice".
+// Returns the cost of the chosen plan, or -1 if the forced values admit none.
+int64_t plan_w8a8_pair(int64_t M, int64_t N, int64_t K, int sms, size_t scratch_bytes, int force_bn,
+                       int force_splits, int* bn_out, int* splits_out) {
+  const int pairs = sms / 2 > 0 ? sms / 2 : 1;
   const int64_t mb = (M + BM_PAIR - 1) / BM_PAIR;
   const int64_t kblocks = (K + BK - 1) / BK;
   auto waves = [pairs](int64_t units) { return (units + pairs - 1) / pairs; };
-  int best_bn = 256, best_splits = 1;
   int64_t best_cost = -1;
-  const int force_bn = [] { const char* e = getenv("PQ_W8A8_BN"); return e ? (e[0] == '1' ? 128 : (e[0] == '2' ? 256 : 0)) : 0; }();
-  const int force_splits = [] { const char* e = getenv("PQ_W8A8_SPLITS"); return e ? atoi(e) : 0; }();
   for (int bn = 256; bn >= 128; bn /= 2) {
     if (force_bn != 0 && bn != force_bn) continue;
-    if (bn == 256 && N <= 128) continue;
+    if (bn == 256 && N <= 128 && force_bn == 0) continue;
     const int64_t tiles = mb * ((N + bn - 1) / bn);
     for (int sp = 1; sp <= 4; ++sp) {
       if (force_splits != 0 && sp != force_splits) continue;
       if (sp > 1) {
-        if (acc != nullptr || kblocks / sp < 8) break;
+        if (kblocks / sp < 8) break;
         const size_t need = static_cast<size_t>(tiles) * 2 * sp * BM_CTA * bn * sizeof(int32_t);
-        if (sc.partials == nullptr || need > sc.partial_bytes || tiles * 2 > kScratchCounters) break;
+        if (need > scratch_bytes || tiles * 2 > kScratchCounters) break;
       }
       const int64_t per_unit = ((kblocks + sp - 1) / sp) * (bn == 256 ? 512 : 550) + (bn == 256 ? 3000 : 1800) +
                                (sp > 1 ? 9000 : 0);   // measured: partial save + fence + reload ~ 4.7 us
       const int64_t cost = waves(tiles * sp) * per_unit;
       if (best_cost < 0 || cost < best_cost) {
         best_cost = cost;
-        best_bn = bn;
-        best_splits = sp;
+        *bn_out = bn;
+        *splits_out = sp;
       }
     }
   }
+  return best_cost;
+}
+
+int launch_gemm_w8a8_pair_with(const Scratch& sc, const int8_t* q, const float* s_tok, const void* wq,
+                               const float* s_ch, int64_t M, int64_t N, int64_t K, void* y, int32_t* acc,
+                               cudaStream_t stream) {
+  const int64_t mb = (M + BM_PAIR - 1) / BM_PAIR;
+  const int64_t kblocks = (K + BK - 1) / BK;
+  const int force_bn = [] { const char* e = getenv("PQ_W8A8_BN"); return e ? (e[0] == '1' ? 128 : (e[0] == '2' ? 256 : 0)) : 0; }();
+  const int force_splits = [] { const char* e = getenv("PQ_W8A8_SPLITS"); return e ? atoi(e) : 0; }();
+  int best_bn = 256, best_splits = 1;
+  const int64_t best_cost = plan_w8a8_pair(M, N, K, sm_count(), acc == nullptr && sc.partials != nullptr ? sc.partial_bytes : 0,
+                                           force_bn, force_splits, &best_bn, &best_splits);
   if (best_cost < 0) return PQ_ERR_SHAPE;   // only reachable through contradictory ablation knobs
   const bool use128 = best_bn == 128;
   const int BN = best_bn;

@@ -48,6 +48,9 @@ int launch_gemm_w8a8(const int8_t* q, const float* s_tok, const void* wq, const 
 // Same contract on CTA pairs (cta_group::2, 256-row tiles); preferred when M > 128.
 int launch_gemm_w8a8_pair(const int8_t* q, const float* s_tok, const void* wq, const float* s_ch, int64_t M,
                           int64_t N, int64_t K, void* y, int32_t* acc, cudaStream_t stream);
+// Host-only: the pair GEMM's choice of tile width and number of K parts (see the definition).
+int64_t plan_w8a8_pair(int64_t M, int64_t N, int64_t K, int sms, size_t scratch_bytes, int force_bn,
+                       int force_splits, int* bn_out, int* splits_out);
 // The same with the split-K scratch given explicitly instead of taken from the device's registry.
 int launch_gemm_w8a8_pair_with(const Scratch& sc, const int8_t* q, const float* s_tok, const void* wq,
                                const float* s_ch, int64_t M, int64_t N, int64_t K, void* y, int32_t* acc,

@@ -38,3 +38,22 @@ def test_argument_errors_come_back_as_status_codes_without_a_device():
     assert L.pq_pack_w4(16, 16, 256, 128, None, 16, None) == PQ_ERR_NULL
     assert L.pq_packed_w8_bytes(8, 256) == 2048 and L.pq_packed_w4_bytes(8, 256) == 1024
     assert L.pq_status_str(0) == b"ok" and b"wait" in L.pq_status_str(6)
+
+
+def test_schedule_choice_for_the_benchmark_shapes():
+    """Host logic of the W8A8 pair GEMM: tile width and K parts, on a 148-SM device."""
+    ws = 64 << 20
+    # many tiles: wide tiles, no split, with or without scratch
+    assert pq.pq_plan_w8a8(4096, 11008, 4096, 148, ws) == (256, 1)
+    assert pq.pq_plan_w8a8(2048, 2048, 2048, 148, ws) == (256, 1)
+    assert pq.pq_plan_w8a8(2048, 2048, 6144, 148, ws) == (256, 1)
+    # 32 tiles and 86 K blocks: two K parts fill the machine -- but only with room for the partials
+    assert pq.pq_plan_w8a8(512, 4096, 11008, 148, ws) == (256, 2)
+    assert pq.pq_plan_w8a8(512, 4096, 11008, 148, 0) == (256, 1)
+    assert pq.pq_plan_w8a8(512, 4096, 11008, 148, 8 << 20)[1] == 1      # 16 MiB needed
+    # short K: the scratch round trip costs more than it saves
+    assert pq.pq_plan_w8a8(512, 4096, 4096, 148, ws) == (256, 1)
+    # a single narrow tile column
+    assert pq.pq_plan_w8a8(300, 128, 2048, 148, ws)[0] == 128
+    # a few tiles with a very long K: up to four parts
+    assert pq.pq_plan_w8a8(257, 264, 8192, 148, ws)[1] == 4
