@@ -77,7 +77,7 @@ __global__ void __launch_bounds__(64 + 32 * EPI_WARPS, MIN_CTAS)
 gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_w,
                       const __grid_constant__ CUtensorMap tm_y, const PairArgs p) {
   using L = PairSmem<BN, STAGES, EPI_BUFS, EPI_WARPS>;
-  static_assert(EPI_WARPS == 4 || EPI_WARPS == 8, "one or two epilogue warps per lane quadrant");
+  static_assert(EPI_WARPS == 4 || EPI_WARPS == 8 || EPI_WARPS == 16, "one, two or four epilogue warps per lane quadrant");
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t smem_base = smem_u32(smem);
@@ -96,8 +96,11 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
   const int num_pairs = gridDim.x >> 1;
   const int num_tiles = p.m_blocks * p.n_blocks;
   const int num_units = num_tiles * p.splits;     // unit u = (tile u / splits, K part u % splits)
-  auto kb_begin = [&](int unit) { return static_cast<int>(static_cast<int64_t>(p.k_blocks) * (unit % p.splits) / p.splits); };
-  auto kb_end = [&](int unit) { return static_cast<int>(static_cast<int64_t>(p.k_blocks) * (unit % p.splits + 1) / p.splits); };
+  // (the unsplit case takes no division: these run on single threads ahead of the first load and MMA)
+  auto tile_of = [&](int unit) { return p.splits == 1 ? unit : unit / p.splits; };
+  auto part_of = [&](int unit) { return p.splits == 1 ? 0 : unit % p.splits; };
+  auto kb_begin = [&](int unit) { return p.splits == 1 ? 0 : (p.k_blocks * part_of(unit)) / p.splits; };
+  auto kb_end = [&](int unit) { return p.splits == 1 ? p.k_blocks : (p.k_blocks * (part_of(unit) + 1)) / p.splits; };
   constexpr uint32_t kTmemCols = ACC_BUFS * BN;
 
   if (threadIdx.x == 0) {
@@ -140,7 +143,7 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
       // negative until the leader's expect_tx, which is allowed.)
       int pre = 0;
       if (pair_id < num_units) {
-        const int tile = pair_id / p.splits, kb0 = kb_begin(pair_id), nkb = kb_end(pair_id) - kb0;
+        const int tile = tile_of(pair_id), kb0 = kb_begin(pair_id), nkb = kb_end(pair_id) - kb0;
         pre = nkb < STAGES ? nkb : STAGES;
         const int n0 = (tile / p.m_blocks) * BN + static_cast<int>(rank) * (BN / 2);
         for (int j = 0; j < pre; ++j) {
@@ -150,7 +153,7 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
       }
       grid_dep_wait();
       if (pair_id < num_units) {
-        const int tile = pair_id / p.splits, kb0 = kb_begin(pair_id);
+        const int tile = tile_of(pair_id), kb0 = kb_begin(pair_id);
         const int m0 = (tile % p.m_blocks) * BM_PAIR + static_cast<int>(rank) * BM_CTA;
         for (int j = 0; j < pre; ++j)
           tma_load_2d_pair(smem_base + j * L::kStageBytes, &tm_q, full0 + j * 8, (kb0 + j) * BK, m0);
@@ -158,7 +161,7 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
       uint32_t it = static_cast<uint32_t>(pre);
       bool ok = true;
       for (int unit = pair_id; unit < num_units && ok; unit += num_pairs) {
-        const int tile = unit / p.splits;
+        const int tile = tile_of(unit);
         const int m0 = (tile % p.m_blocks) * BM_PAIR + static_cast<int>(rank) * BM_CTA;
         const int n0 = (tile / p.m_blocks) * BN + static_cast<int>(rank) * (BN / 2);
         const int kb1 = kb_end(unit);
@@ -217,7 +220,7 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     bool ok = true;
     volatile int* last_flag = reinterpret_cast<volatile int*>(smem + L::kMiscOff + 8);
     for (int unit = pair_id; unit < num_units && ok; unit += num_pairs, ++t) {
-      const int tile = unit / p.splits;
+      const int tile = tile_of(unit);
       const uint32_t b = t % ACC_BUFS;
       const int row0 = (tile % p.m_blocks) * BM_PAIR + static_cast<int>(rank) * BM_CTA + quad * 32;
       const int n0 = (tile / p.m_blocks) * BN + half * HC;
@@ -236,7 +239,7 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
       // Split-K: this CTA's slice of the tile's partials, one slot per K part.  The scratch is
       // private, so it is laid out for coalescing: [4-column piece][row] of 16-byte words -- a warp's
       // store of one piece covers 512 contiguous bytes.
-      const int sp = unit % p.splits;
+      const int sp = part_of(unit);
       const int64_t slot_elems = static_cast<int64_t>(BM_CTA) * BN;
       uint4* ws_tile = nullptr;
       if constexpr (!kExportAcc) {
@@ -484,7 +487,6 @@ int launch_gemm_w8a8_pair_with(const Scratch& sc, const int8_t* q, const float* 
   static const int variant = [] { const char* e = getenv("PQ_W8A8_PAIR_CFG"); return e ? atoi(e) : 0; }();
   if (use128) return launch_pair_cfg<128, 7, 2, 2, 8, 1, false>(tq, tw, ty, a, stream);
   if (variant == 1) return launch_pair_cfg<256, 6, 1, 2, 8, 1, false>(tq, tw, ty, a, stream);
-  if (variant == 2) return launch_pair_cfg<256, 3, 1, 1, 4, 2, false>(tq, tw, ty, a, stream);
   return launch_pair_cfg<256, 5, 2, 2, 8, 1, false>(tq, tw, ty, a, stream);
 }
 
