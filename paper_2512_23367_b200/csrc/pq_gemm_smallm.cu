@@ -78,6 +78,18 @@ __device__ __forceinline__ uint32_t ld_dsmem_u32(uint32_t local_addr, uint32_t r
   return v;
 }
 
+__device__ __forceinline__ uint4 ld_dsmem_v4(uint32_t local_addr, uint32_t rank) {
+  uint4 v;
+  asm volatile(
+      "{\n\t.reg .b32 ra;\n\t"
+      "mapa.shared::cluster.u32 ra, %4, %5;\n\t"
+      "ld.shared::cluster.v4.b32 {%0, %1, %2, %3}, [ra];\n\t}"
+      : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+      : "r"(local_addr), "r"(rank)
+      : "memory");
+  return v;
+}
+
 template <int MPAD>
 __device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t (&r)[MPAD]) {
   if constexpr (MPAD == 16) {
@@ -353,27 +365,58 @@ smallm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   __syncwarp();
   cluster_sync_all();
   if (do_reduce && warp >= 4) {
-    const int n_local = (warp & 3) * 32 + lane;
-    const int n = n0 + n_local;
+    // Thread t owns four consecutive output channels (one 16-byte word of every part's partial
+    // tile) for the rows m = rank + splits * (t / 32 + 4 i): the remote loads of all parts of a row
+    // are issued together, so a row costs one distributed-shared-memory round trip, not `splits`.
+    const int t = threadIdx.x - 128;
+    const int nq = t & 31, msub = t >> 5;
+    const int n = n0 + 4 * nq;
     const uint32_t my_rank = cluster_ctarank();
-    float sc = 0.0f;
-    if (!kW4 && !kExportAcc && n < p.N) sc = __ldg(p.s_ch + n);
-    for (int m = static_cast<int>(my_rank); m < p.M; m += p.splits) {
-      const uint32_t addr = smem_base + static_cast<uint32_t>(m * BW + n_local) * 4u;
+    float sc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    if (!kW4 && !kExportAcc && n < p.N) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) sc[j] = __ldg(p.s_ch + n + j);   // N is a multiple of 8: n < N covers n + 3
+    }
+    for (int m = static_cast<int>(my_rank) + p.splits * msub; m < p.M; m += 4 * p.splits) {
+      const uint32_t addr = smem_base + static_cast<uint32_t>(m * BW + 4 * nq) * 4u;
+      uint4 part[kMaxSplit];
+#pragma unroll
+      for (int r = 0; r < kMaxSplit; ++r) {
+        if (r < p.splits) part[r] = ld_dsmem_v4(addr, static_cast<uint32_t>(r));
+      }
+      if (n >= p.N) continue;
       if constexpr (kW4) {
-        float tot = 0.0f;
-        for (int r = 0; r < p.splits; ++r) tot += __uint_as_float(ld_dsmem_u32(addr, static_cast<uint32_t>(r)));
-        if (n < p.N) p.y[static_cast<int64_t>(m) * p.N + n] = __float2half_rn(tot * __ldg(p.s_tok + m));
-      } else {
-        int32_t tot = 0;
-        for (int r = 0; r < p.splits; ++r) tot += static_cast<int32_t>(ld_dsmem_u32(addr, static_cast<uint32_t>(r)));
-        if (n < p.N) {
-          if constexpr (kExportAcc) {
-            p.acc[static_cast<int64_t>(m) * p.N + n] = tot;
-          } else {
-            const float v = __fmul_rn(__fmul_rn(__int2float_rn(tot), __ldg(p.s_tok + m)), sc);
-            p.y[static_cast<int64_t>(m) * p.N + n] = __float2half_rn(v);
+        float tot[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+        for (int r = 0; r < kMaxSplit; ++r) {
+          if (r < p.splits) {
+            tot[0] += __uint_as_float(part[r].x); tot[1] += __uint_as_float(part[r].y);
+            tot[2] += __uint_as_float(part[r].z); tot[3] += __uint_as_float(part[r].w);
           }
+        }
+        const float st = __ldg(p.s_tok + m);
+        const __half2 h01 = __floats2half2_rn(tot[0] * st, tot[1] * st), h23 = __floats2half2_rn(tot[2] * st, tot[3] * st);
+        *reinterpret_cast<uint2*>(p.y + static_cast<int64_t>(m) * p.N + n) =
+            make_uint2(*reinterpret_cast<const uint32_t*>(&h01), *reinterpret_cast<const uint32_t*>(&h23));
+      } else {
+        int32_t tot[4] = {0, 0, 0, 0};
+#pragma unroll
+        for (int r = 0; r < kMaxSplit; ++r) {
+          if (r < p.splits) {
+            tot[0] += static_cast<int32_t>(part[r].x); tot[1] += static_cast<int32_t>(part[r].y);
+            tot[2] += static_cast<int32_t>(part[r].z); tot[3] += static_cast<int32_t>(part[r].w);
+          }
+        }
+        if constexpr (kExportAcc) {
+          *reinterpret_cast<int4*>(p.acc + static_cast<int64_t>(m) * p.N + n) = make_int4(tot[0], tot[1], tot[2], tot[3]);
+        } else {
+          const float st = __ldg(p.s_tok + m);
+          float v[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) v[j] = __fmul_rn(__fmul_rn(__int2float_rn(tot[j]), st), sc[j]);
+          const __half2 h01 = __floats2half2_rn(v[0], v[1]), h23 = __floats2half2_rn(v[2], v[3]);
+          *reinterpret_cast<uint2*>(p.y + static_cast<int64_t>(m) * p.N + n) =
+              make_uint2(*reinterpret_cast<const uint32_t*>(&h01), *reinterpret_cast<const uint32_t*>(&h23));
         }
       }
     }
