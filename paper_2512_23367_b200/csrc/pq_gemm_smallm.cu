@@ -66,18 +66,6 @@ struct SmallArgs {
   int k_blocks, splits;
 };
 
-__device__ __forceinline__ uint32_t ld_dsmem_u32(uint32_t local_addr, uint32_t rank) {
-  uint32_t v;
-  asm volatile(
-      "{\n\t.reg .b32 ra;\n\t"
-      "mapa.shared::cluster.u32 ra, %1, %2;\n\t"
-      "ld.shared::cluster.b32 %0, [ra];\n\t}"
-      : "=r"(v)
-      : "r"(local_addr), "r"(rank)
-      : "memory");
-  return v;
-}
-
 __device__ __forceinline__ uint4 ld_dsmem_v4(uint32_t local_addr, uint32_t rank) {
   uint4 v;
   asm volatile(
