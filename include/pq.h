@@ -141,6 +141,21 @@ PQ_API int pq_acc_w4a8(const int8_t* q, const void* wp, int32_t group, int64_t M
                 int32_t* acc_g, void* stream);
 
 /*
+ * Several W8A8 linears over the SAME quantized tokens (the q/k/v projections, or gate and up, of
+ * the layers the paper quantizes) as one call.  Result: exactly what `count` calls of pq_gemm_w8a8
+ * with (wq[g], s_ch[g], N[g], y_f16[g]) give, bit for bit.  For M > 128 the members' output tiles
+ * are scheduled together in a single kernel launch, which fills the SMs' waves across the members
+ * and pays the per-launch fixed cost once; other M run one launch per member.
+ *   count: 1..PQ_MAX_GROUP.  wq, s_ch, N, y_f16: HOST arrays of `count` entries (device pointers
+ *   and column counts; read during the call, not retained).  q, s_tok, M, K as in pq_gemm_w8a8.
+ *   The outputs must not overlap each other.  On an argument error nothing is launched.
+ */
+#define PQ_MAX_GROUP 4
+PQ_API int pq_gemm_w8a8_group(const int8_t* q, const float* s_tok, int32_t count, const void* const* wq,
+                              const float* const* s_ch, const int64_t* N, void* const* y_f16, int64_t M,
+                              int64_t K, void* stream);
+
+/*
  * Optional scratch memory for the current device.  With few output tiles and a long K (e.g. a
  * 7B-class layer at M = 512) the W8A8 GEMM cuts K into parts that run on different SMs; the parts'
  * INT32 partial accumulators pass through this scratch and are summed exactly, so results do not

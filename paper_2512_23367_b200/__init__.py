@@ -15,6 +15,7 @@ from .binding import (  # noqa: F401
     pq_device_status,
     pq_gemm_w4a8,
     pq_gemm_w8a8,
+    pq_gemm_w8a8_group,
     pq_gemm_w8a8_noalloc,
     pq_pack_w4,
     pq_pack_w8,

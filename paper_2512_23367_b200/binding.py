@@ -34,7 +34,10 @@ SIGNATURES = {
     "pq_set_workspace": (ctypes.c_int, [_vp, ctypes.c_size_t, _vp]),
     "pq_plan_w8a8": (ctypes.c_int, [_i64, _i64, _i64, _i32, ctypes.c_size_t, ctypes.POINTER(_i32), ctypes.POINTER(_i32)]),
     "pq_gemm_w8a8_noalloc": (ctypes.c_int, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _vp, _vp]),
+    "pq_gemm_w8a8_group": (ctypes.c_int, [_vp, _vp, _i32, ctypes.POINTER(_vp), ctypes.POINTER(_vp),
+                                          ctypes.POINTER(_i64), ctypes.POINTER(_vp), _i64, _i64, _vp]),
 }
+MAX_GROUP = 4
 
 
 class PQError(RuntimeError):
@@ -170,6 +173,30 @@ def pq_gemm_w8a8(q, s_tok, wq, s_ch, N: int, y: torch.Tensor | None = None) -> t
     _check("pq_gemm_w8a8", lib().pq_gemm_w8a8(q.data_ptr(), s_tok.data_ptr(), wq.data_ptr(), s_ch.data_ptr(),
                                               M, N, K, y.data_ptr(), _stream()))
     return y
+
+
+def pq_gemm_w8a8_group(q, s_tok, members, ys=None) -> list[torch.Tensor]:
+    """Several W8A8 linears over the same quantized tokens as one call (one kernel launch when
+    M > 128).  members: sequence of (wq, s_ch, N) from pq_pack_w8; ys: optional outputs f16 [M,N_g].
+    Returns the outputs; each equals pq_gemm_w8a8(q, s_tok, wq, s_ch, N) bit for bit."""
+    q = _dev(q, torch.int8, "q")
+    _ensure_workspace(q.device)
+    M, K = q.shape
+    _dev(s_tok, torch.float32, "s_tok")
+    n = len(members)
+    if ys is None:
+        ys = [torch.empty((M, int(N)), dtype=torch.float16, device=q.device) for (_, _, N) in members]
+    if len(ys) != n:
+        raise ValueError("one output per member")
+    for (wq, s_ch, _), y in zip(members, ys):
+        _dev(wq, torch.uint8, "wq"), _dev(s_ch, torch.float32, "s_ch"), _dev(y, torch.float16, "y")
+    wq_arr = (_vp * max(n, 1))(*[m[0].data_ptr() for m in members])
+    sc_arr = (_vp * max(n, 1))(*[m[1].data_ptr() for m in members])
+    n_arr = (_i64 * max(n, 1))(*[int(m[2]) for m in members])
+    y_arr = (_vp * max(n, 1))(*[y.data_ptr() for y in ys])
+    _check("pq_gemm_w8a8_group", lib().pq_gemm_w8a8_group(q.data_ptr(), s_tok.data_ptr(), n, wq_arr, sc_arr, n_arr,
+                                                          y_arr, M, K, _stream()))
+    return list(ys)
 
 
 def pq_gemm_w8a8_noalloc(q, s_tok, wq, s_ch, N: int, y: torch.Tensor) -> torch.Tensor:

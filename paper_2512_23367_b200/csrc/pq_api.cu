@@ -227,6 +227,32 @@ int pq_gemm_w8a8(const int8_t* q, const float* s_tok, const void* wq, const floa
   return gemm_w8a8_common(q, s_tok, wq, s_ch, M, N, K, y_f16, nullptr, stream);
 }
 
+int pq_gemm_w8a8_group(const int8_t* q, const float* s_tok, int32_t count, const void* const* wq,
+                       const float* const* s_ch, const int64_t* N, void* const* y_f16, int64_t M, int64_t K,
+                       void* stream) {
+  if (!q || !s_tok || !wq || !s_ch || !N || !y_f16) return PQ_ERR_NULL;
+  if (count < 1 || count > PQ_MAX_GROUP) return PQ_ERR_SHAPE;
+  for (int g = 0; g < count; ++g) {
+    if (!wq[g] || !s_ch[g] || !y_f16[g]) return PQ_ERR_NULL;
+    const int rc = check_gemm(M, N[g], K);
+    if (rc != PQ_OK) return rc;
+    if (!aligned16(wq[g]) || !aligned16(y_f16[g])) return PQ_ERR_ALIGN;
+  }
+  if (!aligned16(q)) return PQ_ERR_ALIGN;
+  int rc = check_arch();
+  if (rc != PQ_OK) return rc;
+  if (M <= 128 || count == 1) {
+    // Token counts whose schedules do not group (they reduce inside the SMs): one launch per member.
+    for (int g = 0; g < count; ++g) {
+      rc = gemm_w8a8_common(q, s_tok, wq[g], s_ch[g], M, N[g], K, y_f16[g], nullptr, stream);
+      if (rc != PQ_OK) return rc;
+    }
+    return PQ_OK;
+  }
+  return launch_gemm_w8a8_pair_group(scratch(), q, s_tok, count, wq, s_ch, N, y_f16, M, K, nullptr,
+                                     static_cast<cudaStream_t>(stream));
+}
+
 int pq_acc_w8a8(const int8_t* q, const void* wq, int64_t M, int64_t N, int64_t K, int32_t* acc, void* stream) {
   if (!q || !wq || !acc) return PQ_ERR_NULL;
   return gemm_w8a8_common(q, nullptr, wq, nullptr, M, N, K, nullptr, acc, stream);

@@ -16,14 +16,14 @@
 //               store drains (full 64-byte row segments; ragged edges are clipped by the tensor
 //               map).  The accumulator is handed back to the MMA issuer as soon as its last
 //               column block is in registers.
-// Two ways to overlap a tile's epilogue with the next tile's main loop are compiled:
-//   "wide":  one CTA per SM, two TMEM accumulators, deep stage ring, eight epilogue warps;
-//   "light": two co-resident CTAs per SM, each with one accumulator, a three-stage ring and four
-//            epilogue warps -- while one CTA drains its accumulator the other one multiplies, and
-//            a successor kernel launched with programmatic stream serialization finds room to
-//            set up and prefetch its weights while this kernel's last tiles finish.
+// One CTA per SM with two TMEM accumulators: a tile's epilogue overlaps the next tile's main loop.
 // The weight tiles of a CTA's first ring pass are requested BEFORE the wait on the preceding
 // kernel (weights are constants of the model); everything else comes after it.
+//
+// Grouped launch: up to kMaxGroup linears that share the token codes (q/k/v, gate/up) run as ONE
+// launch.  Their column blocks are concatenated into one tile list, so the persistent scheduler
+// fills its waves across the members and the per-launch fixed cost is paid once; every member
+// keeps its own weights, channel scales and output tensor.
 //
 // Split-K (few tiles, long K -- e.g. M = 512): a work unit is (tile, K part).  Every unit writes
 // its INT32 partial accumulator to global scratch, fences, and bumps the tile's arrival counter;
@@ -48,15 +48,48 @@ constexpr int kOutBoxBytes = 32 * 32 * 2;   // one staged store: 32 rows x 32 FP
 
 struct PairArgs {
   const float* s_tok;
-  const float* s_ch;
+  const float* s_ch[kMaxGroup];   // per member
+  int N[kMaxGroup];               // per member
+  int nb_end[kMaxGroup];          // column blocks of members 0..g (running total); INT_MAX past the last member
+  int count;                      // members in this launch
   int32_t* acc;
   int* status;
   int32_t* ws;              // split-K partial accumulators (global scratch), or nullptr
   unsigned int* counters;   // split-K arrival counters, one per (tile, CTA of the pair); zero between calls
-  int M, N, K;
-  int m_blocks, n_blocks, k_blocks;
+  int M, K;
+  int m_blocks, n_blocks, k_blocks;   // n_blocks: over all members
   int splits;               // K is cut into this many parts; 1 = no split
 };
+
+// Tensor maps of the members' weights and outputs (kernel parameter, indexed by member).
+struct PairMaps {
+  CUtensorMap w[kMaxGroup];
+  CUtensorMap y[kMaxGroup];
+};
+
+// Where a tile lies: its member, the member's column count and channel scales, its first column.
+struct TilePos {
+  int g, m_blk, n0, N;
+  const float* s_ch;
+};
+template <int BN>
+__device__ __forceinline__ TilePos locate_tile(const PairArgs& p, int tile) {
+  TilePos t;
+  int nblk = tile / p.m_blocks;
+  t.m_blk = tile - nblk * p.m_blocks;
+  t.g = 0;
+  t.N = p.N[0];
+  t.s_ch = p.s_ch[0];
+  if (p.count > 1) {
+    // (constant indices: the argument struct stays in the parameter bank)
+    const int e0 = p.nb_end[0], e1 = p.nb_end[1], e2 = p.nb_end[2];
+    if (nblk >= e2) { t.g = 3; t.N = p.N[3]; t.s_ch = p.s_ch[3]; nblk -= e2; }
+    else if (nblk >= e1) { t.g = 2; t.N = p.N[2]; t.s_ch = p.s_ch[2]; nblk -= e1; }
+    else if (nblk >= e0) { t.g = 1; t.N = p.N[1]; t.s_ch = p.s_ch[1]; nblk -= e0; }
+  }
+  t.n0 = nblk * BN;
+  return t;
+}
 
 template <int BN, int STAGES, int EPI_BUFS, int EPI_WARPS>
 struct PairSmem {
@@ -74,8 +107,8 @@ struct PairSmem {
 
 template <int BN, int STAGES, int EPI_BUFS, int ACC_BUFS, int EPI_WARPS, int MIN_CTAS, bool kExportAcc>
 __global__ void __launch_bounds__(64 + 32 * EPI_WARPS, MIN_CTAS)
-gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_w,
-                      const __grid_constant__ CUtensorMap tm_y, const PairArgs p) {
+gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ PairMaps maps,
+                      const PairArgs p) {
   using L = PairSmem<BN, STAGES, EPI_BUFS, EPI_WARPS>;
   static_assert(EPI_WARPS == 4 || EPI_WARPS == 8 || EPI_WARPS == 16, "one, two or four epilogue warps per lane quadrant");
   extern __shared__ uint8_t smem_raw[];
@@ -117,8 +150,10 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
   }
   if (warp == 0 && lane == 0) {
     tma_prefetch_desc(&tm_q);
-    tma_prefetch_desc(&tm_w);
-    if constexpr (!kExportAcc) tma_prefetch_desc(&tm_y);
+    for (int g = 0; g < p.count; ++g) {
+      tma_prefetch_desc(&maps.w[g]);
+      if constexpr (!kExportAcc) tma_prefetch_desc(&maps.y[g]);
+    }
   }
   if (warp == 1) {
     tmem_alloc_pair(smem_u32(tmem_slot), kTmemCols);
@@ -143,12 +178,13 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
       // negative until the leader's expect_tx, which is allowed.)
       int pre = 0;
       if (pair_id < num_units) {
-        const int tile = tile_of(pair_id), kb0 = kb_begin(pair_id), nkb = kb_end(pair_id) - kb0;
+        const int kb0 = kb_begin(pair_id), nkb = kb_end(pair_id) - kb0;
         pre = nkb < STAGES ? nkb : STAGES;
-        const int n0 = (tile / p.m_blocks) * BN + static_cast<int>(rank) * (BN / 2);
+        const TilePos tp = locate_tile<BN>(p, tile_of(pair_id));
+        const int n0 = tp.n0 + static_cast<int>(rank) * (BN / 2);
         for (int j = 0; j < pre; ++j) {
           if (rank == 0) mbar_arrive_expect_tx(bar_full + j * 8, 2 * L::kStageBytes);
-          tma_load_2d_pair(smem_base + j * L::kStageBytes + L::kABytes, &tm_w, full0 + j * 8, (kb0 + j) * BK, n0);
+          tma_load_2d_pair(smem_base + j * L::kStageBytes + L::kABytes, &maps.w[tp.g], full0 + j * 8, (kb0 + j) * BK, n0);
         }
       }
       grid_dep_wait();
@@ -161,9 +197,10 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
       uint32_t it = static_cast<uint32_t>(pre);
       bool ok = true;
       for (int unit = pair_id; unit < num_units && ok; unit += num_pairs) {
-        const int tile = tile_of(unit);
-        const int m0 = (tile % p.m_blocks) * BM_PAIR + static_cast<int>(rank) * BM_CTA;
-        const int n0 = (tile / p.m_blocks) * BN + static_cast<int>(rank) * (BN / 2);
+        const TilePos tp = locate_tile<BN>(p, tile_of(unit));
+        const int m0 = tp.m_blk * BM_PAIR + static_cast<int>(rank) * BM_CTA;
+        const int n0 = tp.n0 + static_cast<int>(rank) * (BN / 2);
+        const CUtensorMap* tm_w = &maps.w[tp.g];
         const int kb1 = kb_end(unit);
         for (int kb = kb_begin(unit) + (unit == pair_id ? pre : 0); kb < kb1; ++kb, ++it) {
           const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
@@ -171,7 +208,7 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
           const uint32_t dst = smem_base + s * L::kStageBytes;
           if (rank == 0) mbar_arrive_expect_tx(bar_full + s * 8, 2 * L::kStageBytes);
           tma_load_2d_pair(dst, &tm_q, full0 + s * 8, kb * BK, m0);
-          tma_load_2d_pair(dst + L::kABytes, &tm_w, full0 + s * 8, kb * BK, n0);
+          tma_load_2d_pair(dst + L::kABytes, tm_w, full0 + s * 8, kb * BK, n0);
         }
       }
       (void)ok;
@@ -221,14 +258,15 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     volatile int* last_flag = reinterpret_cast<volatile int*>(smem + L::kMiscOff + 8);
     for (int unit = pair_id; unit < num_units && ok; unit += num_pairs, ++t) {
       const int tile = tile_of(unit);
+      const TilePos tp = locate_tile<BN>(p, tile);
       const uint32_t b = t % ACC_BUFS;
-      const int row0 = (tile % p.m_blocks) * BM_PAIR + static_cast<int>(rank) * BM_CTA + quad * 32;
-      const int n0 = (tile / p.m_blocks) * BN + half * HC;
+      const int row0 = tp.m_blk * BM_PAIR + static_cast<int>(rank) * BM_CTA + quad * 32;
+      const int n0 = tp.n0 + half * HC;
       const int row = row0 + lane;
       float st = 0.0f;
       if constexpr (!kExportAcc) {
         __syncwarp();
-        for (int c = lane; c < HC; c += 32) sc_warp[c] = (n0 + c < p.N) ? __ldg(p.s_ch + n0 + c) : 0.0f;
+        for (int c = lane; c < HC; c += 32) sc_warp[c] = (n0 + c < tp.N) ? __ldg(tp.s_ch + n0 + c) : 0.0f;
         if (row < p.M) st = __ldg(p.s_tok + row);
         __syncwarp();
       }
@@ -310,10 +348,10 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         }
         if constexpr (kExportAcc) {
           if (row < p.M) {
-            int32_t* dst = p.acc + static_cast<int64_t>(row) * p.N + col0;
+            int32_t* dst = p.acc + static_cast<int64_t>(row) * tp.N + col0;   // export: single member
 #pragma unroll
             for (int j = 0; j < 32; j += 4) {
-              if (col0 + j < p.N) *reinterpret_cast<uint4*>(dst + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+              if (col0 + j < tp.N) *reinterpret_cast<uint4*>(dst + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
             }
           }
         } else {
@@ -338,7 +376,7 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
           fence_proxy_async_smem();
           __syncwarp();
           if (lane == 0) {
-            if (col0 < p.N && row0 < p.M) tma_store_2d(&tm_y, out_warp_u32 + buf * kOutBoxBytes, col0, row0);
+            if (col0 < tp.N && row0 < p.M) tma_store_2d(&maps.y[tp.g], out_warp_u32 + buf * kOutBoxBytes, col0, row0);
             tma_store_commit();  // also when nothing was stored: keeps one group per buffer use
           }
           ++nstore;
@@ -366,8 +404,7 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
 }
 
 template <int BN, int STAGES, int EPI_BUFS, int ACC_BUFS, int EPI_WARPS, int MIN_CTAS, bool kExportAcc>
-int launch_pair_cfg(const CUtensorMap& tq, const CUtensorMap& tw, const CUtensorMap& ty, const PairArgs& a,
-                    cudaStream_t stream) {
+int launch_pair_cfg(const CUtensorMap& tq, const PairMaps& maps, const PairArgs& a, cudaStream_t stream) {
   using L = PairSmem<BN, STAGES, EPI_BUFS, EPI_WARPS>;
   static_assert(MIN_CTAS * (L::kDynamic + 1024) <= 233472, "co-resident CTAs exceed the SM's shared memory");
   static_assert(MIN_CTAS * ACC_BUFS * BN <= 512, "co-resident CTAs exceed the SM's tensor memory");
@@ -395,7 +432,7 @@ int launch_pair_cfg(const CUtensorMap& tq, const CUtensorMap& tw, const CUtensor
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = pdl_enabled() ? 2 : 1;
-  return cuda_status(cudaLaunchKernelEx(&cfg, kern, tq, tw, ty, a));
+  return cuda_status(cudaLaunchKernelEx(&cfg, kern, tq, maps, a));
 }
 
 }  // namespace
@@ -406,18 +443,23 @@ int launch_pair_cfg(const CUtensorMap& tq, const CUtensorMap& tw, const CUtensor
 // Cycles per K block are measured figures: 512 for a 256-wide tile (the tensor-pipe time), 550
 // for a 128-wide one (bound by the bytes each SM pulls per multiply-add, not faster per block).
 // `scratch_bytes` = room for split-K partials (0: never split); force_* = 0 means "free choice".
+// The members' column counts are N[0..count); a launch of one linear has count = 1.
 // Returns the cost of the chosen plan, or -1 if the forced values admit none.
-int64_t plan_w8a8_pair(int64_t M, int64_t N, int64_t K, int sms, size_t scratch_bytes, int force_bn,
-                       int force_splits, int* bn_out, int* splits_out) {
+int64_t plan_w8a8_pair_group(int64_t M, const int64_t* N, int count, int64_t K, int sms, size_t scratch_bytes,
+                             int force_bn, int force_splits, int* bn_out, int* splits_out) {
   const int pairs = sms / 2 > 0 ? sms / 2 : 1;
   const int64_t mb = (M + BM_PAIR - 1) / BM_PAIR;
   const int64_t kblocks = (K + BK - 1) / BK;
   auto waves = [pairs](int64_t units) { return (units + pairs - 1) / pairs; };
+  int64_t n_max = 0;
+  for (int g = 0; g < count; ++g) n_max = N[g] > n_max ? N[g] : n_max;
   int64_t best_cost = -1;
   for (int bn = 256; bn >= 128; bn /= 2) {
     if (force_bn != 0 && bn != force_bn) continue;
-    if (bn == 256 && N <= 128 && force_bn == 0) continue;
-    const int64_t tiles = mb * ((N + bn - 1) / bn);
+    if (bn == 256 && n_max <= 128 && force_bn == 0) continue;
+    int64_t nb = 0;
+    for (int g = 0; g < count; ++g) nb += (N[g] + bn - 1) / bn;
+    const int64_t tiles = mb * nb;
     for (int sp = 1; sp <= 4; ++sp) {
       if (force_splits != 0 && sp != force_splits) continue;
       if (sp > 1) {
@@ -438,56 +480,79 @@ int64_t plan_w8a8_pair(int64_t M, int64_t N, int64_t K, int sms, size_t scratch_
   return best_cost;
 }
 
-int launch_gemm_w8a8_pair_with(const Scratch& sc, const int8_t* q, const float* s_tok, const void* wq,
-                               const float* s_ch, int64_t M, int64_t N, int64_t K, void* y, int32_t* acc,
-                               cudaStream_t stream) {
+int64_t plan_w8a8_pair(int64_t M, int64_t N, int64_t K, int sms, size_t scratch_bytes, int force_bn,
+                       int force_splits, int* bn_out, int* splits_out) {
+  return plan_w8a8_pair_group(M, &N, 1, K, sms, scratch_bytes, force_bn, force_splits, bn_out, splits_out);
+}
+
+int launch_gemm_w8a8_pair_group(const Scratch& sc, const int8_t* q, const float* s_tok, int count,
+                                const void* const* wq, const float* const* s_ch, const int64_t* N, void* const* y,
+                                int64_t M, int64_t K, int32_t* acc, cudaStream_t stream) {
+  if (count < 1 || count > kMaxGroup || (acc != nullptr && count != 1)) return PQ_ERR_SHAPE;
   const int64_t mb = (M + BM_PAIR - 1) / BM_PAIR;
   const int64_t kblocks = (K + BK - 1) / BK;
   const int force_bn = [] { const char* e = getenv("PQ_W8A8_BN"); return e ? (e[0] == '1' ? 128 : (e[0] == '2' ? 256 : 0)) : 0; }();
   const int force_splits = [] { const char* e = getenv("PQ_W8A8_SPLITS"); return e ? atoi(e) : 0; }();
   int best_bn = 256, best_splits = 1;
-  const int64_t best_cost = plan_w8a8_pair(M, N, K, sm_count(), acc == nullptr && sc.partials != nullptr ? sc.partial_bytes : 0,
-                                           force_bn, force_splits, &best_bn, &best_splits);
+  const int64_t best_cost =
+      plan_w8a8_pair_group(M, N, count, K, sm_count(), acc == nullptr && sc.partials != nullptr ? sc.partial_bytes : 0,
+                           force_bn, force_splits, &best_bn, &best_splits);
   if (best_cost < 0) return PQ_ERR_SHAPE;   // only reachable through contradictory ablation knobs
   const bool use128 = best_bn == 128;
   const int BN = best_bn;
 
-  CUtensorMap tq, tw, ty;
+  CUtensorMap tq;
+  PairMaps maps;
   int rc = make_tmap_2d(&tq, q, static_cast<uint64_t>(M), static_cast<uint64_t>(K), BM_CTA, BK, 1, 128);
   if (rc != PQ_OK) return rc;
-  rc = make_tmap_2d(&tw, wq, static_cast<uint64_t>(N), static_cast<uint64_t>(K), static_cast<uint32_t>(BN / 2), BK, 1, 128);
-  if (rc != PQ_OK) return rc;
-  if (y != nullptr) {
-    // FP16 result [M, N]; stores go out as 32 x 32 boxes staged with the 64-byte swizzle.
-    rc = make_tmap_2d(&ty, y, static_cast<uint64_t>(M), static_cast<uint64_t>(N), 32, 32, 2, 64);
-    if (rc != PQ_OK) return rc;
-  } else {
-    ty = tq;  // the accumulator export stores directly; the map is not used
-  }
-
   PairArgs a;
+  int64_t nb_total = 0;
+  for (int g = 0; g < kMaxGroup; ++g) {
+    const int src = g < count ? g : 0;   // unused slots repeat member 0 (never selected)
+    rc = make_tmap_2d(&maps.w[g], wq[src], static_cast<uint64_t>(N[src]), static_cast<uint64_t>(K),
+                      static_cast<uint32_t>(BN / 2), BK, 1, 128);
+    if (rc != PQ_OK) return rc;
+    if (acc == nullptr) {
+      // FP16 result [M, N]; stores go out as 32 x 32 boxes staged with the 64-byte swizzle.
+      rc = make_tmap_2d(&maps.y[g], y[src], static_cast<uint64_t>(M), static_cast<uint64_t>(N[src]), 32, 32, 2, 64);
+      if (rc != PQ_OK) return rc;
+    } else {
+      maps.y[g] = tq;  // the accumulator export stores directly; the map is not used
+    }
+    a.s_ch[g] = s_ch[src];
+    a.N[g] = static_cast<int>(N[src]);
+    if (g < count) nb_total += (N[g] + BN - 1) / BN;
+    a.nb_end[g] = g < count ? static_cast<int>(nb_total) : 0x7fffffff;
+  }
+  if (mb * nb_total > 0x3fffffff) return PQ_ERR_SHAPE;
+
+  a.count = count;
   a.s_tok = s_tok;
-  a.s_ch = s_ch;
   a.acc = acc;
   a.status = device_status_ptr();
   if (a.status == nullptr) return PQ_ERR_CUDA;
   a.M = static_cast<int>(M);
-  a.N = static_cast<int>(N);
   a.K = static_cast<int>(K);
   a.m_blocks = static_cast<int>(mb);
-  a.n_blocks = static_cast<int>((N + BN - 1) / BN);
+  a.n_blocks = static_cast<int>(nb_total);
   a.k_blocks = static_cast<int>(kblocks);
   a.splits = best_splits;
   a.ws = best_splits > 1 ? sc.partials : nullptr;
   a.counters = best_splits > 1 ? sc.counters : nullptr;
   if (acc != nullptr) {
-    return use128 ? launch_pair_cfg<128, 7, 2, 2, 8, 1, true>(tq, tw, ty, a, stream)
-                  : launch_pair_cfg<256, 5, 2, 2, 8, 1, true>(tq, tw, ty, a, stream);
+    return use128 ? launch_pair_cfg<128, 7, 2, 2, 8, 1, true>(tq, maps, a, stream)
+                  : launch_pair_cfg<256, 5, 2, 2, 8, 1, true>(tq, maps, a, stream);
   }
   static const int variant = [] { const char* e = getenv("PQ_W8A8_PAIR_CFG"); return e ? atoi(e) : 0; }();
-  if (use128) return launch_pair_cfg<128, 7, 2, 2, 8, 1, false>(tq, tw, ty, a, stream);
-  if (variant == 1) return launch_pair_cfg<256, 6, 1, 2, 8, 1, false>(tq, tw, ty, a, stream);
-  return launch_pair_cfg<256, 5, 2, 2, 8, 1, false>(tq, tw, ty, a, stream);
+  if (use128) return launch_pair_cfg<128, 7, 2, 2, 8, 1, false>(tq, maps, a, stream);
+  if (variant == 1) return launch_pair_cfg<256, 6, 1, 2, 8, 1, false>(tq, maps, a, stream);
+  return launch_pair_cfg<256, 5, 2, 2, 8, 1, false>(tq, maps, a, stream);
+}
+
+int launch_gemm_w8a8_pair_with(const Scratch& sc, const int8_t* q, const float* s_tok, const void* wq,
+                               const float* s_ch, int64_t M, int64_t N, int64_t K, void* y, int32_t* acc,
+                               cudaStream_t stream) {
+  return launch_gemm_w8a8_pair_group(sc, q, s_tok, 1, &wq, &s_ch, &N, &y, M, K, acc, stream);
 }
 
 int launch_gemm_w8a8_pair(const int8_t* q, const float* s_tok, const void* wq, const float* s_ch, int64_t M,

@@ -48,6 +48,8 @@ int launch_gemm_w8a8(const int8_t* q, const float* s_tok, const void* wq, const 
 // Same contract on CTA pairs (cta_group::2, 256-row tiles); preferred when M > 128.
 int launch_gemm_w8a8_pair(const int8_t* q, const float* s_tok, const void* wq, const float* s_ch, int64_t M,
                           int64_t N, int64_t K, void* y, int32_t* acc, cudaStream_t stream);
+// Linears that share the token codes and run as one launch of the pair GEMM: at most this many.
+constexpr int kMaxGroup = 4;
 // Host-only: the pair GEMM's choice of tile width and number of K parts (see the definition).
 int64_t plan_w8a8_pair(int64_t M, int64_t N, int64_t K, int sms, size_t scratch_bytes, int force_bn,
                        int force_splits, int* bn_out, int* splits_out);
@@ -55,6 +57,13 @@ int64_t plan_w8a8_pair(int64_t M, int64_t N, int64_t K, int sms, size_t scratch_
 int launch_gemm_w8a8_pair_with(const Scratch& sc, const int8_t* q, const float* s_tok, const void* wq,
                                const float* s_ch, int64_t M, int64_t N, int64_t K, void* y, int32_t* acc,
                                cudaStream_t stream);
+// `count` (1..kMaxGroup) linears over the same codes in one launch; arrays are host arrays of
+// device pointers / column counts.  acc (accumulator export) only with count == 1.
+int64_t plan_w8a8_pair_group(int64_t M, const int64_t* N, int count, int64_t K, int sms, size_t scratch_bytes,
+                             int force_bn, int force_splits, int* bn_out, int* splits_out);
+int launch_gemm_w8a8_pair_group(const Scratch& sc, const int8_t* q, const float* s_tok, int count,
+                                const void* const* wq, const float* const* s_ch, const int64_t* N, void* const* y,
+                                int64_t M, int64_t K, int32_t* acc, cudaStream_t stream);
 // Prefill-shaped W4A8 GEMM.  Exactly one of y / acc_g is non-null.
 int launch_gemm_w4a8(const int8_t* q, const float* s_tok, const void* wp, const void* s_grp, int64_t M,
                      int64_t N, int64_t K, void* y, int32_t* acc_g, cudaStream_t stream);

@@ -1,0 +1,80 @@
+"""pq_gemm_w8a8_group: several W8A8 linears over the same quantized tokens in one call.
+
+The contract is "exactly what one pq_gemm_w8a8 call per member gives", so every case checks bit
+equality with those calls, and parity with the CPU oracle (INT32 accumulators are exact, the FP16
+result within the tolerance of the other W8A8 tests) independently of them.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2512_23367_b200 as pq
+from paper_2512_23367_b200 import synth
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+REL, ABS = 2.0 ** -10, 1e-3
+
+
+def _members(K, Ns, seed):
+    ws = [synth.weights(N, K, seed + 1 + i) for i, N in enumerate(Ns)]
+    packed = [pq.pq_pack_w8(torch.from_numpy(w).to(DEV)) for w in ws]
+    return ws, [(wq, s_ch, N) for (wq, s_ch), N in zip(packed, Ns)]
+
+
+# q/k/v-like (equal widths), gate/up-like, ragged widths that end inside a tile, one member wider
+# than the others, four members, M with a ragged last row block, K long enough to split
+@pytest.mark.parametrize("M,K,Ns", [
+    (512, 512, (512, 512, 512)),
+    (300, 256, (520, 264)),
+    (257, 384, (1000, 136, 8)),
+    (2048, 512, (2048, 2048, 2048)),
+    (600, 1024, (256, 768, 264, 128)),
+    (512, 8192, (264, 520)),
+    (129, 128, (16, 24)),
+])
+def test_group_equals_one_call_per_member_and_the_oracle(M, K, Ns):
+    x = synth.activations(M, K, 4000 + M)
+    ws, members = _members(K, Ns, 4100 + M)
+    q, s_tok = pq.pq_quantize_act(torch.from_numpy(x).to(DEV))
+    pad = 512
+    bufs = [torch.full((pad + M * N + pad,), 5.0, dtype=torch.float16, device=DEV) for N in Ns]
+    ys = [b[pad:pad + M * N].view(M, N) for b, N in zip(bufs, Ns)]
+    out = pq.pq_gemm_w8a8_group(q, s_tok, members, ys)
+    torch.cuda.synchronize()
+    assert pq.pq_device_status() == 0
+    qo, so = oracle.quantize_act(x)
+    assert np.array_equal(q.cpu().numpy(), qo)
+    for (wq, s_ch, N), w, y, b in zip(members, ws, out, bufs):
+        single = pq.pq_gemm_w8a8(q, s_tok, wq, s_ch, N)
+        assert torch.equal(y, single)
+        wqo, sco = oracle.pack_w8(w)
+        _, ref = oracle.gemm_w8a8(qo, so, wqo, sco, want_acc=False)
+        g, ref = y.cpu().numpy().astype(np.float64), ref.astype(np.float64)
+        assert np.all(np.abs(g - ref) <= REL * np.abs(ref) + ABS)
+        assert (b[:pad] == 5.0).all() and (b[pad + M * N:] == 5.0).all()   # nothing outside the member's output
+
+
+@pytest.mark.parametrize("M", [1, 16, 64, 100])
+def test_small_token_counts_run_member_by_member_with_the_same_result(M):
+    K, Ns = 512, (256, 520)
+    x = synth.activations(M, K, 4300 + M)
+    _, members = _members(K, Ns, 4400 + M)
+    q, s_tok = pq.pq_quantize_act(torch.from_numpy(x).to(DEV))
+    out = pq.pq_gemm_w8a8_group(q, s_tok, members)
+    for (wq, s_ch, N), y in zip(members, out):
+        assert torch.equal(y, pq.pq_gemm_w8a8(q, s_tok, wq, s_ch, N))
+
+
+def test_two_group_calls_in_a_row_leave_the_split_k_scratch_clean():
+    M, K, Ns = 512, 11008, (512, 512)
+    x = synth.activations(M, K, 4500)
+    _, members = _members(K, Ns, 4501)
+    q, s_tok = pq.pq_quantize_act(torch.from_numpy(x).to(DEV))
+    first = [y.clone() for y in pq.pq_gemm_w8a8_group(q, s_tok, members)]
+    second = pq.pq_gemm_w8a8_group(q, s_tok, members)
+    for a, b, (wq, s_ch, N) in zip(first, second, members):
+        assert torch.equal(a, b)
+        assert torch.equal(a, pq.pq_gemm_w8a8(q, s_tok, wq, s_ch, N))
+    assert pq.pq_device_status() == 0
