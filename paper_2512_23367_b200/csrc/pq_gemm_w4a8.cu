@@ -202,8 +202,7 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         const uint64_t w_desc = umma_desc_k_sw128(smem_base + kW8Off + s * kW8Bytes);   // 256 channel rows (both CTAs)
         const uint64_t q_desc = umma_desc_k_sw128(smem_base + s * kStageBytes);         // 256 token rows (both CTAs)
         const uint32_t d_tmem = tmem_base + a * BT_PAIR;
-        if (!mbar_wait_cluster(bar_w8_full + s * 8, ph, abort_flag) ||
-            !mbar_wait_cluster(bar_acc_empty + a * 8, aph ^ 1u, abort_flag)) break;
+        if (!mbar_wait2_cluster(bar_w8_full + s * 8, ph, bar_acc_empty + a * 8, aph ^ 1u, abort_flag)) break;
         tc_fence_after_sync();
         umma_i8_pair_imm<0>(d_tmem, w_desc, q_desc, idesc);
         umma_i8_pair_imm<1>(d_tmem, w_desc + 2, q_desc + 2, idesc);
@@ -225,9 +224,9 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     for (uint32_t it = s; it < static_cast<uint32_t>(total); it += kUnpackWarps) {
       const uint32_t ph = (it / STAGES) & 1u;
       const uint32_t v = it % SC_SLOTS, vph = (it / SC_SLOTS) & 1u;
-      bool w = mbar_wait(bar_full + s * 8, ph, abort_flag);
-      w = w && mbar_wait(bar_empty + s * 8, ph ^ 1u, abort_flag);       // the slot's previous MMAs are done
-      w = w && mbar_wait(bar_sc_empty + v * 8, vph ^ 1u, abort_flag);
+      // stage landed; the slot's previous MMAs are done; the scale row has been read
+      const bool w = mbar_wait3(bar_full + s * 8, ph, bar_empty + s * 8, ph ^ 1u, bar_sc_empty + v * 8, vph ^ 1u,
+                                abort_flag);
       if (!__all_sync(0xffffffffu, w)) break;
 #pragma unroll 4
       for (int i = 0; i < (BC_CTA * 4) / 32; ++i) {
@@ -274,6 +273,9 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     const uint32_t out_warp_u32 = smem_base + kOutOff + pw * (kOutBufs * kOutBoxBytes);
     uint32_t it = 0, nstore = 0;
     bool ok = true;
+    const float* sc_rows = reinterpret_cast<const float*>(smem + kScOff);
+    bool have_next = false;
+    float sg_next = 0.0f;
     for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs) {
       const int tok0 = (tile % p.m_blocks) * BT_PAIR + half * HT;                          // first token of this warp
       const int ch0 = (tile / p.m_blocks) * BC_PAIR + static_cast<int>(rank) * BC_CTA + quad * 32;   // first channel
@@ -283,15 +285,19 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       for (int g = 0; g < p.k_blocks; ++g, ++it) {
         const uint32_t a = it % ACC_SLOTS, aph = (it / ACC_SLOTS) & 1u;
         const uint32_t v = it % SC_SLOTS, vph = (it / SC_SLOTS) & 1u;
-        bool w = mbar_wait(bar_sc_full + v * 8, vph, abort_flag);
-        w = w && mbar_wait(bar_acc_full + a * 8, aph, abort_flag);
-        ok = __all_sync(0xffffffffu, w);
-        if (!ok) break;
-        tc_fence_after_sync();
         // this thread's channel: one scale for the whole group
-        const float sg = reinterpret_cast<const float*>(smem + kScOff + v * BC_CTA * 4)[c_local];
+        float sg;
+        if (have_next) {
+          sg = sg_next;   // the look-ahead of the previous group saw both barriers complete
+        } else {
+          ok = __all_sync(0xffffffffu, mbar_wait2(bar_sc_full + v * 8, vph, bar_acc_full + a * 8, aph, abort_flag));
+          if (!ok) break;
+          sg = sc_rows[v * BC_CTA + c_local];
+        }
+        tc_fence_after_sync();
         const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + a * BT_PAIR + half * HT;
         uint32_t xb[2][LC];
+        uint32_t look = 0;
         tmem_ld_32x16(t_addr, xb[0]);
 #pragma unroll
         for (int c = 0; c < HT / LC; ++c) {
@@ -304,6 +310,18 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster_addr_relaxed(acc_empty0 + a * 8);
+          }
+          // Look ahead: the MMAs usually run a group ahead, and a barrier round trip costs hundreds
+          // of cycles under tensor-core load -- ask early, use the answer late, so that the arithmetic
+          // in between hides it.
+          if (c == 1) {
+            const uint32_t a1 = (it + 1) % ACC_SLOTS, aph1 = ((it + 1) / ACC_SLOTS) & 1u;
+            const uint32_t v1 = (it + 1) % SC_SLOTS, vph1 = ((it + 1) / SC_SLOTS) & 1u;
+            look = mbar_test2(bar_sc_full + v1 * 8, vph1, bar_acc_full + a1 * 8, aph1);
+          }
+          if (c == HT / LC - 2) {
+            have_next = __all_sync(0xffffffffu, look != 0);
+            if (have_next) sg_next = sc_rows[((it + 1) % SC_SLOTS) * BC_CTA + c_local];
           }
           const uint32_t(&x)[LC] = xb[c & 1];
           if constexpr (kExportAcc) {

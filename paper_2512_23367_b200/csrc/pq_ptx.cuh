@@ -89,6 +89,84 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
   return false;
 }
 
+// Waits on several barriers at once.  Under tensor-core load a single successful try_wait takes a
+// few hundred cycles (it queues behind the operand traffic in shared memory), so waits that follow
+// each other are issued together: their round trips overlap instead of adding up.
+__device__ __forceinline__ bool mbar_wait2(uint32_t bar_a, uint32_t par_a, uint32_t bar_b, uint32_t par_b,
+                                           volatile int* abort_flag) {
+  for (uint32_t i = 0; i < kWaitPollLimit; ++i) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred P, Q;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 P, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 Q, [%3], %4;\n\t"
+        "and.pred P, P, Q;\n\t"
+        "selp.u32 %0, 1, 0, P;\n\t}"
+        : "=r"(ok)
+        : "r"(bar_a), "r"(par_a), "r"(bar_b), "r"(par_b)
+        : "memory");
+    if (ok) return true;
+    if ((i & 255u) == 255u && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
+__device__ __forceinline__ bool mbar_wait3(uint32_t bar_a, uint32_t par_a, uint32_t bar_b, uint32_t par_b,
+                                           uint32_t bar_c, uint32_t par_c, volatile int* abort_flag) {
+  for (uint32_t i = 0; i < kWaitPollLimit; ++i) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred P, Q, R;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 P, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 Q, [%3], %4;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 R, [%5], %6;\n\t"
+        "and.pred P, P, Q;\n\t"
+        "and.pred P, P, R;\n\t"
+        "selp.u32 %0, 1, 0, P;\n\t}"
+        : "=r"(ok)
+        : "r"(bar_a), "r"(par_a), "r"(bar_b), "r"(par_b), "r"(bar_c), "r"(par_c)
+        : "memory");
+    if (ok) return true;
+    if ((i & 255u) == 255u && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
+// Two barriers that CTAs of the cluster arrive on remotely (cluster-scope acquire).
+__device__ __forceinline__ bool mbar_wait2_cluster(uint32_t bar_a, uint32_t par_a, uint32_t bar_b, uint32_t par_b,
+                                                   volatile int* abort_flag) {
+  for (uint32_t i = 0; i < kWaitPollLimit; ++i) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred P, Q;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 P, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 Q, [%3], %4;\n\t"
+        "and.pred P, P, Q;\n\t"
+        "selp.u32 %0, 1, 0, P;\n\t}"
+        : "=r"(ok)
+        : "r"(bar_a), "r"(par_a), "r"(bar_b), "r"(par_b)
+        : "memory");
+    if (ok) return true;
+    if ((i & 255u) == 255u && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
+// Non-blocking look at two barriers: nonzero if both phases have completed (acquire, CTA scope).
+__device__ __forceinline__ uint32_t mbar_test2(uint32_t bar_a, uint32_t par_a, uint32_t bar_b, uint32_t par_b) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred P, Q;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 P, [%1], %2;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 Q, [%3], %4;\n\t"
+      "and.pred P, P, Q;\n\t"
+      "selp.u32 %0, 1, 0, P;\n\t}"
+      : "=r"(ok)
+      : "r"(bar_a), "r"(par_a), "r"(bar_b), "r"(par_b)
+      : "memory");
+  return ok;   // not consumed here: the caller can let the round trip overlap with other work
+}
+
 // ---------------------------------------------------------------- fences
 __device__ __forceinline__ void fence_proxy_async_smem() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
