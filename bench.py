@@ -291,8 +291,8 @@ def run_ours(args, wl: synth.Workload, M: int):
     n_layers = layers_for_rotation(wl, M)
     layers = [LayerBuffers(pq, torch, wl, M, dev, src_x, src_w) for _ in range(n_layers)]
 
-    # The grouped W8A8 call schedules its members in one launch when M > 128.
-    grouped = wl.w_bits == 8 and M > 128 and not args.no_group
+    # The grouped calls schedule their members in one launch (W8A8: M > 128, W4A8: M > 64).
+    grouped = M > (128 if wl.w_bits == 8 else 64) and not args.no_group
 
     def run_layer(L: LayerBuffers, only: str | None = None):
         for gi, (K, idxs) in enumerate(L.groups):
@@ -302,9 +302,9 @@ def run_ours(args, wl: synth.Workload, M: int):
                 continue
             if grouped and len(idxs) > 1:
                 # linears over the same codes (q/k/v, gate/up): one grouped call, one kernel launch
-                pq.pq_gemm_w8a8_group(L.qs[gi], L.s_toks[gi],
-                                      [(L.packed[i][0], L.packed[i][1], wl.linears[i].N) for i in idxs],
-                                      [L.ys[i] for i in idxs])
+                group_call = pq.pq_gemm_w8a8_group if wl.w_bits == 8 else pq.pq_gemm_w4a8_group
+                group_call(L.qs[gi], L.s_toks[gi], [(L.packed[i][0], L.packed[i][1], wl.linears[i].N) for i in idxs],
+                           [L.ys[i] for i in idxs])
                 continue
             for i in idxs:
                 N = wl.linears[i].N

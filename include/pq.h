@@ -155,6 +155,11 @@ PQ_API int pq_gemm_w8a8_group(const int8_t* q, const float* s_tok, int32_t count
                               const float* const* s_ch, const int64_t* N, void* const* y_f16, int64_t M,
                               int64_t K, void* stream);
 
+/* The same for W4A8 linears (pq_gemm_w4a8 per member; grouped into one launch for M > 64). */
+PQ_API int pq_gemm_w4a8_group(const int8_t* q, const float* s_tok, int32_t count, const void* const* wp,
+                              const void* const* s_grp_f16, int32_t group, const int64_t* N,
+                              void* const* y_f16, int64_t M, int64_t K, void* stream);
+
 /*
  * Optional scratch memory for the current device.  With few output tiles and a long K (e.g. a
  * 7B-class layer at M = 512) the W8A8 GEMM cuts K into parts that run on different SMs; the parts'

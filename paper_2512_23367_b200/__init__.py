@@ -14,6 +14,7 @@ from .binding import (  # noqa: F401
     pq_acc_w8a8,
     pq_device_status,
     pq_gemm_w4a8,
+    pq_gemm_w4a8_group,
     pq_gemm_w8a8,
     pq_gemm_w8a8_group,
     pq_gemm_w8a8_noalloc,

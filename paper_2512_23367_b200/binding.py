@@ -36,6 +36,8 @@ SIGNATURES = {
     "pq_gemm_w8a8_noalloc": (ctypes.c_int, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _vp, _vp]),
     "pq_gemm_w8a8_group": (ctypes.c_int, [_vp, _vp, _i32, ctypes.POINTER(_vp), ctypes.POINTER(_vp),
                                           ctypes.POINTER(_i64), ctypes.POINTER(_vp), _i64, _i64, _vp]),
+    "pq_gemm_w4a8_group": (ctypes.c_int, [_vp, _vp, _i32, ctypes.POINTER(_vp), ctypes.POINTER(_vp), _i32,
+                                          ctypes.POINTER(_i64), ctypes.POINTER(_vp), _i64, _i64, _vp]),
 }
 MAX_GROUP = 4
 
@@ -196,6 +198,29 @@ def pq_gemm_w8a8_group(q, s_tok, members, ys=None) -> list[torch.Tensor]:
     y_arr = (_vp * max(n, 1))(*[y.data_ptr() for y in ys])
     _check("pq_gemm_w8a8_group", lib().pq_gemm_w8a8_group(q.data_ptr(), s_tok.data_ptr(), n, wq_arr, sc_arr, n_arr,
                                                           y_arr, M, K, _stream()))
+    return list(ys)
+
+
+def pq_gemm_w4a8_group(q, s_tok, members, ys=None, group: int = GROUP) -> list[torch.Tensor]:
+    """Several W4A8 linears over the same quantized tokens as one call (one kernel launch when
+    M > 64).  members: sequence of (wp, s_grp, N) from pq_pack_w4; ys: optional outputs f16 [M,N_g].
+    Each output equals pq_gemm_w4a8(q, s_tok, wp, s_grp, N) bit for bit."""
+    q = _dev(q, torch.int8, "q")
+    M, K = q.shape
+    _dev(s_tok, torch.float32, "s_tok")
+    n = len(members)
+    if ys is None:
+        ys = [torch.empty((M, int(N)), dtype=torch.float16, device=q.device) for (_, _, N) in members]
+    if len(ys) != n:
+        raise ValueError("one output per member")
+    for (wp, s_grp, _), y in zip(members, ys):
+        _dev(wp, torch.uint8, "wp"), _dev(s_grp, torch.float16, "s_grp"), _dev(y, torch.float16, "y")
+    wp_arr = (_vp * max(n, 1))(*[m[0].data_ptr() for m in members])
+    sg_arr = (_vp * max(n, 1))(*[m[1].data_ptr() for m in members])
+    n_arr = (_i64 * max(n, 1))(*[int(m[2]) for m in members])
+    y_arr = (_vp * max(n, 1))(*[y.data_ptr() for y in ys])
+    _check("pq_gemm_w4a8_group", lib().pq_gemm_w4a8_group(q.data_ptr(), s_tok.data_ptr(), n, wp_arr, sg_arr, group,
+                                                          n_arr, y_arr, M, K, _stream()))
     return list(ys)
 
 

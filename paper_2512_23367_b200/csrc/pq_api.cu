@@ -276,6 +276,33 @@ int pq_gemm_w4a8(const int8_t* q, const float* s_tok, const void* wp, const void
   return gemm_w4a8_common(q, s_tok, wp, s_grp_f16, group, M, N, K, y_f16, nullptr, stream);
 }
 
+int pq_gemm_w4a8_group(const int8_t* q, const float* s_tok, int32_t count, const void* const* wp,
+                       const void* const* s_grp_f16, int32_t group, const int64_t* N, void* const* y_f16, int64_t M,
+                       int64_t K, void* stream) {
+  if (!q || !s_tok || !wp || !s_grp_f16 || !N || !y_f16) return PQ_ERR_NULL;
+  if (count < 1 || count > PQ_MAX_GROUP) return PQ_ERR_SHAPE;
+  if (group != 128 || K % 128 != 0) return PQ_ERR_SHAPE;
+  for (int g = 0; g < count; ++g) {
+    if (!wp[g] || !s_grp_f16[g] || !y_f16[g]) return PQ_ERR_NULL;
+    const int rc = check_gemm(M, N[g], K);
+    if (rc != PQ_OK) return rc;
+    if (!aligned16(wp[g]) || !aligned16(s_grp_f16[g]) || !aligned16(y_f16[g])) return PQ_ERR_ALIGN;
+  }
+  if (!aligned16(q)) return PQ_ERR_ALIGN;
+  int rc = check_arch();
+  if (rc != PQ_OK) return rc;
+  if (M <= kSmallM || count == 1) {
+    // Decode-shaped token counts reduce inside the SMs and do not group: one launch per member.
+    for (int g = 0; g < count; ++g) {
+      rc = gemm_w4a8_common(q, s_tok, wp[g], s_grp_f16[g], group, M, N[g], K, y_f16[g], nullptr, stream);
+      if (rc != PQ_OK) return rc;
+    }
+    return PQ_OK;
+  }
+  return launch_gemm_w4a8_group(q, s_tok, count, wp, s_grp_f16, N, y_f16, M, K, nullptr,
+                                static_cast<cudaStream_t>(stream));
+}
+
 int pq_acc_w4a8(const int8_t* q, const void* wp, int32_t group, int64_t M, int64_t N, int64_t K, int32_t* acc_g,
                 void* stream) {
   if (!q || !wp || !acc_g) return PQ_ERR_NULL;

@@ -208,18 +208,19 @@ smallm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
       for (int j = 0; j < nkb; ++j) {
         const uint32_t it = static_cast<uint32_t>(j);
         const uint32_t s = it % C::STAGES, ph = (it / C::STAGES) & 1u;
-        if (!mbar_wait(bar_full + s * 8, ph, abort_flag)) { ok = false; break; }
         const uint32_t stage = smem_base + s * C::kStageBytes;
         uint64_t w_desc;
         uint32_t d_tmem = tmem_base;
         if constexpr (kW4) {
           const uint32_t u = it % C::A8_SLOTS, uph = (it / C::A8_SLOTS) & 1u;
           const uint32_t a = it % C::ACC_SLOTS, aph = (it / C::ACC_SLOTS) & 1u;
-          if (!mbar_wait(bar_a8_full + u * 8, uph, abort_flag) ||
-              !mbar_wait(bar_acc_empty + a * 8, aph ^ 1u, abort_flag)) { ok = false; break; }
           w_desc = umma_desc_k_sw128(smem_base + C::kA8Off + u * C::kA8Bytes);
           d_tmem = tmem_base + a * MPAD;
+          // (the three waits share their round trips)
+          if (!mbar_wait3(bar_full + s * 8, ph, bar_a8_full + u * 8, uph, bar_acc_empty + a * 8, aph ^ 1u,
+                          abort_flag)) { ok = false; break; }
         } else {
+          if (!mbar_wait(bar_full + s * 8, ph, abort_flag)) { ok = false; break; }
           w_desc = umma_desc_k_sw128(stage);
         }
         tc_fence_after_sync();
@@ -248,9 +249,8 @@ smallm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
         const uint32_t s = it % C::STAGES, ph = (it / C::STAGES) & 1u;
         const uint32_t u = it % C::A8_SLOTS, uph = (it / C::A8_SLOTS) & 1u;
         const uint32_t v = it % C::SC_SLOTS, vph = (it / C::SC_SLOTS) & 1u;
-        bool w = mbar_wait(bar_full + s * 8, ph, abort_flag);
-        w = w && mbar_wait(bar_a8_empty + u * 8, uph ^ 1u, abort_flag);
-        w = w && mbar_wait(bar_sc_empty + v * 8, vph ^ 1u, abort_flag);
+        const bool w = mbar_wait3(bar_full + s * 8, ph, bar_a8_empty + u * 8, uph ^ 1u, bar_sc_empty + v * 8,
+                                  vph ^ 1u, abort_flag);
         ok = __all_sync(0xffffffffu, w);
         if (!ok) break;
         const uint8_t* stage = smem + s * C::kStageBytes;
@@ -295,8 +295,7 @@ smallm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
         const uint32_t it = static_cast<uint32_t>(j);
         const uint32_t a = it % C::ACC_SLOTS, aph = (it / C::ACC_SLOTS) & 1u;
         const uint32_t v = it % C::SC_SLOTS, vph = (it / C::SC_SLOTS) & 1u;
-        bool w = mbar_wait(bar_acc_full + a * 8, aph, abort_flag);
-        w = w && mbar_wait(bar_sc_full + v * 8, vph, abort_flag);
+        const bool w = mbar_wait2(bar_acc_full + a * 8, aph, bar_sc_full + v * 8, vph, abort_flag);
         ok = __all_sync(0xffffffffu, w);
         if (!ok) break;
         tc_fence_after_sync();

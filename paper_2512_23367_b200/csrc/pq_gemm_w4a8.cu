@@ -77,11 +77,41 @@ static_assert(128 * kRegsCtl + 128 * kRegsUnpack + 256 * kRegsPromote <= 65536, 
 
 struct W4Args {
   const float* s_tok;
-  int32_t* acc_g;  // [G, M, N] when exporting
+  int32_t* acc_g;  // [G, M, N] when exporting (single member)
   int* status;
-  int M, N, K;
-  int m_blocks, n_blocks, k_blocks;
+  int N[kMaxGroup];        // per member
+  int nb_end[kMaxGroup];   // channel blocks of members 0..g (running total); INT_MAX past the last member
+  int count;               // members in this launch (linears that share the token codes)
+  int M, K;
+  int m_blocks, n_blocks, k_blocks;   // n_blocks: over all members
 };
+
+// Tensor maps of the members' packed weights, group scales and outputs (indexed by member).
+struct W4Maps {
+  CUtensorMap w[kMaxGroup];
+  CUtensorMap s[kMaxGroup];
+  CUtensorMap y[kMaxGroup];
+};
+
+// Where a tile lies: its member, the member's channel count, its token block and first channel.
+struct W4Tile {
+  int g, m_blk, c0, N;
+};
+__device__ __forceinline__ W4Tile locate_tile(const W4Args& p, int tile) {
+  W4Tile t;
+  int nblk = tile / p.m_blocks;
+  t.m_blk = tile - nblk * p.m_blocks;
+  t.g = 0;
+  t.N = p.N[0];
+  if (p.count > 1) {
+    const int e0 = p.nb_end[0], e1 = p.nb_end[1], e2 = p.nb_end[2];
+    if (nblk >= e2) { t.g = 3; t.N = p.N[3]; nblk -= e2; }
+    else if (nblk >= e1) { t.g = 2; t.N = p.N[2]; nblk -= e1; }
+    else if (nblk >= e0) { t.g = 1; t.N = p.N[1]; nblk -= e0; }
+  }
+  t.c0 = nblk * BC_PAIR;
+  return t;
+}
 
 template <int N>
 __device__ __forceinline__ void setmaxnreg_inc() {
@@ -94,9 +124,7 @@ __device__ __forceinline__ void setmaxnreg_dec() {
 
 template <bool kExportAcc>
 __global__ void __launch_bounds__(kNumThreads, 1)
-gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_w,
-                 const __grid_constant__ CUtensorMap tm_s, const __grid_constant__ CUtensorMap tm_y,
-                 const W4Args p) {
+gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ W4Maps maps, const W4Args p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t smem_base = smem_u32(smem);
@@ -137,9 +165,11 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   }
   if (warp == 0 && lane == 0) {
     tma_prefetch_desc(&tm_q);
-    tma_prefetch_desc(&tm_w);
-    tma_prefetch_desc(&tm_s);
-    if constexpr (!kExportAcc) tma_prefetch_desc(&tm_y);
+    for (int g = 0; g < p.count; ++g) {
+      tma_prefetch_desc(&maps.w[g]);
+      tma_prefetch_desc(&maps.s[g]);
+      if constexpr (!kExportAcc) tma_prefetch_desc(&maps.y[g]);
+    }
   }
   if (warp == 1) {
     tmem_alloc_pair(smem_u32(tmem_slot), kTmemCols);
@@ -157,36 +187,39 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     setmaxnreg_dec<kRegsCtl>();
     if (warp == 0 && lane == 0) {
       // ---------------------------------------------------------- TMA producer (both CTAs)
-      auto load_weights = [&](uint32_t s, int g, int c0) {
+      auto load_weights = [&](uint32_t s, int g, int member, int c0) {
         const uint32_t dst = smem_base + s * kStageBytes;
         mbar_arrive_expect_tx(bar_full + s * 8, kTxBytes);   // the whole stage, codes included
-        tma_load_2d(dst + kQBytes, &tm_w, bar_full + s * 8, g * (BK / 2), c0);
-        tma_load_2d(dst + kQBytes + kPBytes, &tm_s, bar_full + s * 8, c0, g);
+        tma_load_2d(dst + kQBytes, &maps.w[member], bar_full + s * 8, g * (BK / 2), c0);
+        tma_load_2d(dst + kQBytes + kPBytes, &maps.s[member], bar_full + s * 8, c0, g);
       };
       auto load_codes = [&](uint32_t s, int g, int t0) {
         tma_load_2d(smem_base + s * kStageBytes, &tm_q, bar_full + s * 8, g * BK, t0);
       };
-      auto chan0 = [&](int tile) { return (tile / p.m_blocks) * BC_PAIR + static_cast<int>(rank) * BC_CTA; };
-      auto tok0 = [&](int tile) { return (tile % p.m_blocks) * BT_PAIR + static_cast<int>(rank) * BT_CTA; };
+      auto tok0 = [&](const W4Tile& t) { return t.m_blk * BT_PAIR + static_cast<int>(rank) * BT_CTA; };
       // First ring pass of the first tile: weights and scales (constants) before the wait on the
       // preceding kernel, the codes it may have produced after it.
       int pre = 0;
       if (pair_id < num_tiles) {
         pre = p.k_blocks < STAGES ? p.k_blocks : STAGES;
-        for (int g = 0; g < pre; ++g) load_weights(static_cast<uint32_t>(g), g, chan0(pair_id));
+        const W4Tile t = locate_tile(p, pair_id);
+        for (int g = 0; g < pre; ++g)
+          load_weights(static_cast<uint32_t>(g), g, t.g, t.c0 + static_cast<int>(rank) * BC_CTA);
       }
       grid_dep_wait();
       if (pair_id < num_tiles) {
-        for (int g = 0; g < pre; ++g) load_codes(static_cast<uint32_t>(g), g, tok0(pair_id));
+        const W4Tile t = locate_tile(p, pair_id);
+        for (int g = 0; g < pre; ++g) load_codes(static_cast<uint32_t>(g), g, tok0(t));
       }
       uint32_t it = static_cast<uint32_t>(pre);
       bool ok = true;
       for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs) {
-        const int t0 = tok0(tile), c0 = chan0(tile);
+        const W4Tile t = locate_tile(p, tile);
+        const int t0 = tok0(t), c0 = t.c0 + static_cast<int>(rank) * BC_CTA;
         for (int g = (tile == pair_id ? pre : 0); g < p.k_blocks; ++g, ++it) {
           const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
           if (!mbar_wait(bar_empty + s * 8, ph ^ 1u, abort_flag)) { ok = false; break; }
-          load_weights(s, g, c0);
+          load_weights(s, g, t.g, c0);
           load_codes(s, g, t0);
         }
       }
@@ -277,8 +310,9 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     bool have_next = false;
     float sg_next = 0.0f;
     for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs) {
-      const int tok0 = (tile % p.m_blocks) * BT_PAIR + half * HT;                          // first token of this warp
-      const int ch0 = (tile / p.m_blocks) * BC_PAIR + static_cast<int>(rank) * BC_CTA + quad * 32;   // first channel
+      const W4Tile tp = locate_tile(p, tile);
+      const int tok0 = tp.m_blk * BT_PAIR + half * HT;                                // first token of this warp
+      const int ch0 = tp.c0 + static_cast<int>(rank) * BC_CTA + quad * 32;            // first channel (of the member)
       float R[HT];
 #pragma unroll
       for (int j = 0; j < HT; ++j) R[j] = 0.0f;
@@ -329,8 +363,8 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 #pragma unroll
             for (int j = 0; j < LC; ++j) {
               const int m = tok0 + c * LC + j;
-              if (m < p.M && n < p.N)
-                p.acc_g[(static_cast<int64_t>(g) * p.M + m) * p.N + n] = static_cast<int32_t>(x[j]) >> 4;
+              if (m < p.M && n < tp.N)
+                p.acc_g[(static_cast<int64_t>(g) * p.M + m) * tp.N + n] = static_cast<int32_t>(x[j]) >> 4;
             }
           } else {
 #pragma unroll
@@ -367,8 +401,8 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) {
-              if (ch0 < p.N && tok0 + c * CH < p.M)
-                tma_store_2d(&tm_y, out_warp_u32 + buf * kOutBoxBytes, ch0, tok0 + c * CH);
+              if (ch0 < tp.N && tok0 + c * CH < p.M)
+                tma_store_2d(&maps.y[tp.g], out_warp_u32 + buf * kOutBoxBytes, ch0, tok0 + c * CH);
               tma_store_commit();  // also when nothing was stored: keeps one group per buffer use
             }
             ++nstore;
@@ -395,8 +429,7 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 }
 
 template <bool kExportAcc>
-int launch_w4(const CUtensorMap& tq, const CUtensorMap& tw, const CUtensorMap& ts, const CUtensorMap& ty,
-              const W4Args& a, cudaStream_t stream) {
+int launch_w4(const CUtensorMap& tq, const W4Maps& maps, const W4Args& a, cudaStream_t stream) {
   auto kern = gemm_w4a8_kernel<kExportAcc>;
   static int configured = 0;  // 0 = not yet, 1 = ok, -1 = unusable
   if (configured == 0) {
@@ -430,43 +463,56 @@ int launch_w4(const CUtensorMap& tq, const CUtensorMap& tw, const CUtensorMap& t
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = pdl_enabled() ? 2 : 1;
-  return cuda_status(cudaLaunchKernelEx(&cfg, kern, tq, tw, ts, ty, a));
+  return cuda_status(cudaLaunchKernelEx(&cfg, kern, tq, maps, a));
 }
 
 }  // namespace
 
-int launch_gemm_w4a8(const int8_t* q, const float* s_tok, const void* wp, const void* s_grp, int64_t M,
-                     int64_t N, int64_t K, void* y, int32_t* acc_g, cudaStream_t stream) {
-  CUtensorMap tq, tw, ts, ty;
+int launch_gemm_w4a8_group(const int8_t* q, const float* s_tok, int count, const void* const* wp,
+                           const void* const* s_grp, const int64_t* N, void* const* y, int64_t M, int64_t K,
+                           int32_t* acc_g, cudaStream_t stream) {
+  if (count < 1 || count > kMaxGroup || (acc_g != nullptr && count != 1)) return PQ_ERR_SHAPE;
+  CUtensorMap tq;
+  W4Maps maps;
   int rc = make_tmap_2d(&tq, q, static_cast<uint64_t>(M), static_cast<uint64_t>(K), BT_CTA, BK, 1, 128);
   if (rc != PQ_OK) return rc;
-  rc = make_tmap_2d(&tw, wp, static_cast<uint64_t>(N), static_cast<uint64_t>(K / 2), BC_CTA, BK / 2, 1, 0);
-  if (rc != PQ_OK) return rc;
-  // Group scales [K/128, N] FP16; the accumulator-export variant has none and reads a dummy map of Q.
-  if (s_grp != nullptr) {
-    rc = make_tmap_2d(&ts, s_grp, static_cast<uint64_t>(K / 128), static_cast<uint64_t>(N), 1, BC_CTA, 2, 0);
-  } else {
-    rc = make_tmap_2d(&ts, q, static_cast<uint64_t>(M), static_cast<uint64_t>(K / 2), 1, BC_CTA, 2, 0);
-  }
-  if (rc != PQ_OK) return rc;
-  if (y != nullptr) {
-    rc = make_tmap_2d(&ty, y, static_cast<uint64_t>(M), static_cast<uint64_t>(N), 32, 32, 2, 64);
-    if (rc != PQ_OK) return rc;
-  } else {
-    ty = tq;  // not used by the accumulator export
-  }
   W4Args a;
+  int64_t nb_total = 0;
+  for (int g = 0; g < kMaxGroup; ++g) {
+    const int src = g < count ? g : 0;   // unused slots repeat member 0 (never selected)
+    rc = make_tmap_2d(&maps.w[g], wp[src], static_cast<uint64_t>(N[src]), static_cast<uint64_t>(K / 2), BC_CTA, BK / 2, 1, 0);
+    if (rc != PQ_OK) return rc;
+    // Group scales [K/128, N] FP16; the accumulator-export variant has none and reads a dummy map of Q.
+    if (acc_g == nullptr) {
+      rc = make_tmap_2d(&maps.s[g], s_grp[src], static_cast<uint64_t>(K / 128), static_cast<uint64_t>(N[src]), 1, BC_CTA, 2, 0);
+      if (rc != PQ_OK) return rc;
+      rc = make_tmap_2d(&maps.y[g], y[src], static_cast<uint64_t>(M), static_cast<uint64_t>(N[src]), 32, 32, 2, 64);
+    } else {
+      rc = make_tmap_2d(&maps.s[g], q, static_cast<uint64_t>(M), static_cast<uint64_t>(K / 2), 1, BC_CTA, 2, 0);
+      maps.y[g] = tq;  // not used by the accumulator export
+    }
+    if (rc != PQ_OK) return rc;
+    a.N[g] = static_cast<int>(N[src]);
+    if (g < count) nb_total += (N[g] + BC_PAIR - 1) / BC_PAIR;
+    a.nb_end[g] = g < count ? static_cast<int>(nb_total) : 0x7fffffff;
+  }
+  a.m_blocks = static_cast<int>((M + BT_PAIR - 1) / BT_PAIR);
+  if (a.m_blocks * nb_total > 0x3fffffff) return PQ_ERR_SHAPE;
+  a.count = count;
   a.s_tok = s_tok;
   a.acc_g = acc_g;
   a.status = device_status_ptr();
   if (a.status == nullptr) return PQ_ERR_CUDA;
   a.M = static_cast<int>(M);
-  a.N = static_cast<int>(N);
   a.K = static_cast<int>(K);
-  a.m_blocks = static_cast<int>((M + BT_PAIR - 1) / BT_PAIR);
-  a.n_blocks = static_cast<int>((N + BC_PAIR - 1) / BC_PAIR);
+  a.n_blocks = static_cast<int>(nb_total);
   a.k_blocks = static_cast<int>(K / BK);
-  return acc_g != nullptr ? launch_w4<true>(tq, tw, ts, ty, a, stream) : launch_w4<false>(tq, tw, ts, ty, a, stream);
+  return acc_g != nullptr ? launch_w4<true>(tq, maps, a, stream) : launch_w4<false>(tq, maps, a, stream);
+}
+
+int launch_gemm_w4a8(const int8_t* q, const float* s_tok, const void* wp, const void* s_grp, int64_t M,
+                     int64_t N, int64_t K, void* y, int32_t* acc_g, cudaStream_t stream) {
+  return launch_gemm_w4a8_group(q, s_tok, 1, &wp, &s_grp, &N, &y, M, K, acc_g, stream);
 }
 
 }  // namespace pq

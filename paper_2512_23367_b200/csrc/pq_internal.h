@@ -67,6 +67,10 @@ int launch_gemm_w8a8_pair_group(const Scratch& sc, const int8_t* q, const float*
 // Prefill-shaped W4A8 GEMM.  Exactly one of y / acc_g is non-null.
 int launch_gemm_w4a8(const int8_t* q, const float* s_tok, const void* wp, const void* s_grp, int64_t M,
                      int64_t N, int64_t K, void* y, int32_t* acc_g, cudaStream_t stream);
+// `count` (1..kMaxGroup) W4A8 linears over the same codes in one launch (host arrays, as above).
+int launch_gemm_w4a8_group(const int8_t* q, const float* s_tok, int count, const void* const* wp,
+                           const void* const* s_grp, const int64_t* N, void* const* y, int64_t M, int64_t K,
+                           int32_t* acc_g, cudaStream_t stream);
 // Small-M (decode-shaped) weight-streaming variants; same results as the calls above.
 int launch_smallm_w8a8(const int8_t* q, const float* s_tok, const void* wq, const float* s_ch, int64_t M,
                        int64_t N, int64_t K, void* y, int32_t* acc, cudaStream_t stream);

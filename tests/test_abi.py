@@ -46,6 +46,9 @@ def test_argument_errors_come_back_as_status_codes_without_a_device():
     assert L.pq_gemm_w8a8_group(16, 16, 0, ptrs, ptrs, cols, ptrs, 4, 64, None) == PQ_ERR_SHAPE    # empty group
     assert L.pq_gemm_w8a8_group(16, 16, 5, ptrs, ptrs, cols, ptrs, 4, 64, None) == PQ_ERR_SHAPE    # > PQ_MAX_GROUP
     assert L.pq_gemm_w8a8_group(16, 16, 2, ptrs, ptrs, odd, ptrs, 4, 64, None) == PQ_ERR_SHAPE     # N[1] % 8
+    assert L.pq_gemm_w4a8_group(16, 16, 2, ptrs, holes, 128, cols, ptrs, 4, 128, None) == PQ_ERR_NULL
+    assert L.pq_gemm_w4a8_group(16, 16, 2, ptrs, ptrs, 64, cols, ptrs, 4, 128, None) == PQ_ERR_SHAPE    # group != 128
+    assert L.pq_gemm_w4a8_group(16, 16, 5, ptrs, ptrs, 128, cols, ptrs, 4, 128, None) == PQ_ERR_SHAPE   # > PQ_MAX_GROUP
     assert L.pq_packed_w8_bytes(8, 256) == 2048 and L.pq_packed_w4_bytes(8, 256) == 1024
     assert L.pq_status_str(0) == b"ok" and b"wait" in L.pq_status_str(6)
 

@@ -1,4 +1,4 @@
-"""pq_gemm_w8a8_group: several W8A8 linears over the same quantized tokens in one call.
+"""pq_gemm_w8a8_group / pq_gemm_w4a8_group: several linears over the same quantized tokens in one call.
 
 The contract is "exactly what one pq_gemm_w8a8 call per member gives", so every case checks bit
 equality with those calls, and parity with the CPU oracle (INT32 accumulators are exact, the FP16
@@ -78,3 +78,50 @@ def test_two_group_calls_in_a_row_leave_the_split_k_scratch_clean():
         assert torch.equal(a, b)
         assert torch.equal(a, pq.pq_gemm_w8a8(q, s_tok, wq, s_ch, N))
     assert pq.pq_device_status() == 0
+
+
+# ---------------------------------------------------------------------------- W4A8
+
+def _members_w4(K, Ns, seed):
+    ws = [synth.weights(N, K, seed + 1 + i) for i, N in enumerate(Ns)]
+    packed = [pq.pq_pack_w4(torch.from_numpy(w).to(DEV)) for w in ws]
+    return ws, [(wp, sg, N) for (wp, sg), N in zip(packed, Ns)]
+
+
+@pytest.mark.parametrize("M,K,Ns", [
+    (512, 512, (512, 512, 512)),
+    (300, 256, (520, 264)),
+    (257, 384, (1000, 136, 8)),
+    (2048, 512, (2048, 2048, 2048)),
+    (600, 1024, (256, 768, 264, 128)),
+    (65, 128, (16, 24)),
+])
+def test_w4a8_group_equals_one_call_per_member_and_the_oracle(M, K, Ns):
+    x = synth.activations(M, K, 5000 + M)
+    ws, members = _members_w4(K, Ns, 5100 + M)
+    q, s_tok = pq.pq_quantize_act(torch.from_numpy(x).to(DEV))
+    pad = 512
+    bufs = [torch.full((pad + M * N + pad,), 5.0, dtype=torch.float16, device=DEV) for N in Ns]
+    ys = [b[pad:pad + M * N].view(M, N) for b, N in zip(bufs, Ns)]
+    out = pq.pq_gemm_w4a8_group(q, s_tok, members, ys)
+    torch.cuda.synchronize()
+    assert pq.pq_device_status() == 0
+    qo, so = oracle.quantize_act(x)
+    for (wp, sg, N), w, y, b in zip(members, ws, out, bufs):
+        assert torch.equal(y, pq.pq_gemm_w4a8(q, s_tok, wp, sg, N))
+        codes, sgo = oracle.pack_w4(w)
+        _, ref = oracle.gemm_w4a8(qo, so, codes, sgo, want_acc=False)
+        g, ref = y.cpu().numpy().astype(np.float64), ref.astype(np.float64)
+        assert np.all(np.abs(g - ref) <= REL * np.abs(ref) + ABS)
+        assert (b[:pad] == 5.0).all() and (b[pad + M * N:] == 5.0).all()
+
+
+@pytest.mark.parametrize("M", [1, 16, 64])
+def test_w4a8_small_token_counts_run_member_by_member_with_the_same_result(M):
+    K, Ns = 512, (256, 520)
+    x = synth.activations(M, K, 5300 + M)
+    _, members = _members_w4(K, Ns, 5400 + M)
+    q, s_tok = pq.pq_quantize_act(torch.from_numpy(x).to(DEV))
+    out = pq.pq_gemm_w4a8_group(q, s_tok, members)
+    for (wp, sg, N), y in zip(members, out):
+        assert torch.equal(y, pq.pq_gemm_w4a8(q, s_tok, wp, sg, N))
