@@ -107,16 +107,26 @@ def load_peaks():
     return dict(FALLBACK_PEAKS), "fallback"
 
 
-def load_traffic(wl: synth.Workload, M: int):
-    """DRAM bytes per launch of the dominant (GEMM) kernel, averaged over the workload's linears,
-    from the committed ncu summaries (profiles/traffic.json: "gemm_w<bits>a8:MxKxN" -> bytes).
-    None unless every shape of the workload has an entry taken from the current kernel."""
+def load_traffic(wl: synth.Workload, M: int, grouped: bool = False):
+    """DRAM bytes per launch of the dominant (GEMM) kernel, averaged over the step's GEMM launches, from
+    the committed ncu summaries (profiles/traffic.json: "gemm_w<bits>a8:MxKxN" -> bytes of one launch;
+    "...xN*G" for a grouped launch of G linears of width N).  None unless every launch of the step has
+    an entry taken from the current kernel."""
     path = os.path.join(ROOT, "profiles", "traffic.json")
     if not os.path.exists(path):
         return None
     with open(path) as f:
         table = json.load(f)
-    vals = [table.get(f"gemm_w{wl.w_bits}a8:{M}x{lin.K}x{lin.N}") for lin in wl.linears]
+    keys = []
+    for K, idxs in layer_plan(wl):
+        widths = {wl.linears[i].N for i in idxs}
+        if grouped and len(idxs) > 1 and len(widths) == 1:
+            keys.append(f"gemm_w{wl.w_bits}a8:{M}x{K}x{widths.pop()}*{len(idxs)}")
+        elif grouped and len(idxs) > 1:
+            return None
+        else:
+            keys += [f"gemm_w{wl.w_bits}a8:{M}x{K}x{wl.linears[i].N}" for i in idxs]
+    vals = [table.get(k) for k in keys]
     if any(v is None for v in vals):
         return None
     return sum(vals) / len(vals)
@@ -501,7 +511,7 @@ def run_ours(args, wl: synth.Workload, M: int):
         if wl.w_bits and M > 64:
             peak = 2.0 * float(peaks["bf16_tflops"])
             roof = {"bound": "tensor", "achieved": gemm_tops, "peak": peak, "unit": "TOPS",
-                    "frac": gemm_tops / peak, "traffic": load_traffic(wl, M),
+                    "frac": gemm_tops / peak, "traffic": load_traffic(wl, M, grouped),
                     "kernel": f"gemm_w{wl.w_bits}a8 (tcgen05 kind::i8)",
                     "peak_kind": f"2 x bf16_tflops (burst) of {peak_kind}: INT8 peak = bf16 peak x nominal 4.5/2.25",
                     "frac_of_sustained": gemm_tops / (2.0 * float(peaks["bf16_tflops_sustained"])),
@@ -511,7 +521,7 @@ def run_ours(args, wl: synth.Workload, M: int):
             gbs = sbytes["gemm"] / (gemm_avg_ms * gemm_per_layer * 1e-3) / 1e9
             peak = float(peaks["hbm_gbs"])
             roof = {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
-                    "traffic": load_traffic(wl, M),
+                    "traffic": load_traffic(wl, M, grouped),
                     "kernel": f"small-M gemm_w{wl.w_bits}a8", "peak_kind": f"hbm_gbs of {peak_kind}",
                     "avg_launch_us": gemm_avg_ms * 1e3, "launches_timed": gemm_launches}
         decode = M <= 64

@@ -24,6 +24,8 @@ def main(argv=None):
     ap.add_argument("--M", type=int, required=True)
     ap.add_argument("--K", type=int, required=True)
     ap.add_argument("--N", type=int, default=0)
+    ap.add_argument("--group", type=int, default=1,
+                    help="GEMM ops: this many linears of width N over the same tokens in one grouped call")
     ap.add_argument("--sets", type=int, default=0, help="distinct buffer sets (0 = enough to exceed 2 x L2, max 16)")
     ap.add_argument("--launches", type=int, default=16, help="launches per graph replay")
     ap.add_argument("--replays", type=int, default=20)
@@ -31,8 +33,8 @@ def main(argv=None):
     a = ap.parse_args(argv)
     dev = torch.device("cuda", 0)
     torch.manual_seed(0)
-    M, K, N = a.M, a.K, a.N
-    per_set = 2 * M * K + M * K + (N * K if a.op != "quantize" else 0)
+    M, K, N, G = a.M, a.K, a.N, max(a.group, 1)
+    per_set = 2 * M * K + M * K + (G * N * K if a.op != "quantize" else 0)
     sets = a.sets or max(2, min(16, (2 * 126 * 2 ** 20) // max(per_set, 1) + 1))
 
     bufs = []
@@ -42,26 +44,32 @@ def main(argv=None):
         q, s_tok = pq.pq_quantize_act(x)
         entry = {"x": x, "q": q, "s_tok": s_tok}
         if a.op != "quantize":
-            w = (torch.randn((N, K), device=dev, dtype=torch.float32) * 0.02).half()
-            entry["w"] = pq.pq_pack_w8(w) if a.op == "gemm_w8a8" else pq.pq_pack_w4(w)
-            entry["y"] = torch.empty((M, N), device=dev, dtype=torch.float16)
-            del w
+            entry["w"], entry["y"] = [], []
+            for _ in range(G):
+                w = (torch.randn((N, K), device=dev, dtype=torch.float32) * 0.02).half()
+                entry["w"].append(pq.pq_pack_w8(w) if a.op == "gemm_w8a8" else pq.pq_pack_w4(w))
+                entry["y"].append(torch.empty((M, N), device=dev, dtype=torch.float16))
+                del w
         bufs.append(entry)
 
     def launch(i):
         b = bufs[i % sets]
         if a.op == "quantize":
             pq.pq_quantize_act(b["x"], b["q"], b["s_tok"])
+        elif G > 1:
+            call = pq.pq_gemm_w8a8_group if a.op == "gemm_w8a8" else pq.pq_gemm_w4a8_group
+            call(b["q"], b["s_tok"], [(w[0], w[1], N) for w in b["w"]], b["y"])
         elif a.op == "gemm_w8a8":
-            pq.pq_gemm_w8a8(b["q"], b["s_tok"], b["w"][0], b["w"][1], N, y=b["y"])
+            pq.pq_gemm_w8a8(b["q"], b["s_tok"], b["w"][0][0], b["w"][0][1], N, y=b["y"][0])
         else:
-            pq.pq_gemm_w4a8(b["q"], b["s_tok"], b["w"][0], b["w"][1], N, y=b["y"])
+            pq.pq_gemm_w4a8(b["q"], b["s_tok"], b["w"][0][0], b["w"][0][1], N, y=b["y"][0])
 
     if a.eager:
         for i in range(a.eager):
             launch(i)
         torch.cuda.synchronize()
-        print(json.dumps({"op": a.op, "M": M, "K": K, "N": N, "eager_launches": a.eager, "status": pq.pq_device_status()}))
+        print(json.dumps({"op": a.op, "M": M, "K": K, "N": N, "group": G, "eager_launches": a.eager,
+                          "status": pq.pq_device_status()}))
         return
 
     stream = torch.cuda.Stream()
@@ -86,14 +94,14 @@ def main(argv=None):
         stream.synchronize()
     us = sorted(e0.elapsed_time(e1) * 1e3 / a.launches for e0, e1 in times)
     med, best = us[len(us) // 2], us[0]
-    out = {"op": a.op, "M": M, "K": K, "N": N, "sets": sets, "us_median": med, "us_min": best,
+    out = {"op": a.op, "M": M, "K": K, "N": N, "group": G, "sets": sets, "us_median": med, "us_min": best,
            "status": pq.pq_device_status()}
     if a.op == "quantize":
         out["GBps"] = (3 * M * K + 4 * M) / med / 1e3
     else:
-        out["TOPS"] = 2 * M * N * K / med / 1e6
+        out["TOPS"] = 2 * M * G * N * K / med / 1e6
         wbytes = N * K if a.op == "gemm_w8a8" else N * K // 2 + (K // 128) * N * 2
-        out["GBps"] = (wbytes + M * K + 2 * M * N) / med / 1e3
+        out["GBps"] = (G * wbytes + M * K + 2 * M * G * N) / med / 1e3
     print(json.dumps(out))
 
 
