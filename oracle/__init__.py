@@ -49,6 +49,11 @@ def _load():
         lib.pqo_quantize_act.argtypes = [vp, i64, i64, vp, vp]
         lib.pqo_pack_w8.argtypes = [vp, i64, i64, vp, vp]
         lib.pqo_pack_w4.argtypes = [vp, i64, i64, i64, vp, vp]
+        lib.pqo_quantize_act_smooth.argtypes = [vp, vp, i64, i64, vp, vp]
+        lib.pqo_pack_w8_smooth.argtypes = [vp, vp, i64, i64, vp, vp]
+        lib.pqo_pack_w4_smooth.argtypes = [vp, vp, i64, i64, i64, vp, vp]
+        lib.pqo_col_absmax.argtypes = [vp, i64, i64, vp]
+        lib.pqo_smooth_scales.argtypes = [vp, vp, i64, vp, vp]
         lib.pqo_nibble_pack.argtypes = [vp, i64, i64, vp]
         lib.pqo_nibble_unpack.argtypes = [vp, i64, i64, vp]
         lib.pqo_gemm_w8a8.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp, vp]
@@ -96,35 +101,76 @@ def float_to_half_bits(v: float) -> int:
     return int(_load().pqo_float_to_half_rne(float(np.float32(v))))
 
 
-def quantize_act(x: np.ndarray):
-    """x f16 [M,K] -> (q int8 [M,K], s_tok f32 [M]).  Eq. 1-2, n = 8, per token."""
+def _col(col, K: int):
+    col = _c(col, np.float32)
+    if col.shape != (K,):
+        raise OracleError("column factors must have shape [K]")
+    return col
+
+
+def quantize_act(x: np.ndarray, s_inv: np.ndarray | None = None):
+    """x f16 [M,K] -> (q int8 [M,K], s_tok f32 [M]).  Eq. 1-2, n = 8, per token.
+    With s_inv f32 [K]: quantizes X S^-1 (Eq. 3)."""
     x = _c(x, np.float16)
     M, K = x.shape
     q = np.empty((M, K), np.int8)
     s = np.empty((M,), np.float32)
-    _check(_load().pqo_quantize_act(_p(x), M, K, _p(q), _p(s)), "quantize_act")
+    if s_inv is None:
+        _check(_load().pqo_quantize_act(_p(x), M, K, _p(q), _p(s)), "quantize_act")
+    else:
+        s_inv = _col(s_inv, K)
+        _check(_load().pqo_quantize_act_smooth(_p(x), _p(s_inv), M, K, _p(q), _p(s)), "quantize_act_smooth")
     return q, s
 
 
-def pack_w8(w: np.ndarray):
-    """w f16 [N,K] -> (wq int8 [N,K], s_ch f32 [N]).  Eq. 2, n = 8, per output channel."""
+def col_absmax(a: np.ndarray) -> np.ndarray:
+    """a f16 [R,K] -> f32 [K]: max over rows of |a[r,k]| (calibration statistic of Eq. 3)."""
+    a = _c(a, np.float16)
+    R, K = a.shape
+    out = np.empty((K,), np.float32)
+    _check(_load().pqo_col_absmax(_p(a), R, K, _p(out)), "col_absmax")
+    return out
+
+
+def smooth_scales(x_absmax: np.ndarray, w_absmax: np.ndarray):
+    """Eq. 3 with alpha = 0.5: (s, s_inv) f32 [K] from the column maxima of X and W."""
+    xa, wa = _c(x_absmax, np.float32), _c(w_absmax, np.float32)
+    if xa.shape != wa.shape or xa.ndim != 1:
+        raise OracleError("smooth_scales: two vectors of the same length")
+    s, s_inv = np.empty_like(xa), np.empty_like(xa)
+    _check(_load().pqo_smooth_scales(_p(xa), _p(wa), xa.shape[0], _p(s), _p(s_inv)), "smooth_scales")
+    return s, s_inv
+
+
+def pack_w8(w: np.ndarray, smooth: np.ndarray | None = None):
+    """w f16 [N,K] -> (wq int8 [N,K], s_ch f32 [N]).  Eq. 2, n = 8, per output channel.
+    With smooth f32 [K]: quantizes S W (Eq. 3)."""
     w = _c(w, np.float16)
     N, K = w.shape
     wq = np.empty((N, K), np.int8)
     s = np.empty((N,), np.float32)
-    _check(_load().pqo_pack_w8(_p(w), N, K, _p(wq), _p(s)), "pack_w8")
+    if smooth is None:
+        _check(_load().pqo_pack_w8(_p(w), N, K, _p(wq), _p(s)), "pack_w8")
+    else:
+        smooth = _col(smooth, K)
+        _check(_load().pqo_pack_w8_smooth(_p(w), _p(smooth), N, K, _p(wq), _p(s)), "pack_w8_smooth")
     return wq, s
 
 
-def pack_w4(w: np.ndarray, group: int = 128):
-    """w f16 [N,K] -> (codes int8 [N,K] in [-8,7], s_grp f16 [N,K/group]).  Eq. 2, n = 4."""
+def pack_w4(w: np.ndarray, group: int = 128, smooth: np.ndarray | None = None):
+    """w f16 [N,K] -> (codes int8 [N,K] in [-8,7], s_grp f16 [N,K/group]).  Eq. 2, n = 4.
+    With smooth f32 [K]: quantizes S W (Eq. 3)."""
     w = _c(w, np.float16)
     N, K = w.shape
     if K % group:
         raise OracleError("pack_w4: K must be a multiple of the group size")
     codes = np.empty((N, K), np.int8)
     s = np.empty((N, K // group), np.float16)
-    _check(_load().pqo_pack_w4(_p(w), N, K, group, _p(codes), _p(s)), "pack_w4")
+    if smooth is None:
+        _check(_load().pqo_pack_w4(_p(w), N, K, group, _p(codes), _p(s)), "pack_w4")
+    else:
+        smooth = _col(smooth, K)
+        _check(_load().pqo_pack_w4_smooth(_p(w), _p(smooth), N, K, group, _p(codes), _p(s)), "pack_w4_smooth")
     return codes, s
 
 

@@ -18,6 +18,10 @@
  *   - Symmetric quantization (no zero point), as the experimental set-up states.
  *   - The "Unified low-bit inference framework" section: integer matrix product of
  *     the codes followed by dequantization back to FP16.
+ *   - Eq. 3 (SmoothQuant variant of the W4A8 configurations): Y = (X S^-1)(S W) with
+ *     S = diag(s), s_j = max|X_j|^alpha / max|W_j|^(1-alpha), alpha = 0.5.  The column
+ *     factors enter the quantizers as an optional per-k multiplier applied in binary32
+ *     BEFORE the absolute maximum is taken (the *_smooth entry points).
  *
  * Readings taken where the paper is silent (also listed in the design notes):
  *   - ties in the rounding go to even;
@@ -26,7 +30,12 @@
  *     offline weight packers;
  *   - an all-zero row or group has scale 0 and codes 0;
  *   - W4 codes are chosen against the FP16-rounded group scale that is stored;
- *   - dequantization is evaluated in binary64 and rounded once to FP16.
+ *   - dequantization is evaluated in binary64 and rounded once to FP16;
+ *   - Eq. 3 with alpha = 0.5 is evaluated literally as sqrtf(max|X_j|) / sqrtf(max|W_j|)
+ *     (three correctly rounded binary32 operations), s^-1 as the binary32 quotient 1 / s;
+ *     a channel whose activation or weight maximum is 0 gets s = 1;
+ *   - the smoothed value X[m,k] * s^-1[k] (or W[n,k] * s[k]) is one binary32 product of the
+ *     exact FP16 value and the factor; it is NOT rounded back to FP16.
  *
  * Arithmetic notes: integer dot products accumulate in int64 and are checked to
  * fit int32.  All binary32 steps are single IEEE operations (compile with
@@ -102,14 +111,22 @@ static float clampf(float v, float lo, float hi) { return v < lo ? lo : (v > hi 
  *   Q[m,k] = clamp(rne(X[m,k] * (127.5 / a)), -128, 127)
  * x: FP16 bit patterns [M,K] row-major.  q: [M,K].  s_tok: [M].
  */
-int pqo_quantize_act(const uint16_t* x, int64_t M, int64_t K, int8_t* q, float* s_tok) {
+/* The value a quantizer sees: the FP16 element, times the column factor when there is one
+ * (Eq. 3: X S^-1 on the activation side, S W on the weight side). */
+static float smoothed(uint16_t h, const float* col, int64_t k) {
+  float v = pqo_half_to_float(h);
+  return col ? v * col[k] : v;
+}
+
+static int quantize_act_impl(const uint16_t* x, const float* col, int64_t M, int64_t K, int8_t* q,
+                             float* s_tok) {
   if (M < 0 || K <= 0) return PQO_ERR_ARG;
 #pragma omp parallel for schedule(static)
   for (int64_t m = 0; m < M; ++m) {
     const uint16_t* xr = x + m * K;
     float a = 0.0f;
     for (int64_t k = 0; k < K; ++k) {
-      float v = fabsf(pqo_half_to_float(xr[k]));
+      float v = fabsf(smoothed(xr[k], col, k));
       if (v > a) a = v;
     }
     if (a == 0.0f) {
@@ -121,7 +138,7 @@ int pqo_quantize_act(const uint16_t* x, int64_t M, int64_t K, int8_t* q, float* 
     float inv = 127.5f / a;
     s_tok[m] = s;
     for (int64_t k = 0; k < K; ++k) {
-      float t = pqo_half_to_float(xr[k]) * inv;
+      float t = smoothed(xr[k], col, k) * inv;
       float r = nearbyintf(t); /* ties to even */
       q[m * K + k] = (int8_t)clampf(r, -128.0f, 127.0f);
     }
@@ -129,19 +146,30 @@ int pqo_quantize_act(const uint16_t* x, int64_t M, int64_t K, int8_t* q, float* 
   return PQO_OK;
 }
 
+int pqo_quantize_act(const uint16_t* x, int64_t M, int64_t K, int8_t* q, float* s_tok) {
+  return quantize_act_impl(x, 0, M, K, q, s_tok);
+}
+
+/* Eq. 3, activation side: quantize X S^-1.  s_inv: [K] binary32. */
+int pqo_quantize_act_smooth(const uint16_t* x, const float* s_inv, int64_t M, int64_t K, int8_t* q,
+                            float* s_tok) {
+  if (!s_inv) return PQO_ERR_ARG;
+  return quantize_act_impl(x, s_inv, M, K, q, s_tok);
+}
+
 /*
  * Per-output-channel INT8 weight quantization, Eq. 2 with n = 8.
  *   a = max_k |W[n,k]|;  s_ch[n] = a / 127.5;  Wq = clamp(rne(W / s_ch[n]), -128, 127)
  * w: FP16 bit patterns [N,K] (one output channel per row).
  */
-int pqo_pack_w8(const uint16_t* w, int64_t N, int64_t K, int8_t* wq, float* s_ch) {
+static int pack_w8_impl(const uint16_t* w, const float* col, int64_t N, int64_t K, int8_t* wq, float* s_ch) {
   if (N < 0 || K <= 0) return PQO_ERR_ARG;
 #pragma omp parallel for schedule(static)
   for (int64_t n = 0; n < N; ++n) {
     const uint16_t* wr = w + n * K;
     float a = 0.0f;
     for (int64_t k = 0; k < K; ++k) {
-      float v = fabsf(pqo_half_to_float(wr[k]));
+      float v = fabsf(smoothed(wr[k], col, k));
       if (v > a) a = v;
     }
     if (a == 0.0f) {
@@ -152,11 +180,21 @@ int pqo_pack_w8(const uint16_t* w, int64_t N, int64_t K, int8_t* wq, float* s_ch
     float s = a / 127.5f;
     s_ch[n] = s;
     for (int64_t k = 0; k < K; ++k) {
-      float r = nearbyintf(pqo_half_to_float(wr[k]) / s);
+      float r = nearbyintf(smoothed(wr[k], col, k) / s);
       wq[n * K + k] = (int8_t)clampf(r, -128.0f, 127.0f);
     }
   }
   return PQO_OK;
+}
+
+int pqo_pack_w8(const uint16_t* w, int64_t N, int64_t K, int8_t* wq, float* s_ch) {
+  return pack_w8_impl(w, 0, N, K, wq, s_ch);
+}
+
+/* Eq. 3, weight side: quantize S W (W stored [N,K], so s multiplies along k).  s: [K] binary32. */
+int pqo_pack_w8_smooth(const uint16_t* w, const float* s, int64_t N, int64_t K, int8_t* wq, float* s_ch) {
+  if (!s) return PQO_ERR_ARG;
+  return pack_w8_impl(w, s, N, K, wq, s_ch);
 }
 
 /*
@@ -166,8 +204,8 @@ int pqo_pack_w8(const uint16_t* w, int64_t N, int64_t K, int8_t* wq, float* s_ch
  *   code = clamp(rne(W / float(s_grp[n,g])), -8, 7)      (against the stored scale)
  * codes: int8 [N,K] holding values in [-8,7].  s_grp: FP16 bit patterns [N, K/group].
  */
-int pqo_pack_w4(const uint16_t* w, int64_t N, int64_t K, int64_t group, int8_t* codes,
-                uint16_t* s_grp) {
+static int pack_w4_impl(const uint16_t* w, const float* col, int64_t N, int64_t K, int64_t group, int8_t* codes,
+                        uint16_t* s_grp) {
   if (N < 0 || K <= 0 || group <= 0 || K % group) return PQO_ERR_ARG;
   int64_t G = K / group;
 #pragma omp parallel for schedule(static)
@@ -176,7 +214,7 @@ int pqo_pack_w4(const uint16_t* w, int64_t N, int64_t K, int64_t group, int8_t* 
       const uint16_t* wr = w + n * K + g * group;
       float a = 0.0f;
       for (int64_t k = 0; k < group; ++k) {
-        float v = fabsf(pqo_half_to_float(wr[k]));
+        float v = fabsf(smoothed(wr[k], col, g * group + k));
         if (v > a) a = v;
       }
       uint16_t s16 = pqo_float_to_half_rne(a / 7.5f);
@@ -185,12 +223,54 @@ int pqo_pack_w4(const uint16_t* w, int64_t N, int64_t K, int64_t group, int8_t* 
       for (int64_t k = 0; k < group; ++k) {
         int8_t c = 0;
         if (sf != 0.0f) {
-          float r = nearbyintf(pqo_half_to_float(wr[k]) / sf);
+          float r = nearbyintf(smoothed(wr[k], col, g * group + k) / sf);
           c = (int8_t)clampf(r, -8.0f, 7.0f);
         }
         codes[n * K + g * group + k] = c;
       }
     }
+  }
+  return PQO_OK;
+}
+
+int pqo_pack_w4(const uint16_t* w, int64_t N, int64_t K, int64_t group, int8_t* codes,
+                uint16_t* s_grp) {
+  return pack_w4_impl(w, 0, N, K, group, codes, s_grp);
+}
+
+int pqo_pack_w4_smooth(const uint16_t* w, const float* s, int64_t N, int64_t K, int64_t group, int8_t* codes,
+                       uint16_t* s_grp) {
+  if (!s) return PQO_ERR_ARG;
+  return pack_w4_impl(w, s, N, K, group, codes, s_grp);
+}
+
+/* Calibration statistic of Eq. 3: max over rows of |A[r,k]| for every column k.  a: FP16 [R,K]. */
+int pqo_col_absmax(const uint16_t* a, int64_t R, int64_t K, float* out) {
+  if (R < 0 || K <= 0) return PQO_ERR_ARG;
+  for (int64_t k = 0; k < K; ++k) out[k] = 0.0f;
+  for (int64_t r = 0; r < R; ++r) {
+    for (int64_t k = 0; k < K; ++k) {
+      float v = fabsf(pqo_half_to_float(a[r * K + k]));
+      if (v > out[k]) out[k] = v;
+    }
+  }
+  return PQO_OK;
+}
+
+/* Eq. 3 with alpha = 0.5:  s_j = max|X_j|^(1/2) / max|W_j|^(1/2),  s_inv_j = 1 / s_j.
+ * x_absmax, w_absmax: [K] column maxima (pqo_col_absmax of the calibration activations and of W). */
+int pqo_smooth_scales(const float* x_absmax, const float* w_absmax, int64_t K, float* s, float* s_inv) {
+  if (K <= 0) return PQO_ERR_ARG;
+  for (int64_t k = 0; k < K; ++k) {
+    if (!(x_absmax[k] > 0.0f) || !(w_absmax[k] > 0.0f)) {
+      s[k] = 1.0f;
+      s_inv[k] = 1.0f;
+      continue;
+    }
+    float num = sqrtf(x_absmax[k]);
+    float den = sqrtf(w_absmax[k]);
+    s[k] = num / den;
+    s_inv[k] = 1.0f / s[k];
   }
   return PQO_OK;
 }

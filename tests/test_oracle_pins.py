@@ -369,3 +369,95 @@ def test_end_to_end_error_is_consistent_with_half_step_noise():
     # activation half-step noise against outlier-dominated signal gives a few percent for W8A8;
     # 4-bit weights add roughly (1/sqrt(12)) * s/sigma ~ 10 %.
     assert rel8 < 0.10 and rel8 < rel4 < 0.25
+
+
+# ---------------------------------------------------------------------------- Eq. 3 (SmoothQuant variant)
+
+def test_smooth_scales_closed_forms_alpha_one_half():
+    # s_j = sqrt(max|X_j|) / sqrt(max|W_j|): perfect squares give exact values
+    xa = np.array([16.0, 4.0, 9.0, 1.0, 0.25, 0.0, 3.0], np.float32)
+    wa = np.array([4.0, 4.0, 1.0, 4.0, 4.0, 2.0, 0.0], np.float32)
+    s, s_inv = oracle.smooth_scales(xa, wa)
+    assert s.tolist() == [2.0, 1.0, 3.0, 0.5, 0.25, 1.0, 1.0]       # dead channels (a zero maximum) keep s = 1
+    assert s_inv.tolist() == [0.5, 1.0, np.float32(1.0) / np.float32(3.0), 2.0, 4.0, 1.0, 1.0]
+    # the balance Eq. 3 is built for: after smoothing both sides have the same column maximum sqrt(ax * aw)
+    rng = np.random.default_rng(3)
+    xa = rng.uniform(0.1, 60.0, 512).astype(np.float32)
+    wa = rng.uniform(0.01, 0.2, 512).astype(np.float32)
+    s, s_inv = oracle.smooth_scales(xa, wa)
+    geo = np.sqrt(xa.astype(np.float64) * wa.astype(np.float64))
+    assert np.allclose(xa * s_inv, geo, rtol=1e-6) and np.allclose(wa * s, geo, rtol=1e-6)
+
+
+def test_col_absmax_is_the_column_maximum():
+    rng = np.random.default_rng(4)
+    a = (rng.standard_normal((37, 200)) * 3).astype(np.float16)
+    a[5, 7] = -1000.0
+    got = oracle.col_absmax(a)
+    assert np.array_equal(got, np.abs(a.astype(np.float32)).max(axis=0))
+    assert got[7] == 1000.0
+
+
+def test_unit_factors_change_nothing():
+    from paper_2512_23367_b200 import synth
+    x, w = synth.activations(9, 256, seed=11), synth.weights(24, 256, seed=11)
+    one = np.ones(256, np.float32)
+    for plain, smooth in ((oracle.quantize_act(x), oracle.quantize_act(x, one)),
+                          (oracle.pack_w8(w), oracle.pack_w8(w, one)),
+                          (oracle.pack_w4(w, 128), oracle.pack_w4(w, 128, one))):
+        assert np.array_equal(plain[0], smooth[0])
+        assert np.array_equal(plain[1].view(np.uint8), smooth[1].view(np.uint8))
+
+
+def test_power_of_two_factors_reduce_to_the_plain_quantizers():
+    """With s_k = 2^e_k the smoothed values are exactly representable in FP16, so quantizing X S^-1
+    (or S W) must equal the already pinned plain quantizer applied to the pre-multiplied matrix; a
+    factor applied to the wrong axis, inverted, or applied after the maximum fails this."""
+    rng = np.random.default_rng(5)
+    K = 256
+    e = rng.integers(-3, 4, K)
+    f = (2.0 ** e).astype(np.float32)
+    x = rng.integers(-200, 201, (7, K)).astype(np.float16)          # small integers: products stay exact in FP16
+    w = (rng.integers(-60, 61, (12, K)) * 2.0 ** -6).astype(np.float16)
+    for got, want in ((oracle.quantize_act(x, f), oracle.quantize_act((x.astype(np.float32) * f).astype(np.float16))),
+                      (oracle.pack_w8(w, f), oracle.pack_w8((w.astype(np.float32) * f).astype(np.float16))),
+                      (oracle.pack_w4(w, 128, f), oracle.pack_w4((w.astype(np.float32) * f).astype(np.float16), 128))):
+        assert np.array_equal(got[0], want[0])
+        assert np.array_equal(got[1].view(np.uint8), want[1].view(np.uint8))
+    # and the factors really matter here (the test would be vacuous otherwise)
+    assert not np.array_equal(oracle.quantize_act(x, f)[0], oracle.quantize_act(x)[0])
+
+
+def test_smoothed_codes_obey_the_half_step_bound_in_binary32():
+    from paper_2512_23367_b200 import synth
+    x = synth.activations(16, 512, seed=12)
+    s_inv = np.random.default_rng(6).uniform(0.02, 3.0, 512).astype(np.float32)
+    q, s_tok = oracle.quantize_act(x, s_inv)
+    t = x.astype(np.float32) * s_inv                                   # one binary32 product per element
+    err = np.abs(t.astype(np.float64) - q.astype(np.float64) * s_tok[:, None].astype(np.float64))
+    assert (err <= s_tok[:, None].astype(np.float64) * (0.5 + 2.0 ** -14)).all()
+    assert (np.abs(q.astype(np.int16)).max(axis=1) >= 127).all()       # the row maximum maps to the end of the range
+    assert np.array_equal(s_tok, np.abs(t).max(axis=1) / np.float32(127.5))
+
+
+def test_eq3_equivalence_and_smoothing_helps_on_outlier_channels():
+    """Y = (X S^-1)(S W) equals X W exactly in real arithmetic; after quantization the smoothed W4A8
+    product must be CLOSER to X W than the plain one when a few activation channels are outliers
+    (what Eq. 3 is for).  A factor on the wrong side (X S, S^-1 W) would blow the error up instead."""
+    from paper_2512_23367_b200 import synth
+    M, K, N = 64, 1024, 96
+    x, w = synth.activations(M, K, seed=13), synth.weights(N, K, seed=13)
+    exact = x.astype(np.float64) @ w.astype(np.float64).T
+    s, s_inv = oracle.smooth_scales(oracle.col_absmax(x), oracle.col_absmax(w))
+    xs, ws = x.astype(np.float64) * s_inv, w.astype(np.float64) * s
+    assert np.allclose(xs @ ws.T, exact, rtol=0, atol=1e-4 * np.abs(exact).max())   # binary32 factors: s * s_inv ~ 1
+
+    def rel(q, s_tok, codes, sg):
+        _, y = oracle.gemm_w4a8(q, s_tok, codes, sg, 128, want_acc=False)
+        return np.linalg.norm(y.astype(np.float64) - exact) / np.linalg.norm(exact)
+
+    plain = rel(*oracle.quantize_act(x), *oracle.pack_w4(w, 128))
+    smooth = rel(*oracle.quantize_act(x, s_inv), *oracle.pack_w4(w, 128, s))
+    swapped = rel(*oracle.quantize_act(x, s), *oracle.pack_w4(w, 128, s_inv))
+    assert smooth < 0.8 * plain
+    assert swapped > plain
