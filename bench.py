@@ -261,9 +261,11 @@ class LayerBuffers:
     """Device buffers of one decoder layer: inputs, packed weights, scales, outputs."""
 
     def __init__(self, pq, torch, wl, M, dev, src_x, src_w):
-        self.xs, self.qs, self.s_toks, self.groups = [], [], [], layer_plan(wl)
+        self.xs, self.qs, self.s_toks, self.s_invs, self.groups = [], [], [], [], layer_plan(wl)
         for gi, (K, _) in enumerate(self.groups):
             self.xs.append(src_x[gi].clone())
+            # column factors for the Eq. 3 quantizer timing (any positive vector has the same cost)
+            self.s_invs.append(torch.rand((K,), dtype=torch.float32, device=dev) + 0.5)
             self.qs.append(torch.empty((M, K), dtype=torch.int8, device=dev))
             self.s_toks.append(torch.empty((M,), dtype=torch.float32, device=dev))
         self.packed, self.ys = [], []
@@ -306,6 +308,9 @@ def run_ours(args, wl: synth.Workload, M: int):
 
     def run_layer(L: LayerBuffers, only: str | None = None):
         for gi, (K, idxs) in enumerate(L.groups):
+            if only == "quantize_smooth":
+                pq.pq_quantize_act_smooth(L.xs[gi], L.s_invs[gi], L.qs[gi], L.s_toks[gi])
+                continue
             if only != "gemm":
                 pq.pq_quantize_act(L.xs[gi], L.qs[gi], L.s_toks[gi])
             if only == "quantize":
@@ -407,6 +412,7 @@ def run_ours(args, wl: synth.Workload, M: int):
 
     gemm_avg_ms, gemm_launches = time_kind(kind_graphs("gemm"), gemm_per_layer)
     quant_avg_ms, quant_launches = time_kind(kind_graphs("quantize"), len(groups))
+    smooth_avg_ms, _ = time_kind(kind_graphs("quantize_smooth"), len(groups), budget_ms=200.0)
 
     # ---- context (not a target): the same seven shapes as FP16 GEMMs from the vendor library
     # (torch.matmul -> cuBLAS), the comparison the paper's prefill table makes on its own hardware.
@@ -441,6 +447,8 @@ def run_ours(args, wl: synth.Workload, M: int):
     gemm_tops = ops / (gemm_avg_ms * gemm_per_layer * 1e-3) / 1e12
     sbytes = step_bytes(wl, M)
     quant_gbs = sbytes["quantize"] / (quant_avg_ms * len(groups) * 1e-3) / 1e9
+    smooth_bytes = sbytes["quantize"] + sum(4 * K for K, _ in groups)   # + the [K] FP32 factor vector per call
+    smooth_gbs = smooth_bytes / (smooth_avg_ms * len(groups) * 1e-3) / 1e9
 
     # ---- end to end: pinned host inputs -> device -> quantize + GEMMs -> pinned host outputs
     L0 = layers[0]
@@ -549,6 +557,9 @@ def run_ours(args, wl: synth.Workload, M: int):
             "fp16_context": fp16_ctx,
             "quantize": {"achieved_gbs": quant_gbs, "frac_of_hbm": quant_gbs / float(peaks["hbm_gbs"]),
                          "avg_launch_us": quant_avg_ms * 1e3, "launches_timed": quant_launches},
+            "quantize_smooth": {"achieved_gbs": smooth_gbs, "frac_of_hbm": smooth_gbs / float(peaks["hbm_gbs"]),
+                                "avg_launch_us": smooth_avg_ms * 1e3,
+                                "what": "pq_quantize_act_smooth (Eq. 3: X S^-1) on the same inputs; not part of the step"},
             "e2e": {"value": e2e_value, "unit": unit, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps, "overlap": "copy-in, compute and copy-out on three streams"},
             "gpu_launches": launches_per_step * args.steps,

@@ -97,6 +97,32 @@ PQ_API int pq_pack_w8(const void* w_f16, int64_t N, int64_t K, void* wq, float* 
 PQ_API int pq_pack_w4(const void* w_f16, int64_t N, int64_t K, int32_t group, void* wp,
                void* s_grp_f16, void* stream);
 
+/*
+ * SmoothQuant variant (Eq. 3: Y = (X S^-1)(S W), S = diag(s), s_j = max|X_j|^alpha / max|W_j|^(1-alpha),
+ * alpha = 0.5 as in the paper's experiments).  The column factors are computed once, offline, from
+ * calibration activations; at run time they cost one extra [K] FP32 vector read per call.
+ *
+ *   pq_col_absmax:     out[k] = max_r |A[r,k]| for A FP16 [R,K] row-major (R >= 1, K as for the
+ *                      quantizer); out: [K] FP32.  Run it on calibration activations and on W.
+ *   pq_smooth_scales:  s[k] = sqrt(x_absmax[k]) / sqrt(w_absmax[k]),  s_inv[k] = 1 / s[k]  (each a
+ *                      correctly rounded FP32 operation); a channel with a zero maximum gets 1.
+ *   pq_quantize_act_smooth: pq_quantize_act of X S^-1 -- every element is multiplied by s_inv[k] in
+ *                      FP32 (not rounded to FP16) BEFORE the token maximum is taken.
+ *   pq_pack_w8_smooth / pq_pack_w4_smooth: pq_pack_w8 / pq_pack_w4 of S W (W is [N,K], so s[k]
+ *                      multiplies along K), same outputs and layouts.
+ * s, s_inv: [K] FP32 device vectors, 16-byte aligned.  The GEMM calls are unchanged: codes and scales
+ * produced by the smooth variants go into pq_gemm_w8a8 / pq_gemm_w4a8 as they are.
+ */
+PQ_API int pq_col_absmax(const void* a_f16, int64_t R, int64_t K, float* out, void* stream);
+PQ_API int pq_smooth_scales(const float* x_absmax, const float* w_absmax, int64_t K, float* s, float* s_inv,
+                            void* stream);
+PQ_API int pq_quantize_act_smooth(const void* x_f16, const float* s_inv, int64_t M, int64_t K, int8_t* q,
+                                  float* s_tok, void* stream);
+PQ_API int pq_pack_w8_smooth(const void* w_f16, const float* s, int64_t N, int64_t K, void* wq, float* s_ch,
+                             void* stream);
+PQ_API int pq_pack_w4_smooth(const void* w_f16, const float* s, int64_t N, int64_t K, int32_t group, void* wp,
+                             void* s_grp_f16, void* stream);
+
 PQ_API size_t pq_packed_w8_bytes(int64_t N, int64_t K);
 PQ_API size_t pq_packed_w4_bytes(int64_t N, int64_t K);
 

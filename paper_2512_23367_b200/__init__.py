@@ -12,6 +12,7 @@ from .binding import (  # noqa: F401
     lib,
     pq_acc_w4a8,
     pq_acc_w8a8,
+    pq_col_absmax,
     pq_device_status,
     pq_gemm_w4a8,
     pq_gemm_w4a8_group,
@@ -22,7 +23,9 @@ from .binding import (  # noqa: F401
     pq_pack_w8,
     pq_plan_w8a8,
     pq_quantize_act,
+    pq_quantize_act_smooth,
     pq_set_workspace,
+    pq_smooth_scales,
     pq_unpack_w4,
     pq_unpack_w8,
 )

@@ -36,6 +36,11 @@ SIGNATURES = {
     "pq_gemm_w8a8_noalloc": (ctypes.c_int, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _vp, _vp]),
     "pq_gemm_w8a8_group": (ctypes.c_int, [_vp, _vp, _i32, ctypes.POINTER(_vp), ctypes.POINTER(_vp),
                                           ctypes.POINTER(_i64), ctypes.POINTER(_vp), _i64, _i64, _vp]),
+    "pq_col_absmax": (ctypes.c_int, [_vp, _i64, _i64, _vp, _vp]),
+    "pq_smooth_scales": (ctypes.c_int, [_vp, _vp, _i64, _vp, _vp, _vp]),
+    "pq_quantize_act_smooth": (ctypes.c_int, [_vp, _vp, _i64, _i64, _vp, _vp, _vp]),
+    "pq_pack_w8_smooth": (ctypes.c_int, [_vp, _vp, _i64, _i64, _vp, _vp, _vp]),
+    "pq_pack_w4_smooth": (ctypes.c_int, [_vp, _vp, _i64, _i64, _i32, _vp, _vp, _vp]),
     "pq_gemm_w4a8_group": (ctypes.c_int, [_vp, _vp, _i32, ctypes.POINTER(_vp), ctypes.POINTER(_vp), _i32,
                                           ctypes.POINTER(_i64), ctypes.POINTER(_vp), _i64, _i64, _vp]),
 }
@@ -85,6 +90,13 @@ def _check(call: str, status: int) -> None:
         raise PQError(call, status)
 
 
+def _factors(v: torch.Tensor, K: int, name: str) -> torch.Tensor:
+    v = _dev(v, torch.float32, name)
+    if tuple(v.shape) != (K,):
+        raise ValueError(f"{name}: expected shape [{K}]")
+    return v
+
+
 def pq_quantize_act(x: torch.Tensor, q: torch.Tensor | None = None, s_tok: torch.Tensor | None = None):
     """x f16 [M,K] -> (q int8 [M,K], s_tok f32 [M])."""
     x = _dev(x, torch.float16, "x")
@@ -97,23 +109,67 @@ def pq_quantize_act(x: torch.Tensor, q: torch.Tensor | None = None, s_tok: torch
     return q, s_tok
 
 
-def pq_pack_w8(w: torch.Tensor):
-    """w f16 [N,K] -> (wq opaque uint8 buffer, s_ch f32 [N])."""
+def pq_quantize_act_smooth(x: torch.Tensor, s_inv: torch.Tensor, q: torch.Tensor | None = None,
+                           s_tok: torch.Tensor | None = None):
+    """Quantizes X S^-1 (Eq. 3): x f16 [M,K], s_inv f32 [K] -> (q int8 [M,K], s_tok f32 [M])."""
+    x = _dev(x, torch.float16, "x")
+    M, K = x.shape
+    s_inv = _factors(s_inv, K, "s_inv")
+    if q is None:
+        q = torch.empty((M, K), dtype=torch.int8, device=x.device)
+    if s_tok is None:
+        s_tok = torch.empty((M,), dtype=torch.float32, device=x.device)
+    _check("pq_quantize_act_smooth", lib().pq_quantize_act_smooth(x.data_ptr(), s_inv.data_ptr(), M, K, q.data_ptr(),
+                                                                  s_tok.data_ptr(), _stream()))
+    return q, s_tok
+
+
+def pq_col_absmax(a: torch.Tensor) -> torch.Tensor:
+    """a f16 [R,K] -> f32 [K]: column maxima of |a| (calibration statistic of Eq. 3)."""
+    a = _dev(a, torch.float16, "a")
+    R, K = a.shape
+    out = torch.empty((K,), dtype=torch.float32, device=a.device)
+    _check("pq_col_absmax", lib().pq_col_absmax(a.data_ptr(), R, K, out.data_ptr(), _stream()))
+    return out
+
+
+def pq_smooth_scales(x_absmax: torch.Tensor, w_absmax: torch.Tensor):
+    """Eq. 3 with alpha = 0.5: (s, s_inv) f32 [K] from the column maxima of X and of W."""
+    xa = _dev(x_absmax, torch.float32, "x_absmax")
+    wa = _factors(w_absmax, xa.shape[0], "w_absmax")
+    s, s_inv = torch.empty_like(xa), torch.empty_like(xa)
+    _check("pq_smooth_scales", lib().pq_smooth_scales(xa.data_ptr(), wa.data_ptr(), xa.shape[0], s.data_ptr(),
+                                                      s_inv.data_ptr(), _stream()))
+    return s, s_inv
+
+
+def pq_pack_w8(w: torch.Tensor, smooth: torch.Tensor | None = None):
+    """w f16 [N,K] -> (wq opaque uint8 buffer, s_ch f32 [N]).  With smooth f32 [K]: packs S W (Eq. 3)."""
     w = _dev(w, torch.float16, "w")
     N, K = w.shape
     wq = torch.empty((lib().pq_packed_w8_bytes(N, K),), dtype=torch.uint8, device=w.device)
     s_ch = torch.empty((N,), dtype=torch.float32, device=w.device)
-    _check("pq_pack_w8", lib().pq_pack_w8(w.data_ptr(), N, K, wq.data_ptr(), s_ch.data_ptr(), _stream()))
+    if smooth is None:
+        _check("pq_pack_w8", lib().pq_pack_w8(w.data_ptr(), N, K, wq.data_ptr(), s_ch.data_ptr(), _stream()))
+    else:
+        smooth = _factors(smooth, K, "smooth")
+        _check("pq_pack_w8_smooth", lib().pq_pack_w8_smooth(w.data_ptr(), smooth.data_ptr(), N, K, wq.data_ptr(),
+                                                            s_ch.data_ptr(), _stream()))
     return wq, s_ch
 
 
-def pq_pack_w4(w: torch.Tensor, group: int = GROUP):
-    """w f16 [N,K] -> (wp opaque uint8 buffer, s_grp f16 [K/group, N])."""
+def pq_pack_w4(w: torch.Tensor, group: int = GROUP, smooth: torch.Tensor | None = None):
+    """w f16 [N,K] -> (wp opaque uint8 buffer, s_grp f16 [K/group, N]).  With smooth f32 [K]: packs S W (Eq. 3)."""
     w = _dev(w, torch.float16, "w")
     N, K = w.shape
     wp = torch.empty((lib().pq_packed_w4_bytes(N, K),), dtype=torch.uint8, device=w.device)
     s_grp = torch.empty((max(K // max(group, 1), 1), N), dtype=torch.float16, device=w.device)
-    _check("pq_pack_w4", lib().pq_pack_w4(w.data_ptr(), N, K, group, wp.data_ptr(), s_grp.data_ptr(), _stream()))
+    if smooth is None:
+        _check("pq_pack_w4", lib().pq_pack_w4(w.data_ptr(), N, K, group, wp.data_ptr(), s_grp.data_ptr(), _stream()))
+    else:
+        smooth = _factors(smooth, K, "smooth")
+        _check("pq_pack_w4_smooth", lib().pq_pack_w4_smooth(w.data_ptr(), smooth.data_ptr(), N, K, group, wp.data_ptr(),
+                                                            s_grp.data_ptr(), _stream()))
     return wp, s_grp
 
 

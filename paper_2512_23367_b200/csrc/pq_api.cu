@@ -158,35 +158,84 @@ size_t pq_packed_w4_bytes(int64_t N, int64_t K) {
   return (N > 0 && K > 0) ? static_cast<size_t>(N) * static_cast<size_t>(K) / 2 : 0;
 }
 
-int pq_quantize_act(const void* x_f16, int64_t M, int64_t K, int8_t* q, float* s_tok, void* stream) {
+static int quantize_act_common(const void* x_f16, const float* col, int64_t M, int64_t K, int8_t* q, float* s_tok,
+                               void* stream) {
   if (!x_f16 || !q || !s_tok) return PQ_ERR_NULL;
   int rc = check_rows(M, K);
   if (rc != PQ_OK) return rc;
-  if (!aligned16(x_f16) || !aligned16(q)) return PQ_ERR_ALIGN;
+  if (!aligned16(x_f16) || !aligned16(q) || !aligned16(col)) return PQ_ERR_ALIGN;
   if ((rc = check_arch()) != PQ_OK) return rc;
-  return launch_quantize_act(x_f16, M, K, q, s_tok, false, static_cast<cudaStream_t>(stream));
+  return launch_quantize_act(x_f16, M, K, q, s_tok, false, col, static_cast<cudaStream_t>(stream));
 }
 
-int pq_pack_w8(const void* w_f16, int64_t N, int64_t K, void* wq, float* s_ch, void* stream) {
+int pq_quantize_act(const void* x_f16, int64_t M, int64_t K, int8_t* q, float* s_tok, void* stream) {
+  return quantize_act_common(x_f16, nullptr, M, K, q, s_tok, stream);
+}
+
+int pq_quantize_act_smooth(const void* x_f16, const float* s_inv, int64_t M, int64_t K, int8_t* q, float* s_tok,
+                           void* stream) {
+  if (!s_inv) return PQ_ERR_NULL;
+  return quantize_act_common(x_f16, s_inv, M, K, q, s_tok, stream);
+}
+
+static int pack_w8_common(const void* w_f16, const float* col, int64_t N, int64_t K, void* wq, float* s_ch,
+                          void* stream) {
   if (!w_f16 || !wq || !s_ch) return PQ_ERR_NULL;
   int rc = check_gemm(1, N, K);
   if (rc != PQ_OK) return rc;
-  if (!aligned16(w_f16) || !aligned16(wq)) return PQ_ERR_ALIGN;
+  if (!aligned16(w_f16) || !aligned16(wq) || !aligned16(col)) return PQ_ERR_ALIGN;
   if ((rc = check_arch()) != PQ_OK) return rc;
   // The W8 layout the GEMM reads is the row-major code matrix itself (K contiguous per channel).
-  rc = launch_quantize_act(w_f16, N, K, static_cast<int8_t*>(wq), s_ch, true, static_cast<cudaStream_t>(stream));
+  rc = launch_quantize_act(w_f16, N, K, static_cast<int8_t*>(wq), s_ch, true, col, static_cast<cudaStream_t>(stream));
   return rc != PQ_OK ? rc : launch_pack_fence(static_cast<cudaStream_t>(stream));
 }
 
-int pq_pack_w4(const void* w_f16, int64_t N, int64_t K, int32_t group, void* wp, void* s_grp_f16, void* stream) {
+int pq_pack_w8(const void* w_f16, int64_t N, int64_t K, void* wq, float* s_ch, void* stream) {
+  return pack_w8_common(w_f16, nullptr, N, K, wq, s_ch, stream);
+}
+
+int pq_pack_w8_smooth(const void* w_f16, const float* s, int64_t N, int64_t K, void* wq, float* s_ch, void* stream) {
+  if (!s) return PQ_ERR_NULL;
+  return pack_w8_common(w_f16, s, N, K, wq, s_ch, stream);
+}
+
+static int pack_w4_common(const void* w_f16, const float* col, int64_t N, int64_t K, int32_t group, void* wp,
+                          void* s_grp_f16, void* stream) {
   if (!w_f16 || !wp || !s_grp_f16) return PQ_ERR_NULL;
   int rc = check_gemm(1, N, K);
   if (rc != PQ_OK) return rc;
   if (group != 128 || K % 128 != 0) return PQ_ERR_SHAPE;
   if (!aligned16(w_f16) || !aligned16(wp) || !aligned16(s_grp_f16)) return PQ_ERR_ALIGN;
   if ((rc = check_arch()) != PQ_OK) return rc;
-  rc = launch_pack_w4(w_f16, N, K, wp, s_grp_f16, static_cast<cudaStream_t>(stream));
+  rc = launch_pack_w4(w_f16, N, K, wp, s_grp_f16, col, static_cast<cudaStream_t>(stream));
   return rc != PQ_OK ? rc : launch_pack_fence(static_cast<cudaStream_t>(stream));
+}
+
+int pq_pack_w4(const void* w_f16, int64_t N, int64_t K, int32_t group, void* wp, void* s_grp_f16, void* stream) {
+  return pack_w4_common(w_f16, nullptr, N, K, group, wp, s_grp_f16, stream);
+}
+
+int pq_pack_w4_smooth(const void* w_f16, const float* s, int64_t N, int64_t K, int32_t group, void* wp,
+                      void* s_grp_f16, void* stream) {
+  if (!s) return PQ_ERR_NULL;
+  return pack_w4_common(w_f16, s, N, K, group, wp, s_grp_f16, stream);
+}
+
+int pq_col_absmax(const void* a_f16, int64_t R, int64_t K, float* out, void* stream) {
+  if (!a_f16 || !out) return PQ_ERR_NULL;
+  int rc = check_rows(R, K);
+  if (rc != PQ_OK) return rc;
+  if (!aligned16(a_f16)) return PQ_ERR_ALIGN;
+  if ((rc = check_arch()) != PQ_OK) return rc;
+  return launch_col_absmax(a_f16, R, K, out, static_cast<cudaStream_t>(stream));
+}
+
+int pq_smooth_scales(const float* x_absmax, const float* w_absmax, int64_t K, float* s, float* s_inv, void* stream) {
+  if (!x_absmax || !w_absmax || !s || !s_inv) return PQ_ERR_NULL;
+  if (K < 1 || K >= 131072) return PQ_ERR_SHAPE;
+  const int rc = check_arch();
+  if (rc != PQ_OK) return rc;
+  return launch_smooth_scales(x_absmax, w_absmax, K, s, s_inv, static_cast<cudaStream_t>(stream));
 }
 
 int pq_unpack_w8(const void* wq, int64_t N, int64_t K, int8_t* codes, void* stream) {

@@ -36,10 +36,14 @@ int make_tmap_2d(CUtensorMap* out, const void* base, uint64_t rows, uint64_t col
                  uint32_t box_cols, uint32_t elem_bytes, int swizzle_bytes);
 
 // ---- launchers (each returns a pq_status; all are asynchronous on `stream`) ----
+// col (nullable, [K] FP32): per-column factor applied before the maximum is taken (Eq. 3).
 int launch_quantize_act(const void* x, int64_t M, int64_t K, int8_t* q, float* s, bool divide_by_scale,
-                        cudaStream_t stream);
+                        const float* col, cudaStream_t stream);
 int launch_pack_fence(cudaStream_t stream);
-int launch_pack_w4(const void* w, int64_t N, int64_t K, void* wp, void* s_grp, cudaStream_t stream);
+int launch_pack_w4(const void* w, int64_t N, int64_t K, void* wp, void* s_grp, const float* col,
+                   cudaStream_t stream);
+int launch_col_absmax(const void* a, int64_t R, int64_t K, float* out, cudaStream_t stream);
+int launch_smooth_scales(const float* xa, const float* wa, int64_t K, float* s, float* s_inv, cudaStream_t stream);
 int launch_unpack_w4(const void* wp, int64_t N, int64_t K, int8_t* codes, cudaStream_t stream);
 
 // Prefill-shaped W8A8 GEMM (tcgen05 kind::i8).  Exactly one of y / acc is non-null.

@@ -22,20 +22,49 @@ __device__ __forceinline__ float absmax8(const uint4& v) {
 
 // Eq. 1 for one value: round-half-to-even of the scaled value, clamped to [-128, 127].
 template <bool kDivide>
-__device__ __forceinline__ int code8(__half x, float f) {
-  float t = kDivide ? __fdiv_rn(__half2float(x), f) : __fmul_rn(__half2float(x), f);
+__device__ __forceinline__ int code8(float x, float f) {
+  float t = kDivide ? __fdiv_rn(x, f) : __fmul_rn(x, f);
   int r = __float2int_rn(t);
   return max(-128, min(127, r));
 }
 
-template <bool kDivide>
-__device__ __forceinline__ uint2 quantize8(const uint4& v, float f) {
+// The eight values of a 16-byte chunk as the quantizer sees them: the FP16 elements, times the
+// column factors of Eq. 3 (one FP32 product each, not rounded back to FP16) when kSmooth.
+template <bool kSmooth>
+__device__ __forceinline__ void values8(const uint4& v, const float4* __restrict__ col, int chunk, float (&t)[8]) {
   const __half* h = reinterpret_cast<const __half*>(&v);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) t[i] = __half2float(h[i]);
+  if constexpr (kSmooth) {
+    const float4 c0 = __ldg(col + 2 * chunk), c1 = __ldg(col + 2 * chunk + 1);
+    t[0] = __fmul_rn(t[0], c0.x); t[1] = __fmul_rn(t[1], c0.y); t[2] = __fmul_rn(t[2], c0.z); t[3] = __fmul_rn(t[3], c0.w);
+    t[4] = __fmul_rn(t[4], c1.x); t[5] = __fmul_rn(t[5], c1.y); t[6] = __fmul_rn(t[6], c1.z); t[7] = __fmul_rn(t[7], c1.w);
+  }
+}
+
+template <bool kSmooth>
+__device__ __forceinline__ float absmax8v(const uint4& v, const float4* __restrict__ col, int chunk) {
+  if constexpr (!kSmooth) {
+    return absmax8(v);
+  } else {
+    float t[8];
+    values8<true>(v, col, chunk, t);
+    float a = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) a = fmaxf(a, fabsf(t[i]));
+    return a;
+  }
+}
+
+template <bool kDivide, bool kSmooth>
+__device__ __forceinline__ uint2 quantize8(const uint4& v, float f, const float4* __restrict__ col, int chunk) {
+  float t[8];
+  values8<kSmooth>(v, col, chunk, t);
   uint32_t lo = 0, hi = 0;
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    lo |= static_cast<uint32_t>(code8<kDivide>(h[i], f) & 0xff) << (8 * i);
-    hi |= static_cast<uint32_t>(code8<kDivide>(h[4 + i], f) & 0xff) << (8 * i);
+    lo |= static_cast<uint32_t>(code8<kDivide>(t[i], f) & 0xff) << (8 * i);
+    hi |= static_cast<uint32_t>(code8<kDivide>(t[4 + i], f) & 0xff) << (8 * i);
   }
   return make_uint2(lo, hi);
 }
@@ -43,10 +72,12 @@ __device__ __forceinline__ uint2 quantize8(const uint4& v, float f) {
 // T threads cooperate on one row; a block of 256 threads handles 256/T rows.
 //   kDivide = false: activations, code = rne(x * (127.5 / a))
 //   kDivide = true : weights,     code = rne(x / (a / 127.5))
-template <int T, bool kDivide>
+//   kSmooth: x is first multiplied by the per-column factor col[k] (Eq. 3: X S^-1 or S W)
+template <int T, bool kDivide, bool kSmooth>
 __global__ void __launch_bounds__(kThreads) quantize_rows_kernel(const uint4* __restrict__ x, int64_t M,
                                                                  int K8, uint2* __restrict__ q,
-                                                                 float* __restrict__ scale) {
+                                                                 float* __restrict__ scale,
+                                                                 const float4* __restrict__ col) {
   constexpr int kRowsPerBlock = kThreads / T;
   constexpr int kWarpsPerRow = T / 32;
   __shared__ float red[kThreads / 32];
@@ -71,10 +102,10 @@ __global__ void __launch_bounds__(kThreads) quantize_rows_kernel(const uint4* __
       int c = t + i * T;
       if (c < K8) {
         cache[i] = __ldg(xr + c);
-        a = fmaxf(a, absmax8(cache[i]));
+        a = fmaxf(a, absmax8v<kSmooth>(cache[i], col, c));
       }
     }
-    for (int c = t + kCached * T; c < K8; c += T) a = fmaxf(a, absmax8(__ldg(xr + c)));
+    for (int c = t + kCached * T; c < K8; c += T) a = fmaxf(a, absmax8v<kSmooth>(__ldg(xr + c), col, c));
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
@@ -100,13 +131,13 @@ __global__ void __launch_bounds__(kThreads) quantize_rows_kernel(const uint4* __
 #pragma unroll
   for (int i = 0; i < kCached; ++i) {
     int c = t + i * T;
-    if (c < K8) qr[c] = quantize8<kDivide>(cache[i], f);
+    if (c < K8) qr[c] = quantize8<kDivide, kSmooth>(cache[i], f, col, c);
   }
-  for (int c = t + kCached * T; c < K8; c += T) qr[c] = quantize8<kDivide>(__ldg(xr + c), f);
+  for (int c = t + kCached * T; c < K8; c += T) qr[c] = quantize8<kDivide, kSmooth>(__ldg(xr + c), f, col, c);
 }
 
-template <int T, bool kDivide>
-int launch_rows_team(const uint4* xp, int64_t M, int K8, uint2* qp, float* s, cudaStream_t stream) {
+template <int T, bool kDivide, bool kSmooth>
+int launch_rows_team(const uint4* xp, int64_t M, int K8, uint2* qp, float* s, const float4* col, cudaStream_t stream) {
   constexpr int kRowsPerBlock = kThreads / T;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(static_cast<unsigned>((M + kRowsPerBlock - 1) / kRowsPerBlock), 1, 1);
@@ -118,19 +149,20 @@ int launch_rows_team(const uint4* xp, int64_t M, int K8, uint2* qp, float* s, cu
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = (!kDivide && pdl_enabled()) ? 1 : 0;
-  return cuda_status(cudaLaunchKernelEx(&cfg, quantize_rows_kernel<T, kDivide>, xp, M, K8, qp, s));
+  return cuda_status(cudaLaunchKernelEx(&cfg, quantize_rows_kernel<T, kDivide, kSmooth>, xp, M, K8, qp, s, col));
 }
 
-template <bool kDivide>
-int launch_rows(const void* x, int64_t M, int64_t K, int8_t* q, float* s, cudaStream_t stream) {
+template <bool kDivide, bool kSmooth>
+int launch_rows(const void* x, int64_t M, int64_t K, int8_t* q, float* s, const float* col, cudaStream_t stream) {
   const int K8 = static_cast<int>(K / 8);
   const uint4* xp = static_cast<const uint4*>(x);
   uint2* qp = reinterpret_cast<uint2*>(q);
+  const float4* cp = reinterpret_cast<const float4*>(col);
   // Pick the narrowest row team that still keeps the whole row in registers.
-  if (K8 <= 32 * kCached) return launch_rows_team<32, kDivide>(xp, M, K8, qp, s, stream);
-  if (K8 <= 64 * kCached) return launch_rows_team<64, kDivide>(xp, M, K8, qp, s, stream);
-  if (K8 <= 128 * kCached) return launch_rows_team<128, kDivide>(xp, M, K8, qp, s, stream);
-  return launch_rows_team<256, kDivide>(xp, M, K8, qp, s, stream);
+  if (K8 <= 32 * kCached) return launch_rows_team<32, kDivide, kSmooth>(xp, M, K8, qp, s, cp, stream);
+  if (K8 <= 64 * kCached) return launch_rows_team<64, kDivide, kSmooth>(xp, M, K8, qp, s, cp, stream);
+  if (K8 <= 128 * kCached) return launch_rows_team<128, kDivide, kSmooth>(xp, M, K8, qp, s, cp, stream);
+  return launch_rows_team<256, kDivide, kSmooth>(xp, M, K8, qp, s, cp, stream);
 }
 
 // ---------------------------------------------------------------------------- INT4
@@ -142,9 +174,11 @@ int launch_rows(const void* x, int64_t M, int64_t K, int8_t* q, float* s, cudaSt
 
 // One warp per (output channel n, group g of 128 k).  Lane l owns bytes 2*(l%8), 2*(l%8)+1
 // of 32-k run l/8, i.e. codes k0+b, k0+b+1, k0+16+b, k0+16+b+1.
+// col (nullable): the column factors of Eq. 3; the group maximum and the codes are then those of S W.
 __global__ void __launch_bounds__(kThreads) pack_w4_kernel(const __half* __restrict__ w, int64_t N, int K,
                                                            uint8_t* __restrict__ wp,
-                                                           __half* __restrict__ s_grp) {
+                                                           __half* __restrict__ s_grp,
+                                                           const float* __restrict__ col) {
   const int G = K / 128;
   const int64_t warp = static_cast<int64_t>(blockIdx.x) * (kThreads / 32) + (threadIdx.x >> 5);
   if (warp >= N * G) return;
@@ -156,20 +190,26 @@ __global__ void __launch_bounds__(kThreads) pack_w4_kernel(const __half* __restr
   const __half* wr = w + n * K + k0;
   const __half2 lo = *reinterpret_cast<const __half2*>(wr + b);
   const __half2 hi = *reinterpret_cast<const __half2*>(wr + 16 + b);
-  __half2 m2 = __hmax2(__habs2(lo), __habs2(hi));
-  float a = fmaxf(__low2float(m2), __high2float(m2));
+  float v0 = __low2float(lo), v1 = __high2float(lo), v2 = __low2float(hi), v3 = __high2float(hi);
+  if (col != nullptr) {
+    v0 = __fmul_rn(v0, __ldg(col + k0 + b));
+    v1 = __fmul_rn(v1, __ldg(col + k0 + b + 1));
+    v2 = __fmul_rn(v2, __ldg(col + k0 + 16 + b));
+    v3 = __fmul_rn(v3, __ldg(col + k0 + 16 + b + 1));
+  }
+  float a = fmaxf(fmaxf(fabsf(v0), fabsf(v1)), fmaxf(fabsf(v2), fabsf(v3)));
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
   const __half s16 = __float2half_rn(__fdiv_rn(a, 7.5f));
   const float sf = __half2float(s16);
   if (lane == 0) s_grp[static_cast<int64_t>(g) * N + n] = s16;
-  auto code4 = [sf](__half x) -> uint32_t {
+  auto code4 = [sf](float x) -> uint32_t {
     if (sf == 0.0f) return 0u;
-    int r = __float2int_rn(__fdiv_rn(__half2float(x), sf));
+    int r = __float2int_rn(__fdiv_rn(x, sf));
     return static_cast<uint32_t>(max(-8, min(7, r))) & 0xfu;
   };
-  const uint32_t byte0 = code4(__low2half(lo)) | (code4(__low2half(hi)) << 4);
-  const uint32_t byte1 = code4(__high2half(lo)) | (code4(__high2half(hi)) << 4);
+  const uint32_t byte0 = code4(v0) | (code4(v2) << 4);
+  const uint32_t byte1 = code4(v1) | (code4(v3) << 4);
   uint8_t* out = wp + n * (K / 2) + k0 / 2 + b;
   *reinterpret_cast<uint16_t*>(out) = static_cast<uint16_t>(byte0 | (byte1 << 8));
 }
@@ -203,15 +243,85 @@ int launch_pack_fence(cudaStream_t stream) {
 }
 
 int launch_quantize_act(const void* x, int64_t M, int64_t K, int8_t* q, float* s, bool divide_by_scale,
-                        cudaStream_t stream) {
-  return divide_by_scale ? launch_rows<true>(x, M, K, q, s, stream) : launch_rows<false>(x, M, K, q, s, stream);
+                        const float* col, cudaStream_t stream) {
+  if (col != nullptr) {
+    return divide_by_scale ? launch_rows<true, true>(x, M, K, q, s, col, stream)
+                           : launch_rows<false, true>(x, M, K, q, s, col, stream);
+  }
+  return divide_by_scale ? launch_rows<true, false>(x, M, K, q, s, nullptr, stream)
+                         : launch_rows<false, false>(x, M, K, q, s, nullptr, stream);
 }
 
-int launch_pack_w4(const void* w, int64_t N, int64_t K, void* wp, void* s_grp, cudaStream_t stream) {
+int launch_pack_w4(const void* w, int64_t N, int64_t K, void* wp, void* s_grp, const float* col,
+                   cudaStream_t stream) {
   const int64_t warps = N * (K / 128);
   const unsigned blocks = static_cast<unsigned>((warps + kThreads / 32 - 1) / (kThreads / 32));
   pack_w4_kernel<<<blocks, kThreads, 0, stream>>>(static_cast<const __half*>(w), N, static_cast<int>(K),
-                                                  static_cast<uint8_t*>(wp), static_cast<__half*>(s_grp));
+                                                  static_cast<uint8_t*>(wp), static_cast<__half*>(s_grp), col);
+  return cuda_status(cudaGetLastError());
+}
+
+// ---------------------------------------------------------------------------- Eq. 3 calibration
+namespace {
+
+// Column maxima of |A| for A FP16 [R,K]: a thread owns 8 adjacent columns (one 16-byte chunk) of a
+// strip of rows; non-negative floats order like their bit patterns, so strips merge with atomicMax
+// on the patterns.  out must be zero when the kernel starts.
+constexpr int kStripRows = 64;
+__global__ void __launch_bounds__(kThreads) col_absmax_kernel(const uint4* __restrict__ a, int64_t R, int K8,
+                                                              unsigned int* __restrict__ out) {
+  const int c = blockIdx.x * kThreads + threadIdx.x;
+  if (c >= K8) return;
+  const int64_t r0 = static_cast<int64_t>(blockIdx.y) * kStripRows;
+  const int64_t r1 = r0 + kStripRows < R ? r0 + kStripRows : R;
+  __half2 m[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) m[i] = __float2half2_rn(0.0f);
+  for (int64_t r = r0; r < r1; ++r) {
+    const uint4 v = __ldg(a + r * K8 + c);
+    const __half2* h = reinterpret_cast<const __half2*>(&v);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) m[i] = __hmax2(m[i], __habs2(h[i]));
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    atomicMax(out + 8 * c + 2 * i, __float_as_uint(__low2float(m[i])));
+    atomicMax(out + 8 * c + 2 * i + 1, __float_as_uint(__high2float(m[i])));
+  }
+}
+
+// Eq. 3 with alpha = 1/2, literally: sqrt(max|X_j|) / sqrt(max|W_j|), and its reciprocal; three and
+// one correctly rounded FP32 operations.  A channel with a zero maximum keeps s = 1.
+__global__ void __launch_bounds__(kThreads) smooth_scales_kernel(const float* __restrict__ xa,
+                                                                 const float* __restrict__ wa, int64_t K,
+                                                                 float* __restrict__ s, float* __restrict__ s_inv) {
+  const int64_t k = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x;
+  if (k >= K) return;
+  const float x = xa[k], w = wa[k];
+  float sv = 1.0f, si = 1.0f;
+  if (x > 0.0f && w > 0.0f) {
+    sv = __fdiv_rn(__fsqrt_rn(x), __fsqrt_rn(w));
+    si = __fdiv_rn(1.0f, sv);
+  }
+  s[k] = sv;
+  s_inv[k] = si;
+}
+
+}  // namespace
+
+int launch_col_absmax(const void* a, int64_t R, int64_t K, float* out, cudaStream_t stream) {
+  if (cudaMemsetAsync(out, 0, static_cast<size_t>(K) * sizeof(float), stream) != cudaSuccess) return PQ_ERR_CUDA;
+  const int K8 = static_cast<int>(K / 8);
+  const dim3 grid(static_cast<unsigned>((K8 + kThreads - 1) / kThreads),
+                  static_cast<unsigned>((R + kStripRows - 1) / kStripRows), 1);
+  col_absmax_kernel<<<grid, kThreads, 0, stream>>>(static_cast<const uint4*>(a), R, K8,
+                                                   reinterpret_cast<unsigned int*>(out));
+  return cuda_status(cudaGetLastError());
+}
+
+int launch_smooth_scales(const float* xa, const float* wa, int64_t K, float* s, float* s_inv, cudaStream_t stream) {
+  const unsigned blocks = static_cast<unsigned>((K + kThreads - 1) / kThreads);
+  smooth_scales_kernel<<<blocks, kThreads, 0, stream>>>(xa, wa, K, s, s_inv);
   return cuda_status(cudaGetLastError());
 }
 

@@ -49,6 +49,12 @@ def test_argument_errors_come_back_as_status_codes_without_a_device():
     assert L.pq_gemm_w4a8_group(16, 16, 2, ptrs, holes, 128, cols, ptrs, 4, 128, None) == PQ_ERR_NULL
     assert L.pq_gemm_w4a8_group(16, 16, 2, ptrs, ptrs, 64, cols, ptrs, 4, 128, None) == PQ_ERR_SHAPE    # group != 128
     assert L.pq_gemm_w4a8_group(16, 16, 5, ptrs, ptrs, 128, cols, ptrs, 4, 128, None) == PQ_ERR_SHAPE   # > PQ_MAX_GROUP
+    assert L.pq_quantize_act_smooth(16, None, 4, 64, 16, 16, None) == PQ_ERR_NULL
+    assert L.pq_quantize_act_smooth(16, 8, 4, 64, 16, 16, None) == PQ_ERR_ALIGN     # factor vector
+    assert L.pq_pack_w8_smooth(16, None, 16, 64, 16, 16, None) == PQ_ERR_NULL
+    assert L.pq_pack_w4_smooth(16, 16, 16, 256, 64, 16, 16, None) == PQ_ERR_SHAPE   # group != 128
+    assert L.pq_col_absmax(16, 0, 64, 16, None) == PQ_ERR_SHAPE
+    assert L.pq_smooth_scales(16, 16, 0, 16, 16, None) == PQ_ERR_SHAPE
     assert L.pq_packed_w8_bytes(8, 256) == 2048 and L.pq_packed_w4_bytes(8, 256) == 1024
     assert L.pq_status_str(0) == b"ok" and b"wait" in L.pq_status_str(6)
 
