@@ -53,6 +53,12 @@ def _load():
         lib.pqo_pack_w8_smooth.argtypes = [vp, vp, i64, i64, vp, vp]
         lib.pqo_pack_w4_smooth.argtypes = [vp, vp, i64, i64, i64, vp, vp]
         lib.pqo_col_absmax.argtypes = [vp, i64, i64, vp]
+        lib.pqo_hadamard_block.restype = i64
+        lib.pqo_hadamard_block.argtypes = [i64]
+        lib.pqo_rotate_rows.argtypes = [vp, i64, i64, vp]
+        lib.pqo_quantize_act_hadamard.argtypes = [vp, i64, i64, vp, vp]
+        lib.pqo_pack_w8_hadamard.argtypes = [vp, i64, i64, vp, vp]
+        lib.pqo_pack_w4_hadamard.argtypes = [vp, i64, i64, i64, vp, vp]
         lib.pqo_smooth_scales.argtypes = [vp, vp, i64, vp, vp]
         lib.pqo_nibble_pack.argtypes = [vp, i64, i64, vp]
         lib.pqo_nibble_unpack.argtypes = [vp, i64, i64, vp]
@@ -121,6 +127,52 @@ def quantize_act(x: np.ndarray, s_inv: np.ndarray | None = None):
         s_inv = _col(s_inv, K)
         _check(_load().pqo_quantize_act_smooth(_p(x), _p(s_inv), M, K, _p(q), _p(s)), "quantize_act_smooth")
     return q, s
+
+
+def hadamard_block(K: int) -> int:
+    """Order B of the Hadamard blocks used for rows of length K (Eq. 4): largest power of two dividing K, <= 256."""
+    return int(_load().pqo_hadamard_block(int(K)))
+
+
+def rotate_rows(a: np.ndarray) -> np.ndarray:
+    """a f16 [R,K] -> a H in binary32 [R,K], H = I (x) H_B / sqrt(B) (Eq. 4)."""
+    a = _c(a, np.float16)
+    R, K = a.shape
+    out = np.empty((R, K), np.float32)
+    _check(_load().pqo_rotate_rows(_p(a), R, K, _p(out)), "rotate_rows")
+    return out
+
+
+def quantize_act_hadamard(x: np.ndarray):
+    """Per-token INT8 quantization of X H (Eq. 4): x f16 [M,K] -> (q int8 [M,K], s_tok f32 [M])."""
+    x = _c(x, np.float16)
+    M, K = x.shape
+    q = np.empty((M, K), np.int8)
+    s = np.empty((M,), np.float32)
+    _check(_load().pqo_quantize_act_hadamard(_p(x), M, K, _p(q), _p(s)), "quantize_act_hadamard")
+    return q, s
+
+
+def pack_w8_hadamard(w: np.ndarray):
+    """Per-channel INT8 quantization of W H (rows of W rotated, Eq. 4)."""
+    w = _c(w, np.float16)
+    N, K = w.shape
+    wq = np.empty((N, K), np.int8)
+    s = np.empty((N,), np.float32)
+    _check(_load().pqo_pack_w8_hadamard(_p(w), N, K, _p(wq), _p(s)), "pack_w8_hadamard")
+    return wq, s
+
+
+def pack_w4_hadamard(w: np.ndarray, group: int = 128):
+    """Group-wise INT4 quantization of W H (Eq. 4): (codes int8 [N,K], s_grp f16 [N,K/group])."""
+    w = _c(w, np.float16)
+    N, K = w.shape
+    if K % group:
+        raise OracleError("pack_w4_hadamard: K must be a multiple of the group size")
+    codes = np.empty((N, K), np.int8)
+    s = np.empty((N, K // group), np.float16)
+    _check(_load().pqo_pack_w4_hadamard(_p(w), N, K, group, _p(codes), _p(s)), "pack_w4_hadamard")
+    return codes, s
 
 
 def col_absmax(a: np.ndarray) -> np.ndarray:

@@ -22,6 +22,9 @@
  *     S = diag(s), s_j = max|X_j|^alpha / max|W_j|^(1-alpha), alpha = 0.5.  The column
  *     factors enter the quantizers as an optional per-k multiplier applied in binary32
  *     BEFORE the absolute maximum is taken (the *_smooth entry points).
+ *   - Eq. 4 (Hadamard variant): Y = (X H)(H^T W) with H a normalized Hadamard matrix.  With W
+ *     stored [N,K] both sides are rotated along K: rows of X and rows of W are multiplied by H
+ *     (the *_hadamard entry points), so that (X H)(W H)^T = X W^T.
  *
  * Readings taken where the paper is silent (also listed in the design notes):
  *   - ties in the rounding go to even;
@@ -35,7 +38,13 @@
  *     (three correctly rounded binary32 operations), s^-1 as the binary32 quotient 1 / s;
  *     a channel whose activation or weight maximum is 0 gets s = 1;
  *   - the smoothed value X[m,k] * s^-1[k] (or W[n,k] * s[k]) is one binary32 product of the
- *     exact FP16 value and the factor; it is NOT rounded back to FP16.
+ *     exact FP16 value and the factor; it is NOT rounded back to FP16;
+ *   - Eq. 4 needs a Hadamard matrix of order K, which does not exist for every K of the paper's
+ *     layers (11008 = 2^8 * 43): H is taken block-diagonal, H = I (x) H_B / sqrt(B), with H_B the
+ *     Sylvester matrix of order B = the largest power of two that divides K, at most 256.  It is
+ *     applied as the textbook in-place butterfly (distances 1, 2, 4, ..., B/2 in this order, each
+ *     step a' = a + b, b' = a - b in binary32), then one binary32 product with
+ *     1 / sqrtf(B); the rotated values stay in binary32.
  *
  * Arithmetic notes: integer dot products accumulate in int64 and are checked to
  * fit int32.  All binary32 steps are single IEEE operations (compile with
@@ -48,6 +57,7 @@
  */
 #include <math.h>
 #include <stdint.h>
+#include <stdlib.h>
 #include <string.h>
 #ifdef _OPENMP
 #include <omp.h>
@@ -116,6 +126,129 @@ static float clampf(float v, float lo, float hi) { return v < lo ? lo : (v > hi 
 static float smoothed(uint16_t h, const float* col, int64_t k) {
   float v = pqo_half_to_float(h);
   return col ? v * col[k] : v;
+}
+
+/* Eq. 4: order of the Hadamard blocks for a row of length K (see the readings above). */
+int64_t pqo_hadamard_block(int64_t K) {
+  int64_t B = 1;
+  while (B < 256 && K % (2 * B) == 0) B *= 2;
+  return B;
+}
+
+/* v[0..B) <- v H_B (Sylvester order; H_B is symmetric), unnormalized, in place. */
+static void butterfly(float* v, int64_t B) {
+  for (int64_t h = 1; h < B; h *= 2) {
+    for (int64_t i = 0; i < B; i += 2 * h) {
+      for (int64_t j = i; j < i + h; ++j) {
+        float a = v[j], b = v[j + h];
+        v[j] = a + b;
+        v[j + h] = a - b;
+      }
+    }
+  }
+}
+
+/* out[r,:] = A[r,:] H  for A FP16 [R,K], out binary32 [R,K]. */
+int pqo_rotate_rows(const uint16_t* a, int64_t R, int64_t K, float* out) {
+  if (R < 0 || K <= 0) return PQO_ERR_ARG;
+  int64_t B = pqo_hadamard_block(K);
+  float norm = 1.0f / sqrtf((float)B);
+#pragma omp parallel for schedule(static)
+  for (int64_t r = 0; r < R; ++r) {
+    float* o = out + r * K;
+    for (int64_t k = 0; k < K; ++k) o[k] = pqo_half_to_float(a[r * K + k]);
+    for (int64_t k0 = 0; k0 < K; k0 += B) {
+      butterfly(o + k0, B);
+      for (int64_t k = k0; k < k0 + B; ++k) o[k] = o[k] * norm;
+    }
+  }
+  return PQO_OK;
+}
+
+/* Eq. 1-2 per row on values that are already binary32 (the rotated rows of Eq. 4). */
+static void quantize_row_f32(const float* t, int64_t K, int as_weight, int8_t* q, float* scale) {
+  float a = 0.0f;
+  for (int64_t k = 0; k < K; ++k) {
+    float v = fabsf(t[k]);
+    if (v > a) a = v;
+  }
+  if (a == 0.0f) {
+    *scale = 0.0f;
+    for (int64_t k = 0; k < K; ++k) q[k] = 0;
+    return;
+  }
+  float s = a / 127.5f;
+  float inv = 127.5f / a;
+  *scale = s;
+  for (int64_t k = 0; k < K; ++k) {
+    float r = nearbyintf(as_weight ? t[k] / s : t[k] * inv);   /* the same two forms as the plain quantizers */
+    float c = r < -128.0f ? -128.0f : (r > 127.0f ? 127.0f : r);
+    q[k] = (int8_t)c;
+  }
+}
+
+/* Eq. 4, activation side: per-token INT8 quantization of X H. */
+int pqo_quantize_act_hadamard(const uint16_t* x, int64_t M, int64_t K, int8_t* q, float* s_tok) {
+  if (M < 0 || K <= 0) return PQO_ERR_ARG;
+  float* t = (float*)malloc((size_t)(M > 0 ? M : 1) * (size_t)K * sizeof(float));
+  if (!t) return PQO_ERR_ARG;
+  int rc = pqo_rotate_rows(x, M, K, t);
+  if (rc == PQO_OK) {
+#pragma omp parallel for schedule(static)
+    for (int64_t m = 0; m < M; ++m) quantize_row_f32(t + m * K, K, 0, q + m * K, s_tok + m);
+  }
+  free(t);
+  return rc;
+}
+
+/* Eq. 4, weight side, W8: per-output-channel INT8 quantization of W H (rows of W rotated). */
+int pqo_pack_w8_hadamard(const uint16_t* w, int64_t N, int64_t K, int8_t* wq, float* s_ch) {
+  if (N < 0 || K <= 0) return PQO_ERR_ARG;
+  float* t = (float*)malloc((size_t)(N > 0 ? N : 1) * (size_t)K * sizeof(float));
+  if (!t) return PQO_ERR_ARG;
+  int rc = pqo_rotate_rows(w, N, K, t);
+  if (rc == PQO_OK) {
+#pragma omp parallel for schedule(static)
+    for (int64_t n = 0; n < N; ++n) quantize_row_f32(t + n * K, K, 1, wq + n * K, s_ch + n);
+  }
+  free(t);
+  return rc;
+}
+
+/* Eq. 4, weight side, W4: group-wise INT4 quantization of W H against the stored FP16 scale. */
+int pqo_pack_w4_hadamard(const uint16_t* w, int64_t N, int64_t K, int64_t group, int8_t* codes,
+                         uint16_t* s_grp) {
+  if (N < 0 || K <= 0 || group <= 0 || K % group) return PQO_ERR_ARG;
+  float* t = (float*)malloc((size_t)(N > 0 ? N : 1) * (size_t)K * sizeof(float));
+  if (!t) return PQO_ERR_ARG;
+  int rc = pqo_rotate_rows(w, N, K, t);
+  int64_t G = K / group;
+  if (rc == PQO_OK) {
+#pragma omp parallel for schedule(static)
+    for (int64_t n = 0; n < N; ++n) {
+      for (int64_t g = 0; g < G; ++g) {
+        const float* tr = t + n * K + g * group;
+        float a = 0.0f;
+        for (int64_t k = 0; k < group; ++k) {
+          float v = fabsf(tr[k]);
+          if (v > a) a = v;
+        }
+        uint16_t s16 = pqo_float_to_half_rne(a / 7.5f);
+        float sf = pqo_half_to_float(s16);
+        s_grp[n * G + g] = s16;
+        for (int64_t k = 0; k < group; ++k) {
+          int8_t c = 0;
+          if (sf != 0.0f) {
+            float r = nearbyintf(tr[k] / sf);
+            c = (int8_t)(r < -8.0f ? -8.0f : (r > 7.0f ? 7.0f : r));
+          }
+          codes[n * K + g * group + k] = c;
+        }
+      }
+    }
+  }
+  free(t);
+  return rc;
 }
 
 static int quantize_act_impl(const uint16_t* x, const float* col, int64_t M, int64_t K, int8_t* q,

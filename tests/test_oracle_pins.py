@@ -461,3 +461,88 @@ def test_eq3_equivalence_and_smoothing_helps_on_outlier_channels():
     swapped = rel(*oracle.quantize_act(x, s), *oracle.pack_w4(w, 128, s_inv))
     assert smooth < 0.8 * plain
     assert swapped > plain
+
+
+# ---------------------------------------------------------------------------- Eq. 4 (Hadamard variant)
+
+def test_hadamard_block_order():
+    assert [oracle.hadamard_block(K) for K in (16, 48, 208, 256, 2048, 4096, 6144, 11008)] == \
+        [16, 16, 16, 256, 256, 256, 256, 256]
+
+
+def test_rotation_of_unit_rows_is_the_library_hadamard_matrix():
+    """Row e_k times H is row k of H: compare the whole matrix with scipy's Sylvester construction."""
+    from scipy.linalg import hadamard
+    for K, B in ((16, 16), (64, 64), (256, 256), (48, 16), (512, 256)):
+        eye = np.eye(K, dtype=np.float16)
+        H = oracle.rotate_rows(eye).astype(np.float64)
+        want = np.kron(np.eye(K // B), hadamard(B).astype(np.float64) / np.sqrt(B))
+        assert np.allclose(H, want, rtol=0, atol=1e-7)
+        assert np.allclose(H @ H.T, np.eye(K), atol=1e-6)                 # orthogonal
+        if B in (16, 64, 256):                                           # 1/sqrt(B) is a power of two: exact
+            assert np.array_equal(H, want)
+
+
+def test_rotation_matches_the_dense_product_and_preserves_norms():
+    from scipy.linalg import hadamard
+    rng = np.random.default_rng(21)
+    a = (rng.standard_normal((5, 768)) * 4).astype(np.float16)
+    got = oracle.rotate_rows(a).astype(np.float64)
+    H = np.kron(np.eye(3), hadamard(256) / 16.0)
+    want = a.astype(np.float64) @ H
+    assert np.allclose(got, want, rtol=0, atol=2e-5 * np.abs(want).max())
+    assert np.allclose(np.linalg.norm(got, axis=1), np.linalg.norm(a.astype(np.float64), axis=1), rtol=1e-6)
+    # a lone spike of height A in a block becomes +-A/16 across that block (exactly), nothing elsewhere
+    spike = np.zeros((1, 512), np.float16)
+    spike[0, 300] = 48.0
+    r = oracle.rotate_rows(spike)
+    assert (np.abs(r[0, 256:]) == 3.0).all() and (r[0, :256] == 0).all()
+
+
+def test_hadamard_quantizers_are_the_plain_rule_on_the_rotated_values():
+    """Integer-valued rows keep the rotation exact in binary32 (and, scaled by 16, representable in
+    FP16), so quantizing X H must equal the pinned plain quantizer applied to the rotated matrix."""
+    from scipy.linalg import hadamard
+    rng = np.random.default_rng(22)
+    K = 512
+    H = np.kron(np.eye(2), hadamard(256))
+    x = rng.integers(-3, 4, (6, K)).astype(np.float16) * 16                 # x H / 16 is an integer below 2048
+    xr = (x.astype(np.float64) @ H / 16.0)
+    assert np.array_equal(xr, np.round(xr)) and np.abs(xr).max() < 2048
+    q, s = oracle.quantize_act_hadamard(x)
+    q2, s2 = oracle.quantize_act(xr.astype(np.float16))
+    assert np.array_equal(q, q2) and np.array_equal(s, s2)
+    w = rng.integers(-2, 3, (10, K)).astype(np.float16) * 16
+    wr = (w.astype(np.float64) @ H / 16.0).astype(np.float16)
+    for got, want in ((oracle.pack_w8_hadamard(w), oracle.pack_w8(wr)),
+                      (oracle.pack_w4_hadamard(w, 128), oracle.pack_w4(wr, 128))):
+        assert np.array_equal(got[0], want[0])
+        assert np.array_equal(got[1].view(np.uint8), want[1].view(np.uint8))
+
+
+def test_eq4_equivalence_and_rotation_helps_on_outlier_channels():
+    from paper_2512_23367_b200 import synth
+    M, K, N = 64, 1024, 96
+    x, w = synth.activations(M, K, seed=23), synth.weights(N, K, seed=23)
+    exact = x.astype(np.float64) @ w.astype(np.float64).T
+    xr, wr = oracle.rotate_rows(x).astype(np.float64), oracle.rotate_rows(w).astype(np.float64)
+    assert np.allclose(xr @ wr.T, exact, rtol=0, atol=1e-5 * np.abs(exact).max())    # (X H)(W H)^T = X W^T
+
+    def rel8(q, s_tok, wq, s_ch):
+        _, y = oracle.gemm_w8a8(q, s_tok, wq, s_ch, want_acc=False)
+        return np.linalg.norm(y.astype(np.float64) - exact) / np.linalg.norm(exact)
+
+    def rel4(q, s_tok, codes, sg):
+        _, y = oracle.gemm_w4a8(q, s_tok, codes, sg, 128, want_acc=False)
+        return np.linalg.norm(y.astype(np.float64) - exact) / np.linalg.norm(exact)
+
+    # INT8 x INT8: the error is the activations' (outlier channels set the token scale); spreading every
+    # outlier over its block of 256 removes most of it
+    plain8 = rel8(*oracle.quantize_act(x), *oracle.pack_w8(w))
+    rotated8 = rel8(*oracle.quantize_act_hadamard(x), *oracle.pack_w8_hadamard(w))
+    assert rotated8 < 0.5 * plain8
+    # INT4 weights: Gaussian weights gain nothing from the rotation, so the total only improves a little
+    assert rel4(*oracle.quantize_act_hadamard(x), *oracle.pack_w4_hadamard(w, 128)) < \
+        rel4(*oracle.quantize_act(x), *oracle.pack_w4(w, 128))
+    # rotating only one operand destroys the product
+    assert rel8(*oracle.quantize_act_hadamard(x), *oracle.pack_w8(w)) > 0.5
