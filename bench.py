@@ -311,6 +311,9 @@ def run_ours(args, wl: synth.Workload, M: int):
             if only == "quantize_smooth":
                 pq.pq_quantize_act_smooth(L.xs[gi], L.s_invs[gi], L.qs[gi], L.s_toks[gi])
                 continue
+            if only == "quantize_hadamard":
+                pq.pq_quantize_act_hadamard(L.xs[gi], L.qs[gi], L.s_toks[gi])
+                continue
             if only != "gemm":
                 pq.pq_quantize_act(L.xs[gi], L.qs[gi], L.s_toks[gi])
             if only == "quantize":
@@ -413,6 +416,7 @@ def run_ours(args, wl: synth.Workload, M: int):
     gemm_avg_ms, gemm_launches = time_kind(kind_graphs("gemm"), gemm_per_layer)
     quant_avg_ms, quant_launches = time_kind(kind_graphs("quantize"), len(groups))
     smooth_avg_ms, _ = time_kind(kind_graphs("quantize_smooth"), len(groups), budget_ms=200.0)
+    hadamard_avg_ms, _ = time_kind(kind_graphs("quantize_hadamard"), len(groups), budget_ms=200.0)
 
     # ---- context (not a target): the same seven shapes as FP16 GEMMs from the vendor library
     # (torch.matmul -> cuBLAS), the comparison the paper's prefill table makes on its own hardware.
@@ -449,6 +453,7 @@ def run_ours(args, wl: synth.Workload, M: int):
     quant_gbs = sbytes["quantize"] / (quant_avg_ms * len(groups) * 1e-3) / 1e9
     smooth_bytes = sbytes["quantize"] + sum(4 * K for K, _ in groups)   # + the [K] FP32 factor vector per call
     smooth_gbs = smooth_bytes / (smooth_avg_ms * len(groups) * 1e-3) / 1e9
+    hadamard_gbs = sbytes["quantize"] / (hadamard_avg_ms * len(groups) * 1e-3) / 1e9
 
     # ---- end to end: pinned host inputs -> device -> quantize + GEMMs -> pinned host outputs
     L0 = layers[0]
@@ -560,6 +565,9 @@ def run_ours(args, wl: synth.Workload, M: int):
             "quantize_smooth": {"achieved_gbs": smooth_gbs, "frac_of_hbm": smooth_gbs / float(peaks["hbm_gbs"]),
                                 "avg_launch_us": smooth_avg_ms * 1e3,
                                 "what": "pq_quantize_act_smooth (Eq. 3: X S^-1) on the same inputs; not part of the step"},
+            "quantize_hadamard": {"achieved_gbs": hadamard_gbs, "frac_of_hbm": hadamard_gbs / float(peaks["hbm_gbs"]),
+                                  "avg_launch_us": hadamard_avg_ms * 1e3,
+                                  "what": "pq_quantize_act_hadamard (Eq. 4: X H) on the same inputs; not part of the step"},
             "e2e": {"value": e2e_value, "unit": unit, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps, "overlap": "copy-in, compute and copy-out on three streams"},
             "gpu_launches": launches_per_step * args.steps,

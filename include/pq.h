@@ -123,6 +123,25 @@ PQ_API int pq_pack_w8_smooth(const void* w_f16, const float* s, int64_t N, int64
 PQ_API int pq_pack_w4_smooth(const void* w_f16, const float* s, int64_t N, int64_t K, int32_t group, void* wp,
                              void* s_grp_f16, void* stream);
 
+/*
+ * Hadamard variant (Eq. 4: Y = (X H)(H^T W), H a normalized Hadamard matrix).  With W stored [N,K]
+ * both operands are rotated along K: (X H)(W H)^T = X W^T.  A Hadamard matrix of order K does not
+ * exist for every layer width (11008 = 2^8 * 43), so H = I (x) H_B / sqrt(B) is block diagonal, H_B
+ * the Sylvester matrix of order B = pq_hadamard_block(K) = the largest power of two dividing K, at
+ * most 256.  The rotation is the in-place butterfly (distances 1, 2, ..., B/2 in this order) in FP32
+ * on the exact FP16 inputs, times 1/sqrt(B); the rotated values are quantized from FP32.
+ *   pq_quantize_act_hadamard: pq_quantize_act of X H (on line, fused into the quantizer kernel);
+ *   pq_pack_w8_hadamard / pq_pack_w4_hadamard: pq_pack_w8 / pq_pack_w4 of W H (off line).
+ * Same arguments, outputs and layouts as the plain calls; K <= 16384 (PQ_ERR_SHAPE beyond).  The
+ * GEMM calls are unchanged.  pq_hadamard_block is a host-only query (0 for a K the quantizer rejects).
+ */
+PQ_API int32_t pq_hadamard_block(int64_t K);
+PQ_API int pq_quantize_act_hadamard(const void* x_f16, int64_t M, int64_t K, int8_t* q, float* s_tok,
+                                    void* stream);
+PQ_API int pq_pack_w8_hadamard(const void* w_f16, int64_t N, int64_t K, void* wq, float* s_ch, void* stream);
+PQ_API int pq_pack_w4_hadamard(const void* w_f16, int64_t N, int64_t K, int32_t group, void* wp,
+                               void* s_grp_f16, void* stream);
+
 PQ_API size_t pq_packed_w8_bytes(int64_t N, int64_t K);
 PQ_API size_t pq_packed_w4_bytes(int64_t N, int64_t K);
 

@@ -19,10 +19,14 @@ from .binding import (  # noqa: F401
     pq_gemm_w8a8,
     pq_gemm_w8a8_group,
     pq_gemm_w8a8_noalloc,
+    pq_hadamard_block,
     pq_pack_w4,
+    pq_pack_w4_hadamard,
     pq_pack_w8,
+    pq_pack_w8_hadamard,
     pq_plan_w8a8,
     pq_quantize_act,
+    pq_quantize_act_hadamard,
     pq_quantize_act_smooth,
     pq_set_workspace,
     pq_smooth_scales,

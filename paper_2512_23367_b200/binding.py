@@ -36,6 +36,10 @@ SIGNATURES = {
     "pq_gemm_w8a8_noalloc": (ctypes.c_int, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _vp, _vp]),
     "pq_gemm_w8a8_group": (ctypes.c_int, [_vp, _vp, _i32, ctypes.POINTER(_vp), ctypes.POINTER(_vp),
                                           ctypes.POINTER(_i64), ctypes.POINTER(_vp), _i64, _i64, _vp]),
+    "pq_hadamard_block": (_i32, [_i64]),
+    "pq_quantize_act_hadamard": (ctypes.c_int, [_vp, _i64, _i64, _vp, _vp, _vp]),
+    "pq_pack_w8_hadamard": (ctypes.c_int, [_vp, _i64, _i64, _vp, _vp, _vp]),
+    "pq_pack_w4_hadamard": (ctypes.c_int, [_vp, _i64, _i64, _i32, _vp, _vp, _vp]),
     "pq_col_absmax": (ctypes.c_int, [_vp, _i64, _i64, _vp, _vp]),
     "pq_smooth_scales": (ctypes.c_int, [_vp, _vp, _i64, _vp, _vp, _vp]),
     "pq_quantize_act_smooth": (ctypes.c_int, [_vp, _vp, _i64, _i64, _vp, _vp, _vp]),
@@ -122,6 +126,45 @@ def pq_quantize_act_smooth(x: torch.Tensor, s_inv: torch.Tensor, q: torch.Tensor
     _check("pq_quantize_act_smooth", lib().pq_quantize_act_smooth(x.data_ptr(), s_inv.data_ptr(), M, K, q.data_ptr(),
                                                                   s_tok.data_ptr(), _stream()))
     return q, s_tok
+
+
+def pq_hadamard_block(K: int) -> int:
+    """Order of the Hadamard blocks the Eq. 4 calls use for rows of length K (host-only query)."""
+    return int(lib().pq_hadamard_block(int(K)))
+
+
+def pq_quantize_act_hadamard(x: torch.Tensor, q: torch.Tensor | None = None, s_tok: torch.Tensor | None = None):
+    """Quantizes X H (Eq. 4): x f16 [M,K] -> (q int8 [M,K], s_tok f32 [M])."""
+    x = _dev(x, torch.float16, "x")
+    M, K = x.shape
+    if q is None:
+        q = torch.empty((M, K), dtype=torch.int8, device=x.device)
+    if s_tok is None:
+        s_tok = torch.empty((M,), dtype=torch.float32, device=x.device)
+    _check("pq_quantize_act_hadamard", lib().pq_quantize_act_hadamard(x.data_ptr(), M, K, q.data_ptr(),
+                                                                      s_tok.data_ptr(), _stream()))
+    return q, s_tok
+
+
+def pq_pack_w8_hadamard(w: torch.Tensor):
+    """Packs W H (Eq. 4): w f16 [N,K] -> (wq opaque uint8 buffer, s_ch f32 [N])."""
+    w = _dev(w, torch.float16, "w")
+    N, K = w.shape
+    wq = torch.empty((lib().pq_packed_w8_bytes(N, K),), dtype=torch.uint8, device=w.device)
+    s_ch = torch.empty((N,), dtype=torch.float32, device=w.device)
+    _check("pq_pack_w8_hadamard", lib().pq_pack_w8_hadamard(w.data_ptr(), N, K, wq.data_ptr(), s_ch.data_ptr(), _stream()))
+    return wq, s_ch
+
+
+def pq_pack_w4_hadamard(w: torch.Tensor, group: int = GROUP):
+    """Packs W H (Eq. 4): w f16 [N,K] -> (wp opaque uint8 buffer, s_grp f16 [K/group, N])."""
+    w = _dev(w, torch.float16, "w")
+    N, K = w.shape
+    wp = torch.empty((lib().pq_packed_w4_bytes(N, K),), dtype=torch.uint8, device=w.device)
+    s_grp = torch.empty((max(K // max(group, 1), 1), N), dtype=torch.float16, device=w.device)
+    _check("pq_pack_w4_hadamard", lib().pq_pack_w4_hadamard(w.data_ptr(), N, K, group, wp.data_ptr(), s_grp.data_ptr(),
+                                                            _stream()))
+    return wp, s_grp
 
 
 def pq_col_absmax(a: torch.Tensor) -> torch.Tensor:

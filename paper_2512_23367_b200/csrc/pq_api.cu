@@ -221,6 +221,41 @@ int pq_pack_w4_smooth(const void* w_f16, const float* s, int64_t N, int64_t K, i
   return pack_w4_common(w_f16, s, N, K, group, wp, s_grp_f16, stream);
 }
 
+int32_t pq_hadamard_block(int64_t K) { return (K >= 16 && K % 16 == 0) ? hadamard_block_order(K) : 0; }
+
+int pq_quantize_act_hadamard(const void* x_f16, int64_t M, int64_t K, int8_t* q, float* s_tok, void* stream) {
+  if (!x_f16 || !q || !s_tok) return PQ_ERR_NULL;
+  int rc = check_rows(M, K);
+  if (rc != PQ_OK) return rc;
+  if (K > 16384) return PQ_ERR_SHAPE;
+  if (!aligned16(x_f16) || !aligned16(q)) return PQ_ERR_ALIGN;
+  if ((rc = check_arch()) != PQ_OK) return rc;
+  return launch_quantize_act_hadamard(x_f16, M, K, q, s_tok, false, static_cast<cudaStream_t>(stream));
+}
+
+int pq_pack_w8_hadamard(const void* w_f16, int64_t N, int64_t K, void* wq, float* s_ch, void* stream) {
+  if (!w_f16 || !wq || !s_ch) return PQ_ERR_NULL;
+  int rc = check_gemm(1, N, K);
+  if (rc != PQ_OK) return rc;
+  if (K > 16384) return PQ_ERR_SHAPE;
+  if (!aligned16(w_f16) || !aligned16(wq)) return PQ_ERR_ALIGN;
+  if ((rc = check_arch()) != PQ_OK) return rc;
+  rc = launch_quantize_act_hadamard(w_f16, N, K, static_cast<int8_t*>(wq), s_ch, true, static_cast<cudaStream_t>(stream));
+  return rc != PQ_OK ? rc : launch_pack_fence(static_cast<cudaStream_t>(stream));
+}
+
+int pq_pack_w4_hadamard(const void* w_f16, int64_t N, int64_t K, int32_t group, void* wp, void* s_grp_f16,
+                        void* stream) {
+  if (!w_f16 || !wp || !s_grp_f16) return PQ_ERR_NULL;
+  int rc = check_gemm(1, N, K);
+  if (rc != PQ_OK) return rc;
+  if (group != 128 || K % 128 != 0) return PQ_ERR_SHAPE;
+  if (!aligned16(w_f16) || !aligned16(wp) || !aligned16(s_grp_f16)) return PQ_ERR_ALIGN;
+  if ((rc = check_arch()) != PQ_OK) return rc;
+  rc = launch_pack_w4_hadamard(w_f16, N, K, wp, s_grp_f16, static_cast<cudaStream_t>(stream));
+  return rc != PQ_OK ? rc : launch_pack_fence(static_cast<cudaStream_t>(stream));
+}
+
 int pq_col_absmax(const void* a_f16, int64_t R, int64_t K, float* out, void* stream) {
   if (!a_f16 || !out) return PQ_ERR_NULL;
   int rc = check_rows(R, K);

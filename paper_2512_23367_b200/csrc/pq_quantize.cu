@@ -5,10 +5,20 @@
 //   - group-wise INT4 weight quantization + nibble packing (offline), and its inverse.
 #include <cuda_fp16.h>
 
+#include <cmath>
+
 #include "pq_internal.h"
 #include "pq_ptx.cuh"
 
 namespace pq {
+
+// Order of the Hadamard blocks for rows of length K (Eq. 4): the largest power of two dividing K, at most 256.
+int hadamard_block_order(int64_t K) {
+  int B = 1;
+  while (B < 256 && K % (2 * B) == 0) B *= 2;
+  return B;
+}
+
 namespace {
 
 constexpr int kThreads = 256;
@@ -136,6 +146,140 @@ __global__ void __launch_bounds__(kThreads) quantize_rows_kernel(const uint4* __
   for (int c = t + kCached * T; c < K8; c += T) qr[c] = quantize8<kDivide, kSmooth>(__ldg(xr + c), f, col, c);
 }
 
+// ---------------------------------------------------------------------------- Eq. 4 (Hadamard variant)
+// Rows are multiplied by H = I (x) H_B / sqrt(B) before they are quantized: H_B the Sylvester matrix
+// of order B = largest power of two dividing K (at most 256), applied as the in-place butterfly with
+// distances 1, 2, 4, ..., B/2 in this order.  A thread holds 16-byte chunks (8 consecutive k) and the
+// 32 lanes of a warp hold 32 consecutive chunks, so distances 1, 2, 4 stay inside a thread and
+// 8 .. 128 are lane exchanges at XOR distance 1 .. 16; a block never leaves its warp.
+
+// One chunk: v[0..8) are elements 8*lane .. 8*lane+7 of the warp's 256-element span.
+__device__ __forceinline__ void hadamard_chunk(float (&v)[8], int lane, int chunks_per_block, float norm) {
+#pragma unroll
+  for (int h = 1; h < 8; h <<= 1) {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      if ((j & h) == 0) {
+        const float a = v[j], b = v[j + h];
+        v[j] = __fadd_rn(a, b);
+        v[j + h] = __fsub_rn(a, b);
+      }
+    }
+  }
+  for (int d = 1; d < chunks_per_block; d <<= 1) {
+    const bool upper = (lane & d) != 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const float other = __shfl_xor_sync(0xffffffffu, v[j], d);
+      v[j] = upper ? __fsub_rn(other, v[j]) : __fadd_rn(v[j], other);   // a' = a + b (lower), b' = a - b (upper)
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < 8; ++j) v[j] = __fmul_rn(v[j], norm);
+}
+
+// The row quantizer on rotated rows.  The whole row stays in registers as FP32 (K <= 8 * kCached * T).
+template <int T, bool kDivide>
+__global__ void __launch_bounds__(kThreads) quantize_rows_rot_kernel(const uint4* __restrict__ x, int64_t M,
+                                                                     int K8, uint2* __restrict__ q,
+                                                                     float* __restrict__ scale,
+                                                                     int chunks_per_block, float norm) {
+  constexpr int kRowsPerBlock = kThreads / T;
+  constexpr int kWarpsPerRow = T / 32;
+  __shared__ float red[kThreads / 32];
+
+  const int tid = threadIdx.x;
+  const int t = tid % T;
+  const int lane = tid & 31;
+  const int64_t row = static_cast<int64_t>(blockIdx.x) * kRowsPerBlock + tid / T;
+  const bool live = row < M;          // uniform per warp: a warp never spans two rows
+  const uint4* xr = x + row * K8;
+
+  if constexpr (!kDivide) grid_dep_launch();
+  grid_dep_wait();
+
+  float v[kCached][8];
+  float a = 0.0f;
+#pragma unroll
+  for (int i = 0; i < kCached; ++i) {
+    const int c = t + i * T;
+    uint4 raw = make_uint4(0u, 0u, 0u, 0u);
+    if (live && c < K8) raw = __ldg(xr + c);
+    const __half* h = reinterpret_cast<const __half*>(&raw);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) v[i][j] = __half2float(h[j]);
+    hadamard_chunk(v[i], lane, chunks_per_block, norm);   // all lanes take part in the exchanges
+#pragma unroll
+    for (int j = 0; j < 8; ++j) a = fmaxf(a, fabsf(v[i][j]));
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
+  if constexpr (kWarpsPerRow > 1) {
+    if ((tid & 31) == 0) red[tid >> 5] = a;
+    __syncthreads();
+    const int w0 = (tid / T) * kWarpsPerRow;
+#pragma unroll
+    for (int w = 0; w < kWarpsPerRow; ++w) a = fmaxf(a, red[w0 + w]);
+  }
+  if (!live) return;
+
+  const float s = __fdiv_rn(a, 127.5f);
+  float f;
+  if (kDivide) {
+    f = (a == 0.0f) ? 1.0f : s;
+  } else {
+    f = (a == 0.0f) ? 0.0f : __fdiv_rn(127.5f, a);
+  }
+  if (t == 0) scale[row] = s;
+
+  uint2* qr = q + row * K8;
+#pragma unroll
+  for (int i = 0; i < kCached; ++i) {
+    const int c = t + i * T;
+    if (c < K8) {
+      uint32_t lo = 0, hi = 0;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        lo |= static_cast<uint32_t>(code8<kDivide>(v[i][j], f) & 0xff) << (8 * j);
+        hi |= static_cast<uint32_t>(code8<kDivide>(v[i][4 + j], f) & 0xff) << (8 * j);
+      }
+      qr[c] = make_uint2(lo, hi);
+    }
+  }
+}
+
+template <int T, bool kDivide>
+int launch_rows_rot_team(const uint4* xp, int64_t M, int K8, uint2* qp, float* s, int chunks_per_block, float norm,
+                         cudaStream_t stream) {
+  constexpr int kRowsPerBlock = kThreads / T;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>((M + kRowsPerBlock - 1) / kRowsPerBlock), 1, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = (!kDivide && pdl_enabled()) ? 1 : 0;
+  return cuda_status(cudaLaunchKernelEx(&cfg, quantize_rows_rot_kernel<T, kDivide>, xp, M, K8, qp, s,
+                                        chunks_per_block, norm));
+}
+
+template <bool kDivide>
+int launch_rows_rot(const void* x, int64_t M, int64_t K, int8_t* q, float* s, cudaStream_t stream) {
+  const int K8 = static_cast<int>(K / 8);
+  if (K8 > 256 * kCached) return PQ_ERR_SHAPE;   // the rotated row has to fit the team's registers
+  const int B = hadamard_block_order(K);
+  const float norm = 1.0f / sqrtf(static_cast<float>(B));   // both correctly rounded: the value the butterfly is scaled by
+  const uint4* xp = static_cast<const uint4*>(x);
+  uint2* qp = reinterpret_cast<uint2*>(q);
+  if (K8 <= 32 * kCached) return launch_rows_rot_team<32, kDivide>(xp, M, K8, qp, s, B / 8, norm, stream);
+  if (K8 <= 64 * kCached) return launch_rows_rot_team<64, kDivide>(xp, M, K8, qp, s, B / 8, norm, stream);
+  if (K8 <= 128 * kCached) return launch_rows_rot_team<128, kDivide>(xp, M, K8, qp, s, B / 8, norm, stream);
+  return launch_rows_rot_team<256, kDivide>(xp, M, K8, qp, s, B / 8, norm, stream);
+}
+
 template <int T, bool kDivide, bool kSmooth>
 int launch_rows_team(const uint4* xp, int64_t M, int K8, uint2* qp, float* s, const float4* col, cudaStream_t stream) {
   constexpr int kRowsPerBlock = kThreads / T;
@@ -230,6 +374,65 @@ __global__ void __launch_bounds__(kThreads) unpack_w4_kernel(const uint8_t* __re
   codes[n * K + k0 + 16 + b] = static_cast<int8_t>(hi);
 }
 
+// Group-wise INT4 packing of W H (Eq. 4).  One warp per (output channel n, span of 256 k): lane l holds
+// k = k0 + 8 l .. + 7, rotates with its block (order 128 or 256: K is a multiple of 128), then the two
+// groups of the span (lanes 0-15, 16-31) are quantized like pack_w4_kernel does and the codes are
+// exchanged between lanes l and l ^ 2 to form the packed bytes (byte b of a 32-k run = code(b) |
+// code(16 + b) << 4).
+__global__ void __launch_bounds__(kThreads) pack_w4_rot_kernel(const __half* __restrict__ w, int64_t N, int K,
+                                                               uint8_t* __restrict__ wp,
+                                                               __half* __restrict__ s_grp, int chunks_per_block,
+                                                               float norm) {
+  const int spans = (K + 255) / 256;
+  const int64_t warp = static_cast<int64_t>(blockIdx.x) * (kThreads / 32) + (threadIdx.x >> 5);
+  if (warp >= N * spans) return;
+  const int lane = threadIdx.x & 31;
+  const int64_t n = warp / spans;
+  const int k0 = static_cast<int>(warp % spans) * 256;
+  const int k = k0 + 8 * lane;
+  const bool inside = k < K;                      // K is a multiple of 128: a half-span is all in or all out
+  uint4 raw = make_uint4(0u, 0u, 0u, 0u);
+  if (inside) raw = *reinterpret_cast<const uint4*>(w + n * K + k);
+  const __half* h = reinterpret_cast<const __half*>(&raw);
+  float v[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) v[j] = __half2float(h[j]);
+  hadamard_chunk(v, lane, chunks_per_block, norm);
+  float a = 0.0f;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) a = fmaxf(a, fabsf(v[j]));
+#pragma unroll
+  for (int o = 8; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));   // over the group's 16 lanes
+  const __half s16 = __float2half_rn(__fdiv_rn(a, 7.5f));
+  const float sf = __half2float(s16);
+  const int G = K / 128;
+  if (inside && (lane & 15) == 0) s_grp[static_cast<int64_t>(k / 128) * N + n] = s16;
+  uint32_t mine = 0;                               // eight 4-bit codes, code j in bits 4j .. 4j+3
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    uint32_t c = 0;
+    if (sf != 0.0f) {
+      const int r = __float2int_rn(__fdiv_rn(v[j], sf));
+      c = static_cast<uint32_t>(max(-8, min(7, r))) & 0xfu;
+    }
+    mine |= c << (4 * j);
+  }
+  const uint32_t theirs = __shfl_xor_sync(0xffffffffu, mine, 2);
+  if (inside && (lane & 2) == 0) {
+    // this lane holds positions 8 (l % 4) .. + 7 of its 32-k run, the partner the positions 16 higher
+    uint32_t lo = 0, hi = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      lo |= (((mine >> (4 * j)) & 0xfu) | (((theirs >> (4 * j)) & 0xfu) << 4)) << (8 * j);
+      hi |= (((mine >> (4 * (j + 4))) & 0xfu) | (((theirs >> (4 * (j + 4))) & 0xfu) << 4)) << (8 * j);
+    }
+    const int run = lane >> 2;
+    uint8_t* out = wp + n * (K / 2) + k0 / 2 + run * 16 + (lane & 1) * 8;
+    *reinterpret_cast<uint2*>(out) = make_uint2(lo, hi);
+  }
+  (void)G;
+}
+
 // Launched (plainly, stream-ordered) behind the offline weight kernels.  A GEMM that follows in
 // the stream may request weight tiles before its own wait on its predecessor; with this kernel
 // in between, that predecessor starts only after the packed weights are complete and visible.
@@ -258,6 +461,22 @@ int launch_pack_w4(const void* w, int64_t N, int64_t K, void* wp, void* s_grp, c
   const unsigned blocks = static_cast<unsigned>((warps + kThreads / 32 - 1) / (kThreads / 32));
   pack_w4_kernel<<<blocks, kThreads, 0, stream>>>(static_cast<const __half*>(w), N, static_cast<int>(K),
                                                   static_cast<uint8_t*>(wp), static_cast<__half*>(s_grp), col);
+  return cuda_status(cudaGetLastError());
+}
+
+int launch_quantize_act_hadamard(const void* x, int64_t M, int64_t K, int8_t* q, float* s, bool divide_by_scale,
+                                 cudaStream_t stream) {
+  return divide_by_scale ? launch_rows_rot<true>(x, M, K, q, s, stream) : launch_rows_rot<false>(x, M, K, q, s, stream);
+}
+
+int launch_pack_w4_hadamard(const void* w, int64_t N, int64_t K, void* wp, void* s_grp, cudaStream_t stream) {
+  const int B = hadamard_block_order(K);
+  const float norm = 1.0f / sqrtf(static_cast<float>(B));
+  const int64_t warps = N * ((K + 255) / 256);
+  const unsigned blocks = static_cast<unsigned>((warps + kThreads / 32 - 1) / (kThreads / 32));
+  pack_w4_rot_kernel<<<blocks, kThreads, 0, stream>>>(static_cast<const __half*>(w), N, static_cast<int>(K),
+                                                      static_cast<uint8_t*>(wp), static_cast<__half*>(s_grp), B / 8,
+                                                      norm);
   return cuda_status(cudaGetLastError());
 }
 
