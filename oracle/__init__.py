@@ -52,6 +52,7 @@ def _load():
         lib.pqo_quantize_act_smooth.argtypes = [vp, vp, i64, i64, vp, vp]
         lib.pqo_pack_w8_smooth.argtypes = [vp, vp, i64, i64, vp, vp]
         lib.pqo_pack_w4_smooth.argtypes = [vp, vp, i64, i64, i64, vp, vp]
+        lib.pqo_quantize_act_static.argtypes = [vp, ctypes.c_float, i64, i64, vp, vp]
         lib.pqo_col_absmax.argtypes = [vp, i64, i64, vp]
         lib.pqo_hadamard_block.restype = i64
         lib.pqo_hadamard_block.argtypes = [i64]
@@ -126,6 +127,16 @@ def quantize_act(x: np.ndarray, s_inv: np.ndarray | None = None):
     else:
         s_inv = _col(s_inv, K)
         _check(_load().pqo_quantize_act_smooth(_p(x), _p(s_inv), M, K, _p(q), _p(s)), "quantize_act_smooth")
+    return q, s
+
+
+def quantize_act_static(x: np.ndarray, scale: float):
+    """INT8 codes of x against ONE calibrated scale (static quantization): (q int8 [M,K], s_tok f32 [M] = scale)."""
+    x = _c(x, np.float16)
+    M, K = x.shape
+    q = np.empty((M, K), np.int8)
+    s = np.empty((M,), np.float32)
+    _check(_load().pqo_quantize_act_static(_p(x), float(np.float32(scale)), M, K, _p(q), _p(s)), "quantize_act_static")
     return q, s
 
 

@@ -283,6 +283,26 @@ int pqo_quantize_act(const uint16_t* x, int64_t M, int64_t K, int8_t* q, float* 
   return quantize_act_impl(x, 0, M, K, q, s_tok);
 }
 
+/*
+ * Static (calibrated) activation scale: Eq. 1 with a scale fixed ahead of time instead of the
+ * token's own maximum (the paper's accuracy runs use "calibrated scales"); one scale for the whole
+ * tensor.  code = clamp(rne(X * (1 / s)), -128, 127), 1 / s one binary32 division, the product one
+ * binary32 multiplication; values beyond the calibrated range saturate.  s <= 0 gives codes 0.
+ * s_tok[m] = s for every token, so that the GEMM calls are used unchanged.
+ */
+int pqo_quantize_act_static(const uint16_t* x, float s, int64_t M, int64_t K, int8_t* q, float* s_tok) {
+  if (M < 0 || K <= 0) return PQO_ERR_ARG;
+  float inv = s > 0.0f ? 1.0f / s : 0.0f;
+  for (int64_t m = 0; m < M; ++m) {
+    s_tok[m] = s > 0.0f ? s : 0.0f;
+    for (int64_t k = 0; k < K; ++k) {
+      float r = nearbyintf(pqo_half_to_float(x[m * K + k]) * inv);
+      q[m * K + k] = (int8_t)clampf(r, -128.0f, 127.0f);
+    }
+  }
+  return PQO_OK;
+}
+
 /* Eq. 3, activation side: quantize X S^-1.  s_inv: [K] binary32. */
 int pqo_quantize_act_smooth(const uint16_t* x, const float* s_inv, int64_t M, int64_t K, int8_t* q,
                             float* s_tok) {

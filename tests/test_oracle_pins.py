@@ -546,3 +546,31 @@ def test_eq4_equivalence_and_rotation_helps_on_outlier_channels():
         rel4(*oracle.quantize_act(x), *oracle.pack_w4(w, 128))
     # rotating only one operand destroys the product
     assert rel8(*oracle.quantize_act_hadamard(x), *oracle.pack_w8(w)) > 0.5
+
+
+# ---------------------------------------------------------------------------- static (calibrated) activation scale
+
+def test_static_scale_closed_forms_and_saturation():
+    # s = 2^-2: codes are rne(4 x); ties to even; beyond +-127/4 the codes saturate
+    x = np.array([[0.0, 0.125, 0.375, 0.625, -0.125, -0.375, 1.0, -1.0, 31.75, 31.875, 40.0, -32.0, -32.125, -100.0]],
+                 np.float16)
+    q, s_tok = oracle.quantize_act_static(x, 0.25)
+    assert q[0].tolist() == [0, 0, 2, 2, 0, -2, 4, -4, 127, 127, 127, -128, -128, -128]
+    assert s_tok.tolist() == [0.25]
+    # a scale that is not positive: nothing can be represented
+    q0, s0 = oracle.quantize_act_static(x, 0.0)
+    assert (q0 == 0).all() and s0[0] == 0.0
+
+
+def test_static_scale_error_bound_inside_the_calibrated_range():
+    from paper_2512_23367_b200 import synth
+    x = synth.activations(8, 512, seed=31)
+    s = np.float32(np.abs(x.astype(np.float32)).max() / 127.5)       # calibrated on the data itself: nothing saturates low
+    q, s_tok = oracle.quantize_act_static(x, s)
+    assert (s_tok == s).all()
+    err = np.abs(x.astype(np.float64) - q.astype(np.float64) * float(s))
+    inside = np.abs(x.astype(np.float64)) <= 127.0 * float(s)
+    assert (err[inside] <= float(s) * (0.5 + 2.0 ** -12)).all()
+    # one scale for all tokens: rows without an outlier lose resolution against the per-token rule of Eq. 2
+    qd, sd = oracle.quantize_act(x)
+    assert (sd <= s * (1 + 1e-6)).all()
