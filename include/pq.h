@@ -124,6 +124,18 @@ PQ_API int pq_pack_w4_smooth(const void* w_f16, const float* s, int64_t N, int64
                              void* s_grp_f16, void* stream);
 
 /*
+ * Static (calibrated) activation scale: the paper's accuracy runs quantize with "calibrated scales"
+ * fixed ahead of time instead of the token's own maximum.  One scale for the whole tensor:
+ *   code = clamp(rne(X[m,k] * (1 / s)), -128, 127)   (FP32; values beyond the range saturate),
+ *   s_tok[m] = s for every token, so that the GEMM calls are used unchanged.
+ * scale: DEVICE pointer to one FP32 value (it may be produced by a preceding kernel); s <= 0 gives
+ * codes 0 and token scales 0.  No maximum pass: the kernel reads X once and is launched like
+ * pq_quantize_act.
+ */
+PQ_API int pq_quantize_act_static(const void* x_f16, const float* scale, int64_t M, int64_t K, int8_t* q,
+                                  float* s_tok, void* stream);
+
+/*
  * Hadamard variant (Eq. 4: Y = (X H)(H^T W), H a normalized Hadamard matrix).  With W stored [N,K]
  * both operands are rotated along K: (X H)(W H)^T = X W^T.  A Hadamard matrix of order K does not
  * exist for every layer width (11008 = 2^8 * 43), so H = I (x) H_B / sqrt(B) is block diagonal, H_B

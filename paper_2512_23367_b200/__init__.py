@@ -28,6 +28,7 @@ from .binding import (  # noqa: F401
     pq_quantize_act,
     pq_quantize_act_hadamard,
     pq_quantize_act_smooth,
+    pq_quantize_act_static,
     pq_set_workspace,
     pq_smooth_scales,
     pq_unpack_w4,

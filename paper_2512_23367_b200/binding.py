@@ -36,6 +36,7 @@ SIGNATURES = {
     "pq_gemm_w8a8_noalloc": (ctypes.c_int, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _vp, _vp]),
     "pq_gemm_w8a8_group": (ctypes.c_int, [_vp, _vp, _i32, ctypes.POINTER(_vp), ctypes.POINTER(_vp),
                                           ctypes.POINTER(_i64), ctypes.POINTER(_vp), _i64, _i64, _vp]),
+    "pq_quantize_act_static": (ctypes.c_int, [_vp, _vp, _i64, _i64, _vp, _vp, _vp]),
     "pq_hadamard_block": (_i32, [_i64]),
     "pq_quantize_act_hadamard": (ctypes.c_int, [_vp, _i64, _i64, _vp, _vp, _vp]),
     "pq_pack_w8_hadamard": (ctypes.c_int, [_vp, _i64, _i64, _vp, _vp, _vp]),
@@ -124,6 +125,24 @@ def pq_quantize_act_smooth(x: torch.Tensor, s_inv: torch.Tensor, q: torch.Tensor
     if s_tok is None:
         s_tok = torch.empty((M,), dtype=torch.float32, device=x.device)
     _check("pq_quantize_act_smooth", lib().pq_quantize_act_smooth(x.data_ptr(), s_inv.data_ptr(), M, K, q.data_ptr(),
+                                                                  s_tok.data_ptr(), _stream()))
+    return q, s_tok
+
+
+def pq_quantize_act_static(x: torch.Tensor, scale: torch.Tensor, q: torch.Tensor | None = None,
+                           s_tok: torch.Tensor | None = None):
+    """INT8 codes against one calibrated scale: x f16 [M,K], scale f32 device tensor with one element
+    -> (q int8 [M,K], s_tok f32 [M] filled with the scale)."""
+    x = _dev(x, torch.float16, "x")
+    M, K = x.shape
+    scale = _dev(scale, torch.float32, "scale")
+    if scale.numel() != 1:
+        raise ValueError("scale: one element")
+    if q is None:
+        q = torch.empty((M, K), dtype=torch.int8, device=x.device)
+    if s_tok is None:
+        s_tok = torch.empty((M,), dtype=torch.float32, device=x.device)
+    _check("pq_quantize_act_static", lib().pq_quantize_act_static(x.data_ptr(), scale.data_ptr(), M, K, q.data_ptr(),
                                                                   s_tok.data_ptr(), _stream()))
     return q, s_tok
 

@@ -221,6 +221,16 @@ int pq_pack_w4_smooth(const void* w_f16, const float* s, int64_t N, int64_t K, i
   return pack_w4_common(w_f16, s, N, K, group, wp, s_grp_f16, stream);
 }
 
+int pq_quantize_act_static(const void* x_f16, const float* scale, int64_t M, int64_t K, int8_t* q, float* s_tok,
+                           void* stream) {
+  if (!x_f16 || !scale || !q || !s_tok) return PQ_ERR_NULL;
+  int rc = check_rows(M, K);
+  if (rc != PQ_OK) return rc;
+  if (!aligned16(x_f16) || !aligned16(q)) return PQ_ERR_ALIGN;
+  if ((rc = check_arch()) != PQ_OK) return rc;
+  return launch_quantize_act_static(x_f16, scale, M, K, q, s_tok, static_cast<cudaStream_t>(stream));
+}
+
 int32_t pq_hadamard_block(int64_t K) { return (K >= 16 && K % 16 == 0) ? hadamard_block_order(K) : 0; }
 
 int pq_quantize_act_hadamard(const void* x_f16, int64_t M, int64_t K, int8_t* q, float* s_tok, void* stream) {

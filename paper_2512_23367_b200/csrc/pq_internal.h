@@ -47,6 +47,8 @@ int hadamard_block_order(int64_t K);
 int launch_quantize_act_hadamard(const void* x, int64_t M, int64_t K, int8_t* q, float* s, bool divide_by_scale,
                                  cudaStream_t stream);
 int launch_pack_w4_hadamard(const void* w, int64_t N, int64_t K, void* wp, void* s_grp, cudaStream_t stream);
+int launch_quantize_act_static(const void* x, const float* s_ptr, int64_t M, int64_t K, int8_t* q, float* s_tok,
+                               cudaStream_t stream);
 int launch_col_absmax(const void* a, int64_t R, int64_t K, float* out, cudaStream_t stream);
 int launch_smooth_scales(const float* xa, const float* wa, int64_t K, float* s, float* s_inv, cudaStream_t stream);
 int launch_unpack_w4(const void* wp, int64_t N, int64_t K, int8_t* codes, cudaStream_t stream);

@@ -480,6 +480,49 @@ int launch_pack_w4_hadamard(const void* w, int64_t N, int64_t K, void* wp, void*
   return cuda_status(cudaGetLastError());
 }
 
+// ---------------------------------------------------------------------------- static activation scale
+namespace {
+
+// Eq. 1 against ONE calibrated scale (no maximum pass): a thread owns a 16-byte chunk of 8 elements.
+// *s_ptr is the scale; the token scale vector is filled with it so that the GEMMs run unchanged.
+__global__ void __launch_bounds__(kThreads) quantize_static_kernel(const uint4* __restrict__ x, int64_t M, int K8,
+                                                                   uint2* __restrict__ q, float* __restrict__ s_tok,
+                                                                   const float* __restrict__ s_ptr) {
+  grid_dep_launch();
+  grid_dep_wait();   // x (and possibly the scale) come from the preceding kernel
+  const float s = __ldg(s_ptr);
+  const float sc = s > 0.0f ? s : 0.0f;
+  const float inv = s > 0.0f ? __fdiv_rn(1.0f, s) : 0.0f;
+  const int64_t total = M * K8;
+  for (int64_t i = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x; i < total;
+       i += static_cast<int64_t>(gridDim.x) * kThreads) {
+    q[i] = quantize8<false, false>(__ldg(x + i), inv, nullptr, 0);
+    if (i % K8 == 0) s_tok[i / K8] = sc;
+  }
+}
+
+}  // namespace
+
+int launch_quantize_act_static(const void* x, const float* s_ptr, int64_t M, int64_t K, int8_t* q, float* s_tok,
+                               cudaStream_t stream) {
+  const int K8 = static_cast<int>(K / 8);
+  const int64_t total = M * K8;
+  int64_t blocks = (total + kThreads - 1) / kThreads;
+  const int64_t cap = static_cast<int64_t>(sm_count()) * 16;   // grid-stride beyond a few waves
+  if (blocks > cap) blocks = cap;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(blocks), 1, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl_enabled() ? 1 : 0;
+  return cuda_status(cudaLaunchKernelEx(&cfg, quantize_static_kernel, static_cast<const uint4*>(x), M, K8,
+                                        reinterpret_cast<uint2*>(q), s_tok, s_ptr));
+}
+
 // ---------------------------------------------------------------------------- Eq. 3 calibration
 namespace {
 
