@@ -178,12 +178,15 @@ __device__ __forceinline__ void hadamard_chunk(float (&v)[8], int lane, int chun
   for (int j = 0; j < 8; ++j) v[j] = __fmul_rn(v[j], norm);
 }
 
-// The row quantizer on rotated rows.  The whole row stays in registers as FP32 (K <= 8 * kCached * T).
-template <int T, bool kDivide>
+// The row quantizer on transformed rows: the whole row stays in registers as FP32 (K <= 8 * kCached * T),
+// so the transform is evaluated once.  kRotate: Eq. 4 (block Hadamard rotation); otherwise Eq. 3 (times
+// the column factor col[k]).
+template <int T, bool kDivide, bool kRotate>
 __global__ void __launch_bounds__(kThreads) quantize_rows_rot_kernel(const uint4* __restrict__ x, int64_t M,
                                                                      int K8, uint2* __restrict__ q,
                                                                      float* __restrict__ scale,
-                                                                     int chunks_per_block, float norm) {
+                                                                     int chunks_per_block, float norm,
+                                                                     const float4* __restrict__ col) {
   constexpr int kRowsPerBlock = kThreads / T;
   constexpr int kWarpsPerRow = T / 32;
   __shared__ float red[kThreads / 32];
@@ -205,10 +208,19 @@ __global__ void __launch_bounds__(kThreads) quantize_rows_rot_kernel(const uint4
     const int c = t + i * T;
     uint4 raw = make_uint4(0u, 0u, 0u, 0u);
     if (live && c < K8) raw = __ldg(xr + c);
-    const __half* h = reinterpret_cast<const __half*>(&raw);
+    if constexpr (kRotate) {
+      const __half* h = reinterpret_cast<const __half*>(&raw);
 #pragma unroll
-    for (int j = 0; j < 8; ++j) v[i][j] = __half2float(h[j]);
-    hadamard_chunk(v[i], lane, chunks_per_block, norm);   // all lanes take part in the exchanges
+      for (int j = 0; j < 8; ++j) v[i][j] = __half2float(h[j]);
+      hadamard_chunk(v[i], lane, chunks_per_block, norm);   // all lanes take part in the exchanges
+    } else {
+      if (live && c < K8) {
+        values8<true>(raw, col, c, v[i]);
+      } else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) v[i][j] = 0.0f;
+      }
+    }
 #pragma unroll
     for (int j = 0; j < 8; ++j) a = fmaxf(a, fabsf(v[i][j]));
   }
@@ -248,9 +260,9 @@ __global__ void __launch_bounds__(kThreads) quantize_rows_rot_kernel(const uint4
   }
 }
 
-template <int T, bool kDivide>
+template <int T, bool kDivide, bool kRotate>
 int launch_rows_rot_team(const uint4* xp, int64_t M, int K8, uint2* qp, float* s, int chunks_per_block, float norm,
-                         cudaStream_t stream) {
+                         const float4* col, cudaStream_t stream) {
   constexpr int kRowsPerBlock = kThreads / T;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(static_cast<unsigned>((M + kRowsPerBlock - 1) / kRowsPerBlock), 1, 1);
@@ -262,22 +274,24 @@ int launch_rows_rot_team(const uint4* xp, int64_t M, int K8, uint2* qp, float* s
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = (!kDivide && pdl_enabled()) ? 1 : 0;
-  return cuda_status(cudaLaunchKernelEx(&cfg, quantize_rows_rot_kernel<T, kDivide>, xp, M, K8, qp, s,
-                                        chunks_per_block, norm));
+  return cuda_status(cudaLaunchKernelEx(&cfg, quantize_rows_rot_kernel<T, kDivide, kRotate>, xp, M, K8, qp, s,
+                                        chunks_per_block, norm, col));
 }
 
-template <bool kDivide>
-int launch_rows_rot(const void* x, int64_t M, int64_t K, int8_t* q, float* s, cudaStream_t stream) {
+// col == nullptr: Eq. 4 rotation; otherwise Eq. 3 column factors.
+template <bool kDivide, bool kRotate>
+int launch_rows_f32(const void* x, int64_t M, int64_t K, int8_t* q, float* s, const float* col, cudaStream_t stream) {
   const int K8 = static_cast<int>(K / 8);
-  if (K8 > 256 * kCached) return PQ_ERR_SHAPE;   // the rotated row has to fit the team's registers
+  if (K8 > 256 * kCached) return PQ_ERR_SHAPE;   // the transformed row has to fit the team's registers
   const int B = hadamard_block_order(K);
   const float norm = 1.0f / sqrtf(static_cast<float>(B));   // both correctly rounded: the value the butterfly is scaled by
   const uint4* xp = static_cast<const uint4*>(x);
   uint2* qp = reinterpret_cast<uint2*>(q);
-  if (K8 <= 32 * kCached) return launch_rows_rot_team<32, kDivide>(xp, M, K8, qp, s, B / 8, norm, stream);
-  if (K8 <= 64 * kCached) return launch_rows_rot_team<64, kDivide>(xp, M, K8, qp, s, B / 8, norm, stream);
-  if (K8 <= 128 * kCached) return launch_rows_rot_team<128, kDivide>(xp, M, K8, qp, s, B / 8, norm, stream);
-  return launch_rows_rot_team<256, kDivide>(xp, M, K8, qp, s, B / 8, norm, stream);
+  const float4* cp = reinterpret_cast<const float4*>(col);
+  if (K8 <= 32 * kCached) return launch_rows_rot_team<32, kDivide, kRotate>(xp, M, K8, qp, s, B / 8, norm, cp, stream);
+  if (K8 <= 64 * kCached) return launch_rows_rot_team<64, kDivide, kRotate>(xp, M, K8, qp, s, B / 8, norm, cp, stream);
+  if (K8 <= 128 * kCached) return launch_rows_rot_team<128, kDivide, kRotate>(xp, M, K8, qp, s, B / 8, norm, cp, stream);
+  return launch_rows_rot_team<256, kDivide, kRotate>(xp, M, K8, qp, s, B / 8, norm, cp, stream);
 }
 
 template <int T, bool kDivide, bool kSmooth>
@@ -448,6 +462,11 @@ int launch_pack_fence(cudaStream_t stream) {
 int launch_quantize_act(const void* x, int64_t M, int64_t K, int8_t* q, float* s, bool divide_by_scale,
                         const float* col, cudaStream_t stream) {
   if (col != nullptr) {
+    if (K / 8 <= 256 * kCached) {
+      // the row fits the team's registers as FP32: evaluate x * col[k] once
+      return divide_by_scale ? launch_rows_f32<true, false>(x, M, K, q, s, col, stream)
+                             : launch_rows_f32<false, false>(x, M, K, q, s, col, stream);
+    }
     return divide_by_scale ? launch_rows<true, true>(x, M, K, q, s, col, stream)
                            : launch_rows<false, true>(x, M, K, q, s, col, stream);
   }
@@ -466,7 +485,8 @@ int launch_pack_w4(const void* w, int64_t N, int64_t K, void* wp, void* s_grp, c
 
 int launch_quantize_act_hadamard(const void* x, int64_t M, int64_t K, int8_t* q, float* s, bool divide_by_scale,
                                  cudaStream_t stream) {
-  return divide_by_scale ? launch_rows_rot<true>(x, M, K, q, s, stream) : launch_rows_rot<false>(x, M, K, q, s, stream);
+  return divide_by_scale ? launch_rows_f32<true, true>(x, M, K, q, s, nullptr, stream)
+                         : launch_rows_f32<false, true>(x, M, K, q, s, nullptr, stream);
 }
 
 int launch_pack_w4_hadamard(const void* w, int64_t N, int64_t K, void* wp, void* s_grp, cudaStream_t stream) {
