@@ -12,7 +12,9 @@
 //
 //   warp 0      TMA producer (weights + token tile per 128-deep K block)
 //   warp 1      MMA issuer
-//   warps 2-3   W4 only: nibble -> INT8 widening into the swizzled operand layout
+//   warps 2-3, 8-9   W4 only: nibble -> INT8 widening into the swizzled operand layout; the two
+//               pairs of warps take the K blocks in turn (even / odd), each into its own slot, so
+//               that one pair's proxy fence and hand-over overlap with the other pair's work
 //   warps 4-7   TMEM -> registers (W4: per-group promotion with the row's own group scale),
 //               cross-CTA reduction, dequantization, FP16 store
 #include <cuda_fp16.h>
@@ -26,8 +28,9 @@ namespace {
 constexpr int BW = 128;   // weight rows per tile (TMEM lanes)
 constexpr int BK = 128;   // K per block = one W4 group
 constexpr int UMMA_K = 32;
-constexpr int kNumThreads = 256;
-constexpr int kUnpackThreads = 64;
+constexpr int kNumThreads = 256;      // W8 and 64-token W4; the other W4 variants add two widening warps
+constexpr int kNumThreadsW4 = 320;
+constexpr int kUnpackThreads = 64;    // per K block (one pair of warps)
 constexpr int kMaxSplit = 8;  // portable cluster size
 
 template <int MPAD, bool kW4>
@@ -40,8 +43,12 @@ struct Cfg {
   // Short rings and small footprints: three or four CTAs fit on an SM, so the CTAs of the NEXT
   // launch become resident (and stream their weights) while this launch reduces and stores.
   static constexpr int STAGES = MPAD == 64 ? 4 : 3;
-  static constexpr int kMinCtasPerSm = MPAD == 64 ? 2 : (kW4 ? 3 : 4);
-  static constexpr int A8_SLOTS = kW4 ? 2 : 0;                   // widened weight tiles
+  // W4 with up to 32 tokens: two pairs of widening warps (the 64-token variant needs its registers
+  // for the per-thread partial results and keeps one pair and two co-resident CTAs)
+  static constexpr int kUnpackPairs = (kW4 && MPAD < 64) ? 2 : 1;
+  static constexpr int kThreads = kUnpackPairs == 2 ? kNumThreadsW4 : kNumThreads;
+  static constexpr int kMinCtasPerSm = MPAD == 64 ? 2 : (kW4 ? 2 : 4);
+  static constexpr int A8_SLOTS = kW4 ? 2 : 0;                   // widened weight tiles: one per pair of widening warps
   static constexpr int kA8Bytes = BW * BK;
   static constexpr int SC_SLOTS = kW4 ? 6 : 0;                   // FP32 scale rows (128 floats)
   static constexpr int ACC_SLOTS = kW4 ? 4 : 1;
@@ -93,7 +100,7 @@ __device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t (&r)[MPAD]
 }
 
 template <int MPAD, bool kW4, bool kExportAcc>
-__global__ void __launch_bounds__(kNumThreads, Cfg<MPAD, kW4>::kMinCtasPerSm)
+__global__ void __launch_bounds__(Cfg<MPAD, kW4>::kThreads, Cfg<MPAD, kW4>::kMinCtasPerSm)
 smallm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_q,
               const __grid_constant__ CUtensorMap tm_s, const SmallArgs p) {
   using C = Cfg<MPAD, kW4>;
@@ -240,11 +247,12 @@ smallm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
         if (ok) umma_commit(bar_acc_full);
       }
     }
-  } else if (warp < 4) {
+  } else if (warp < 4 || warp >= 8) {
     // ------------------------------------------------------------ W4: widen nibbles to INT8
     if constexpr (kW4) {
-      const int ut = threadIdx.x - 64;
-      for (int j = 0; j < nkb; ++j) {
+      const int pair = warp >= 8 ? 1 : 0;                      // warps 2-3: even K blocks, warps 8-9: odd ones
+      const int ut = threadIdx.x - (pair ? 256 : 64);
+      for (int j = pair; j < nkb; j += C::kUnpackPairs) {
         const uint32_t it = static_cast<uint32_t>(j);
         const uint32_t s = it % C::STAGES, ph = (it / C::STAGES) & 1u;
         const uint32_t u = it % C::A8_SLOTS, uph = (it / C::A8_SLOTS) & 1u;
@@ -343,7 +351,7 @@ smallm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   // stage ring is free and holds this CTA's partial tile as red[m][n] (32-bit words).
   uint32_t* red = reinterpret_cast<uint32_t*>(smem);
   const bool do_reduce = !(kW4 && kExportAcc);
-  if (do_reduce && warp >= 4) {
+  if (do_reduce && warp >= 4 && warp < 8) {
     const int n_local = (warp & 3) * 32 + lane;
 #pragma unroll
     for (int m = 0; m < MPAD; ++m) red[m * BW + n_local] = P[m];
@@ -351,7 +359,7 @@ smallm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   tc_fence_before_sync();
   __syncwarp();
   cluster_sync_all();
-  if (do_reduce && warp >= 4) {
+  if (do_reduce && warp >= 4 && warp < 8) {
     // Thread t owns four consecutive output channels (one 16-byte word of every part's partial
     // tile) for the rows m = rank + splits * (t / 32 + 4 i): the remote loads of all parts of a row
     // are issued together, so a row costs one distributed-shared-memory round trip, not `splits`.
@@ -431,7 +439,7 @@ int launch_cfg(const CUtensorMap& tw, const CUtensorMap& tq, const CUtensorMap& 
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(static_cast<unsigned>(n_tiles), static_cast<unsigned>(a.splits), 1);
-  cfg.blockDim = dim3(kNumThreads, 1, 1);
+  cfg.blockDim = dim3(C::kThreads, 1, 1);
   cfg.dynamicSmemBytes = C::kDynamic;
   cfg.stream = stream;
   cudaLaunchAttribute attr[2];
