@@ -178,10 +178,68 @@ __device__ __forceinline__ void hadamard_chunk(float (&v)[8], int lane, int chun
   for (int j = 0; j < 8; ++j) v[j] = __fmul_rn(v[j], norm);
 }
 
+// The same transform for a thread that holds C chunks of ONE block: an 8-lane group owns 8*C
+// consecutive chunks (C/4 blocks of 32), lane l' of the group the chunks l' + 8 i.  Element index inside
+// the block = j + 8 l' + 64 (i mod 4): distances 1-4 stay inside a chunk, 8-32 are lane exchanges at XOR
+// distance 1-4, 64 and 128 pair chunks of the same thread -- three exchanges per element instead of five.
+template <int C>
+__device__ __forceinline__ void hadamard_rows(float (&v)[C][8], int lane, int chunks_per_block, float norm) {
+#pragma unroll
+  for (int i = 0; i < C; ++i) {
+#pragma unroll
+    for (int h = 1; h < 8; h <<= 1) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        if ((j & h) == 0) {
+          const float a = v[i][j], b = v[i][j + h];
+          v[i][j] = __fadd_rn(a, b);
+          v[i][j + h] = __fsub_rn(a, b);
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int d = 1; d < 8; d <<= 1) {
+    if (d < chunks_per_block) {
+      const bool upper = (lane & d) != 0;
+#pragma unroll
+      for (int i = 0; i < C; ++i) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const float other = __shfl_xor_sync(0xffffffffu, v[i][j], d);
+          v[i][j] = upper ? __fsub_rn(other, v[i][j]) : __fadd_rn(v[i][j], other);
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int di = 1; di < 4; di <<= 1) {
+    if (8 * di < chunks_per_block) {
+#pragma unroll
+      for (int i = 0; i < C; ++i) {
+        if ((i & di) == 0) {
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const float a = v[i][j], b = v[i + di][j];
+            v[i][j] = __fadd_rn(a, b);
+            v[i + di][j] = __fsub_rn(a, b);
+          }
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < C; ++i) {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) v[i][j] = __fmul_rn(v[i][j], norm);
+  }
+}
+
 // The row quantizer on transformed rows: the whole row stays in registers as FP32 (K <= 8 * kCached * T),
 // so the transform is evaluated once.  kRotate: Eq. 4 (block Hadamard rotation); otherwise Eq. 3 (times
 // the column factor col[k]).
-template <int T, bool kDivide, bool kRotate>
+// C = chunks per thread: 4 where the row allows it (fewer registers, more resident warps), else 8.
+template <int T, int C, bool kDivide, bool kRotate>
 __global__ void __launch_bounds__(kThreads) quantize_rows_rot_kernel(const uint4* __restrict__ x, int64_t M,
                                                                      int K8, uint2* __restrict__ q,
                                                                      float* __restrict__ scale,
@@ -201,18 +259,21 @@ __global__ void __launch_bounds__(kThreads) quantize_rows_rot_kernel(const uint4
   if constexpr (!kDivide) grid_dep_launch();
   grid_dep_wait();
 
-  float v[kCached][8];
+  // Chunk i of this thread.  Eq. 3: chunks t, t + T, ...  Eq. 4: an 8-lane group owns 8 C consecutive chunks
+  // (see hadamard_rows).
+  const int chunk0 = kRotate ? (t & ~31) * C + (lane >> 3) * (8 * C) + (lane & 7) : t;
+  constexpr int kChunkStep = kRotate ? 8 : T;
+  float v[C][8];
   float a = 0.0f;
 #pragma unroll
-  for (int i = 0; i < kCached; ++i) {
-    const int c = t + i * T;
+  for (int i = 0; i < C; ++i) {
+    const int c = chunk0 + i * kChunkStep;
     uint4 raw = make_uint4(0u, 0u, 0u, 0u);
     if (live && c < K8) raw = __ldg(xr + c);
     if constexpr (kRotate) {
       const __half* h = reinterpret_cast<const __half*>(&raw);
 #pragma unroll
       for (int j = 0; j < 8; ++j) v[i][j] = __half2float(h[j]);
-      hadamard_chunk(v[i], lane, chunks_per_block, norm);   // all lanes take part in the exchanges
     } else {
       if (live && c < K8) {
         values8<true>(raw, col, c, v[i]);
@@ -221,6 +282,10 @@ __global__ void __launch_bounds__(kThreads) quantize_rows_rot_kernel(const uint4
         for (int j = 0; j < 8; ++j) v[i][j] = 0.0f;
       }
     }
+  }
+  if constexpr (kRotate) hadamard_rows<C>(v, lane, chunks_per_block, norm);   // all lanes take part in the exchanges
+#pragma unroll
+  for (int i = 0; i < C; ++i) {
 #pragma unroll
     for (int j = 0; j < 8; ++j) a = fmaxf(a, fabsf(v[i][j]));
   }
@@ -246,8 +311,8 @@ __global__ void __launch_bounds__(kThreads) quantize_rows_rot_kernel(const uint4
 
   uint2* qr = q + row * K8;
 #pragma unroll
-  for (int i = 0; i < kCached; ++i) {
-    const int c = t + i * T;
+  for (int i = 0; i < C; ++i) {
+    const int c = chunk0 + i * kChunkStep;
     if (c < K8) {
       uint32_t lo = 0, hi = 0;
 #pragma unroll
@@ -260,7 +325,7 @@ __global__ void __launch_bounds__(kThreads) quantize_rows_rot_kernel(const uint4
   }
 }
 
-template <int T, bool kDivide, bool kRotate>
+template <int T, int C, bool kDivide, bool kRotate>
 int launch_rows_rot_team(const uint4* xp, int64_t M, int K8, uint2* qp, float* s, int chunks_per_block, float norm,
                          const float4* col, cudaStream_t stream) {
   constexpr int kRowsPerBlock = kThreads / T;
@@ -274,7 +339,7 @@ int launch_rows_rot_team(const uint4* xp, int64_t M, int K8, uint2* qp, float* s
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = (!kDivide && pdl_enabled()) ? 1 : 0;
-  return cuda_status(cudaLaunchKernelEx(&cfg, quantize_rows_rot_kernel<T, kDivide, kRotate>, xp, M, K8, qp, s,
+  return cuda_status(cudaLaunchKernelEx(&cfg, quantize_rows_rot_kernel<T, C, kDivide, kRotate>, xp, M, K8, qp, s,
                                         chunks_per_block, norm, col));
 }
 
@@ -288,10 +353,12 @@ int launch_rows_f32(const void* x, int64_t M, int64_t K, int8_t* q, float* s, co
   const uint4* xp = static_cast<const uint4*>(x);
   uint2* qp = reinterpret_cast<uint2*>(q);
   const float4* cp = reinterpret_cast<const float4*>(col);
-  if (K8 <= 32 * kCached) return launch_rows_rot_team<32, kDivide, kRotate>(xp, M, K8, qp, s, B / 8, norm, cp, stream);
-  if (K8 <= 64 * kCached) return launch_rows_rot_team<64, kDivide, kRotate>(xp, M, K8, qp, s, B / 8, norm, cp, stream);
-  if (K8 <= 128 * kCached) return launch_rows_rot_team<128, kDivide, kRotate>(xp, M, K8, qp, s, B / 8, norm, cp, stream);
-  return launch_rows_rot_team<256, kDivide, kRotate>(xp, M, K8, qp, s, B / 8, norm, cp, stream);
+  // the narrowest team that holds the row with four chunks per thread; eight only for the longest rows
+  if (K8 <= 32 * 4) return launch_rows_rot_team<32, 4, kDivide, kRotate>(xp, M, K8, qp, s, B / 8, norm, cp, stream);
+  if (K8 <= 64 * 4) return launch_rows_rot_team<64, 4, kDivide, kRotate>(xp, M, K8, qp, s, B / 8, norm, cp, stream);
+  if (K8 <= 128 * 4) return launch_rows_rot_team<128, 4, kDivide, kRotate>(xp, M, K8, qp, s, B / 8, norm, cp, stream);
+  if (K8 <= 256 * 4) return launch_rows_rot_team<256, 4, kDivide, kRotate>(xp, M, K8, qp, s, B / 8, norm, cp, stream);
+  return launch_rows_rot_team<256, kCached, kDivide, kRotate>(xp, M, K8, qp, s, B / 8, norm, cp, stream);
 }
 
 template <int T, bool kDivide, bool kSmooth>

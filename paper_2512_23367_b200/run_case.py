@@ -15,7 +15,8 @@ import torch
 
 from . import binding as pq
 
-OPS = ("quantize", "gemm_w8a8", "gemm_w4a8")
+QUANT_OPS = ("quantize", "quantize_smooth", "quantize_hadamard", "quantize_static")
+OPS = QUANT_OPS + ("gemm_w8a8", "gemm_w4a8")
 
 
 def main(argv=None):
@@ -34,7 +35,7 @@ def main(argv=None):
     dev = torch.device("cuda", 0)
     torch.manual_seed(0)
     M, K, N, G = a.M, a.K, a.N, max(a.group, 1)
-    per_set = 2 * M * K + M * K + (G * N * K if a.op != "quantize" else 0)
+    per_set = 2 * M * K + M * K + (G * N * K if a.op not in QUANT_OPS else 0)
     sets = a.sets or max(2, min(16, (2 * 126 * 2 ** 20) // max(per_set, 1) + 1))
 
     bufs = []
@@ -42,8 +43,10 @@ def main(argv=None):
         x = torch.randn((M, K), device=dev, dtype=torch.float16)
         x[:, :: max(K // 41, 1)] *= 50
         q, s_tok = pq.pq_quantize_act(x)
-        entry = {"x": x, "q": q, "s_tok": s_tok}
-        if a.op != "quantize":
+        entry = {"x": x, "q": q, "s_tok": s_tok,
+                 "s_inv": torch.rand((K,), device=dev, dtype=torch.float32) + 0.5,
+                 "scale": torch.full((1,), 0.05, device=dev, dtype=torch.float32)}
+        if a.op not in QUANT_OPS:
             entry["w"], entry["y"] = [], []
             for _ in range(G):
                 w = (torch.randn((N, K), device=dev, dtype=torch.float32) * 0.02).half()
@@ -56,6 +59,12 @@ def main(argv=None):
         b = bufs[i % sets]
         if a.op == "quantize":
             pq.pq_quantize_act(b["x"], b["q"], b["s_tok"])
+        elif a.op == "quantize_smooth":
+            pq.pq_quantize_act_smooth(b["x"], b["s_inv"], b["q"], b["s_tok"])
+        elif a.op == "quantize_hadamard":
+            pq.pq_quantize_act_hadamard(b["x"], b["q"], b["s_tok"])
+        elif a.op == "quantize_static":
+            pq.pq_quantize_act_static(b["x"], b["scale"], b["q"], b["s_tok"])
         elif G > 1:
             call = pq.pq_gemm_w8a8_group if a.op == "gemm_w8a8" else pq.pq_gemm_w4a8_group
             call(b["q"], b["s_tok"], [(w[0], w[1], N) for w in b["w"]], b["y"])
@@ -96,8 +105,8 @@ def main(argv=None):
     med, best = us[len(us) // 2], us[0]
     out = {"op": a.op, "M": M, "K": K, "N": N, "group": G, "sets": sets, "us_median": med, "us_min": best,
            "status": pq.pq_device_status()}
-    if a.op == "quantize":
-        out["GBps"] = (3 * M * K + 4 * M) / med / 1e3
+    if a.op in QUANT_OPS:
+        out["GBps"] = (3 * M * K + 4 * M + (4 * K if a.op == "quantize_smooth" else 0)) / med / 1e3
     else:
         out["TOPS"] = 2 * M * G * N * K / med / 1e6
         wbytes = N * K if a.op == "gemm_w8a8" else N * K // 2 + (K // 128) * N * 2
