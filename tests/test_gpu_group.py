@@ -125,3 +125,41 @@ def test_w4a8_small_token_counts_run_member_by_member_with_the_same_result(M):
     out = pq.pq_gemm_w4a8_group(q, s_tok, members)
     for (wp, sg, N), y in zip(members, out):
         assert torch.equal(y, pq.pq_gemm_w4a8(q, s_tok, wp, sg, N))
+
+
+# ---------------------------------------------------------------------------- the benchmark's grouped launches
+
+@pytest.mark.parametrize("bits,M,K,Ns", [
+    (8, 2048, 2048, (2048, 2048, 2048)),      # 1B-class q/k/v
+    (8, 2048, 2048, (6144, 6144)),            # 1B-class gate/up
+    (8, 4096, 4096, (4096, 4096, 4096)),      # 7B-class q/k/v
+    (8, 512, 4096, (11008, 11008)),           # 7B-class gate/up at M = 512
+    (4, 2048, 4096, (4096, 4096, 4096)),      # W4A8 q/k/v
+    (4, 2048, 4096, (11008, 11008)),          # W4A8 gate/up
+])
+def test_benchmark_groups_at_full_size_on_sampled_rows(bits, M, K, Ns):
+    """The grouped launches exactly as bench.py issues them; the oracle checks a seeded sample of token
+    rows (all channels of every member: every tile column, first / last / interior row blocks)."""
+    rng = np.random.default_rng(4600 + M + len(Ns))
+    rows = np.unique(np.concatenate([[0, 127, 128, 255, 256, M - 1], rng.integers(0, M, 10)]))
+    x = synth.activations(M, K, 4700 + M)
+    ws = [synth.weights(N, K, 4800 + i) for i, N in enumerate(Ns)]
+    q, s_tok = pq.pq_quantize_act(torch.from_numpy(x).to(DEV))
+    qo, so = oracle.quantize_act(x[rows])
+    assert np.array_equal(q.cpu().numpy()[rows], qo)
+    if bits == 8:
+        members = [(*pq.pq_pack_w8(torch.from_numpy(w).to(DEV)), N) for w, N in zip(ws, Ns)]
+        out = pq.pq_gemm_w8a8_group(q, s_tok, members)
+    else:
+        members = [(*pq.pq_pack_w4(torch.from_numpy(w).to(DEV)), N) for w, N in zip(ws, Ns)]
+        out = pq.pq_gemm_w4a8_group(q, s_tok, members)
+    torch.cuda.synchronize()
+    assert pq.pq_device_status() == 0
+    for w, y in zip(ws, out):
+        if bits == 8:
+            _, ref = oracle.gemm_w8a8(qo, so, *oracle.pack_w8(w), want_acc=False)
+        else:
+            _, ref = oracle.gemm_w4a8(qo, so, *oracle.pack_w4(w, 128), 128, want_acc=False)
+        g, ref = y.cpu().numpy()[rows].astype(np.float64), ref.astype(np.float64)
+        assert np.isfinite(g).all()
+        assert np.all(np.abs(g - ref) <= REL * np.abs(ref) + ABS)
