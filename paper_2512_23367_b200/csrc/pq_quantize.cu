@@ -34,8 +34,9 @@ __device__ __forceinline__ float absmax8(const uint4& v) {
 template <bool kDivide>
 __device__ __forceinline__ int code8(float x, float f) {
   float t = kDivide ? __fdiv_rn(x, f) : __fmul_rn(x, f);
-  int r = __float2int_rn(t);
-  return max(-128, min(127, r));
+  int r;   // round to nearest even and saturate to [-128, 127] in one conversion
+  asm("cvt.rni.sat.s8.f32 %0, %1;" : "=r"(r) : "f"(t));
+  return r;
 }
 
 // The eight values of a 16-byte chunk as the quantizer sees them: the FP16 elements, times the
