@@ -168,11 +168,13 @@ __device__ __forceinline__ void hadamard_chunk(float (&v)[8], int lane, int chun
     }
   }
   for (int d = 1; d < chunks_per_block; d <<= 1) {
-    const bool upper = (lane & d) != 0;
+    // a' = a + b in the lower lane, b' = a - b in the upper one: other + sign * v, one exactly rounded
+    // fused multiply-add with sign = +-1 (the product is exact, so this IS the sum / difference)
+    const float sign = (lane & d) != 0 ? -1.0f : 1.0f;
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
       const float other = __shfl_xor_sync(0xffffffffu, v[j], d);
-      v[j] = upper ? __fsub_rn(other, v[j]) : __fadd_rn(v[j], other);   // a' = a + b (lower), b' = a - b (upper)
+      v[j] = __fmaf_rn(sign, v[j], other);
     }
   }
 #pragma unroll
@@ -202,13 +204,13 @@ __device__ __forceinline__ void hadamard_rows(float (&v)[C][8], int lane, int ch
 #pragma unroll
   for (int d = 1; d < 8; d <<= 1) {
     if (d < chunks_per_block) {
-      const bool upper = (lane & d) != 0;
+      const float sign = (lane & d) != 0 ? -1.0f : 1.0f;   // other + sign * v: the sum below, the difference above
 #pragma unroll
       for (int i = 0; i < C; ++i) {
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
           const float other = __shfl_xor_sync(0xffffffffu, v[i][j], d);
-          v[i][j] = upper ? __fsub_rn(other, v[i][j]) : __fadd_rn(v[i][j], other);
+          v[i][j] = __fmaf_rn(sign, v[i][j], other);
         }
       }
     }
