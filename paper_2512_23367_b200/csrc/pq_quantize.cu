@@ -30,13 +30,19 @@ __device__ __forceinline__ float absmax8(const uint4& v) {
   return fmaxf(__low2float(m), __high2float(m));
 }
 
-// Eq. 1 for one value: round-half-to-even of the scaled value, clamped to [-128, 127].
+// Eq. 1 for four values at a time.
+// Four scaled values -> four INT8 codes in one word (code i in byte i): round to nearest even, then two
+// packing conversions that saturate to [-128, 127].
 template <bool kDivide>
-__device__ __forceinline__ int code8(float x, float f) {
-  float t = kDivide ? __fdiv_rn(x, f) : __fmul_rn(x, f);
-  int r;   // round to nearest even and saturate to [-128, 127] in one conversion
-  asm("cvt.rni.sat.s8.f32 %0, %1;" : "=r"(r) : "f"(t));
-  return r;
+__device__ __forceinline__ uint32_t codes4(float x0, float x1, float x2, float x3, float f) {
+  const int a0 = __float2int_rn(kDivide ? __fdiv_rn(x0, f) : __fmul_rn(x0, f));
+  const int a1 = __float2int_rn(kDivide ? __fdiv_rn(x1, f) : __fmul_rn(x1, f));
+  const int a2 = __float2int_rn(kDivide ? __fdiv_rn(x2, f) : __fmul_rn(x2, f));
+  const int a3 = __float2int_rn(kDivide ? __fdiv_rn(x3, f) : __fmul_rn(x3, f));
+  uint32_t hi, out;
+  asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(a3), "r"(a2), "r"(0));
+  asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(out) : "r"(a1), "r"(a0), "r"(hi));
+  return out;
 }
 
 // The eight values of a 16-byte chunk as the quantizer sees them: the FP16 elements, times the
@@ -71,13 +77,7 @@ template <bool kDivide, bool kSmooth>
 __device__ __forceinline__ uint2 quantize8(const uint4& v, float f, const float4* __restrict__ col, int chunk) {
   float t[8];
   values8<kSmooth>(v, col, chunk, t);
-  uint32_t lo = 0, hi = 0;
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    lo |= static_cast<uint32_t>(code8<kDivide>(t[i], f) & 0xff) << (8 * i);
-    hi |= static_cast<uint32_t>(code8<kDivide>(t[4 + i], f) & 0xff) << (8 * i);
-  }
-  return make_uint2(lo, hi);
+  return make_uint2(codes4<kDivide>(t[0], t[1], t[2], t[3], f), codes4<kDivide>(t[4], t[5], t[6], t[7], f));
 }
 
 // T threads cooperate on one row; a block of 256 threads handles 256/T rows.
@@ -317,13 +317,8 @@ __global__ void __launch_bounds__(kThreads) quantize_rows_rot_kernel(const uint4
   for (int i = 0; i < C; ++i) {
     const int c = chunk0 + i * kChunkStep;
     if (c < K8) {
-      uint32_t lo = 0, hi = 0;
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        lo |= static_cast<uint32_t>(code8<kDivide>(v[i][j], f) & 0xff) << (8 * j);
-        hi |= static_cast<uint32_t>(code8<kDivide>(v[i][4 + j], f) & 0xff) << (8 * j);
-      }
-      qr[c] = make_uint2(lo, hi);
+      qr[c] = make_uint2(codes4<kDivide>(v[i][0], v[i][1], v[i][2], v[i][3], f),
+                         codes4<kDivide>(v[i][4], v[i][5], v[i][6], v[i][7], f));
     }
   }
 }
