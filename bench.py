@@ -9,8 +9,13 @@ its operands cached.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
 
-Prints ONE JSON line (see the design doc for the field definitions).  `--impl reference` times the
-CPU oracle instead (a deliberately plain program; a baseline, not a target).
+Prints ONE JSON line: `value` = whole-step throughput with inputs resident on the device (TOPS for
+prefill workloads, GB/s of algorithmic bytes for decode workloads); `roofline` = the GEMM launches alone
+against the measured peak; `quantize*` = the quantizer and its variants against the measured copy rate;
+`e2e` = the same step with pinned-host inputs copied in and outputs copied out; `cpu_baseline` = the CPU
+oracle on a row sample; `clocks` = SM clocks and throttle reasons sampled during the timed region.
+`--impl reference` times the CPU oracle instead (a deliberately plain program; a baseline, not a target).
+Linears that share their input are issued as one grouped call (`--no-group`: one call per linear).
 """
 from __future__ import annotations
 
