@@ -458,6 +458,37 @@ def run_ours(args, wl: synth.Workload, M: int):
                     "int8_over_fp16_speedup": (fp16_avg_ms * len(wl.linears)) / (gemm_avg_ms * gemm_per_layer),
                     "paper_context": "the paper reports 1.2x-1.5x INT8 over FP16 end-to-end prefill on Atlas A2"}
         del xs16, ws16, ys16, gs16
+        # The vendor library's own INT8 GEMM (torch._int_mm -> cuBLASLt, INT32 output, no dequantization)
+        # on the same shapes: a second context figure, not a target either.
+        try:
+            xs8 = [torch.randint(-127, 128, (M, K), dtype=torch.int8, device=dev) for K, _ in groups]
+            ws8 = [[torch.randint(-127, 128, (lin.N, lin.K), dtype=torch.int8, device=dev) for lin in wl.linears]
+                   for _ in range(n_layers)]
+            ys8 = [torch.empty((M, lin.N), dtype=torch.int32, device=dev) for lin in wl.linears]
+
+            def int8_layer(ws):
+                for gi, (K, idxs) in enumerate(groups):
+                    for i in idxs:
+                        torch._int_mm(xs8[gi], ws[i].t(), out=ys8[i])
+
+            with torch.cuda.stream(stream):
+                for ws in ws8:
+                    int8_layer(ws)
+            stream.synchronize()
+            gs8 = []
+            for ws in ws8:
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=stream):
+                    int8_layer(ws)
+                gs8.append(g)
+            lib8_avg_ms, _ = time_kind(gs8, len(wl.linears), budget_ms=200.0)
+            fp16_ctx["library_int8"] = {
+                "kernel": "torch._int_mm (cuBLASLt INT8 -> INT32, no dequantization), same shapes",
+                "tops": ops / (lib8_avg_ms * len(wl.linears) * 1e-3) / 1e12,
+                "ours_over_library": (lib8_avg_ms * len(wl.linears)) / (gemm_avg_ms * gemm_per_layer)}
+            del xs8, ws8, ys8, gs8
+        except Exception as e:   # the library call is context only: its absence must not fail the benchmark
+            fp16_ctx["library_int8"] = {"unavailable": f"{type(e).__name__}: {str(e)[:120]}"}
     gemm_tops = ops / (gemm_avg_ms * gemm_per_layer * 1e-3) / 1e12
     sbytes = step_bytes(wl, M)
     quant_gbs = sbytes["quantize"] / (quant_avg_ms * len(groups) * 1e-3) / 1e9
