@@ -14,7 +14,8 @@ __device__ int g_status_word = 0;
 namespace {
 
 constexpr int kMaxDevices = 64;
-constexpr int64_t kSmallM = 64;  // M at or below this takes the weight-streaming schedule
+constexpr int64_t kSmallM = 64;      // W4A8: M at or below this takes the weight-streaming schedule
+constexpr int64_t kSmallM_W8 = 128;  // W8A8
 
 struct DeviceInfo {
   bool probed = false;
@@ -308,11 +309,10 @@ static int gemm_w8a8_common(const int8_t* q, const float* s_tok, const void* wq,
   if (!aligned16(q) || !aligned16(wq) || !aligned16(y) || !aligned16(acc)) return PQ_ERR_ALIGN;
   if ((rc = check_arch()) != PQ_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (M <= kSmallM) return launch_smallm_w8a8(q, s_tok, wq, s_ch, M, N, K, y, acc, st);
-  bool pair = M > 128;  // below that the second CTA of a pair would only hold padding rows
-  if (const char* e = getenv("PQ_W8A8_PAIR")) pair = (e[0] != '0');  // ablation knob
-  if (pair) return launch_gemm_w8a8_pair(q, s_tok, wq, s_ch, M, N, K, y, acc, st);
-  return launch_gemm_w8a8(q, s_tok, wq, s_ch, M, N, K, y, acc, st);
+  // Up to 128 tokens: the weight-streaming schedule (tokens are the narrow MMA dimension, K split over a
+  // cluster); beyond that the second CTA of a pair no longer holds only padding rows.
+  if (M <= kSmallM_W8) return launch_smallm_w8a8(q, s_tok, wq, s_ch, M, N, K, y, acc, st);
+  return launch_gemm_w8a8_pair(q, s_tok, wq, s_ch, M, N, K, y, acc, st);
 }
 
 int pq_gemm_w8a8(const int8_t* q, const float* s_tok, const void* wq, const float* s_ch, int64_t M, int64_t N,

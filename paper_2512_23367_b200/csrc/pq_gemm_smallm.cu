@@ -1,8 +1,8 @@
-// Small-M (decode-shaped, M <= 64) W8A8 / W4A8 linear for sm_100a: a weight-streaming schedule
+// Small-M (decode-shaped; W8A8: M <= 128, W4A8: M <= 64) linear for sm_100a: a weight-streaming schedule
 // that computes the same result as the prefill kernels.
 //
 // The roles of the two operands are swapped: a tile of 128 WEIGHT rows is the 128-lane operand
-// of tcgen05.mma and the (zero-padded) tokens are the narrow N dimension (16, 32 or 64), so one
+// of tcgen05.mma and the (zero-padded) tokens are the narrow N dimension (16, 32, 64 or 128), so one
 // instruction consumes 4 KB of weights and the tensor pipe stays far below its limit while the
 // weights stream from HBM exactly once.  The K dimension is split over the CTAs of a thread-block
 // cluster (up to 8) so that ~2 CTAs per SM pull weights concurrently; the partial results are
@@ -43,11 +43,12 @@ struct Cfg {
   // Short rings and small footprints: three or four CTAs fit on an SM, so the CTAs of the NEXT
   // launch become resident (and stream their weights) while this launch reduces and stores.
   static constexpr int STAGES = MPAD == 64 ? 4 : 3;
+  static_assert(!(kW4 && MPAD > 64), "the W4 variant keeps MPAD partial results per thread in registers");
   // W4 with up to 32 tokens: two pairs of widening warps (the 64-token variant needs its registers
   // for the per-thread partial results and keeps one pair and two co-resident CTAs)
   static constexpr int kUnpackPairs = (kW4 && MPAD < 64) ? 2 : 1;
   static constexpr int kThreads = kUnpackPairs == 2 ? kNumThreadsW4 : kNumThreads;
-  static constexpr int kMinCtasPerSm = MPAD == 64 ? 2 : (kW4 ? 2 : 4);
+  static constexpr int kMinCtasPerSm = MPAD >= 64 ? 2 : (kW4 ? 2 : 4);
   static constexpr int A8_SLOTS = kW4 ? 2 : 0;                   // widened weight tiles: one per pair of widening warps
   static constexpr int kA8Bytes = BW * BK;
   static constexpr int SC_SLOTS = kW4 ? 6 : 0;                   // FP32 scale rows (128 floats)
@@ -181,10 +182,12 @@ smallm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
 
-  // Per-thread partial results of the epilogue warps: P[m] for weight row n0 + 32*quad + lane.
-  uint32_t P[MPAD];
+  // W4: per-thread partial results of the epilogue warps, P[m] for weight row n0 + 32*quad + lane.
+  // (W8 copies its one accumulator from tensor memory straight into the reduction tile.)
+  constexpr int kPartials = kW4 ? MPAD : 1;
+  uint32_t P[kPartials];
 #pragma unroll
-  for (int m = 0; m < MPAD; ++m) P[m] = 0u;
+  for (int m = 0; m < kPartials; ++m) P[m] = 0u;
   bool ok = true;
 
   if (warp == 0) {
@@ -334,15 +337,26 @@ smallm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
         }
       }
     } else {
-      if (nkb > 0) {
-        ok = __all_sync(0xffffffffu, mbar_wait(bar_acc_full, 0u, abort_flag));
-        if (ok) {
-          tc_fence_after_sync();
-          tmem_ld_cols<MPAD>(lane_addr, P);
+      // All K blocks of this CTA are consumed once the accumulator is complete, so the stage ring is
+      // free: the partial tile goes there as red[m][n] (32-bit words), 32 token columns at a time.
+      uint32_t* red_w8 = reinterpret_cast<uint32_t*>(smem);
+      if (nkb > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar_acc_full, 0u, abort_flag));
+      if (ok) tc_fence_after_sync();
+      constexpr int CW = MPAD < 32 ? MPAD : 32;
+#pragma unroll
+      for (int c0 = 0; c0 < MPAD; c0 += CW) {
+        uint32_t r[CW];
+        if (ok && nkb > 0) {
+          tmem_ld_cols<CW>(lane_addr + c0, r);
           tmem_ld_wait();
-          tc_fence_before_sync();
+        } else {
+#pragma unroll
+          for (int m = 0; m < CW; ++m) r[m] = 0u;
         }
+#pragma unroll
+        for (int m = 0; m < CW; ++m) red_w8[(c0 + m) * BW + n_local] = r[m];
       }
+      tc_fence_before_sync();
     }
   }
 
@@ -351,10 +365,10 @@ smallm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   // stage ring is free and holds this CTA's partial tile as red[m][n] (32-bit words).
   uint32_t* red = reinterpret_cast<uint32_t*>(smem);
   const bool do_reduce = !(kW4 && kExportAcc);
-  if (do_reduce && warp >= 4 && warp < 8) {
+  if (do_reduce && kW4 && warp >= 4 && warp < 8) {
     const int n_local = (warp & 3) * 32 + lane;
 #pragma unroll
-    for (int m = 0; m < MPAD; ++m) red[m * BW + n_local] = P[m];
+    for (int m = 0; m < kPartials; ++m) red[m * BW + n_local] = P[m];
   }
   tc_fence_before_sync();
   __syncwarp();
@@ -457,12 +471,20 @@ int launch_cfg(const CUtensorMap& tw, const CUtensorMap& tq, const CUtensorMap& 
 template <bool kW4>
 int launch_smallm(const int8_t* q, const float* s_tok, const void* w, const float* s_ch, const void* s_grp,
                   int64_t M, int64_t N, int64_t K, void* y, int32_t* acc, cudaStream_t stream) {
-  const int mpad = M <= 16 ? 16 : (M <= 32 ? 32 : 64);
+  const int mpad = M <= 16 ? 16 : (M <= 32 ? 32 : (M <= 64 ? 64 : 128));
+  if (kW4 && mpad > 64) return PQ_ERR_SHAPE;   // (the W4A8 dispatch sends M > 64 to the pair kernel)
   const int n_tiles = static_cast<int>((N + BW - 1) / BW);
   const int k_blocks = static_cast<int>((K + BK - 1) / BK);
   // Aim at two resident CTAs per SM; the split is the cluster size (<= 8) and <= K blocks.
   int splits = (2 * sm_count()) / n_tiles;
   splits = splits < 1 ? 1 : (splits > kMaxSplit ? kMaxSplit : splits);
+  // Variants with two CTAs per SM have no room to spare: a cluster has to fit one GPC, so a grid that
+  // nearly fills the device leaves clusters for a second wave (2048 -> 6144 at M = 64: 12.8 us with
+  // clusters of 6, 7.4 us with clusters of 4).  Stay below 90 % of the resident capacity, and off the
+  // cluster sizes 5 and 7.
+  const int ctas_per_sm = mpad >= 64 ? 2 : (kW4 ? 2 : 4);
+  while (splits > 1 && n_tiles * splits * 10 > ctas_per_sm * sm_count() * 9) --splits;
+  if (splits == 5 || splits == 7) --splits;
   if (splits > k_blocks) splits = k_blocks;
 
   CUtensorMap tw, tq, ts;
@@ -499,7 +521,13 @@ int launch_smallm(const int8_t* q, const float* s_tok, const void* w, const floa
   switch (mpad) {
     case 16: return ex ? launch_cfg<16, kW4, true>(tw, tq, ts, a, n_tiles, stream) : launch_cfg<16, kW4, false>(tw, tq, ts, a, n_tiles, stream);
     case 32: return ex ? launch_cfg<32, kW4, true>(tw, tq, ts, a, n_tiles, stream) : launch_cfg<32, kW4, false>(tw, tq, ts, a, n_tiles, stream);
-    default: return ex ? launch_cfg<64, kW4, true>(tw, tq, ts, a, n_tiles, stream) : launch_cfg<64, kW4, false>(tw, tq, ts, a, n_tiles, stream);
+    case 64: return ex ? launch_cfg<64, kW4, true>(tw, tq, ts, a, n_tiles, stream) : launch_cfg<64, kW4, false>(tw, tq, ts, a, n_tiles, stream);
+    default:
+      if constexpr (kW4) {
+        return PQ_ERR_SHAPE;
+      } else {
+        return ex ? launch_cfg<128, false, true>(tw, tq, ts, a, n_tiles, stream) : launch_cfg<128, false, false>(tw, tq, ts, a, n_tiles, stream);
+      }
   }
 }
 

@@ -53,10 +53,8 @@ int launch_col_absmax(const void* a, int64_t R, int64_t K, float* out, cudaStrea
 int launch_smooth_scales(const float* xa, const float* wa, int64_t K, float* s, float* s_inv, cudaStream_t stream);
 int launch_unpack_w4(const void* wp, int64_t N, int64_t K, int8_t* codes, cudaStream_t stream);
 
-// Prefill-shaped W8A8 GEMM (tcgen05 kind::i8).  Exactly one of y / acc is non-null.
-int launch_gemm_w8a8(const int8_t* q, const float* s_tok, const void* wq, const float* s_ch, int64_t M,
-                     int64_t N, int64_t K, void* y, int32_t* acc, cudaStream_t stream);
-// Same contract on CTA pairs (cta_group::2, 256-row tiles); preferred when M > 128.
+// Prefill-shaped W8A8 GEMM (tcgen05 kind::i8) on CTA pairs (cta_group::2, 256-row tiles), for M > 128.
+// Exactly one of y / acc is non-null.
 int launch_gemm_w8a8_pair(const int8_t* q, const float* s_tok, const void* wq, const float* s_ch, int64_t M,
                           int64_t N, int64_t K, void* y, int32_t* acc, cudaStream_t stream);
 // Linears that share the token codes and run as one launch of the pair GEMM: at most this many.
