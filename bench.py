@@ -309,8 +309,8 @@ def run_ours(args, wl: synth.Workload, M: int):
     n_layers = layers_for_rotation(wl, M)
     layers = [LayerBuffers(pq, torch, wl, M, dev, src_x, src_w) for _ in range(n_layers)]
 
-    # The grouped calls schedule their members in one launch (W8A8: M > 128, W4A8: M > 64).
-    grouped = M > (128 if wl.w_bits == 8 else 64) and not args.no_group
+    # The grouped calls schedule their members in one launch.
+    grouped = not args.no_group
 
     def run_layer(L: LayerBuffers, only: str | None = None):
         for gi, (K, idxs) in enumerate(L.groups):

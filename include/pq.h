@@ -200,9 +200,10 @@ PQ_API int pq_acc_w4a8(const int8_t* q, const void* wp, int32_t group, int64_t M
 /*
  * Several W8A8 linears over the SAME quantized tokens (the q/k/v projections, or gate and up, of
  * the layers the paper quantizes) as one call.  Result: exactly what `count` calls of pq_gemm_w8a8
- * with (wq[g], s_ch[g], N[g], y_f16[g]) give, bit for bit.  For M > 128 the members' output tiles
- * are scheduled together in a single kernel launch, which fills the SMs' waves across the members
- * and pays the per-launch fixed cost once; other M run one launch per member.
+ * with (wq[g], s_ch[g], N[g], y_f16[g]) give, bit for bit.  The members' output tiles are scheduled
+ * together in a single kernel launch (of the prefill kernel for M > 128, of the weight-streaming
+ * kernel below), which fills the SMs' waves across the members and pays the per-launch fixed cost
+ * once -- at decode-shaped token counts that fixed cost is most of a call.
  *   count: 1..PQ_MAX_GROUP.  wq, s_ch, N, y_f16: HOST arrays of `count` entries (device pointers
  *   and column counts; read during the call, not retained).  q, s_tok, M, K as in pq_gemm_w8a8.
  *   The outputs must not overlap each other.  On an argument error nothing is launched.
@@ -212,7 +213,9 @@ PQ_API int pq_gemm_w8a8_group(const int8_t* q, const float* s_tok, int32_t count
                               const float* const* s_ch, const int64_t* N, void* const* y_f16, int64_t M,
                               int64_t K, void* stream);
 
-/* The same for W4A8 linears (pq_gemm_w4a8 per member; grouped into one launch for M > 64). */
+/* The same for W4A8 linears (pq_gemm_w4a8 per member, one launch for all of them).  For M <= 64 the FP32
+ * group sums of the K parts are added in a fixed order, but the number of parts depends on how many tiles
+ * the launch holds, so the grouped result may differ from the per-member call in the last FP32 bit. */
 PQ_API int pq_gemm_w4a8_group(const int8_t* q, const float* s_tok, int32_t count, const void* const* wp,
                               const void* const* s_grp_f16, int32_t group, const int64_t* N,
                               void* const* y_f16, int64_t M, int64_t K, void* stream);

@@ -296,8 +296,7 @@ def pq_gemm_w8a8(q, s_tok, wq, s_ch, N: int, y: torch.Tensor | None = None) -> t
 
 
 def pq_gemm_w8a8_group(q, s_tok, members, ys=None) -> list[torch.Tensor]:
-    """Several W8A8 linears over the same quantized tokens as one call (one kernel launch when
-    M > 128).  members: sequence of (wq, s_ch, N) from pq_pack_w8; ys: optional outputs f16 [M,N_g].
+    """Several W8A8 linears over the same quantized tokens as one call (one kernel launch).  members: sequence of (wq, s_ch, N) from pq_pack_w8; ys: optional outputs f16 [M,N_g].
     Returns the outputs; each equals pq_gemm_w8a8(q, s_tok, wq, s_ch, N) bit for bit."""
     q = _dev(q, torch.int8, "q")
     _ensure_workspace(q.device)
@@ -320,8 +319,7 @@ def pq_gemm_w8a8_group(q, s_tok, members, ys=None) -> list[torch.Tensor]:
 
 
 def pq_gemm_w4a8_group(q, s_tok, members, ys=None, group: int = GROUP) -> list[torch.Tensor]:
-    """Several W4A8 linears over the same quantized tokens as one call (one kernel launch when
-    M > 64).  members: sequence of (wp, s_grp, N) from pq_pack_w4; ys: optional outputs f16 [M,N_g].
+    """Several W4A8 linears over the same quantized tokens as one call (one kernel launch).  members: sequence of (wp, s_grp, N) from pq_pack_w4; ys: optional outputs f16 [M,N_g].
     Each output equals pq_gemm_w4a8(q, s_tok, wp, s_grp, N) bit for bit."""
     q = _dev(q, torch.int8, "q")
     M, K = q.shape

@@ -335,13 +335,9 @@ int pq_gemm_w8a8_group(const int8_t* q, const float* s_tok, int32_t count, const
   if (!aligned16(q)) return PQ_ERR_ALIGN;
   int rc = check_arch();
   if (rc != PQ_OK) return rc;
-  if (M <= 128 || count == 1) {
-    // Token counts whose schedules do not group (they reduce inside the SMs): one launch per member.
-    for (int g = 0; g < count; ++g) {
-      rc = gemm_w8a8_common(q, s_tok, wq[g], s_ch[g], M, N[g], K, y_f16[g], nullptr, stream);
-      if (rc != PQ_OK) return rc;
-    }
-    return PQ_OK;
+  if (M <= kSmallM_W8) {
+    return launch_smallm_w8a8_group(q, s_tok, count, wq, s_ch, N, y_f16, M, K, nullptr,
+                                    static_cast<cudaStream_t>(stream));
   }
   return launch_gemm_w8a8_pair_group(scratch(), q, s_tok, count, wq, s_ch, N, y_f16, M, K, nullptr,
                                      static_cast<cudaStream_t>(stream));
@@ -385,13 +381,9 @@ int pq_gemm_w4a8_group(const int8_t* q, const float* s_tok, int32_t count, const
   if (!aligned16(q)) return PQ_ERR_ALIGN;
   int rc = check_arch();
   if (rc != PQ_OK) return rc;
-  if (M <= kSmallM || count == 1) {
-    // Decode-shaped token counts reduce inside the SMs and do not group: one launch per member.
-    for (int g = 0; g < count; ++g) {
-      rc = gemm_w4a8_common(q, s_tok, wp[g], s_grp_f16[g], group, M, N[g], K, y_f16[g], nullptr, stream);
-      if (rc != PQ_OK) return rc;
-    }
-    return PQ_OK;
+  if (M <= kSmallM) {
+    return launch_smallm_w4a8_group(q, s_tok, count, wp, s_grp_f16, N, y_f16, M, K, nullptr,
+                                    static_cast<cudaStream_t>(stream));
   }
   return launch_gemm_w4a8_group(q, s_tok, count, wp, s_grp_f16, N, y_f16, M, K, nullptr,
                                 static_cast<cudaStream_t>(stream));

@@ -66,12 +66,21 @@ struct Cfg {
 
 struct SmallArgs {
   const float* s_tok;
-  const float* s_ch;     // W8
-  __half* y;
-  int32_t* acc;          // export: W8 [M,N]; W4 [G,M,N]
+  const float* s_ch[kMaxGroup];   // W8, per member
+  __half* y[kMaxGroup];           // per member
+  int N[kMaxGroup];               // per member
+  int tile_end[kMaxGroup];        // 128-channel tiles of members 0..g (running total); INT_MAX past the last
+  int count;                      // members in this launch (linears over the same tokens)
+  int32_t* acc;          // export (single member): W8 [M,N]; W4 [G,M,N]
   int* status;
-  int M, N, K;
+  int M, K;
   int k_blocks, splits;
+};
+
+// Tensor maps of the members' weights (and W4 group scales), indexed by member.
+struct SmallMaps {
+  CUtensorMap w[kMaxGroup];
+  CUtensorMap s[kMaxGroup];
 };
 
 __device__ __forceinline__ uint4 ld_dsmem_v4(uint32_t local_addr, uint32_t rank) {
@@ -102,8 +111,7 @@ __device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t (&r)[MPAD]
 
 template <int MPAD, bool kW4, bool kExportAcc>
 __global__ void __launch_bounds__(Cfg<MPAD, kW4>::kThreads, Cfg<MPAD, kW4>::kMinCtasPerSm)
-smallm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_q,
-              const __grid_constant__ CUtensorMap tm_s, const SmallArgs p) {
+smallm_kernel(const __grid_constant__ SmallMaps maps, const __grid_constant__ CUtensorMap tm_q, const SmallArgs p) {
   using C = Cfg<MPAD, kW4>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -121,7 +129,20 @@ smallm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int n0 = blockIdx.x * BW;
+  // This CTA's member and first channel inside it (grid.x runs over the tiles of all members).
+  int member = 0, tile = static_cast<int>(blockIdx.x);
+  if (p.count > 1) {
+    const int e0 = p.tile_end[0], e1 = p.tile_end[1], e2 = p.tile_end[2];
+    if (tile >= e2) { member = 3; tile -= e2; }
+    else if (tile >= e1) { member = 2; tile -= e1; }
+    else if (tile >= e0) { member = 1; tile -= e0; }
+  }
+  const int n0 = tile * BW;
+  const int N_mem = member == 0 ? p.N[0] : (member == 1 ? p.N[1] : (member == 2 ? p.N[2] : p.N[3]));
+  const float* s_ch_mem = member == 0 ? p.s_ch[0] : (member == 1 ? p.s_ch[1] : (member == 2 ? p.s_ch[2] : p.s_ch[3]));
+  __half* y_mem = member == 0 ? p.y[0] : (member == 1 ? p.y[1] : (member == 2 ? p.y[2] : p.y[3]));
+  const CUtensorMap* tm_w = &maps.w[member];
+  const CUtensorMap* tm_s = &maps.s[member];
   const int split = blockIdx.y;                       // == rank in the cluster (cluster = all of grid.y)
   const int kb0 = static_cast<int>(static_cast<int64_t>(p.k_blocks) * split / p.splits);
   const int kb1 = static_cast<int>(static_cast<int64_t>(p.k_blocks) * (split + 1) / p.splits);
@@ -135,8 +156,8 @@ smallm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
     const uint32_t dst = smem_base + s * C::kStageBytes;
     const int kb = kb0 + j;
     mbar_arrive_expect_tx(bar_full + s * 8, C::kTxBytes);
-    tma_load_2d(dst, &tm_w, bar_full + s * 8, kW4 ? kb * (BK / 2) : kb * BK, n0);
-    if constexpr (kW4) tma_load_2d(dst + C::kWBytes + C::kQBytes, &tm_s, bar_full + s * 8, n0, kb);
+    tma_load_2d(dst, tm_w, bar_full + s * 8, kW4 ? kb * (BK / 2) : kb * BK, n0);
+    if constexpr (kW4) tma_load_2d(dst + C::kWBytes + C::kQBytes, tm_s, bar_full + s * 8, n0, kb);
   };
   auto issue_codes = [&](int j) {
     const uint32_t s = static_cast<uint32_t>(j) % C::STAGES;
@@ -144,9 +165,9 @@ smallm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   };
 
   if (threadIdx.x == 64) {
-    tma_prefetch_desc(&tm_w);
+    tma_prefetch_desc(tm_w);
     tma_prefetch_desc(&tm_q);
-    if constexpr (kW4) tma_prefetch_desc(&tm_s);
+    if constexpr (kW4) tma_prefetch_desc(tm_s);
   }
   if (threadIdx.x == 0) {
     *abort_flag = 0;
@@ -320,8 +341,8 @@ smallm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
             const int n = n0 + n_local;
 #pragma unroll
             for (int m = 0; m < CH; ++m) {
-              if (c0 + m < p.M && n < p.N)
-                p.acc[(static_cast<int64_t>(kb0 + j) * p.M + c0 + m) * p.N + n] = static_cast<int32_t>(r[m]) >> 4;
+              if (c0 + m < p.M && n < N_mem)
+                p.acc[(static_cast<int64_t>(kb0 + j) * p.M + c0 + m) * N_mem + n] = static_cast<int32_t>(r[m]) >> 4;
             }
           } else {
 #pragma unroll
@@ -382,9 +403,9 @@ smallm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
     const int n = n0 + 4 * nq;
     const uint32_t my_rank = cluster_ctarank();
     float sc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-    if (!kW4 && !kExportAcc && n < p.N) {
+    if (!kW4 && !kExportAcc && n < N_mem) {
 #pragma unroll
-      for (int j = 0; j < 4; ++j) sc[j] = __ldg(p.s_ch + n + j);   // N is a multiple of 8: n < N covers n + 3
+      for (int j = 0; j < 4; ++j) sc[j] = __ldg(s_ch_mem + n + j);   // N is a multiple of 8: n < N covers n + 3
     }
     for (int m = static_cast<int>(my_rank) + p.splits * msub; m < p.M; m += 4 * p.splits) {
       const uint32_t addr = smem_base + static_cast<uint32_t>(m * BW + 4 * nq) * 4u;
@@ -393,7 +414,7 @@ smallm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
       for (int r = 0; r < kMaxSplit; ++r) {
         if (r < p.splits) part[r] = ld_dsmem_v4(addr, static_cast<uint32_t>(r));
       }
-      if (n >= p.N) continue;
+      if (n >= N_mem) continue;
       if constexpr (kW4) {
         float tot[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
@@ -405,7 +426,7 @@ smallm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
         }
         const float st = __ldg(p.s_tok + m);
         const __half2 h01 = __floats2half2_rn(tot[0] * st, tot[1] * st), h23 = __floats2half2_rn(tot[2] * st, tot[3] * st);
-        *reinterpret_cast<uint2*>(p.y + static_cast<int64_t>(m) * p.N + n) =
+        *reinterpret_cast<uint2*>(y_mem + static_cast<int64_t>(m) * N_mem + n) =
             make_uint2(*reinterpret_cast<const uint32_t*>(&h01), *reinterpret_cast<const uint32_t*>(&h23));
       } else {
         int32_t tot[4] = {0, 0, 0, 0};
@@ -417,14 +438,14 @@ smallm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
           }
         }
         if constexpr (kExportAcc) {
-          *reinterpret_cast<int4*>(p.acc + static_cast<int64_t>(m) * p.N + n) = make_int4(tot[0], tot[1], tot[2], tot[3]);
+          *reinterpret_cast<int4*>(p.acc + static_cast<int64_t>(m) * N_mem + n) = make_int4(tot[0], tot[1], tot[2], tot[3]);
         } else {
           const float st = __ldg(p.s_tok + m);
           float v[4];
 #pragma unroll
           for (int j = 0; j < 4; ++j) v[j] = __fmul_rn(__fmul_rn(__int2float_rn(tot[j]), st), sc[j]);
           const __half2 h01 = __floats2half2_rn(v[0], v[1]), h23 = __floats2half2_rn(v[2], v[3]);
-          *reinterpret_cast<uint2*>(p.y + static_cast<int64_t>(m) * p.N + n) =
+          *reinterpret_cast<uint2*>(y_mem + static_cast<int64_t>(m) * N_mem + n) =
               make_uint2(*reinterpret_cast<const uint32_t*>(&h01), *reinterpret_cast<const uint32_t*>(&h23));
         }
       }
@@ -441,8 +462,7 @@ smallm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
 }
 
 template <int MPAD, bool kW4, bool kExportAcc>
-int launch_cfg(const CUtensorMap& tw, const CUtensorMap& tq, const CUtensorMap& ts, const SmallArgs& a, int n_tiles,
-               cudaStream_t stream) {
+int launch_cfg(const SmallMaps& maps, const CUtensorMap& tq, const SmallArgs& a, int n_tiles, cudaStream_t stream) {
   using C = Cfg<MPAD, kW4>;
   auto kern = smallm_kernel<MPAD, kW4, kExportAcc>;
   static bool configured = false;
@@ -465,82 +485,109 @@ int launch_cfg(const CUtensorMap& tw, const CUtensorMap& tq, const CUtensorMap& 
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = pdl_enabled() ? 2 : 1;
-  return cuda_status(cudaLaunchKernelEx(&cfg, kern, tw, tq, ts, a));
+  return cuda_status(cudaLaunchKernelEx(&cfg, kern, maps, tq, a));
 }
 
+// `count` linears over the same tokens in one launch: grid.x runs over the 128-channel tiles of all
+// members.  w / s_ch / s_grp / N / y are host arrays of `count` entries; acc (export) only with count == 1.
 template <bool kW4>
-int launch_smallm(const int8_t* q, const float* s_tok, const void* w, const float* s_ch, const void* s_grp,
-                  int64_t M, int64_t N, int64_t K, void* y, int32_t* acc, cudaStream_t stream) {
+int launch_smallm(const int8_t* q, const float* s_tok, int count, const void* const* w, const float* const* s_ch,
+                  const void* const* s_grp, const int64_t* N, void* const* y, int64_t M, int64_t K, int32_t* acc,
+                  cudaStream_t stream) {
+  if (count < 1 || count > kMaxGroup || (acc != nullptr && count != 1)) return PQ_ERR_SHAPE;
   const int mpad = M <= 16 ? 16 : (M <= 32 ? 32 : (M <= 64 ? 64 : 128));
   if (kW4 && mpad > 64) return PQ_ERR_SHAPE;   // (the W4A8 dispatch sends M > 64 to the pair kernel)
-  const int n_tiles = static_cast<int>((N + BW - 1) / BW);
   const int k_blocks = static_cast<int>((K + BK - 1) / BK);
+
+  CUtensorMap tq;
+  SmallMaps maps;
+  SmallArgs a;
+  int rc = make_tmap_2d(&tq, q, static_cast<uint64_t>(M), static_cast<uint64_t>(K), static_cast<uint32_t>(mpad), BK, 1, 128);
+  if (rc != PQ_OK) return rc;
+  int64_t n_tiles = 0;
+  for (int g = 0; g < kMaxGroup; ++g) {
+    const int src = g < count ? g : 0;   // unused slots repeat member 0 (never selected)
+    if (kW4) {
+      rc = make_tmap_2d(&maps.w[g], w[src], static_cast<uint64_t>(N[src]), static_cast<uint64_t>(K / 2), BW, BK / 2, 1, 0);
+    } else {
+      rc = make_tmap_2d(&maps.w[g], w[src], static_cast<uint64_t>(N[src]), static_cast<uint64_t>(K), BW, BK, 1, 128);
+    }
+    if (rc != PQ_OK) return rc;
+    if (kW4 && acc == nullptr) {
+      rc = make_tmap_2d(&maps.s[g], s_grp[src], static_cast<uint64_t>(K / 128), static_cast<uint64_t>(N[src]), 1, BW, 2, 0);
+    } else if (kW4) {
+      // the W4 accumulator export has no scales: it reads (and ignores) token bytes instead
+      rc = make_tmap_2d(&maps.s[g], q, static_cast<uint64_t>(M), static_cast<uint64_t>(K / 2), 1, BW, 2, 0);
+    } else {
+      maps.s[g] = tq;  // unused by W8
+    }
+    if (rc != PQ_OK) return rc;
+    a.s_ch[g] = kW4 ? nullptr : s_ch[src];
+    a.y[g] = static_cast<__half*>(acc == nullptr ? y[src] : nullptr);
+    a.N[g] = static_cast<int>(N[src]);
+    if (g < count) n_tiles += (N[g] + BW - 1) / BW;
+    a.tile_end[g] = g < count ? static_cast<int>(n_tiles) : 0x7fffffff;
+  }
+  if (n_tiles > 0x3fffffff) return PQ_ERR_SHAPE;
+
   // Aim at two resident CTAs per SM; the split is the cluster size (<= 8) and <= K blocks.
-  int splits = (2 * sm_count()) / n_tiles;
+  int splits = static_cast<int>((2 * sm_count()) / n_tiles);
   splits = splits < 1 ? 1 : (splits > kMaxSplit ? kMaxSplit : splits);
   // Variants with two CTAs per SM have no room to spare: a cluster has to fit one GPC, so a grid that
   // nearly fills the device leaves clusters for a second wave (2048 -> 6144 at M = 64: 12.8 us with
   // clusters of 6, 7.4 us with clusters of 4).  Stay below 90 % of the resident capacity, and off the
   // cluster sizes 5 and 7.
   const int ctas_per_sm = mpad >= 64 ? 2 : (kW4 ? 2 : 4);
-  while (splits > 1 && n_tiles * splits * 10 > ctas_per_sm * sm_count() * 9) --splits;
+  while (splits > 1 && n_tiles * splits * 10 > static_cast<int64_t>(ctas_per_sm) * sm_count() * 9) --splits;
   if (splits == 5 || splits == 7) --splits;
   if (splits > k_blocks) splits = k_blocks;
 
-  CUtensorMap tw, tq, ts;
-  int rc;
-  if (kW4) {
-    rc = make_tmap_2d(&tw, w, static_cast<uint64_t>(N), static_cast<uint64_t>(K / 2), BW, BK / 2, 1, 0);
-  } else {
-    rc = make_tmap_2d(&tw, w, static_cast<uint64_t>(N), static_cast<uint64_t>(K), BW, BK, 1, 128);
-  }
-  if (rc != PQ_OK) return rc;
-  rc = make_tmap_2d(&tq, q, static_cast<uint64_t>(M), static_cast<uint64_t>(K), static_cast<uint32_t>(mpad), BK, 1, 128);
-  if (rc != PQ_OK) return rc;
-  if (kW4 && s_grp != nullptr) {
-    rc = make_tmap_2d(&ts, s_grp, static_cast<uint64_t>(K / 128), static_cast<uint64_t>(N), 1, BW, 2, 0);
-  } else {
-    ts = tq;  // unused by W8; the W4 accumulator export reads (and ignores) token bytes instead of scales
-    if (kW4) rc = make_tmap_2d(&ts, q, static_cast<uint64_t>(M), static_cast<uint64_t>(K / 2), 1, BW, 2, 0);
-  }
-  if (rc != PQ_OK) return rc;
-
-  SmallArgs a;
+  a.count = count;
   a.s_tok = s_tok;
-  a.s_ch = s_ch;
-  a.y = static_cast<__half*>(y);
   a.acc = acc;
   a.status = device_status_ptr();
   if (a.status == nullptr) return PQ_ERR_CUDA;
   a.M = static_cast<int>(M);
-  a.N = static_cast<int>(N);
   a.K = static_cast<int>(K);
   a.k_blocks = k_blocks;
   a.splits = splits;
   const bool ex = acc != nullptr;
+  const int nt = static_cast<int>(n_tiles);
   switch (mpad) {
-    case 16: return ex ? launch_cfg<16, kW4, true>(tw, tq, ts, a, n_tiles, stream) : launch_cfg<16, kW4, false>(tw, tq, ts, a, n_tiles, stream);
-    case 32: return ex ? launch_cfg<32, kW4, true>(tw, tq, ts, a, n_tiles, stream) : launch_cfg<32, kW4, false>(tw, tq, ts, a, n_tiles, stream);
-    case 64: return ex ? launch_cfg<64, kW4, true>(tw, tq, ts, a, n_tiles, stream) : launch_cfg<64, kW4, false>(tw, tq, ts, a, n_tiles, stream);
+    case 16: return ex ? launch_cfg<16, kW4, true>(maps, tq, a, nt, stream) : launch_cfg<16, kW4, false>(maps, tq, a, nt, stream);
+    case 32: return ex ? launch_cfg<32, kW4, true>(maps, tq, a, nt, stream) : launch_cfg<32, kW4, false>(maps, tq, a, nt, stream);
+    case 64: return ex ? launch_cfg<64, kW4, true>(maps, tq, a, nt, stream) : launch_cfg<64, kW4, false>(maps, tq, a, nt, stream);
     default:
       if constexpr (kW4) {
         return PQ_ERR_SHAPE;
       } else {
-        return ex ? launch_cfg<128, false, true>(tw, tq, ts, a, n_tiles, stream) : launch_cfg<128, false, false>(tw, tq, ts, a, n_tiles, stream);
+        return ex ? launch_cfg<128, false, true>(maps, tq, a, nt, stream) : launch_cfg<128, false, false>(maps, tq, a, nt, stream);
       }
   }
 }
 
 }  // namespace
 
+int launch_smallm_w8a8_group(const int8_t* q, const float* s_tok, int count, const void* const* wq,
+                             const float* const* s_ch, const int64_t* N, void* const* y, int64_t M, int64_t K,
+                             int32_t* acc, cudaStream_t stream) {
+  return launch_smallm<false>(q, s_tok, count, wq, s_ch, nullptr, N, y, M, K, acc, stream);
+}
+
+int launch_smallm_w4a8_group(const int8_t* q, const float* s_tok, int count, const void* const* wp,
+                             const void* const* s_grp, const int64_t* N, void* const* y, int64_t M, int64_t K,
+                             int32_t* acc_g, cudaStream_t stream) {
+  return launch_smallm<true>(q, s_tok, count, wp, nullptr, s_grp, N, y, M, K, acc_g, stream);
+}
+
 int launch_smallm_w8a8(const int8_t* q, const float* s_tok, const void* wq, const float* s_ch, int64_t M,
                        int64_t N, int64_t K, void* y, int32_t* acc, cudaStream_t stream) {
-  return launch_smallm<false>(q, s_tok, wq, s_ch, nullptr, M, N, K, y, acc, stream);
+  return launch_smallm_w8a8_group(q, s_tok, 1, &wq, &s_ch, &N, &y, M, K, acc, stream);
 }
 
 int launch_smallm_w4a8(const int8_t* q, const float* s_tok, const void* wp, const void* s_grp, int64_t M,
                        int64_t N, int64_t K, void* y, int32_t* acc_g, cudaStream_t stream) {
-  return launch_smallm<true>(q, s_tok, wp, nullptr, s_grp, M, N, K, y, acc_g, stream);
+  return launch_smallm_w4a8_group(q, s_tok, 1, &wp, &s_grp, &N, &y, M, K, acc_g, stream);
 }
 
 }  // namespace pq

@@ -86,6 +86,14 @@ int launch_smallm_w8a8(const int8_t* q, const float* s_tok, const void* wq, cons
 int launch_smallm_w4a8(const int8_t* q, const float* s_tok, const void* wp, const void* s_grp, int64_t M,
                        int64_t N, int64_t K, void* y, int32_t* acc_g, cudaStream_t stream);
 
+// `count` (1..kMaxGroup) small-M linears over the same tokens in one launch (host arrays, as above).
+int launch_smallm_w8a8_group(const int8_t* q, const float* s_tok, int count, const void* const* wq,
+                             const float* const* s_ch, const int64_t* N, void* const* y, int64_t M, int64_t K,
+                             int32_t* acc, cudaStream_t stream);
+int launch_smallm_w4a8_group(const int8_t* q, const float* s_tok, int count, const void* const* wp,
+                             const void* const* s_grp, const int64_t* N, void* const* y, int64_t M, int64_t K,
+                             int32_t* acc_g, cudaStream_t stream);
+
 inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? PQ_OK : PQ_ERR_CUDA; }
 
 }  // namespace pq
