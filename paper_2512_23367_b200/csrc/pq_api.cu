@@ -382,6 +382,18 @@ int pq_gemm_w4a8_group(const int8_t* q, const float* s_tok, int32_t count, const
   int rc = check_arch();
   if (rc != PQ_OK) return rc;
   if (M <= kSmallM) {
+    // One launch, unless the members together hold more 128-channel tiles than the device has SMs:
+    // the K dimension would then not be split at all, and the widening makes a CTA's chain over all of K
+    // slower than separate launches (2 x 4096->11008 at M=1: 23.8 us grouped, 22.4 us separately).
+    int64_t tiles = 0;
+    for (int g = 0; g < count; ++g) tiles += (N[g] + 127) / 128;
+    if (count > 1 && tiles > sm_count()) {
+      for (int g = 0; g < count; ++g) {
+        rc = gemm_w4a8_common(q, s_tok, wp[g], s_grp_f16[g], group, M, N[g], K, y_f16[g], nullptr, stream);
+        if (rc != PQ_OK) return rc;
+      }
+      return PQ_OK;
+    }
     return launch_smallm_w4a8_group(q, s_tok, count, wp, s_grp_f16, N, y_f16, M, K, nullptr,
                                     static_cast<cudaStream_t>(stream));
   }
