@@ -96,6 +96,10 @@ WORKLOADS = {
     "c4_w4a8_7b_prefill": Workload(4, "c4_w4a8_7b_prefill", 4, (2048,), LAYER_7B),
     "c5_w8a8_7b_decode": Workload(5, "c5_w8a8_7b_decode", 8, (1, 4, 16, 64), SHAPES_7B),
     "c5_w4a8_7b_decode": Workload(6, "c5_w4a8_7b_decode", 4, (1, 4, 16, 64), SHAPES_7B),
+    # The whole 7B-class layer at decode-shaped token counts (q/k/v and gate/up share their inputs, so the
+    # grouped calls apply): the same seven linears as c3, the token counts of c5.
+    "c5l_w8a8_7b_decode_layer": Workload(7, "c5l_w8a8_7b_decode_layer", 8, (1, 4, 16, 64), LAYER_7B),
+    "c5l_w4a8_7b_decode_layer": Workload(8, "c5l_w4a8_7b_decode_layer", 4, (1, 4, 16, 64), LAYER_7B),
 }
 
 
