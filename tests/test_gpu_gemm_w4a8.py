@@ -24,7 +24,16 @@ def assert_y_close(y_gpu, y_ref):
     assert not bad.any(), (int(bad.sum()), np.argwhere(bad)[:5], g[bad][:5], r[bad][:5])
 
 
-def run_case(M, N, K, seed, n_out=None, rows=None, check_acc=True):
+def stratified(n, block, rng, extra=()):
+    """Sorted sample of range(n): one seeded index in every block of `block`, the edges, and `extra`."""
+    starts = np.arange(0, n, block)
+    picks = np.minimum(starts + rng.integers(0, block, len(starts)), n - 1)
+    return np.unique(np.concatenate([picks, [0, n - 1], np.asarray(extra, dtype=np.int64)])).astype(np.int64)
+
+
+def run_case(M, N, K, seed, n_out=None, rows=None, cols=None):
+    """rows: compare these token rows x all N; cols (with rows): also all M rows x these output channels.
+    Without either, every element is compared.  The per-group INT32 accumulators are always compared."""
     x = synth.activations(M, K, seed, n_out)
     w = synth.weights(N, K, seed)
     if N > 2 and K >= 256:
@@ -32,17 +41,23 @@ def run_case(M, N, K, seed, n_out=None, rows=None, check_acc=True):
     q, s_tok = pq.pq_quantize_act(torch.from_numpy(x).to(DEV))
     wp, s_grp = pq.pq_pack_w4(torch.from_numpy(w).to(DEV))
     y = pq.pq_gemm_w4a8(q, s_tok, wp, s_grp, N)
-    acc = pq.pq_acc_w4a8(q, wp, N) if check_acc else None
+    acc = pq.pq_acc_w4a8(q, wp, N)
     assert pq.pq_device_status() == 0
     q_ref, s_tok_ref = oracle.quantize_act(x)
     codes_ref, sg_ref = oracle.pack_w4(w, 128)
     assert np.array_equal(_np(q), q_ref)
     assert np.array_equal(_np(pq.pq_unpack_w4(wp, N, K)), codes_ref)
+    assert np.array_equal(_np(s_grp).view(np.uint16), np.ascontiguousarray(sg_ref.T).view(np.uint16))   # device layout [K/128, N]
     sel = np.arange(M) if rows is None else rows
-    acc_ref, y_ref = oracle.gemm_w4a8(q_ref[sel], s_tok_ref[sel], codes_ref, sg_ref, 128, want_acc=check_acc)
-    if check_acc:
-        assert np.array_equal(_np(acc)[:, sel, :], np.transpose(acc_ref, (2, 0, 1)))
-    assert_y_close(_np(y)[sel], y_ref)
+    sel_d = torch.from_numpy(sel).to(DEV)
+    acc_ref, y_ref = oracle.gemm_w4a8(q_ref[sel], s_tok_ref[sel], codes_ref, sg_ref, 128)
+    assert np.array_equal(_np(acc[:, sel_d, :]), np.transpose(acc_ref, (2, 0, 1)))
+    assert_y_close(_np(y[sel_d]), y_ref)
+    if cols is not None:
+        cols_d = torch.from_numpy(cols).to(DEV)
+        acc_ref, y_ref = oracle.gemm_w4a8(q_ref, s_tok_ref, codes_ref[cols], sg_ref[cols], 128)
+        assert np.array_equal(_np(acc[:, :, cols_d]), np.transpose(acc_ref, (2, 0, 1)))
+        assert_y_close(_np(y[:, cols_d]), y_ref)
 
 
 @pytest.mark.parametrize("M", [16, 200])
@@ -86,7 +101,11 @@ def test_equal_power_of_two_group_scales_reduce_to_integer_sum():
 
 
 @pytest.mark.parametrize("M,K,N", [(2048, 4096, 11008), (2048, 11008, 4096), (2048, 4096, 4096)])
-def test_full_size_layers_on_sampled_rows(M, K, N):
+def test_full_size_layers_touch_every_tile(M, K, N):
+    """The benchmarked shapes: a token row out of every block of 128 x all N channels, and all M rows x a
+    channel out of every block of 64 (at least 256 channels): every output tile is compared, the per-group
+    INT32 accumulators bit for bit."""
     rng = np.random.default_rng(M + K + N)
-    rows = np.unique(np.concatenate([[0, 127, 128, M - 129, M - 1], rng.integers(0, M, 11)]))
-    run_case(M, N, K, seed=4000 + N % 97, rows=rows, check_acc=False)
+    rows = stratified(M, 128, rng, extra=[127, 128, M - 129])
+    cols = stratified(N, 64, rng, extra=rng.integers(0, N, max(0, 256 - N // 64)))
+    run_case(M, N, K, seed=4000 + N % 97, rows=rows, cols=cols)

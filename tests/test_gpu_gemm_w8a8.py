@@ -24,7 +24,17 @@ def assert_y_close(y_gpu, y_ref):
     assert not bad.any(), (int(bad.sum()), np.argwhere(bad)[:5], g[bad][:5], r[bad][:5])
 
 
-def run_case(M, N, K, seed, n_out=None, rows=None):
+def stratified(n, block, rng, extra=()):
+    """Sorted sample of range(n): one seeded index in every block of `block`, the edges, and `extra`."""
+    starts = np.arange(0, n, block)
+    picks = starts + rng.integers(0, block, len(starts))
+    picks = np.minimum(picks, n - 1)
+    return np.unique(np.concatenate([picks, [0, n - 1], np.asarray(extra, dtype=np.int64)])).astype(np.int64)
+
+
+def run_case(M, N, K, seed, n_out=None, rows=None, cols=None):
+    """rows: compare these token rows x all N; cols (with rows): also all M rows x these output channels.
+    Without either, every element is compared."""
     x = synth.activations(M, K, seed, n_out)
     w = synth.weights(N, K, seed)
     xd, wd = torch.from_numpy(x).to(DEV), torch.from_numpy(w).to(DEV)
@@ -36,10 +46,18 @@ def run_case(M, N, K, seed, n_out=None, rows=None):
     q_ref, s_tok_ref = oracle.quantize_act(x)
     wq_ref, s_ch_ref = oracle.pack_w8(w)
     assert np.array_equal(_np(q), q_ref)
+    assert np.array_equal(_np(s_tok), s_tok_ref)
+    assert np.array_equal(_np(pq.pq_unpack_w8(wq, N, K)), wq_ref)
     sel = np.arange(M) if rows is None else rows
     acc_ref, y_ref = oracle.gemm_w8a8(q_ref[sel], s_tok_ref[sel], wq_ref, s_ch_ref)
-    assert np.array_equal(_np(acc)[sel], acc_ref)
-    assert_y_close(_np(y)[sel], y_ref)
+    sel_d = torch.from_numpy(sel).to(DEV)
+    assert np.array_equal(_np(acc[sel_d]), acc_ref)
+    assert_y_close(_np(y[sel_d]), y_ref)
+    if cols is not None:
+        acc_ref, y_ref = oracle.gemm_w8a8(q_ref, s_tok_ref, wq_ref[cols], s_ch_ref[cols])
+        cols_d = torch.from_numpy(cols).to(DEV)
+        assert np.array_equal(_np(acc[:, cols_d]), acc_ref)
+        assert_y_close(_np(y[:, cols_d]), y_ref)
 
 
 def test_config1_tiny_linear_every_element():
@@ -94,11 +112,19 @@ def test_output_guard_bands_stay_untouched():
     assert (buf[:pad] == 7.0).all() and (buf[pad + M * N:] == 7.0).all()
 
 
-@pytest.mark.parametrize("M,K,N", [(2048, 2048, 6144), (4096, 4096, 11008), (512, 11008, 4096)])
-def test_full_size_layers_on_sampled_rows(M, K, N):
+# every (K, N) of the 1B-class layer at M = 2048 and of the 7B-class layer at M = 512 and M = 4096
+@pytest.mark.parametrize("M,K,N", [(2048, 2048, 2048), (2048, 2048, 6144), (2048, 6144, 2048),
+                                   (512, 4096, 4096), (512, 4096, 11008), (512, 11008, 4096),
+                                   (4096, 4096, 4096), (4096, 4096, 11008), (4096, 11008, 4096)])
+def test_full_size_layers_touch_every_tile(M, K, N):
+    """The benchmarked shapes: a token row out of every block of 128 rows x all N channels, and all M rows
+    x a channel out of every block of 64 (at least 256 channels) -- every output tile of every tiling the
+    kernel may choose is compared, the INT32 accumulators bit for bit."""
     rng = np.random.default_rng(M + K + N)
-    rows = np.unique(np.concatenate([[0, 127, 128, M - 129, M - 1], rng.integers(0, M, 19)]))
-    run_case(M, N, K, seed=2000 + N % 97, rows=rows)
+    rows = stratified(M, 128, rng, extra=[127, 128, M - 129])
+    cols = stratified(N, 64, rng, extra=rng.integers(0, N, max(0, 256 - N // 64)))
+    assert len(cols) >= min(N, 200)
+    run_case(M, N, K, seed=2000 + N % 97, rows=rows, cols=cols)
 
 
 @pytest.mark.parametrize("M,K,N", [(512, 11008, 1024), (300, 11008, 520), (140, 6144, 136), (257, 8192, 264)])

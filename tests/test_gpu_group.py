@@ -149,16 +149,18 @@ def test_w4a8_small_token_counts_group_on_the_weight_streaming_kernel(M, K, Ns):
     (4, 2048, 4096, (4096, 4096, 4096)),      # W4A8 q/k/v
     (4, 2048, 4096, (11008, 11008)),          # W4A8 gate/up
 ])
-def test_benchmark_groups_at_full_size_on_sampled_rows(bits, M, K, Ns):
-    """The grouped launches exactly as bench.py issues them; the oracle checks a seeded sample of token
-    rows (all channels of every member: every tile column, first / last / interior row blocks)."""
+def test_benchmark_groups_at_full_size_touch_every_tile(bits, M, K, Ns):
+    """The grouped launches exactly as bench.py issues them.  The oracle checks a token row out of every
+    block of 128 x all channels of every member, and all token rows x a channel out of every block of 64
+    of every member: every output tile of the launch is compared."""
     rng = np.random.default_rng(4600 + M + len(Ns))
-    rows = np.unique(np.concatenate([[0, 127, 128, 255, 256, M - 1], rng.integers(0, M, 10)]))
+    starts = np.arange(0, M, 128)
+    rows = np.unique(np.concatenate([[0, 127, 128, 255, 256, M - 1], np.minimum(starts + rng.integers(0, 128, len(starts)), M - 1)]))
     x = synth.activations(M, K, 4700 + M)
     ws = [synth.weights(N, K, 4800 + i) for i, N in enumerate(Ns)]
     q, s_tok = pq.pq_quantize_act(torch.from_numpy(x).to(DEV))
-    qo, so = oracle.quantize_act(x[rows])
-    assert np.array_equal(q.cpu().numpy()[rows], qo)
+    qo, so = oracle.quantize_act(x)
+    assert np.array_equal(q.cpu().numpy(), qo)
     if bits == 8:
         members = [(*pq.pq_pack_w8(torch.from_numpy(w).to(DEV)), N) for w, N in zip(ws, Ns)]
         out = pq.pq_gemm_w8a8_group(q, s_tok, members)
@@ -167,11 +169,22 @@ def test_benchmark_groups_at_full_size_on_sampled_rows(bits, M, K, Ns):
         out = pq.pq_gemm_w4a8_group(q, s_tok, members)
     torch.cuda.synchronize()
     assert pq.pq_device_status() == 0
-    for w, y in zip(ws, out):
+
+    def close(g, ref):
+        g, ref = g.astype(np.float64), ref.astype(np.float64)
+        return np.isfinite(g).all() and np.all(np.abs(g - ref) <= REL * np.abs(ref) + ABS)
+
+    for w, y, N in zip(ws, out, Ns):
+        cstarts = np.arange(0, N, 64)
+        cols = np.unique(np.concatenate([[0, N - 1], np.minimum(cstarts + rng.integers(0, 64, len(cstarts)), N - 1)]))
+        yh = y.cpu().numpy()
         if bits == 8:
-            _, ref = oracle.gemm_w8a8(qo, so, *oracle.pack_w8(w), want_acc=False)
+            wq, sc = oracle.pack_w8(w)
+            _, ref_r = oracle.gemm_w8a8(qo[rows], so[rows], wq, sc, want_acc=False)
+            _, ref_c = oracle.gemm_w8a8(qo, so, wq[cols], sc[cols], want_acc=False)
         else:
-            _, ref = oracle.gemm_w4a8(qo, so, *oracle.pack_w4(w, 128), 128, want_acc=False)
-        g, ref = y.cpu().numpy()[rows].astype(np.float64), ref.astype(np.float64)
-        assert np.isfinite(g).all()
-        assert np.all(np.abs(g - ref) <= REL * np.abs(ref) + ABS)
+            codes, sg = oracle.pack_w4(w, 128)
+            _, ref_r = oracle.gemm_w4a8(qo[rows], so[rows], codes, sg, 128, want_acc=False)
+            _, ref_c = oracle.gemm_w4a8(qo, so, codes[cols], sg[cols], 128, want_acc=False)
+        assert close(yh[rows], ref_r)
+        assert close(yh[:, cols], ref_c)
