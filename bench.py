@@ -9,13 +9,24 @@ its operands cached.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
 
-Prints ONE JSON line: `value` = whole-step throughput with inputs resident on the device (TOPS for
-prefill workloads, GB/s of algorithmic bytes for decode workloads); `roofline` = the GEMM launches alone
-against the measured peak; `quantize*` = the quantizer and its variants against the measured copy rate;
-`e2e` = the same step with pinned-host inputs copied in and outputs copied out; `cpu_baseline` = the CPU
-oracle on a row sample; `clocks` = SM clocks and throttle reasons sampled during the timed region.
+Prints ONE JSON line.  The timed region of K steps is repeated (each repetition bracketed by a barrier
+and a device synchronization) until at least half a second has been timed; `ms_per_step` is the median
+over the repetitions and `value` the whole-step throughput that follows from it, inputs resident on the
+device (TOPS for prefill workloads, GB/s of algorithmic bytes for decode workloads).  `roofline` = the
+GEMM launches alone against the measured peak (and against the datasheet figure); `workloads` = the same
+two figures for the other benchmark configurations (1B-class layer, 7B-class layer at M = 512, W4A8, the
+decode sweep for both weight formats), each timed for at least 0.3 s; `quantize*` = the quantizer and its
+variants against the measured copy rate; `e2e` = the same step with pinned-host inputs copied in and
+outputs copied out; `cpu_baseline` = the CPU oracle on a row sample; `clocks` = SM clocks and throttle
+reasons sampled over the whole timed span.
 `--impl reference` times the CPU oracle instead (a deliberately plain program; a baseline, not a target).
 Linears that share their input are issued as one grouped call (`--no-group`: one call per linear).
+
+    python bench.py --one-op gemm_w8a8 --shape M,K,N [--members G] [--eager 3]
+
+runs ONE operation on one seeded shape: with --eager a few plain launches (for profilers: one kernel, few
+launches, bounded memory), otherwise a timed CUDA-graph replay of back-to-back launches that rotate over
+buffer sets larger than twice the L2.
 """
 from __future__ import annotations
 
@@ -37,7 +48,14 @@ import numpy as np  # noqa: E402
 from paper_2512_23367_b200 import synth  # noqa: E402
 
 L2_BYTES = 126 * 1024 * 1024
-DEFAULT_WORKLOAD = "c2_w8a8_1b_prefill"
+DEFAULT_WORKLOAD = "c3_w8a8_7b_prefill"      # at its largest token count (M = 4096): the largest single-GPU configuration
+# The other benchmark configurations, reported in the `workloads` block of the same JSON line.
+SIDE_WORKLOADS = (
+    [("c2_w8a8_1b_prefill", 2048), ("c3_w8a8_7b_prefill", 512), ("c4_w4a8_7b_prefill", 2048)]
+    + [("c5_w8a8_7b_decode", m) for m in (1, 4, 16, 64)]
+    + [("c5_w4a8_7b_decode", m) for m in (1, 4, 16, 64)]
+)
+NOMINAL_HBM_GBS = 8000.0
 DATASHEET_INT8_TOPS = 4500.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
@@ -110,6 +128,17 @@ def load_peaks():
         with open(path) as f:
             return json.load(f), "measured"
     return dict(FALLBACK_PEAKS), "fallback"
+
+
+def gemm_launches(wl: synth.Workload, grouped: bool):
+    """The GEMM launches of one step: [(K, [widths])] -- one entry per kernel launch."""
+    out = []
+    for K, idxs in layer_plan(wl):
+        if grouped and len(idxs) > 1:
+            out.append((K, [wl.linears[i].N for i in idxs]))
+        else:
+            out += [(K, [wl.linears[i].N]) for i in idxs]
+    return out
 
 
 def load_traffic(wl: synth.Workload, M: int, grouped: bool = False):
@@ -265,7 +294,7 @@ def run_reference(args, wl: synth.Workload, M: int):
 class LayerBuffers:
     """Device buffers of one decoder layer: inputs, packed weights, scales, outputs."""
 
-    def __init__(self, pq, torch, wl, M, dev, src_x, src_w):
+    def __init__(self, torch, wl, M, dev, src_x, src_w):
         self.xs, self.qs, self.s_toks, self.s_invs, self.groups = [], [], [], [], layer_plan(wl)
         for gi, (K, _) in enumerate(self.groups):
             self.xs.append(src_x[gi].clone())
@@ -278,6 +307,160 @@ class LayerBuffers:
         for i, lin in enumerate(wl.linears):
             self.packed.append(tuple(t.clone() for t in src_w[i]))
             self.ys.append(torch.empty((M, lin.N), dtype=torch.float16, device=dev))
+
+
+class GpuWorkload:
+    """One benchmark configuration resident on the device: seeded inputs, packed weights, the rotation of
+    layer buffer sets, the workspace of the compute stream, and CUDA graphs of the step and of its parts."""
+
+    def __init__(self, pq, torch, wl: synth.Workload, M: int, dev, stream, grouped: bool, use_graphs: bool = True):
+        self.pq, self.torch, self.wl, self.M, self.dev, self.stream = pq, torch, wl, M, dev, stream
+        self.grouped, self.groups = grouped, layer_plan(wl)
+        # One layer of seeded inputs, packed once (offline step); further layers of the rotation are
+        # copies in distinct buffers -- only their addresses matter for cache behaviour.
+        src_x = [torch.from_numpy(synth.activations(M, K, wl.seed(idxs[0]), wl.n_outlier)).to(dev) for K, idxs in self.groups]
+        src_w = []
+        for i, lin in enumerate(wl.linears):
+            w = torch.from_numpy(synth.weights(lin.N, lin.K, wl.seed(i))).to(dev)
+            src_w.append(pq.pq_pack_w8(w) if wl.w_bits == 8 else pq.pq_pack_w4(w))
+            del w
+        self.n_layers = layers_for_rotation(wl, M)
+        self.layers = [LayerBuffers(torch, wl, M, dev, src_x, src_w) for _ in range(self.n_layers)]
+        self.launches = gemm_launches(wl, grouped)
+        self.gemm_per_layer = len(self.launches)
+        self.launches_per_step = len(self.groups) + self.gemm_per_layer
+        # Split-K scratch of the compute stream (W8A8 with few tiles and a long K): the caller's to
+        # provide, sized for the largest need among the step's launches; None when no launch splits.
+        need = max([pq.pq_workspace_bytes(M, Ns, K) for K, Ns in self.launches]) if wl.w_bits == 8 else 0
+        self.workspace = pq.pq_workspace_init(torch.empty((need,), dtype=torch.uint8, device=dev)) if need else None
+        self.workspace_bytes = need
+        # Eager warm-up (also sets kernel attributes), then one CUDA graph per layer buffer set.
+        with torch.cuda.stream(stream):
+            for L in self.layers:
+                self.run_layer(L)
+        stream.synchronize()
+        self.use_graphs = use_graphs
+        self.graphs = self.kind_graphs(None) if use_graphs else []
+
+    def run_layer(self, L: LayerBuffers, only: str | None = None):
+        pq, wl = self.pq, self.wl
+        for gi, (K, idxs) in enumerate(L.groups):
+            if only == "quantize_smooth":
+                pq.pq_quantize_act_smooth(L.xs[gi], L.s_invs[gi], L.qs[gi], L.s_toks[gi])
+                continue
+            if only == "quantize_static":
+                pq.pq_quantize_act_static(L.xs[gi], L.static_scale, L.qs[gi], L.s_toks[gi])
+                continue
+            if only == "quantize_hadamard":
+                pq.pq_quantize_act_hadamard(L.xs[gi], L.qs[gi], L.s_toks[gi])
+                continue
+            if only != "gemm":
+                pq.pq_quantize_act(L.xs[gi], L.qs[gi], L.s_toks[gi])
+            if only == "quantize":
+                continue
+            if self.grouped and len(idxs) > 1:
+                # linears over the same codes (q/k/v, gate/up): one grouped call, one kernel launch
+                members = [(L.packed[i][0], L.packed[i][1], wl.linears[i].N) for i in idxs]
+                if wl.w_bits == 8:
+                    pq.pq_gemm_w8a8_group(L.qs[gi], L.s_toks[gi], members, [L.ys[i] for i in idxs], workspace=self.workspace)
+                else:
+                    pq.pq_gemm_w4a8_group(L.qs[gi], L.s_toks[gi], members, [L.ys[i] for i in idxs])
+                continue
+            for i in idxs:
+                N = wl.linears[i].N
+                a, b = L.packed[i]
+                if wl.w_bits == 8:
+                    pq.pq_gemm_w8a8(L.qs[gi], L.s_toks[gi], a, b, N, y=L.ys[i], workspace=self.workspace)
+                else:
+                    pq.pq_gemm_w4a8(L.qs[gi], L.s_toks[gi], a, b, N, y=L.ys[i])
+
+    def kind_graphs(self, which: str | None):
+        """One CUDA graph per layer buffer set holding the whole step (which=None) or only its GEMMs /
+        only its quantizers (same buffers, same launch configuration)."""
+        torch, gs = self.torch, []
+        for L in self.layers:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=self.stream):
+                self.run_layer(L, only=which)
+            gs.append(g)
+        return gs
+
+    def step(self, i: int):
+        if self.graphs:
+            self.graphs[i % self.n_layers].replay()
+        else:
+            self.run_layer(self.layers[i % self.n_layers])
+
+    def time_replays(self, gs, launches_per_replay: int, min_ms: float):
+        """Average launch duration (ms) of the kernels in `gs`, replayed back to back on the launching
+        stream and timed with CUDA events there: event time / launches (launch gaps included, so the
+        figure is conservative).  Repeats until at least `min_ms` have been timed."""
+        torch, stream = self.torch, self.stream
+        with torch.cuda.stream(stream):
+            for _ in range(3):
+                for g in gs:
+                    g.replay()
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for g in gs:
+                g.replay()
+            b.record(stream)
+            torch.cuda.synchronize()
+            rounds = int(max(3, min(20000, 1.1 * min_ms / max(a.elapsed_time(b), 1e-3))))
+            a.record(stream)
+            for _ in range(rounds):
+                for g in gs:
+                    g.replay()
+            b.record(stream)
+            torch.cuda.synchronize()
+        n = rounds * len(gs) * launches_per_replay
+        return a.elapsed_time(b) / n, n
+
+    def roofline(self, gemm_avg_ms: float, gemm_launches_timed: int, peaks: dict, peak_kind: str) -> dict:
+        """The GEMM launches of the step against the roofline that bounds them."""
+        wl, M = self.wl, self.M
+        if M > 64:
+            tops = step_ops(wl, M) / (gemm_avg_ms * self.gemm_per_layer * 1e-3) / 1e12
+            peak = 2.0 * float(peaks["bf16_tflops"])
+            return {"bound": "tensor", "achieved": tops, "peak": peak, "unit": "TOPS", "frac": tops / peak,
+                    "traffic": load_traffic(wl, M, self.grouped),
+                    "kernel": f"gemm_w{wl.w_bits}a8 (tcgen05 kind::i8)",
+                    "peak_kind": f"2 x bf16_tflops (burst) of {peak_kind}: INT8 peak = bf16 peak x nominal 4.5/2.25",
+                    "frac_of_sustained": tops / (2.0 * float(peaks["bf16_tflops_sustained"])),
+                    "frac_of_datasheet_4500": tops / DATASHEET_INT8_TOPS,
+                    "avg_launch_us": gemm_avg_ms * 1e3, "launches_timed": gemm_launches_timed}
+        gbs = step_bytes(wl, M)["gemm"] / (gemm_avg_ms * self.gemm_per_layer * 1e-3) / 1e9
+        peak = float(peaks["hbm_gbs"])
+        return {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
+                "traffic": load_traffic(wl, M, self.grouped),
+                "kernel": f"small-M gemm_w{wl.w_bits}a8", "peak_kind": f"hbm_gbs of {peak_kind}",
+                "frac_of_nominal_8000": gbs / NOMINAL_HBM_GBS,
+                "avg_launch_us": gemm_avg_ms * 1e3, "launches_timed": gemm_launches_timed}
+
+    def value_of(self, ms_per_step: float, world: int = 1):
+        """(metric, unit, value) of the whole job for a step time."""
+        wl, M = self.wl, self.M
+        if M <= 64:
+            b = step_bytes(wl, M)
+            return "quantized_linear_gbs", "GB/s", (b["gemm"] + b["quantize"]) * world / (ms_per_step * 1e-3) / 1e9
+        return "quantized_linear_tops", "TOPS", step_ops(wl, M) * world / (ms_per_step * 1e-3) / 1e12
+
+
+def side_workload(pq, torch, name: str, M: int, dev, stream, grouped: bool, peaks, peak_kind, min_ms: float = 300.0) -> dict:
+    """Whole-step throughput and GEMM-only roofline of one more benchmark configuration."""
+    wl = synth.WORKLOADS[name]
+    w = GpuWorkload(pq, torch, wl, M, dev, stream, grouped)
+    step_ms, _ = w.time_replays(w.graphs, 1, min_ms)
+    gemm_ms, n = w.time_replays(w.kind_graphs("gemm"), w.gemm_per_layer, min_ms)
+    quant_ms, _ = w.time_replays(w.kind_graphs("quantize"), len(w.groups), min_ms / 3)
+    _, unit, value = w.value_of(step_ms)
+    roof = w.roofline(gemm_ms, n, peaks, peak_kind)
+    quant_gbs = step_bytes(wl, M)["quantize"] / (quant_ms * len(w.groups) * 1e-3) / 1e9
+    return {"workload": name, "M": M, "w_bits": wl.w_bits, "value": value, "unit": unit, "ms_per_step": step_ms,
+            "launches_per_step": w.launches_per_step, "frac": roof["frac"], "avg_launch_us": roof["avg_launch_us"],
+            "roofline": roof, "quantize_frac_of_hbm": quant_gbs / float(peaks["hbm_gbs"]),
+            "rotation_layers": w.n_layers}
 
 
 def run_ours(args, wl: synth.Workload, M: int):
@@ -296,137 +479,57 @@ def run_ours(args, wl: synth.Workload, M: int):
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
     pq.lib()
+    peaks, peak_kind = load_peaks()
 
-    # One layer of seeded inputs, packed once (offline step); further layers of the rotation are
-    # copies in distinct buffers -- only their addresses matter for cache behaviour.
-    groups = layer_plan(wl)
-    src_x = [torch.from_numpy(synth.activations(M, K, wl.seed(idxs[0]), wl.n_outlier)).to(dev) for K, idxs in groups]
-    src_w = []
-    for i, lin in enumerate(wl.linears):
-        w = torch.from_numpy(synth.weights(lin.N, lin.K, wl.seed(i))).to(dev)
-        src_w.append(pq.pq_pack_w8(w) if wl.w_bits == 8 else pq.pq_pack_w4(w))
-        del w
-    n_layers = layers_for_rotation(wl, M)
-    layers = [LayerBuffers(pq, torch, wl, M, dev, src_x, src_w) for _ in range(n_layers)]
-
-    # The grouped calls schedule their members in one launch.
     grouped = not args.no_group
-
-    def run_layer(L: LayerBuffers, only: str | None = None):
-        for gi, (K, idxs) in enumerate(L.groups):
-            if only == "quantize_smooth":
-                pq.pq_quantize_act_smooth(L.xs[gi], L.s_invs[gi], L.qs[gi], L.s_toks[gi])
-                continue
-            if only == "quantize_static":
-                pq.pq_quantize_act_static(L.xs[gi], L.static_scale, L.qs[gi], L.s_toks[gi])
-                continue
-            if only == "quantize_hadamard":
-                pq.pq_quantize_act_hadamard(L.xs[gi], L.qs[gi], L.s_toks[gi])
-                continue
-            if only != "gemm":
-                pq.pq_quantize_act(L.xs[gi], L.qs[gi], L.s_toks[gi])
-            if only == "quantize":
-                continue
-            if grouped and len(idxs) > 1:
-                # linears over the same codes (q/k/v, gate/up): one grouped call, one kernel launch
-                group_call = pq.pq_gemm_w8a8_group if wl.w_bits == 8 else pq.pq_gemm_w4a8_group
-                group_call(L.qs[gi], L.s_toks[gi], [(L.packed[i][0], L.packed[i][1], wl.linears[i].N) for i in idxs],
-                           [L.ys[i] for i in idxs])
-                continue
-            for i in idxs:
-                N = wl.linears[i].N
-                a, b = L.packed[i]
-                if wl.w_bits == 8:
-                    pq.pq_gemm_w8a8(L.qs[gi], L.s_toks[gi], a, b, N, y=L.ys[i])
-                else:
-                    pq.pq_gemm_w4a8(L.qs[gi], L.s_toks[gi], a, b, N, y=L.ys[i])
-
-    gemm_per_layer = sum(1 if grouped and len(idxs) > 1 else len(idxs) for _, idxs in groups)   # GEMM launches
-    launches_per_step = len(groups) + gemm_per_layer
-
-    # Eager warm-up (also sets kernel attributes), then one CUDA graph per layer buffer set.
     stream = torch.cuda.Stream(device=dev)
-    with torch.cuda.stream(stream):
-        for L in layers:
-            run_layer(L)
-    stream.synchronize()
-    graphs = []
-    if not args.no_graph:
-        for L in layers:
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g, stream=stream):
-                run_layer(L)
-            graphs.append(g)
-
-    def step(i: int):
-        if graphs:
-            graphs[i % n_layers].replay()
-        else:
-            run_layer(layers[i % n_layers])
+    W = GpuWorkload(pq, torch, wl, M, dev, stream, grouped, use_graphs=not args.no_graph)
+    groups, n_layers, layers = W.groups, W.n_layers, W.layers
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- device-resident throughput
+    # ---- device-resident throughput: rounds of exactly `steps` steps, each bracketed by a barrier and a
+    # device synchronization and timed with CUDA events on the launching stream, repeated until at least
+    # MIN_TIMED_MS have been timed; the clock sampler runs over the whole span.
+    MIN_TIMED_MS, MAX_ROUNDS = 500.0, 400
     sampler = ClockSampler(local_rank)
+    round_ms = []
     with torch.cuda.stream(stream):
         for i in range(args.warmup):
-            step(i)
+            W.step(i)
         barrier()
         if rank == 0:
             sampler.start()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for i in range(args.steps):
-            step(args.warmup + i)
-        e1.record(stream)
-        barrier()
+        it = args.warmup
+        while True:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            barrier()
+            e0.record(stream)
+            for i in range(args.steps):
+                W.step(it + i)
+            e1.record(stream)
+            barrier()
+            it += args.steps
+            local = e0.elapsed_time(e1)
+            total_ms, _ = aggregate_over_ranks(local, 0.0, world)     # max over ranks: the same on every rank
+            round_ms.append(total_ms)
+            if sum(round_ms) >= MIN_TIMED_MS or len(round_ms) >= MAX_ROUNDS:
+                break
     clocks = sampler.stop() if rank == 0 else None
-    local_ms = e0.elapsed_time(e1)
+    ms_per_step = statistics.median(round_ms) / args.steps
     ops = step_ops(wl, M)
-    total_ms, total_ops = aggregate_over_ranks(local_ms, float(ops) * args.steps, world)
 
     # ---- per-kernel durations: the same launches on the same buffers, replayed as graphs that hold
-    # only the GEMMs (or only the quantizers) of a layer, timed with CUDA events on the launching
-    # stream.  Event time / launches = average launch duration of that kernel inside a back-to-back
-    # stream of its own kind (launch gaps included, so the figure is conservative).
-    def kind_graphs(which: str):
-        gs = []
-        for L in layers:
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g, stream=stream):
-                run_layer(L, only=which)
-            gs.append(g)
-        return gs
-
-    def time_kind(gs, launches_per_replay: int, budget_ms: float = 400.0):
-        with torch.cuda.stream(stream):
-            for g in gs:
-                g.replay()
-            torch.cuda.synchronize()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream)
-            for g in gs:
-                g.replay()
-            b.record(stream)
-            torch.cuda.synchronize()
-            rounds = int(max(3, min(2000, budget_ms / max(a.elapsed_time(b), 1e-3))))
-            a.record(stream)
-            for _ in range(rounds):
-                for g in gs:
-                    g.replay()
-            b.record(stream)
-            torch.cuda.synchronize()
-        n = rounds * len(gs) * launches_per_replay
-        return a.elapsed_time(b) / n, n
-
-    gemm_avg_ms, gemm_launches = time_kind(kind_graphs("gemm"), gemm_per_layer)
-    quant_avg_ms, quant_launches = time_kind(kind_graphs("quantize"), len(groups))
-    smooth_avg_ms, _ = time_kind(kind_graphs("quantize_smooth"), len(groups), budget_ms=200.0)
-    hadamard_avg_ms, _ = time_kind(kind_graphs("quantize_hadamard"), len(groups), budget_ms=200.0)
-    static_avg_ms, _ = time_kind(kind_graphs("quantize_static"), len(groups), budget_ms=200.0)
+    # only the GEMMs (or only the quantizers) of a layer.
+    gemm_per_layer = W.gemm_per_layer
+    gemm_avg_ms, gemm_launches_timed = W.time_replays(W.kind_graphs("gemm"), gemm_per_layer, 400.0)
+    quant_avg_ms, quant_launches = W.time_replays(W.kind_graphs("quantize"), len(groups), 300.0)
+    smooth_avg_ms, _ = W.time_replays(W.kind_graphs("quantize_smooth"), len(groups), 150.0)
+    hadamard_avg_ms, _ = W.time_replays(W.kind_graphs("quantize_hadamard"), len(groups), 150.0)
+    static_avg_ms, _ = W.time_replays(W.kind_graphs("quantize_static"), len(groups), 150.0)
 
     # ---- context (not a target): the same seven shapes as FP16 GEMMs from the vendor library
     # (torch.matmul -> cuBLAS), the comparison the paper's prefill table makes on its own hardware.
@@ -452,7 +555,7 @@ def run_ours(args, wl: synth.Workload, M: int):
             with torch.cuda.graph(g, stream=stream):
                 fp16_layer(ws)
             gs16.append(g)
-        fp16_avg_ms, _ = time_kind(gs16, len(wl.linears), budget_ms=200.0)
+        fp16_avg_ms, _ = W.time_replays(gs16, len(wl.linears), 200.0)
         fp16_ctx = {"kernel": "torch.matmul FP16 (cuBLAS), same shapes", "avg_launch_us": fp16_avg_ms * 1e3,
                     "tflops": ops / (fp16_avg_ms * len(wl.linears) * 1e-3) / 1e12,
                     "int8_over_fp16_speedup": (fp16_avg_ms * len(wl.linears)) / (gemm_avg_ms * gemm_per_layer),
@@ -481,7 +584,7 @@ def run_ours(args, wl: synth.Workload, M: int):
                 with torch.cuda.graph(g, stream=stream):
                     int8_layer(ws)
                 gs8.append(g)
-            lib8_avg_ms, _ = time_kind(gs8, len(wl.linears), budget_ms=200.0)
+            lib8_avg_ms, _ = W.time_replays(gs8, len(wl.linears), 200.0)
             fp16_ctx["library_int8"] = {
                 "kernel": "torch._int_mm (cuBLASLt INT8 -> INT32, no dequantization), same shapes",
                 "tops": ops / (lib8_avg_ms * len(wl.linears) * 1e-3) / 1e12,
@@ -489,7 +592,6 @@ def run_ours(args, wl: synth.Workload, M: int):
             del xs8, ws8, ys8, gs8
         except Exception as e:   # the library call is context only: its absence must not fail the benchmark
             fp16_ctx["library_int8"] = {"unavailable": f"{type(e).__name__}: {str(e)[:120]}"}
-    gemm_tops = ops / (gemm_avg_ms * gemm_per_layer * 1e-3) / 1e12
     sbytes = step_bytes(wl, M)
     quant_gbs = sbytes["quantize"] / (quant_avg_ms * len(groups) * 1e-3) / 1e9
     smooth_bytes = sbytes["quantize"] + sum(4 * K for K, _ in groups)   # + the [K] FP32 factor vector per call
@@ -526,7 +628,7 @@ def run_ours(args, wl: synth.Workload, M: int):
             stream.wait_event(in_done)
             if prev in out_done:
                 stream.wait_event(out_done[prev])       # the set's outputs have been copied out
-            run_layer(L)
+            W.run_layer(L)
             comp_done[i] = torch.cuda.Event()
             comp_done[i].record(stream)
         with torch.cuda.stream(s_out):
@@ -555,67 +657,63 @@ def run_ours(args, wl: synth.Workload, M: int):
     join_all()
     f1.record(stream)
     barrier()
-    e2e_ms, e2e_ops = aggregate_over_ranks(f0.elapsed_time(f1), float(ops) * e2e_steps, world)
+    e2e_ms, _ = aggregate_over_ranks(f0.elapsed_time(f1), 0.0, world)
 
     status = pq.pq_device_status()
     if status != 0:
         raise SystemExit(f"bench.py: device status {status} after the timed region")
 
+    # ---- the other benchmark configurations (single GPU only: a scaling run repeats the main workload)
+    side = None
+    if world == 1 and not args.no_side_workloads:
+        del host_x, host_y
+        side = []
+        for name, m in SIDE_WORKLOADS:
+            if name == wl.name and m == M:
+                continue
+            torch.cuda.empty_cache()
+            side.append(side_workload(pq, torch, name, m, dev, stream, grouped, peaks, peak_kind))
+        status = pq.pq_device_status()
+        if status != 0:
+            raise SystemExit(f"bench.py: device status {status} after the side workloads")
+
     if rank == 0:
-        peaks, peak_kind = load_peaks()
-        if wl.w_bits and M > 64:
-            peak = 2.0 * float(peaks["bf16_tflops"])
-            roof = {"bound": "tensor", "achieved": gemm_tops, "peak": peak, "unit": "TOPS",
-                    "frac": gemm_tops / peak, "traffic": load_traffic(wl, M, grouped),
-                    "kernel": f"gemm_w{wl.w_bits}a8 (tcgen05 kind::i8)",
-                    "peak_kind": f"2 x bf16_tflops (burst) of {peak_kind}: INT8 peak = bf16 peak x nominal 4.5/2.25",
-                    "frac_of_sustained": gemm_tops / (2.0 * float(peaks["bf16_tflops_sustained"])),
-                    "frac_of_datasheet_4500": gemm_tops / DATASHEET_INT8_TOPS,
-                    "avg_launch_us": gemm_avg_ms * 1e3, "launches_timed": gemm_launches}
-        else:
-            gbs = sbytes["gemm"] / (gemm_avg_ms * gemm_per_layer * 1e-3) / 1e9
-            peak = float(peaks["hbm_gbs"])
-            roof = {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
-                    "traffic": load_traffic(wl, M, grouped),
-                    "kernel": f"small-M gemm_w{wl.w_bits}a8", "peak_kind": f"hbm_gbs of {peak_kind}",
-                    "avg_launch_us": gemm_avg_ms * 1e3, "launches_timed": gemm_launches}
-        decode = M <= 64
-        if decode:
-            metric, unit = "quantized_linear_gbs", "GB/s"
-            per_step = sbytes["gemm"] + sbytes["quantize"]
-            value = per_step * args.steps * world / (total_ms * 1e-3) / 1e9
-            e2e_value = per_step * e2e_steps * world / (e2e_ms * 1e-3) / 1e9
-        else:
-            metric, unit = "quantized_linear_tops", "TOPS"
-            value = total_ops / (total_ms * 1e-3) / 1e12
-            e2e_value = e2e_ops / (e2e_ms * 1e-3) / 1e12
+        roof = W.roofline(gemm_avg_ms, gemm_launches_timed, peaks, peak_kind)
+        metric, unit, value = W.value_of(ms_per_step, world)
+        _, _, e2e_value = W.value_of(e2e_ms / e2e_steps, world)
+        hbm = float(peaks["hbm_gbs"])
         out = {
             "metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
             "config": {"workload": wl.name, "M": M, "w_bits": wl.w_bits,
                        "linears": [[lin.name, lin.K, lin.N] for lin in wl.linears],
                        "step": f"{len(groups)} activation quantizations + {len(wl.linears)} quantized linears "
-                               f"(one decoder layer) in {launches_per_step} kernel launches",
+                               f"(one decoder layer) in {W.launches_per_step} kernel launches",
                        "grouped_calls": bool(grouped),
                        "cache": f"rotation over {n_layers} distinct layer buffer sets (> 2 x L2)",
-                       "launch": "cuda_graph_per_layer" if graphs else "eager", "parallelism": "replicas"},
+                       "launch": "cuda_graph_per_layer" if W.graphs else "eager", "parallelism": "replicas",
+                       "workspace_bytes": W.workspace_bytes},
+            "timing": {"rounds": len(round_ms), "steps_per_round": args.steps, "timed_ms_total": sum(round_ms),
+                       "ms_per_step_min": min(round_ms) / args.steps, "ms_per_step_max": max(round_ms) / args.steps,
+                       "ms_per_step": "median over rounds"},
             "roofline": roof,
+            "workloads": side,
             "fp16_context": fp16_ctx,
-            "quantize": {"achieved_gbs": quant_gbs, "frac_of_hbm": quant_gbs / float(peaks["hbm_gbs"]),
+            "quantize": {"achieved_gbs": quant_gbs, "frac_of_hbm": quant_gbs / hbm,
                          "avg_launch_us": quant_avg_ms * 1e3, "launches_timed": quant_launches},
-            "quantize_smooth": {"achieved_gbs": smooth_gbs, "frac_of_hbm": smooth_gbs / float(peaks["hbm_gbs"]),
+            "quantize_smooth": {"achieved_gbs": smooth_gbs, "frac_of_hbm": smooth_gbs / hbm,
                                 "avg_launch_us": smooth_avg_ms * 1e3,
                                 "what": "pq_quantize_act_smooth (Eq. 3: X S^-1) on the same inputs; not part of the step"},
-            "quantize_hadamard": {"achieved_gbs": hadamard_gbs, "frac_of_hbm": hadamard_gbs / float(peaks["hbm_gbs"]),
+            "quantize_hadamard": {"achieved_gbs": hadamard_gbs, "frac_of_hbm": hadamard_gbs / hbm,
                                   "avg_launch_us": hadamard_avg_ms * 1e3,
                                   "what": "pq_quantize_act_hadamard (Eq. 4: X H) on the same inputs; not part of the step"},
-            "quantize_static": {"achieved_gbs": static_gbs, "frac_of_hbm": static_gbs / float(peaks["hbm_gbs"]),
+            "quantize_static": {"achieved_gbs": static_gbs, "frac_of_hbm": static_gbs / hbm,
                                 "avg_launch_us": static_avg_ms * 1e3,
                                 "what": "pq_quantize_act_static (one calibrated scale) on the same inputs; not part of the step"},
             "e2e": {"value": e2e_value, "unit": unit, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps, "overlap": "copy-in, compute and copy-out on three streams"},
-            "gpu_launches": launches_per_step * args.steps,
+            "gpu_launches": W.launches_per_step * args.steps,
             "clocks": clocks,
         }
         if not args.no_cpu_baseline and world == 1:
@@ -625,11 +723,112 @@ def run_ours(args, wl: synth.Workload, M: int):
         dist.destroy_process_group()
 
 
+# --------------------------------------------------------------------------- one operation (profilers, per-shape timing)
+
+QUANT_OPS = ("quantize", "quantize_smooth", "quantize_hadamard", "quantize_static")
+ONE_OPS = QUANT_OPS + ("gemm_w8a8", "gemm_w4a8")
+
+
+def run_one_op(args):
+    """ONE operation on one seeded shape.  --eager n: n plain launches and exit (for profilers);
+    otherwise a CUDA graph of back-to-back launches rotating over buffer sets > 2 x L2, timed with events."""
+    import torch
+
+    import paper_2512_23367_b200 as pq
+
+    op = args.one_op
+    dims = [int(v) for v in args.shape.split(",")]
+    M, K = dims[0], dims[1]
+    N = dims[2] if len(dims) > 2 else 0
+    G = max(args.members, 1)
+    if op not in QUANT_OPS and N <= 0:
+        raise SystemExit("bench.py --one-op gemm_*: --shape M,K,N")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    per_set = 3 * M * K + (G * N * K if op not in QUANT_OPS else 0)
+    sets = args.sets or max(2, min(16, (2 * L2_BYTES) // max(per_set, 1) + 1))
+    x = torch.from_numpy(synth.activations(M, K, 9000)).to(dev)
+    packed = []
+    for g in range(G if op not in QUANT_OPS else 0):
+        w = torch.from_numpy(synth.weights(N, K, 9001 + g)).to(dev)
+        packed.append(pq.pq_pack_w8(w) if op == "gemm_w8a8" else pq.pq_pack_w4(w))
+        del w
+    need = pq.pq_workspace_bytes(M, [N] * G, K) if op == "gemm_w8a8" else 0
+    ws = pq.pq_workspace_init(torch.empty((need,), dtype=torch.uint8, device=dev)) if need else None
+    bufs = []
+    for _ in range(sets):
+        xc = x.clone()
+        q, s_tok = pq.pq_quantize_act(xc)
+        b = {"x": xc, "q": q, "s_tok": s_tok, "s_inv": torch.rand((K,), device=dev, dtype=torch.float32) + 0.5,
+             "scale": torch.full((1,), 0.05, device=dev, dtype=torch.float32),
+             "w": [tuple(t.clone() for t in p) for p in packed],
+             "y": [torch.empty((M, N), device=dev, dtype=torch.float16) for _ in packed]}
+        bufs.append(b)
+
+    def launch(i):
+        b = bufs[i % sets]
+        if op == "quantize":
+            pq.pq_quantize_act(b["x"], b["q"], b["s_tok"])
+        elif op == "quantize_smooth":
+            pq.pq_quantize_act_smooth(b["x"], b["s_inv"], b["q"], b["s_tok"])
+        elif op == "quantize_hadamard":
+            pq.pq_quantize_act_hadamard(b["x"], b["q"], b["s_tok"])
+        elif op == "quantize_static":
+            pq.pq_quantize_act_static(b["x"], b["scale"], b["q"], b["s_tok"])
+        elif G > 1 and op == "gemm_w8a8":
+            pq.pq_gemm_w8a8_group(b["q"], b["s_tok"], [(w[0], w[1], N) for w in b["w"]], b["y"], workspace=ws)
+        elif G > 1:
+            pq.pq_gemm_w4a8_group(b["q"], b["s_tok"], [(w[0], w[1], N) for w in b["w"]], b["y"])
+        elif op == "gemm_w8a8":
+            pq.pq_gemm_w8a8(b["q"], b["s_tok"], b["w"][0][0], b["w"][0][1], N, y=b["y"][0], workspace=ws)
+        else:
+            pq.pq_gemm_w4a8(b["q"], b["s_tok"], b["w"][0][0], b["w"][0][1], N, y=b["y"][0])
+
+    base = {"op": op, "M": M, "K": K, "N": N, "members": G, "sets": sets}
+    if args.eager:
+        for i in range(args.eager):
+            launch(i)
+        torch.cuda.synchronize()
+        print(json.dumps({**base, "eager_launches": args.eager, "status": pq.pq_device_status()}))
+        return
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        for i in range(sets):
+            launch(i)
+    stream.synchronize()
+    n_launch = 16
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=stream):
+        for i in range(n_launch):
+            launch(i)
+    times = []
+    with torch.cuda.stream(stream):
+        for _ in range(3):
+            g.replay()
+        for _ in range(20):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            g.replay()
+            e1.record(stream)
+            times.append((e0, e1))
+        stream.synchronize()
+    us = sorted(e0.elapsed_time(e1) * 1e3 / n_launch for e0, e1 in times)
+    med = us[len(us) // 2]
+    out = {**base, "us_median": med, "us_min": us[0], "status": pq.pq_device_status()}
+    if op in QUANT_OPS:
+        out["GBps"] = (3 * M * K + 4 * M + (4 * K if op == "quantize_smooth" else 0)) / med / 1e3
+    else:
+        out["TOPS"] = 2 * M * G * N * K / med / 1e6
+        wbytes = N * K + 4 * N if op == "gemm_w8a8" else N * K // 2 + (K // 128) * N * 2
+        out["GBps"] = (G * wbytes + M * K + 4 * M + 2 * M * G * N) / med / 1e3
+    print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20000)
-    ap.add_argument("--warmup", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(synth.WORKLOADS))
     ap.add_argument("--M", type=int, default=None, help="token count (default: the workload's largest)")
@@ -638,7 +837,15 @@ def main():
     ap.add_argument("--no-group", action="store_true",
                     help="one GEMM call per linear instead of grouped calls for linears that share their input")
     ap.add_argument("--no-fp16-context", action="store_true", help="skip the cuBLAS FP16 same-shape timing")
+    ap.add_argument("--no-side-workloads", action="store_true", help="skip the `workloads` block (the other configurations)")
+    ap.add_argument("--one-op", choices=ONE_OPS, default=None, help="run one operation on one shape instead of a workload")
+    ap.add_argument("--shape", default="", help="--one-op: M,K[,N]")
+    ap.add_argument("--members", type=int, default=1, help="--one-op gemm_*: this many linears of width N in one grouped call")
+    ap.add_argument("--sets", type=int, default=0, help="--one-op: distinct buffer sets (0 = enough to exceed 2 x L2, max 16)")
+    ap.add_argument("--eager", type=int, default=0, help="--one-op: run this many plain launches and exit (for profilers)")
     args = ap.parse_args()
+    if args.one_op:
+        return run_one_op(args)
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     wl = synth.WORKLOADS[args.workload]
     M = args.M if args.M is not None else max(wl.Ms)

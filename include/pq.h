@@ -26,8 +26,12 @@
  *     is launched.  Nothing aborts, throws or traps; non-finite inputs are memory
  *     safe with unspecified results.
  *   - Every wait inside a kernel is bounded; if one expires the kernel records
- *     PQ_ERR_TIMEOUT in a device status word, drains and returns.  pq_device_status()
- *     reads that word.
+ *     PQ_ERR_TIMEOUT in a device status word, waits (bounded) for the copies and MMAs it has
+ *     in flight, and returns; the outputs of that call are then unspecified.
+ *     pq_device_status() reads that word.
+ *   - The library keeps no per-call state on the host: calls may be made from several host
+ *     threads and on several streams at once.  The only memory a call shares with other calls
+ *     is what the caller passes in (see `workspace` below).
  *   - Requires compute capability 10.0; anything else returns PQ_ERR_ARCH (there is
  *     no fallback path).
  */
@@ -172,9 +176,24 @@ PQ_API int pq_unpack_w4(const void* wp, int64_t N, int64_t K, int8_t* codes, voi
  *   y_f16 [M,N] FP16 out.
  * Any M is accepted; small M (decode shapes) is routed to a weight-streaming schedule
  * that computes the same result.
+ *
+ * workspace / workspace_bytes: optional scratch of THIS call (NULL / 0 = none).  With few output
+ * tiles and a long K (e.g. a 7B-class layer at M = 512) the GEMM cuts K into parts that run on
+ * different SMs; the parts' INT32 partial accumulators pass through the workspace and are summed
+ * exactly, so the result does not depend on it.  Without a workspace, or with one too small for the
+ * shape, K is simply not split.  (The paper's "matrix multiplication ... within the operator
+ * template library" leaves scheduling to the kernel; this is scheduling only.)
+ *   - Device memory owned by the caller, 256-byte aligned (else PQ_ERR_ALIGN), of at least
+ *     pq_workspace_bytes(...) bytes for the shape to be served in full.
+ *   - Before its first use it is prepared once with pq_workspace_init (which zeroes its first
+ *     64 KB, the arrival counters); every call that completes leaves it prepared for the next.
+ *     After a PQ_ERR_TIMEOUT prepare it again.
+ *   - Calls that may overlap on the GPU (different streams, parallel graph branches) must be
+ *     given different workspaces; calls ordered in one stream may share one.
  */
 PQ_API int pq_gemm_w8a8(const int8_t* q, const float* s_tok, const void* wq, const float* s_ch,
-                 int64_t M, int64_t N, int64_t K, void* y_f16, void* stream);
+                 int64_t M, int64_t N, int64_t K, void* y_f16, void* workspace, size_t workspace_bytes,
+                 void* stream);
 
 /*
  * W4A8 linear: INT4 codes are widened to INT8 inside the kernel, multiplied in
@@ -207,11 +226,12 @@ PQ_API int pq_acc_w4a8(const int8_t* q, const void* wp, int32_t group, int64_t M
  *   count: 1..PQ_MAX_GROUP.  wq, s_ch, N, y_f16: HOST arrays of `count` entries (device pointers
  *   and column counts; read during the call, not retained).  q, s_tok, M, K as in pq_gemm_w8a8.
  *   The outputs must not overlap each other.  On an argument error nothing is launched.
+ *   workspace / workspace_bytes: as for pq_gemm_w8a8 (sized with pq_workspace_bytes for the group).
  */
 #define PQ_MAX_GROUP 4
 PQ_API int pq_gemm_w8a8_group(const int8_t* q, const float* s_tok, int32_t count, const void* const* wq,
                               const float* const* s_ch, const int64_t* N, void* const* y_f16, int64_t M,
-                              int64_t K, void* stream);
+                              int64_t K, void* workspace, size_t workspace_bytes, void* stream);
 
 /* The same for W4A8 linears (pq_gemm_w4a8 per member; one launch for all of them, except at M <= 64 when
  * the members together hold more 128-channel tiles than the device has SMs).  For M <= 64 the FP32
@@ -222,22 +242,23 @@ PQ_API int pq_gemm_w4a8_group(const int8_t* q, const float* s_tok, int32_t count
                               void* const* y_f16, int64_t M, int64_t K, void* stream);
 
 /*
- * Optional scratch memory for the current device.  With few output tiles and a long K (e.g. a
- * 7B-class layer at M = 512) the W8A8 GEMM cuts K into parts that run on different SMs; the parts'
- * INT32 partial accumulators pass through this scratch and are summed exactly, so results do not
- * change.  Without registered scratch (or when it is too small for a shape) the GEMM simply does
- * not split.  (The paper's "matrix multiplication ... within the operator template library" leaves
- * scheduling to the kernel; this is scheduling only.)
- *   workspace: device pointer, 256-byte aligned, owned by the caller, at least 64 KB + 1 MB
- *   (64 MB serves every 7B-class shape); NULL or 0 bytes unregisters.  Its first 64 KB are cleared
- *   on `stream`; GEMM calls enqueued afterwards on that stream (or after a synchronization) may use
- *   it.  Calls that overlap on the GPU must not share one workspace.
+ * Workspace of the W8A8 calls (see pq_gemm_w8a8).
+ *   pq_workspace_bytes: host-only (touches no device).  The number of bytes with which
+ *     pq_gemm_w8a8 (count = 1) or pq_gemm_w8a8_group over the column counts N[0..count) at these M
+ *     and K runs the schedule it would pick with unlimited room, on a GPU with `sms`
+ *     multiprocessors (148 on a B200); 0 when that schedule does not split K (then no workspace is
+ *     of any use) or when an argument is invalid.  The maximum over the shapes a caller issues
+ *     serves all of them.  pq_gemm_w4a8 and every decode-shaped call (M <= 128) need none.
+ *   pq_workspace_init: zeroes the first 64 KB of `workspace` on `stream` (bytes >= 65536, 256-byte
+ *     aligned).  GEMM calls enqueued afterwards on that stream (or after a synchronization) may
+ *     use the workspace.  A buffer the caller has zero-filled by other means is equally good.
  */
-PQ_API int pq_set_workspace(void* workspace, size_t bytes, void* stream);
+PQ_API size_t pq_workspace_bytes(int64_t M, const int64_t* N, int32_t count, int64_t K, int32_t sms);
+PQ_API int pq_workspace_init(void* workspace, size_t bytes, void* stream);
 
 /*
  * Host-only query (touches no device): the schedule pq_gemm_w8a8 picks for M > 128 on a GPU with
- * `sms` multiprocessors and a registered workspace of `scratch_bytes` (0 = none): the output tile
+ * `sms` multiprocessors and a workspace of `scratch_bytes` (0 = none): the output tile
  * width (*tile_n = 256 or 128 columns) and the number of parts K is cut into (*k_parts, 1 = no
  * split).  For capacity planning and tests; the result has no effect on later calls.
  */
@@ -248,8 +269,8 @@ PQ_API int pq_plan_w8a8(int64_t M, int64_t N, int64_t K, int32_t sms, size_t scr
  * W8A8 linear for callers that cannot allocate device memory (the paper has no counterpart to
  * this call; it exists for deployment constraints, not for the method).
  *
- * Same arguments, same result as pq_gemm_w8a8.  The difference is where the split-K scratch comes
- * from: not from a buffer registered with pq_set_workspace -- which somebody had to cudaMalloc --
+ * Same result as pq_gemm_w8a8, same arguments without the workspace.  The difference is where the
+ * split-K scratch comes from: not from a workspace argument -- which somebody had to cudaMalloc --
  * but from a fixed 32 MiB + 64 KiB array inside the library, held by every GPU that loads the
  * library until the process exits.  Meant for hosts that hand a plug-in nothing but its inputs and
  * outputs, for serving loops and capture regions in which cudaMalloc (a synchronizing call) is
@@ -257,11 +278,14 @@ PQ_API int pq_plan_w8a8(int64_t M, int64_t N, int64_t K, int32_t sms, size_t scr
  * itself invokes no allocation or free routine of any kind.
  *   - Limit: M and N each rounded up to a multiple of 256, multiplied, may not exceed 2,097,152
  *     (e.g. 512 x 4096, 1024 x 2048, 256 x 8192); beyond that the call returns PQ_ERR_LIMIT and
- *     launches nothing.  M <= 128 needs no scratch and is simply forwarded to pq_gemm_w8a8.
+ *     launches nothing.  M <= 128 needs no scratch: such calls are forwarded to pq_gemm_w8a8
+ *     whatever N is, and the limit does not apply to them.
  *   - The first call on each device looks up the array's device address; make that first call
  *     outside any stream capture.
  *   - All calls on a device share the one array, and it keeps whatever the last call left in it
- *     (the kernel restores the few words that must read zero).  Two calls that overlap on the GPU
+ *     (a call that completes restores the few words that must read zero; after a call that ended
+ *     in PQ_ERR_TIMEOUT, pq_device_status() -- the call that reports it -- clears them with a memset
+ *     on the array, so read the status before going on).  Two calls that overlap on the GPU
  *     -- different streams, parallel graph branches -- would race on it: keep them ordered.
  */
 PQ_API int pq_gemm_w8a8_noalloc(const int8_t* q, const float* s_tok, const void* wq, const float* s_ch,
@@ -273,6 +297,16 @@ PQ_API int pq_gemm_w8a8_noalloc(const int8_t* q, const float* s_tok, const void*
  * regions.
  */
 PQ_API int pq_device_status(int* host_status);
+
+/*
+ * The poll bound of the waits inside the kernels launched from now on (process-wide; 0 restores
+ * the default of 2^24 polls, about a second).  For tests of the give-up path: with PQ_WAIT_NONE no
+ * wait polls at all, so every role of a kernel gives up at its first wait although nothing is
+ * wrong; with a bound of a few polls some wait runs out somewhere in the middle.  Either way the
+ * kernel reports PQ_ERR_TIMEOUT through the status word and returns with unspecified outputs.
+ */
+#define PQ_WAIT_NONE 0xFFFFFFFFu
+PQ_API int pq_set_wait_limit(uint32_t polls);
 
 #ifdef __cplusplus
 }

@@ -29,8 +29,10 @@ from .binding import (  # noqa: F401
     pq_quantize_act_hadamard,
     pq_quantize_act_smooth,
     pq_quantize_act_static,
-    pq_set_workspace,
+    pq_set_wait_limit,
     pq_smooth_scales,
     pq_unpack_w4,
     pq_unpack_w8,
+    pq_workspace_bytes,
+    pq_workspace_init,
 )

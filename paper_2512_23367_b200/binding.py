@@ -26,16 +26,19 @@ SIGNATURES = {
     "pq_pack_w4": (ctypes.c_int, [_vp, _i64, _i64, _i32, _vp, _vp, _vp]),
     "pq_unpack_w8": (ctypes.c_int, [_vp, _i64, _i64, _vp, _vp]),
     "pq_unpack_w4": (ctypes.c_int, [_vp, _i64, _i64, _vp, _vp]),
-    "pq_gemm_w8a8": (ctypes.c_int, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _vp, _vp]),
+    "pq_gemm_w8a8": (ctypes.c_int, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _vp, _vp, ctypes.c_size_t, _vp]),
     "pq_gemm_w4a8": (ctypes.c_int, [_vp, _vp, _vp, _vp, _i32, _i64, _i64, _i64, _vp, _vp]),
     "pq_acc_w8a8": (ctypes.c_int, [_vp, _vp, _i64, _i64, _i64, _vp, _vp]),
     "pq_acc_w4a8": (ctypes.c_int, [_vp, _vp, _i32, _i64, _i64, _i64, _vp, _vp]),
     "pq_device_status": (ctypes.c_int, [ctypes.POINTER(ctypes.c_int)]),
-    "pq_set_workspace": (ctypes.c_int, [_vp, ctypes.c_size_t, _vp]),
+    "pq_workspace_bytes": (ctypes.c_size_t, [_i64, ctypes.POINTER(_i64), _i32, _i64, _i32]),
+    "pq_workspace_init": (ctypes.c_int, [_vp, ctypes.c_size_t, _vp]),
+    "pq_set_wait_limit": (ctypes.c_int, [ctypes.c_uint32]),
     "pq_plan_w8a8": (ctypes.c_int, [_i64, _i64, _i64, _i32, ctypes.c_size_t, ctypes.POINTER(_i32), ctypes.POINTER(_i32)]),
     "pq_gemm_w8a8_noalloc": (ctypes.c_int, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _vp, _vp]),
     "pq_gemm_w8a8_group": (ctypes.c_int, [_vp, _vp, _i32, ctypes.POINTER(_vp), ctypes.POINTER(_vp),
-                                          ctypes.POINTER(_i64), ctypes.POINTER(_vp), _i64, _i64, _vp]),
+                                          ctypes.POINTER(_i64), ctypes.POINTER(_vp), _i64, _i64, _vp,
+                                          ctypes.c_size_t, _vp]),
     "pq_quantize_act_static": (ctypes.c_int, [_vp, _vp, _i64, _i64, _vp, _vp, _vp]),
     "pq_hadamard_block": (_i32, [_i64]),
     "pq_quantize_act_hadamard": (ctypes.c_int, [_vp, _i64, _i64, _vp, _vp, _vp]),
@@ -95,21 +98,76 @@ def _check(call: str, status: int) -> None:
         raise PQError(call, status)
 
 
+def _sized(t: torch.Tensor, dtype: torch.dtype, numel: int, what: str) -> torch.Tensor:
+    """A contiguous tensor of `dtype` with exactly `numel` elements.  The C calls take raw pointers and trust
+    the sizes they are given, so a short buffer would become an out-of-bounds device access: every operand is
+    measured here, before anything is launched (and before the devices are looked at, so that a wrong size is
+    reported as such wherever the tensor lives)."""
+    if t.dtype != dtype:
+        raise TypeError(f"{what}: expected {dtype}, got {t.dtype}")
+    if t.numel() != int(numel):
+        raise ValueError(f"{what}: expected {int(numel)} elements, got {t.numel()}")
+    if not t.is_contiguous():
+        raise ValueError(f"{what}: expected a contiguous tensor")
+    return t
+
+
+def _together(first: torch.Tensor, *others: torch.Tensor | None) -> None:
+    """All operands of a call live on one CUDA device."""
+    if not first.is_cuda:
+        raise ValueError("expected CUDA tensors (this library has no CPU path)")
+    for t in others:
+        if t is not None and t.device != first.device:
+            raise ValueError(f"operands on different devices: {t.device} and {first.device}")
+
+
+def _tokens(q: torch.Tensor, s_tok: torch.Tensor) -> tuple[int, int]:
+    """Measures the quantized tokens (q int8 [M,K], s_tok f32 [M]); returns (M, K)."""
+    if q.dim() != 2:
+        raise ValueError("q: expected a 2-D tensor [M,K]")
+    M, K = q.shape
+    _sized(q, torch.int8, M * K, "q")
+    _sized(s_tok, torch.float32, M, "s_tok")
+    return int(M), int(K)
+
+
+def _out(y: torch.Tensor | None, M: int, N: int, like: torch.Tensor) -> torch.Tensor:
+    if y is None:
+        return torch.empty((M, N), dtype=torch.float16, device=like.device)
+    return _sized(y, torch.float16, M * N, "y")
+
+
+def _ws(workspace: torch.Tensor | None) -> tuple[int | None, int]:
+    if workspace is None:
+        return None, 0
+    _sized(workspace, torch.uint8, workspace.numel(), "workspace")
+    return workspace.data_ptr(), workspace.numel()
+
+
 def _factors(v: torch.Tensor, K: int, name: str) -> torch.Tensor:
-    v = _dev(v, torch.float32, name)
-    if tuple(v.shape) != (K,):
-        raise ValueError(f"{name}: expected shape [{K}]")
-    return v
+    """A per-column factor vector f32 [K] on the device."""
+    return _dev(_sized(v, torch.float32, K, name), torch.float32, name)
+
+
+def _rows(x: torch.Tensor, q: torch.Tensor | None, s_tok: torch.Tensor | None):
+    """Outputs of a row quantizer for x f16 [M,K]: created when absent, measured when given."""
+    if x.dim() != 2:
+        raise ValueError("x: expected a 2-D tensor [M,K]")
+    M, K = x.shape
+    _sized(x, torch.float16, M * K, "x")
+    if q is not None:
+        _sized(q, torch.int8, M * K, "q")
+    if s_tok is not None:
+        _sized(s_tok, torch.float32, M, "s_tok")
+    _together(x, q, s_tok)
+    q = torch.empty((M, K), dtype=torch.int8, device=x.device) if q is None else q
+    s_tok = torch.empty((M,), dtype=torch.float32, device=x.device) if s_tok is None else s_tok
+    return int(M), int(K), q, s_tok
 
 
 def pq_quantize_act(x: torch.Tensor, q: torch.Tensor | None = None, s_tok: torch.Tensor | None = None):
     """x f16 [M,K] -> (q int8 [M,K], s_tok f32 [M])."""
-    x = _dev(x, torch.float16, "x")
-    M, K = x.shape
-    if q is None:
-        q = torch.empty((M, K), dtype=torch.int8, device=x.device)
-    if s_tok is None:
-        s_tok = torch.empty((M,), dtype=torch.float32, device=x.device)
+    M, K, q, s_tok = _rows(x, q, s_tok)
     _check("pq_quantize_act", lib().pq_quantize_act(x.data_ptr(), M, K, q.data_ptr(), s_tok.data_ptr(), _stream()))
     return q, s_tok
 
@@ -117,13 +175,8 @@ def pq_quantize_act(x: torch.Tensor, q: torch.Tensor | None = None, s_tok: torch
 def pq_quantize_act_smooth(x: torch.Tensor, s_inv: torch.Tensor, q: torch.Tensor | None = None,
                            s_tok: torch.Tensor | None = None):
     """Quantizes X S^-1 (Eq. 3): x f16 [M,K], s_inv f32 [K] -> (q int8 [M,K], s_tok f32 [M])."""
-    x = _dev(x, torch.float16, "x")
-    M, K = x.shape
+    M, K, q, s_tok = _rows(x, q, s_tok)
     s_inv = _factors(s_inv, K, "s_inv")
-    if q is None:
-        q = torch.empty((M, K), dtype=torch.int8, device=x.device)
-    if s_tok is None:
-        s_tok = torch.empty((M,), dtype=torch.float32, device=x.device)
     _check("pq_quantize_act_smooth", lib().pq_quantize_act_smooth(x.data_ptr(), s_inv.data_ptr(), M, K, q.data_ptr(),
                                                                   s_tok.data_ptr(), _stream()))
     return q, s_tok
@@ -133,15 +186,9 @@ def pq_quantize_act_static(x: torch.Tensor, scale: torch.Tensor, q: torch.Tensor
                            s_tok: torch.Tensor | None = None):
     """INT8 codes against one calibrated scale: x f16 [M,K], scale f32 device tensor with one element
     -> (q int8 [M,K], s_tok f32 [M] filled with the scale)."""
-    x = _dev(x, torch.float16, "x")
-    M, K = x.shape
-    scale = _dev(scale, torch.float32, "scale")
-    if scale.numel() != 1:
-        raise ValueError("scale: one element")
-    if q is None:
-        q = torch.empty((M, K), dtype=torch.int8, device=x.device)
-    if s_tok is None:
-        s_tok = torch.empty((M,), dtype=torch.float32, device=x.device)
+    M, K, q, s_tok = _rows(x, q, s_tok)
+    scale = _sized(scale, torch.float32, 1, "scale")
+    _together(x, scale)
     _check("pq_quantize_act_static", lib().pq_quantize_act_static(x.data_ptr(), scale.data_ptr(), M, K, q.data_ptr(),
                                                                   s_tok.data_ptr(), _stream()))
     return q, s_tok
@@ -154,12 +201,7 @@ def pq_hadamard_block(K: int) -> int:
 
 def pq_quantize_act_hadamard(x: torch.Tensor, q: torch.Tensor | None = None, s_tok: torch.Tensor | None = None):
     """Quantizes X H (Eq. 4): x f16 [M,K] -> (q int8 [M,K], s_tok f32 [M])."""
-    x = _dev(x, torch.float16, "x")
-    M, K = x.shape
-    if q is None:
-        q = torch.empty((M, K), dtype=torch.int8, device=x.device)
-    if s_tok is None:
-        s_tok = torch.empty((M,), dtype=torch.float32, device=x.device)
+    M, K, q, s_tok = _rows(x, q, s_tok)
     _check("pq_quantize_act_hadamard", lib().pq_quantize_act_hadamard(x.data_ptr(), M, K, q.data_ptr(),
                                                                       s_tok.data_ptr(), _stream()))
     return q, s_tok
@@ -236,14 +278,14 @@ def pq_pack_w4(w: torch.Tensor, group: int = GROUP, smooth: torch.Tensor | None 
 
 
 def pq_unpack_w8(wq: torch.Tensor, N: int, K: int) -> torch.Tensor:
-    wq = _dev(wq, torch.uint8, "wq")
+    wq = _dev(_sized(wq, torch.uint8, N * K, "wq"), torch.uint8, "wq")
     codes = torch.empty((N, K), dtype=torch.int8, device=wq.device)
     _check("pq_unpack_w8", lib().pq_unpack_w8(wq.data_ptr(), N, K, codes.data_ptr(), _stream()))
     return codes
 
 
 def pq_unpack_w4(wp: torch.Tensor, N: int, K: int) -> torch.Tensor:
-    wp = _dev(wp, torch.uint8, "wp")
+    wp = _dev(_sized(wp, torch.uint8, N * K // 2, "wp"), torch.uint8, "wp")
     codes = torch.empty((N, K), dtype=torch.int8, device=wp.device)
     _check("pq_unpack_w4", lib().pq_unpack_w4(wp.data_ptr(), N, K, codes.data_ptr(), _stream()))
     return codes
@@ -256,99 +298,102 @@ def pq_plan_w8a8(M: int, N: int, K: int, sms: int = 148, scratch_bytes: int = 0)
     return int(bn.value), int(sp.value)
 
 
-_workspaces: dict[int, torch.Tensor] = {}
-WORKSPACE_BYTES = int(os.environ.get("PQ_WORKSPACE_MB", "64")) << 20
+def pq_workspace_bytes(M: int, Ns, K: int, sms: int = 148) -> int:
+    """Bytes of workspace with which pq_gemm_w8a8 (Ns = one width) or pq_gemm_w8a8_group (Ns = the members'
+    widths) at these M and K runs the schedule it would pick with unlimited room; 0 if that schedule does not
+    split K.  Host-only, needs no GPU."""
+    Ns = [int(Ns)] if isinstance(Ns, int) else [int(n) for n in Ns]
+    arr = (_i64 * max(len(Ns), 1))(*Ns)
+    return int(lib().pq_workspace_bytes(int(M), arr, len(Ns), int(K), int(sms)))
 
 
-def pq_set_workspace(workspace: torch.Tensor | None) -> None:
-    """Registers (or, with None, unregisters) scratch memory for the current device: a uint8 CUDA
-    tensor the caller keeps alive.  The W8A8 GEMM uses it to split K on shapes with few tiles."""
-    if workspace is None:
-        _check("pq_set_workspace", lib().pq_set_workspace(None, 0, _stream()))
-        return
+def pq_workspace_init(workspace: torch.Tensor) -> torch.Tensor:
+    """Prepares a caller-owned workspace (uint8 CUDA tensor, 256-byte aligned, >= 64 KiB) for the W8A8 calls
+    on the current stream: zeroes its arrival counters.  Returns the tensor."""
     workspace = _dev(workspace, torch.uint8, "workspace")
-    _check("pq_set_workspace", lib().pq_set_workspace(workspace.data_ptr(), workspace.numel(), _stream()))
+    with torch.cuda.device(workspace.device):
+        _check("pq_workspace_init", lib().pq_workspace_init(workspace.data_ptr(), workspace.numel(), _stream()))
+    return workspace
 
 
-def _ensure_workspace(device: torch.device) -> None:
-    """Gives each device one scratch buffer on first use (torch owns the memory; the library never
-    allocates).  PQ_WORKSPACE_MB=0 turns this off."""
-    idx = device.index if device.index is not None else torch.cuda.current_device()
-    if idx in _workspaces or WORKSPACE_BYTES <= 0:
-        return
-    with torch.cuda.device(idx):
-        buf = torch.empty((WORKSPACE_BYTES,), dtype=torch.uint8, device=device)
-        pq_set_workspace(buf)
-    _workspaces[idx] = buf
+def pq_set_wait_limit(polls: int) -> None:
+    """Poll bound of the waits inside kernels launched from now on (0 = the default).  Test hook."""
+    _check("pq_set_wait_limit", lib().pq_set_wait_limit(int(polls)))
 
 
-def pq_gemm_w8a8(q, s_tok, wq, s_ch, N: int, y: torch.Tensor | None = None) -> torch.Tensor:
-    """q int8 [M,K], s_tok f32 [M], wq/s_ch from pq_pack_w8 -> y f16 [M,N]."""
-    q = _dev(q, torch.int8, "q")
-    _ensure_workspace(q.device)
-    M, K = q.shape
-    _dev(s_tok, torch.float32, "s_tok"), _dev(wq, torch.uint8, "wq"), _dev(s_ch, torch.float32, "s_ch")
-    if y is None:
-        y = torch.empty((M, N), dtype=torch.float16, device=q.device)
+def pq_gemm_w8a8(q, s_tok, wq, s_ch, N: int, y: torch.Tensor | None = None,
+                 workspace: torch.Tensor | None = None) -> torch.Tensor:
+    """q int8 [M,K], s_tok f32 [M], wq/s_ch from pq_pack_w8 -> y f16 [M,N].  workspace: optional prepared
+    scratch of this call (pq_workspace_bytes / pq_workspace_init); without it K is never split."""
+    M, K = _tokens(q, s_tok)
+    _sized(wq, torch.uint8, N * K, "wq"), _sized(s_ch, torch.float32, N, "s_ch")
+    ws, ws_bytes = _ws(workspace)
+    if y is not None:
+        _sized(y, torch.float16, M * N, "y")
+    _together(q, s_tok, wq, s_ch, y, workspace)
+    y = _out(y, M, N, q)
     _check("pq_gemm_w8a8", lib().pq_gemm_w8a8(q.data_ptr(), s_tok.data_ptr(), wq.data_ptr(), s_ch.data_ptr(),
-                                              M, N, K, y.data_ptr(), _stream()))
+                                              M, N, K, y.data_ptr(), ws, ws_bytes, _stream()))
     return y
 
 
-def pq_gemm_w8a8_group(q, s_tok, members, ys=None) -> list[torch.Tensor]:
-    """Several W8A8 linears over the same quantized tokens as one call (one kernel launch).  members: sequence of (wq, s_ch, N) from pq_pack_w8; ys: optional outputs f16 [M,N_g].
-    Returns the outputs; each equals pq_gemm_w8a8(q, s_tok, wq, s_ch, N) bit for bit."""
-    q = _dev(q, torch.int8, "q")
-    _ensure_workspace(q.device)
-    M, K = q.shape
-    _dev(s_tok, torch.float32, "s_tok")
+def _group_arrays(q, s_tok, members, ys, w_dtype, w_numel, s_dtype, s_numel, M, workspace=None):
     n = len(members)
+    if not 1 <= n <= MAX_GROUP:
+        raise ValueError(f"a group holds 1..{MAX_GROUP} members")
     if ys is None:
-        ys = [torch.empty((M, int(N)), dtype=torch.float16, device=q.device) for (_, _, N) in members]
+        ys = [None] * n
     if len(ys) != n:
         raise ValueError("one output per member")
-    for (wq, s_ch, _), y in zip(members, ys):
-        _dev(wq, torch.uint8, "wq"), _dev(s_ch, torch.float32, "s_ch"), _dev(y, torch.float16, "y")
-    wq_arr = (_vp * max(n, 1))(*[m[0].data_ptr() for m in members])
-    sc_arr = (_vp * max(n, 1))(*[m[1].data_ptr() for m in members])
-    n_arr = (_i64 * max(n, 1))(*[int(m[2]) for m in members])
-    y_arr = (_vp * max(n, 1))(*[y.data_ptr() for y in ys])
+    for i, ((w, sc, N), y) in enumerate(zip(members, ys)):
+        N = int(N)
+        _sized(w, w_dtype, w_numel(N), f"members[{i}] weights")
+        _sized(sc, s_dtype, s_numel(N), f"members[{i}] scales")
+        if y is not None:
+            _sized(y, torch.float16, M * N, f"ys[{i}]")
+    _together(q, s_tok, workspace, *[m[0] for m in members], *[m[1] for m in members], *ys)
+    outs = [_out(y, M, int(m[2]), q) for m, y in zip(members, ys)]
+    w_arr = (_vp * n)(*[m[0].data_ptr() for m in members])
+    s_arr = (_vp * n)(*[m[1].data_ptr() for m in members])
+    n_arr = (_i64 * n)(*[int(m[2]) for m in members])
+    y_arr = (_vp * n)(*[y.data_ptr() for y in outs])
+    return n, w_arr, s_arr, n_arr, y_arr, outs
+
+
+def pq_gemm_w8a8_group(q, s_tok, members, ys=None, workspace: torch.Tensor | None = None) -> list[torch.Tensor]:
+    """Several W8A8 linears over the same quantized tokens as one call (one kernel launch).  members: sequence of (wq, s_ch, N) from pq_pack_w8; ys: optional outputs f16 [M,N_g]; workspace: as for pq_gemm_w8a8.
+    Returns the outputs; each equals pq_gemm_w8a8(q, s_tok, wq, s_ch, N) bit for bit."""
+    M, K = _tokens(q, s_tok)
+    ws, ws_bytes = _ws(workspace)
+    n, wq_arr, sc_arr, n_arr, y_arr, outs = _group_arrays(q, s_tok, members, ys, torch.uint8, lambda N: N * K,
+                                                          torch.float32, lambda N: N, M, workspace)
     _check("pq_gemm_w8a8_group", lib().pq_gemm_w8a8_group(q.data_ptr(), s_tok.data_ptr(), n, wq_arr, sc_arr, n_arr,
-                                                          y_arr, M, K, _stream()))
-    return list(ys)
+                                                          y_arr, M, K, ws, ws_bytes, _stream()))
+    return outs
 
 
 def pq_gemm_w4a8_group(q, s_tok, members, ys=None, group: int = GROUP) -> list[torch.Tensor]:
     """Several W4A8 linears over the same quantized tokens as one call (one kernel launch).  members: sequence of (wp, s_grp, N) from pq_pack_w4; ys: optional outputs f16 [M,N_g].
     Each output equals pq_gemm_w4a8(q, s_tok, wp, s_grp, N) bit for bit."""
-    q = _dev(q, torch.int8, "q")
-    M, K = q.shape
-    _dev(s_tok, torch.float32, "s_tok")
-    n = len(members)
-    if ys is None:
-        ys = [torch.empty((M, int(N)), dtype=torch.float16, device=q.device) for (_, _, N) in members]
-    if len(ys) != n:
-        raise ValueError("one output per member")
-    for (wp, s_grp, _), y in zip(members, ys):
-        _dev(wp, torch.uint8, "wp"), _dev(s_grp, torch.float16, "s_grp"), _dev(y, torch.float16, "y")
-    wp_arr = (_vp * max(n, 1))(*[m[0].data_ptr() for m in members])
-    sg_arr = (_vp * max(n, 1))(*[m[1].data_ptr() for m in members])
-    n_arr = (_i64 * max(n, 1))(*[int(m[2]) for m in members])
-    y_arr = (_vp * max(n, 1))(*[y.data_ptr() for y in ys])
+    M, K = _tokens(q, s_tok)
+    n, wp_arr, sg_arr, n_arr, y_arr, outs = _group_arrays(q, s_tok, members, ys, torch.uint8, lambda N: N * K // 2,
+                                                          torch.float16, lambda N: (K // max(group, 1)) * N, M)
     _check("pq_gemm_w4a8_group", lib().pq_gemm_w4a8_group(q.data_ptr(), s_tok.data_ptr(), n, wp_arr, sg_arr, group,
                                                           n_arr, y_arr, M, K, _stream()))
-    return list(ys)
+    return outs
 
 
 def pq_gemm_w8a8_noalloc(q, s_tok, wq, s_ch, N: int, y: torch.Tensor) -> torch.Tensor:
     """Same product as pq_gemm_w8a8, for callers that may not allocate: the output tensor is
     required (this wrapper creates none) and the library's built-in scratch array is used instead of
-    a registered workspace.  Raises PQError with status 7 when the padded output exceeds 2 Mi
+    a workspace.  Raises PQError with status 7 when M > 128 and the padded output exceeds 2 Mi
     elements.  Calls on one device must not overlap on the GPU."""
-    q = _dev(q, torch.int8, "q")
-    M, K = q.shape
-    _dev(s_tok, torch.float32, "s_tok"), _dev(wq, torch.uint8, "wq"), _dev(s_ch, torch.float32, "s_ch")
-    _dev(y, torch.float16, "y")
+    M, K = _tokens(q, s_tok)
+    _sized(wq, torch.uint8, N * K, "wq"), _sized(s_ch, torch.float32, N, "s_ch")
+    if y is None:
+        raise ValueError("y: required (this entry point creates no tensor)")
+    _sized(y, torch.float16, M * N, "y")
+    _together(q, s_tok, wq, s_ch, y)
     _check("pq_gemm_w8a8_noalloc", lib().pq_gemm_w8a8_noalloc(q.data_ptr(), s_tok.data_ptr(), wq.data_ptr(),
                                                               s_ch.data_ptr(), M, N, K, y.data_ptr(), _stream()))
     return y
@@ -356,11 +401,12 @@ def pq_gemm_w8a8_noalloc(q, s_tok, wq, s_ch, N: int, y: torch.Tensor) -> torch.T
 
 def pq_gemm_w4a8(q, s_tok, wp, s_grp, N: int, group: int = GROUP, y: torch.Tensor | None = None) -> torch.Tensor:
     """q int8 [M,K], s_tok f32 [M], wp/s_grp from pq_pack_w4 -> y f16 [M,N]."""
-    q = _dev(q, torch.int8, "q")
-    M, K = q.shape
-    _dev(s_tok, torch.float32, "s_tok"), _dev(wp, torch.uint8, "wp"), _dev(s_grp, torch.float16, "s_grp")
-    if y is None:
-        y = torch.empty((M, N), dtype=torch.float16, device=q.device)
+    M, K = _tokens(q, s_tok)
+    _sized(wp, torch.uint8, N * K // 2, "wp"), _sized(s_grp, torch.float16, (K // max(group, 1)) * N, "s_grp")
+    if y is not None:
+        _sized(y, torch.float16, M * N, "y")
+    _together(q, s_tok, wp, s_grp, y)
+    y = _out(y, M, N, q)
     _check("pq_gemm_w4a8", lib().pq_gemm_w4a8(q.data_ptr(), s_tok.data_ptr(), wp.data_ptr(), s_grp.data_ptr(),
                                               group, M, N, K, y.data_ptr(), _stream()))
     return y
@@ -368,9 +414,11 @@ def pq_gemm_w4a8(q, s_tok, wp, s_grp, N: int, group: int = GROUP, y: torch.Tenso
 
 def pq_acc_w8a8(q, wq, N: int) -> torch.Tensor:
     """Exact INT32 accumulators [M,N] of the W8A8 product."""
-    q = _dev(q, torch.int8, "q")
+    if q.dim() != 2:
+        raise ValueError("q: expected a 2-D tensor [M,K]")
     M, K = q.shape
-    _dev(wq, torch.uint8, "wq")
+    _sized(q, torch.int8, M * K, "q"), _sized(wq, torch.uint8, N * K, "wq")
+    _together(q, wq)
     acc = torch.empty((M, N), dtype=torch.int32, device=q.device)
     _check("pq_acc_w8a8", lib().pq_acc_w8a8(q.data_ptr(), wq.data_ptr(), M, N, K, acc.data_ptr(), _stream()))
     return acc
@@ -378,9 +426,11 @@ def pq_acc_w8a8(q, wq, N: int) -> torch.Tensor:
 
 def pq_acc_w4a8(q, wp, N: int, group: int = GROUP) -> torch.Tensor:
     """Exact INT32 per-group accumulators [K/group, M, N] of the W4A8 product."""
-    q = _dev(q, torch.int8, "q")
+    if q.dim() != 2:
+        raise ValueError("q: expected a 2-D tensor [M,K]")
     M, K = q.shape
-    _dev(wp, torch.uint8, "wp")
+    _sized(q, torch.int8, M * K, "q"), _sized(wp, torch.uint8, N * K // 2, "wp")
+    _together(q, wp)
     acc = torch.empty((K // group, M, N), dtype=torch.int32, device=q.device)
     _check("pq_acc_w4a8", lib().pq_acc_w4a8(q.data_ptr(), wp.data_ptr(), group, M, N, K, acc.data_ptr(), _stream()))
     return acc

@@ -3,9 +3,12 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <atomic>
 #include <cstdlib>
+#include <mutex>
 
 #include "pq_internal.h"
+#include "pq_ptx.cuh"
 
 namespace pq {
 
@@ -17,32 +20,38 @@ constexpr int kMaxDevices = 64;
 constexpr int64_t kSmallM = 64;      // W4A8: M at or below this takes the weight-streaming schedule
 constexpr int64_t kSmallM_W8 = 128;  // W8A8
 
+// Facts about a device, filled in by the first call on it.  Host threads may make that first call
+// concurrently: the fill happens under a mutex and `probed` is published last.
 struct DeviceInfo {
-  bool probed = false;
+  std::atomic<bool> probed{false};
   bool ok = false;
   int sms = 0;
   int* status = nullptr;
-  Scratch scratch;
 };
 DeviceInfo g_dev[kMaxDevices];
+std::mutex g_dev_mutex;
+std::atomic<uint32_t> g_wait_limit{kWaitPollLimit};
 
 DeviceInfo* current_device() {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
   DeviceInfo& d = g_dev[dev];
-  if (!d.probed) {
-    int major = 0, minor = 0, sms = 0;
-    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return nullptr;
-    if (cudaDeviceGetAttribute(&minor, cudaDevAttrComputeCapabilityMinor, dev) != cudaSuccess) return nullptr;
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return nullptr;
-    d.sms = sms;
-    d.ok = (major == 10 && minor == 0);
-    if (d.ok) {
-      void* p = nullptr;
-      if (cudaGetSymbolAddress(&p, g_status_word) != cudaSuccess) return nullptr;
-      d.status = static_cast<int*>(p);
+  if (!d.probed.load(std::memory_order_acquire)) {
+    std::lock_guard<std::mutex> lock(g_dev_mutex);
+    if (!d.probed.load(std::memory_order_relaxed)) {
+      int major = 0, minor = 0, sms = 0;
+      if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return nullptr;
+      if (cudaDeviceGetAttribute(&minor, cudaDevAttrComputeCapabilityMinor, dev) != cudaSuccess) return nullptr;
+      if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return nullptr;
+      d.sms = sms;
+      d.ok = (major == 10 && minor == 0);
+      if (d.ok) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_status_word) != cudaSuccess) return nullptr;
+        d.status = static_cast<int*>(p);
+      }
+      d.probed.store(true, std::memory_order_release);
     }
-    d.probed = true;
   }
   return &d;
 }
@@ -76,7 +85,20 @@ using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t
                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
                                    CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
                                    CUtensorMapFloatOOBfill);
-EncodeTiledFn g_encode = nullptr;
+// cuTensorMapEncodeTiled, looked up once (thread-safe: initialisation of a function-local static).
+EncodeTiledFn encode_fn() {
+  static const EncodeTiledFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess) {
+      cudaGetLastError();
+      p = nullptr;
+    }
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
 
 }  // namespace
 
@@ -85,10 +107,7 @@ int* device_status_ptr() {
   return d ? d->status : nullptr;
 }
 
-Scratch scratch() {
-  DeviceInfo* d = current_device();
-  return d ? d->scratch : Scratch();
-}
+uint32_t wait_limit() { return g_wait_limit.load(std::memory_order_relaxed); }
 
 int sm_count() {
   DeviceInfo* d = current_device();
@@ -105,16 +124,8 @@ bool pdl_enabled() {
 
 int make_tmap_2d(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows,
                  uint32_t box_cols, uint32_t elem_bytes, int swizzle_bytes) {
-  if (g_encode == nullptr) {
-    void* fn = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
-        qres != cudaDriverEntryPointSuccess || fn == nullptr) {
-      cudaGetLastError();
-      return PQ_ERR_CUDA;
-    }
-    g_encode = reinterpret_cast<EncodeTiledFn>(fn);
-  }
+  const EncodeTiledFn g_encode = encode_fn();
+  if (g_encode == nullptr) return PQ_ERR_CUDA;
   CUtensorMapDataType dt = elem_bytes == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8
                            : elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_UINT16
                                              : CU_TENSOR_MAP_DATA_TYPE_UINT32;
@@ -302,28 +313,31 @@ int pq_unpack_w4(const void* wp, int64_t N, int64_t K, int8_t* codes, void* stre
   return launch_unpack_w4(wp, N, K, codes, static_cast<cudaStream_t>(stream));
 }
 
+static bool aligned256(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
+
 static int gemm_w8a8_common(const int8_t* q, const float* s_tok, const void* wq, const float* s_ch, int64_t M,
-                            int64_t N, int64_t K, void* y, int32_t* acc, void* stream) {
+                            int64_t N, int64_t K, void* y, int32_t* acc, void* workspace, size_t workspace_bytes,
+                            void* stream) {
   int rc = check_gemm(M, N, K);
   if (rc != PQ_OK) return rc;
-  if (!aligned16(q) || !aligned16(wq) || !aligned16(y) || !aligned16(acc)) return PQ_ERR_ALIGN;
+  if (!aligned16(q) || !aligned16(wq) || !aligned16(y) || !aligned16(acc) || !aligned256(workspace)) return PQ_ERR_ALIGN;
   if ((rc = check_arch()) != PQ_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   // Up to 128 tokens: the weight-streaming schedule (tokens are the narrow MMA dimension, K split over a
   // cluster); beyond that the second CTA of a pair no longer holds only padding rows.
   if (M <= kSmallM_W8) return launch_smallm_w8a8(q, s_tok, wq, s_ch, M, N, K, y, acc, st);
-  return launch_gemm_w8a8_pair(q, s_tok, wq, s_ch, M, N, K, y, acc, st);
+  return launch_gemm_w8a8_pair(scratch_from(workspace, workspace_bytes), q, s_tok, wq, s_ch, M, N, K, y, acc, st);
 }
 
 int pq_gemm_w8a8(const int8_t* q, const float* s_tok, const void* wq, const float* s_ch, int64_t M, int64_t N,
-                 int64_t K, void* y_f16, void* stream) {
+                 int64_t K, void* y_f16, void* workspace, size_t workspace_bytes, void* stream) {
   if (!q || !s_tok || !wq || !s_ch || !y_f16) return PQ_ERR_NULL;
-  return gemm_w8a8_common(q, s_tok, wq, s_ch, M, N, K, y_f16, nullptr, stream);
+  return gemm_w8a8_common(q, s_tok, wq, s_ch, M, N, K, y_f16, nullptr, workspace, workspace_bytes, stream);
 }
 
 int pq_gemm_w8a8_group(const int8_t* q, const float* s_tok, int32_t count, const void* const* wq,
                        const float* const* s_ch, const int64_t* N, void* const* y_f16, int64_t M, int64_t K,
-                       void* stream) {
+                       void* workspace, size_t workspace_bytes, void* stream) {
   if (!q || !s_tok || !wq || !s_ch || !N || !y_f16) return PQ_ERR_NULL;
   if (count < 1 || count > PQ_MAX_GROUP) return PQ_ERR_SHAPE;
   for (int g = 0; g < count; ++g) {
@@ -332,20 +346,20 @@ int pq_gemm_w8a8_group(const int8_t* q, const float* s_tok, int32_t count, const
     if (rc != PQ_OK) return rc;
     if (!aligned16(wq[g]) || !aligned16(y_f16[g])) return PQ_ERR_ALIGN;
   }
-  if (!aligned16(q)) return PQ_ERR_ALIGN;
+  if (!aligned16(q) || !aligned256(workspace)) return PQ_ERR_ALIGN;
   int rc = check_arch();
   if (rc != PQ_OK) return rc;
   if (M <= kSmallM_W8) {
     return launch_smallm_w8a8_group(q, s_tok, count, wq, s_ch, N, y_f16, M, K, nullptr,
                                     static_cast<cudaStream_t>(stream));
   }
-  return launch_gemm_w8a8_pair_group(scratch(), q, s_tok, count, wq, s_ch, N, y_f16, M, K, nullptr,
-                                     static_cast<cudaStream_t>(stream));
+  return launch_gemm_w8a8_pair_group(scratch_from(workspace, workspace_bytes), q, s_tok, count, wq, s_ch, N, y_f16,
+                                     M, K, nullptr, static_cast<cudaStream_t>(stream));
 }
 
 int pq_acc_w8a8(const int8_t* q, const void* wq, int64_t M, int64_t N, int64_t K, int32_t* acc, void* stream) {
   if (!q || !wq || !acc) return PQ_ERR_NULL;
-  return gemm_w8a8_common(q, nullptr, wq, nullptr, M, N, K, nullptr, acc, stream);
+  return gemm_w8a8_common(q, nullptr, wq, nullptr, M, N, K, nullptr, acc, nullptr, 0, stream);
 }
 
 static int gemm_w4a8_common(const int8_t* q, const float* s_tok, const void* wp, const void* s_grp, int32_t group,
@@ -421,27 +435,32 @@ int pq_plan_w8a8(int64_t M, int64_t N, int64_t K, int32_t sms, size_t scratch_by
   return PQ_OK;
 }
 
-int pq_set_workspace(void* workspace, size_t bytes, void* stream) {
-  int rc = check_arch();
-  if (rc != PQ_OK) return rc;
-  DeviceInfo* d = current_device();
-  if (d == nullptr) return PQ_ERR_CUDA;
-  if (workspace == nullptr || bytes == 0) {
-    d->scratch = Scratch();
-    return PQ_OK;
+size_t pq_workspace_bytes(int64_t M, const int64_t* N, int32_t count, int64_t K, int32_t sms) {
+  if (!N || count < 1 || count > PQ_MAX_GROUP || sms < 2) return 0;
+  for (int g = 0; g < count; ++g) {
+    if (check_gemm(M, N[g], K) != PQ_OK) return 0;
   }
-  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return PQ_ERR_ALIGN;
-  if (bytes < kScratchHeaderBytes + (size_t(1) << 20)) return PQ_ERR_SHAPE;
+  if (M <= kSmallM_W8) return 0;   // the weight-streaming schedule reduces inside the SMs
+  int bn = 256, sp = 1;
+  // the schedule chosen when room is no constraint
+  if (plan_w8a8_pair_group(M, N, count, K, sms, ~size_t(0), 0, 0, &bn, &sp) < 0 || sp <= 1) return 0;
+  return kScratchHeaderBytes + w8a8_pair_partial_bytes(M, N, count, bn, sp);
+}
+
+int pq_workspace_init(void* workspace, size_t bytes, void* stream) {
+  if (!workspace) return PQ_ERR_NULL;
+  if (!aligned256(workspace)) return PQ_ERR_ALIGN;
+  if (bytes < kScratchHeaderBytes) return PQ_ERR_SHAPE;
   // the arrival counters must read zero when a GEMM first uses them
   if (cudaMemsetAsync(workspace, 0, kScratchHeaderBytes, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
     cudaGetLastError();
     return PQ_ERR_CUDA;
   }
-  Scratch sc;
-  sc.counters = static_cast<unsigned int*>(workspace);
-  sc.partials = reinterpret_cast<int32_t*>(static_cast<uint8_t*>(workspace) + kScratchHeaderBytes);
-  sc.partial_bytes = bytes - kScratchHeaderBytes;
-  d->scratch = sc;
+  return PQ_OK;
+}
+
+int pq_set_wait_limit(uint32_t polls) {
+  g_wait_limit.store(polls == 0 ? kWaitPollLimit : (polls == PQ_WAIT_NONE ? 0u : polls), std::memory_order_relaxed);
   return PQ_OK;
 }
 
@@ -454,7 +473,11 @@ int pq_device_status(int* host_status) {
   if (cudaDeviceSynchronize() != cudaSuccess) return PQ_ERR_CUDA;
   int v = 0;
   if (cudaMemcpy(&v, p, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return PQ_ERR_CUDA;
-  if (v != 0 && cudaMemset(p, 0, sizeof(int)) != cudaSuccess) return PQ_ERR_CUDA;
+  if (v != 0) {
+    if (cudaMemset(p, 0, sizeof(int)) != cudaSuccess) return PQ_ERR_CUDA;
+    // A call that gave up may have left arrival counters of the built-in scratch array non-zero.
+    if ((rc = reset_static_scratch()) != PQ_OK) return rc;
+  }
   *host_status = v;
   return PQ_OK;
 }

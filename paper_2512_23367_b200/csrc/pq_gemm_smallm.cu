@@ -58,7 +58,7 @@ struct Cfg {
   static constexpr int kRingEnd = kScOff + SC_SLOTS * BW * 4;
   static constexpr int kRedBytes = MPAD * BW * 4;                // aliases the stage ring
   static constexpr int kBarOff = (kRingEnd > kRedBytes ? kRingEnd : kRedBytes);
-  static constexpr int kNumBars = 2 * STAGES + 2 * A8_SLOTS + 2 * SC_SLOTS + 2 * ACC_SLOTS;
+  static constexpr int kNumBars = 2 * STAGES + 2 * A8_SLOTS + 2 * SC_SLOTS + 2 * ACC_SLOTS + 1;   // + the MMA issuer's drain barrier
   static constexpr int kMiscOff = kBarOff + kNumBars * 8;
   static constexpr int kDynamic = kMiscOff + 16 + 1024;
   static constexpr uint32_t kTmemCols = (ACC_SLOTS * MPAD) < 32 ? 32 : (ACC_SLOTS * MPAD);
@@ -75,6 +75,7 @@ struct SmallArgs {
   int* status;
   int M, K;
   int k_blocks, splits;
+  uint32_t wait_limit;   // poll bound of every wait
 };
 
 // Tensor maps of the members' weights (and W4 group scales), indexed by member.
@@ -124,8 +125,10 @@ smallm_kernel(const __grid_constant__ SmallMaps maps, const __grid_constant__ CU
   const uint32_t bar_sc_empty = bar_sc_full + C::SC_SLOTS * 8;
   const uint32_t bar_acc_full = bar_sc_empty + C::SC_SLOTS * 8;
   const uint32_t bar_acc_empty = bar_acc_full + C::ACC_SLOTS * 8;
+  const uint32_t bar_drain = bar_acc_empty + C::ACC_SLOTS * 8;   // give-up path of the MMA issuer only
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + C::kMiscOff);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + C::kMiscOff + 4);
+  const WaitCtx wc{abort_flag, p.wait_limit};
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -171,6 +174,7 @@ smallm_kernel(const __grid_constant__ SmallMaps maps, const __grid_constant__ CU
   }
   if (threadIdx.x == 0) {
     *abort_flag = 0;
+    mbar_init(bar_drain, 1);
     for (int s = 0; s < C::STAGES; ++s) {
       mbar_init(bar_full + s * 8, 1);
       mbar_init(bar_empty + s * 8, kW4 ? 1 + kUnpackThreads / 32 : 1);
@@ -210,6 +214,7 @@ smallm_kernel(const __grid_constant__ SmallMaps maps, const __grid_constant__ CU
 #pragma unroll
   for (int m = 0; m < kPartials; ++m) P[m] = 0u;
   bool ok = true;
+  int issued = 0;   // producer thread: K blocks it has requested (for the give-up path)
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer (remaining blocks)
@@ -220,17 +225,11 @@ smallm_kernel(const __grid_constant__ SmallMaps maps, const __grid_constant__ CU
       int j = C::STAGES;
       for (; j < nkb; ++j) {
         const uint32_t s = static_cast<uint32_t>(j) % C::STAGES, ph = (static_cast<uint32_t>(j) / C::STAGES) & 1u;
-        if (!mbar_wait(bar_empty + s * 8, ph ^ 1u, abort_flag)) { ok = false; break; }
+        if (!mbar_wait(bar_empty + s * 8, ph ^ 1u, wc)) { ok = false; break; }
         issue_weights(j);
         issue_codes(j);
       }
-      if (!ok) {
-        const int first = j >= C::STAGES ? j - C::STAGES : 0;
-        for (int i = first; i < j; ++i) {
-          const uint32_t s = static_cast<uint32_t>(i) % C::STAGES, ph = (static_cast<uint32_t>(i) / C::STAGES) & 1u;
-          for (uint32_t w = 0; w < (1u << 16) && !mbar_try_wait(bar_full + s * 8, ph); ++w) {}
-        }
-      }
+      issued = j < nkb ? j : nkb;
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
@@ -249,9 +248,9 @@ smallm_kernel(const __grid_constant__ SmallMaps maps, const __grid_constant__ CU
           d_tmem = tmem_base + a * MPAD;
           // (the three waits share their round trips)
           if (!mbar_wait3(bar_full + s * 8, ph, bar_a8_full + u * 8, uph, bar_acc_empty + a * 8, aph ^ 1u,
-                          abort_flag)) { ok = false; break; }
+                          wc)) { ok = false; break; }
         } else {
-          if (!mbar_wait(bar_full + s * 8, ph, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(bar_full + s * 8, ph, wc)) { ok = false; break; }
           w_desc = umma_desc_k_sw128(stage);
         }
         tc_fence_after_sync();
@@ -282,7 +281,7 @@ smallm_kernel(const __grid_constant__ SmallMaps maps, const __grid_constant__ CU
         const uint32_t u = it % C::A8_SLOTS, uph = (it / C::A8_SLOTS) & 1u;
         const uint32_t v = it % C::SC_SLOTS, vph = (it / C::SC_SLOTS) & 1u;
         const bool w = mbar_wait3(bar_full + s * 8, ph, bar_a8_empty + u * 8, uph ^ 1u, bar_sc_empty + v * 8,
-                                  vph ^ 1u, abort_flag);
+                                  vph ^ 1u, wc);
         ok = __all_sync(0xffffffffu, w);
         if (!ok) break;
         const uint8_t* stage = smem + s * C::kStageBytes;
@@ -327,7 +326,7 @@ smallm_kernel(const __grid_constant__ SmallMaps maps, const __grid_constant__ CU
         const uint32_t it = static_cast<uint32_t>(j);
         const uint32_t a = it % C::ACC_SLOTS, aph = (it / C::ACC_SLOTS) & 1u;
         const uint32_t v = it % C::SC_SLOTS, vph = (it / C::SC_SLOTS) & 1u;
-        const bool w = mbar_wait2(bar_acc_full + a * 8, aph, bar_sc_full + v * 8, vph, abort_flag);
+        const bool w = mbar_wait2(bar_acc_full + a * 8, aph, bar_sc_full + v * 8, vph, wc);
         ok = __all_sync(0xffffffffu, w);
         if (!ok) break;
         tc_fence_after_sync();
@@ -361,7 +360,7 @@ smallm_kernel(const __grid_constant__ SmallMaps maps, const __grid_constant__ CU
       // All K blocks of this CTA are consumed once the accumulator is complete, so the stage ring is
       // free: the partial tile goes there as red[m][n] (32-bit words), 32 token columns at a time.
       uint32_t* red_w8 = reinterpret_cast<uint32_t*>(smem);
-      if (nkb > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar_acc_full, 0u, abort_flag));
+      if (nkb > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar_acc_full, 0u, wc));
       if (ok) tc_fence_after_sync();
       constexpr int CW = MPAD < 32 ? MPAD : 32;
 #pragma unroll
@@ -394,6 +393,20 @@ smallm_kernel(const __grid_constant__ SmallMaps maps, const __grid_constant__ CU
   tc_fence_before_sync();
   __syncwarp();
   cluster_sync_all();
+  if (*abort_flag) {
+    // Some role of this CTA gave up (every role is past its loop here).  Work already handed to the
+    // hardware still completes by itself and must have done so before this CTA's shared and tensor
+    // memory go away: the producer's loads and the issuer's MMAs.  (The other threads go on to the
+    // reduction, whose result is unspecified after a give-up, and meet these two at the next barrier.)
+    if (threadIdx.x == 0) {
+      const int first = issued > C::STAGES ? issued - C::STAGES : 0;
+      for (int i = first; i < issued; ++i)
+        mbar_drain(bar_full + (static_cast<uint32_t>(i) % C::STAGES) * 8, (static_cast<uint32_t>(i) / C::STAGES) & 1u);
+    } else if (threadIdx.x == 32) {
+      umma_commit(bar_drain);
+      mbar_drain(bar_drain, 0u);
+    }
+  }
   if (do_reduce && warp >= 4 && warp < 8) {
     // Thread t owns four consecutive output channels (one 16-byte word of every part's partial
     // tile) for the rows m = rank + splits * (t / 32 + 4 i): the remote loads of all parts of a row
@@ -465,12 +478,8 @@ template <int MPAD, bool kW4, bool kExportAcc>
 int launch_cfg(const SmallMaps& maps, const CUtensorMap& tq, const SmallArgs& a, int n_tiles, cudaStream_t stream) {
   using C = Cfg<MPAD, kW4>;
   auto kern = smallm_kernel<MPAD, kW4, kExportAcc>;
-  static bool configured = false;
-  if (!configured) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kDynamic) != cudaSuccess)
-      return PQ_ERR_CUDA;
-    configured = true;
-  }
+  static PerDeviceOnce once;   // one per kernel variant
+  if (const int rc = set_dynamic_smem_once(once, kern, C::kDynamic); rc != PQ_OK) return rc;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(static_cast<unsigned>(n_tiles), static_cast<unsigned>(a.splits), 1);
   cfg.blockDim = dim3(C::kThreads, 1, 1);
@@ -551,6 +560,7 @@ int launch_smallm(const int8_t* q, const float* s_tok, int count, const void* co
   a.K = static_cast<int>(K);
   a.k_blocks = k_blocks;
   a.splits = splits;
+  a.wait_limit = wait_limit();
   const bool ex = acc != nullptr;
   const int nt = static_cast<int>(n_tiles);
   switch (mpad) {

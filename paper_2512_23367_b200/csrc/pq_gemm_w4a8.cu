@@ -67,7 +67,7 @@ constexpr int kW8Off = STAGES * kStageBytes;
 constexpr int kScOff = kW8Off + STAGES * kW8Bytes;
 constexpr int kOutOff = kScOff + SC_SLOTS * BC_CTA * 4;
 constexpr int kBarOff = kOutOff + kPromoteWarps * kOutBufs * kOutBoxBytes;
-constexpr int kNumBars = 3 * STAGES + 2 * SC_SLOTS + 2 * ACC_SLOTS;
+constexpr int kNumBars = 3 * STAGES + 2 * SC_SLOTS + 2 * ACC_SLOTS + 1;   // + the MMA issuer's drain barrier
 constexpr int kMiscOff = kBarOff + kNumBars * 8;
 constexpr int kDynamicSmem = kMiscOff + 16 + 1024;
 static_assert(kDynamicSmem <= 232448, "exceeds the shared memory of one CTA");
@@ -84,6 +84,7 @@ struct W4Args {
   int count;               // members in this launch (linears that share the token codes)
   int M, K;
   int m_blocks, n_blocks, k_blocks;   // n_blocks: over all members
+  uint32_t wait_limit;     // poll bound of every wait
 };
 
 // Tensor maps of the members' packed weights, group scales and outputs (indexed by member).
@@ -136,7 +137,9 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const uint32_t bar_acc_full = bar_sc_empty + SC_SLOTS * 8;  // local: group accumulator complete
   const uint32_t bar_acc_empty = bar_acc_full + ACC_SLOTS * 8;  // LEADER: both CTAs' promotion drained it
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kMiscOff);
+  const uint32_t bar_drain = bar_acc_empty + ACC_SLOTS * 8;     // give-up path of the MMA issuer only
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kMiscOff + 4);
+  const WaitCtx wc{abort_flag, p.wait_limit};
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -148,6 +151,7 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 
   if (threadIdx.x == 0) {
     *abort_flag = 0;
+    mbar_init(bar_drain, 1);
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(bar_full + s * 8, 1);
       mbar_init(bar_empty + s * 8, 1);    // the MMAs' commit: by then the widening has read the stage too
@@ -182,6 +186,7 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const uint32_t tmem_base = *tmem_slot;
 
   grid_dep_launch();   // nothing above touched global data; the successor may begin its set-up
+  uint32_t issued = 0;   // producer thread: ring passes it has requested (for the give-up path)
 
   if (warp < 4) {
     setmaxnreg_dec<kRegsCtl>();
@@ -218,16 +223,18 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         const int t0 = tok0(t), c0 = t.c0 + static_cast<int>(rank) * BC_CTA;
         for (int g = (tile == pair_id ? pre : 0); g < p.k_blocks; ++g, ++it) {
           const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
-          if (!mbar_wait(bar_empty + s * 8, ph ^ 1u, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(bar_empty + s * 8, ph ^ 1u, wc)) { ok = false; break; }
           load_weights(s, g, t.g, c0);
           load_codes(s, g, t0);
         }
       }
+      issued = it;
       (void)ok;
     } else if (warp == 1 && lane == 0 && rank == 0) {
       // ---------------------------------------------------------- MMA issuer (leader only)
       constexpr uint32_t idesc = umma_idesc_s8(BC_PAIR, BT_PAIR);
       const int total = pair_id < num_tiles ? ((num_tiles - pair_id + num_pairs - 1) / num_pairs) * p.k_blocks : 0;   // groups of this pair
+      bool ok = true;
       for (uint32_t it = 0; it < static_cast<uint32_t>(total); ++it) {
         const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
         const uint32_t a = it % ACC_SLOTS, aph = (it / ACC_SLOTS) & 1u;
@@ -235,7 +242,7 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         const uint64_t w_desc = umma_desc_k_sw128(smem_base + kW8Off + s * kW8Bytes);   // 256 channel rows (both CTAs)
         const uint64_t q_desc = umma_desc_k_sw128(smem_base + s * kStageBytes);         // 256 token rows (both CTAs)
         const uint32_t d_tmem = tmem_base + a * BT_PAIR;
-        if (!mbar_wait2_cluster(bar_w8_full + s * 8, ph, bar_acc_empty + a * 8, aph ^ 1u, abort_flag)) break;
+        if (!mbar_wait2_cluster(bar_w8_full + s * 8, ph, bar_acc_empty + a * 8, aph ^ 1u, wc)) { ok = false; break; }
         tc_fence_after_sync();
         umma_i8_pair_imm<0>(d_tmem, w_desc, q_desc, idesc);
         umma_i8_pair_imm<1>(d_tmem, w_desc + 2, q_desc + 2, idesc);
@@ -244,6 +251,7 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         umma_commit_pair_mcast(bar_acc_full + a * 8, 0x3);
         umma_commit_pair_mcast(bar_empty + s * 8, 0x3);   // frees the stage and the widened slot in both CTAs
       }
+      (void)ok;
     }
   } else if (warp < 8) {
     // ------------------------------------------------------------ widen nibbles (warps 4..7)
@@ -259,7 +267,7 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       const uint32_t v = it % SC_SLOTS, vph = (it / SC_SLOTS) & 1u;
       // stage landed; the slot's previous MMAs are done; the scale row has been read
       const bool w = mbar_wait3(bar_full + s * 8, ph, bar_empty + s * 8, ph ^ 1u, bar_sc_empty + v * 8, vph ^ 1u,
-                                abort_flag);
+                                wc);
       if (!__all_sync(0xffffffffu, w)) break;
 #pragma unroll 4
       for (int i = 0; i < (BC_CTA * 4) / 32; ++i) {
@@ -324,7 +332,7 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         if (have_next) {
           sg = sg_next;   // the look-ahead of the previous group saw both barriers complete
         } else {
-          ok = __all_sync(0xffffffffu, mbar_wait2(bar_sc_full + v * 8, vph, bar_acc_full + a * 8, aph, abort_flag));
+          ok = __all_sync(0xffffffffu, mbar_wait2(bar_sc_full + v * 8, vph, bar_acc_full + a * 8, aph, wc));
           if (!ok) break;
           sg = sc_rows[v * BC_CTA + c_local];
         }
@@ -418,6 +426,18 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   // ------------------------------------------------------------ teardown
   tc_fence_before_sync();
   __syncthreads();
+  if (*abort_flag) {
+    // Somebody gave up.  Work already handed to the hardware still completes by itself and must have
+    // done so before this CTA's shared and tensor memory go away: the producer's loads (their barriers
+    // are local) and the leader's MMAs (they read both CTAs' shared memory and write both tensor memories).
+    if (threadIdx.x == 0) {
+      const uint32_t first = issued > static_cast<uint32_t>(STAGES) ? issued - STAGES : 0u;
+      for (uint32_t i = first; i < issued; ++i) mbar_drain(bar_full + (i % STAGES) * 8, (i / STAGES) & 1u);
+    } else if (threadIdx.x == 32 && rank == 0) {
+      umma_commit_pair_mcast(bar_drain, 0x1);
+      mbar_drain(bar_drain, 0u);
+    }
+  }
   __syncwarp();
   cluster_sync_all();  // neither CTA leaves while its peer may still signal or read it
   tc_fence_after_sync();
@@ -431,21 +451,20 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 template <bool kExportAcc>
 int launch_w4(const CUtensorMap& tq, const W4Maps& maps, const W4Args& a, cudaStream_t stream) {
   auto kern = gemm_w4a8_kernel<kExportAcc>;
-  static int configured = 0;  // 0 = not yet, 1 = ok, -1 = unusable
-  if (configured == 0) {
+  // The promotion warps raise their register budget with setmaxnreg; that only terminates if the
+  // CTA's allocation (registers per thread at launch x 512) holds the sum of the three budgets.  The
+  // register count is a property of the compiled kernel: checked once per process.
+  static const int regs_ok = [kern] {
     cudaFuncAttributes fa;
-    if (cudaFuncGetAttributes(&fa, kern) != cudaSuccess) return PQ_ERR_CUDA;
-    // The promotion warps raise their register budget with setmaxnreg; that only terminates if the
-    // CTA's allocation (registers per thread at launch x 512) holds the sum of the three budgets.
-    if (fa.numRegs * kNumThreads < 128 * kRegsCtl + 128 * kRegsUnpack + 256 * kRegsPromote) {
-      configured = -1;
-    } else if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kDynamicSmem) != cudaSuccess) {
-      return PQ_ERR_CUDA;
-    } else {
-      configured = 1;
-    }
+    if (cudaFuncGetAttributes(&fa, kern) != cudaSuccess) return -1;
+    return fa.numRegs * kNumThreads >= 128 * kRegsCtl + 128 * kRegsUnpack + 256 * kRegsPromote ? 1 : 0;
+  }();
+  if (regs_ok <= 0) {
+    cudaGetLastError();
+    return PQ_ERR_CUDA;
   }
-  if (configured < 0) return PQ_ERR_CUDA;
+  static PerDeviceOnce once;
+  if (const int rc = set_dynamic_smem_once(once, kern, kDynamicSmem); rc != PQ_OK) return rc;
   const int tiles = a.m_blocks * a.n_blocks;
   const int max_pairs = sm_count() / 2;
   const int pairs = tiles < max_pairs ? tiles : max_pairs;
@@ -507,6 +526,7 @@ int launch_gemm_w4a8_group(const int8_t* q, const float* s_tok, int count, const
   a.K = static_cast<int>(K);
   a.n_blocks = static_cast<int>(nb_total);
   a.k_blocks = static_cast<int>(K / BK);
+  a.wait_limit = wait_limit();
   return acc_g != nullptr ? launch_w4<true>(tq, maps, a, stream) : launch_w4<false>(tq, maps, a, stream);
 }
 

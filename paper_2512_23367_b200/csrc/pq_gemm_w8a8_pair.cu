@@ -59,6 +59,7 @@ struct PairArgs {
   int M, K;
   int m_blocks, n_blocks, k_blocks;   // n_blocks: over all members
   int splits;               // K is cut into this many parts; 1 = no split
+  uint32_t wait_limit;      // poll bound of every wait
 };
 
 // Tensor maps of the members' weights and outputs (kernel parameter, indexed by member).
@@ -99,7 +100,7 @@ struct PairSmem {
   static constexpr int kOutOff = STAGES * kStageBytes;                     // staging, 2 KB boxes
   static constexpr int kScaleOff = kOutOff + EPI_WARPS * EPI_BUFS * kOutBoxBytes;
   static constexpr int kBarOff = kScaleOff + 4 * BN * 4;   // each warp's own copy of its columns' scales
-  static constexpr int kNumBars = 2 * STAGES + 4;
+  static constexpr int kNumBars = 2 * STAGES + 4 + 1;   // + the MMA issuer's drain barrier
   static constexpr int kMiscOff = kBarOff + kNumBars * 8;
   static constexpr int kDynamic = kMiscOff + 16 + 1024;
   static_assert(kDynamic <= 232448, "exceeds the shared memory of one CTA");
@@ -119,8 +120,11 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
   const uint32_t bar_empty = bar_full + STAGES * 8;     // per CTA: the pair's MMAs released the stage
   const uint32_t bar_tfull = bar_empty + STAGES * 8;    // per CTA: accumulator complete
   const uint32_t bar_tempty = bar_tfull + ACC_BUFS * 8;        // used in the leader: both epilogues drained it
+  const uint32_t bar_drain = bar_tempty + ACC_BUFS * 8;        // give-up path of the MMA issuer only
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::kMiscOff);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::kMiscOff + 4);
+  volatile int* fail_flag = reinterpret_cast<volatile int*>(smem + L::kMiscOff + 12);   // split-K epilogue: a warp's wait ran out
+  const WaitCtx wc{abort_flag, p.wait_limit};
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -138,6 +142,8 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
 
   if (threadIdx.x == 0) {
     *abort_flag = 0;
+    *fail_flag = 0;
+    mbar_init(bar_drain, 1);
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(bar_full + s * 8, 1);    // the leader's producer posts the byte count of BOTH CTAs
       mbar_init(bar_empty + s * 8, 1);
@@ -167,6 +173,7 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
 
   // Everything above touched no global data.  The successor kernel may start its own set-up now.
   grid_dep_launch();
+  uint32_t issued = 0;   // producer thread: ring passes it has requested (for the give-up path)
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer (both CTAs)
@@ -204,14 +211,14 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         const int kb1 = kb_end(unit);
         for (int kb = kb_begin(unit) + (unit == pair_id ? pre : 0); kb < kb1; ++kb, ++it) {
           const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
-          if (!mbar_wait(bar_empty + s * 8, ph ^ 1u, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(bar_empty + s * 8, ph ^ 1u, wc)) { ok = false; break; }
           const uint32_t dst = smem_base + s * L::kStageBytes;
           if (rank == 0) mbar_arrive_expect_tx(bar_full + s * 8, 2 * L::kStageBytes);
           tma_load_2d_pair(dst, &tm_q, full0 + s * 8, kb * BK, m0);
           tma_load_2d_pair(dst + L::kABytes, tm_w, full0 + s * 8, kb * BK, n0);
         }
       }
-      (void)ok;
+      issued = it;
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer (leader only)
@@ -221,13 +228,13 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
       bool ok = true;
       for (int unit = pair_id; unit < num_units && ok; unit += num_pairs, ++t) {
         const uint32_t b = t % ACC_BUFS;
-        if (!mbar_wait(bar_tempty + b * 8, ((t / ACC_BUFS) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+        if (!mbar_wait(bar_tempty + b * 8, ((t / ACC_BUFS) & 1u) ^ 1u, wc)) { ok = false; break; }
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + b * BN;
         const int kb0 = kb_begin(unit), kb1 = kb_end(unit);
         for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
-          if (!mbar_wait(bar_full + s * 8, ph, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(bar_full + s * 8, ph, wc)) { ok = false; break; }
           tc_fence_after_sync();
           const uint32_t a_addr = smem_base + s * L::kStageBytes;
           const uint64_t a_desc = umma_desc_k_sw128(a_addr);
@@ -270,9 +277,13 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         if (row < p.M) st = __ldg(p.s_tok + row);
         __syncwarp();
       }
-      ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + b * 8, (t / ACC_BUFS) & 1u, abort_flag));
-      if (!ok) break;
-      tc_fence_after_sync();
+      const bool got = __all_sync(0xffffffffu, mbar_wait(bar_tfull + b * 8, (t / ACC_BUFS) & 1u, wc));
+      const bool split_unit = !kExportAcc && p.splits > 1;
+      // Without a K split a warp that gave up just leaves.  With one, the epilogue warps of the CTA meet
+      // at named barriers below, so they decide TOGETHER: every warp reaches the first barrier whatever
+      // its own wait said, and all leave after it if any of them failed.
+      if (!got && !split_unit) { ok = false; break; }
+      if (got) tc_fence_after_sync();
       const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + b * BN + half * HC;
       // Split-K: this CTA's slice of the tile's partials, one slot per K part.  The scratch is
       // private, so it is laid out for coalescing: [4-column piece][row] of 16-byte words -- a warp's
@@ -285,25 +296,33 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
           ws_tile = reinterpret_cast<uint4*>(p.ws + (static_cast<int64_t>(tile) * 2 + rank) * p.splits * slot_elems) +
                     static_cast<int64_t>(half * (HC / 4)) * BM_CTA + (quad * 32 + lane);
           uint4* mine = ws_tile + sp * (slot_elems / 4);
+          if (!got) {
+            if (lane == 0) *fail_flag = 1;
+          } else {
 #pragma unroll 1
-          for (int c = 0; c < NCH; ++c) {
-            uint32_t v[32];
-            tmem_ld_32x32(t_addr + c * 32, v);
-            tmem_ld_wait();
+            for (int c = 0; c < NCH; ++c) {
+              uint32_t v[32];
+              tmem_ld_32x32(t_addr + c * 32, v);
+              tmem_ld_wait();
 #pragma unroll
-            for (int j = 0; j < 32; j += 4)
-              __stcg(mine + (c * 8 + j / 4) * BM_CTA, make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]));
+              for (int j = 0; j < 32; j += 4)
+                __stcg(mine + (c * 8 + j / 4) * BM_CTA, make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]));
+            }
           }
           __threadfence();                               // the partial is visible before the arrival
           named_bar_sync(1, EPI_WARPS * 32);
           if (warp == 2 && lane == 0) {
-            unsigned int* ctr = p.counters + (tile * 2 + static_cast<int>(rank));
-            const unsigned int old = atomicAdd(ctr, 1u);
-            const int last = (old == static_cast<unsigned int>(p.splits - 1));
-            if (last) *ctr = 0u;                         // nobody else touches it in this call; zero for the next
+            int last = 0;
+            if (*fail_flag == 0) {
+              unsigned int* ctr = p.counters + (tile * 2 + static_cast<int>(rank));
+              const unsigned int old = atomicAdd(ctr, 1u);
+              last = (old == static_cast<unsigned int>(p.splits - 1));
+              if (last) *ctr = 0u;                       // nobody else touches it in this call; zero for the next
+            }
             *last_flag = last;
           }
           named_bar_sync(1, EPI_WARPS * 32);
+          if (*fail_flag != 0) { ok = false; break; }    // the same answer in every warp
           const bool last = *last_flag != 0;
           __threadfence();                               // the other parts' partials are read after the arrival count
           if (!last) {
@@ -393,6 +412,25 @@ gemm_w8a8_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
   // ------------------------------------------------------------ teardown
   tc_fence_before_sync();
   __syncthreads();
+  if (*abort_flag) {
+    // Somebody gave up.  Work already handed to the hardware still completes by itself and must have
+    // done so before this CTA's shared and tensor memory go away:
+    if (threadIdx.x == 0) {
+      // loads requested by this CTA's producer.  The leader sees them on its "stage landed" barriers;
+      // the peer's loads are counted on the leader's barriers too, which it cannot poll -- it waits a
+      // time that covers any load in flight.
+      if (rank == 0) {
+        const uint32_t first = issued > static_cast<uint32_t>(STAGES) ? issued - STAGES : 0u;
+        for (uint32_t i = first; i < issued; ++i) mbar_drain(bar_full + (i % STAGES) * 8, (i / STAGES) & 1u);
+      } else {
+        drain_sleep_us(100);
+      }
+    } else if (threadIdx.x == 32 && rank == 0) {
+      // MMAs issued by the leader (they read both CTAs' shared memory and write both tensor memories)
+      umma_commit_pair_mcast(bar_drain, 0x1);
+      mbar_drain(bar_drain, 0u);
+    }
+  }
   __syncwarp();
   cluster_sync_all();  // neither CTA leaves while its peer may still signal or read it
   tc_fence_after_sync();
@@ -409,12 +447,8 @@ int launch_pair_cfg(const CUtensorMap& tq, const PairMaps& maps, const PairArgs&
   static_assert(MIN_CTAS * (L::kDynamic + 1024) <= 233472, "co-resident CTAs exceed the SM's shared memory");
   static_assert(MIN_CTAS * ACC_BUFS * BN <= 512, "co-resident CTAs exceed the SM's tensor memory");
   auto kern = gemm_w8a8_pair_kernel<BN, STAGES, EPI_BUFS, ACC_BUFS, EPI_WARPS, MIN_CTAS, kExportAcc>;
-  static bool configured = false;
-  if (!configured) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamic) != cudaSuccess)
-      return PQ_ERR_CUDA;
-    configured = true;
-  }
+  static PerDeviceOnce once;   // one per kernel variant
+  if (const int rc = set_dynamic_smem_once(once, kern, L::kDynamic); rc != PQ_OK) return rc;
   const int units = a.m_blocks * a.n_blocks * a.splits;
   const int max_pairs = MIN_CTAS * (sm_count() / 2);
   const int pairs = units < max_pairs ? units : max_pairs;
@@ -485,14 +519,24 @@ int64_t plan_w8a8_pair(int64_t M, int64_t N, int64_t K, int sms, size_t scratch_
   return plan_w8a8_pair_group(M, &N, 1, K, sms, scratch_bytes, force_bn, force_splits, bn_out, splits_out);
 }
 
+// Bytes of split-K partial sums the plan (bn, splits) needs for these members; 0 when K is not split.
+size_t w8a8_pair_partial_bytes(int64_t M, const int64_t* N, int count, int bn, int splits) {
+  if (splits <= 1) return 0;
+  const int64_t mb = (M + BM_PAIR - 1) / BM_PAIR;
+  int64_t nb = 0;
+  for (int g = 0; g < count; ++g) nb += (N[g] + bn - 1) / bn;
+  return static_cast<size_t>(mb * nb) * 2 * splits * BM_CTA * bn * sizeof(int32_t);
+}
+
 int launch_gemm_w8a8_pair_group(const Scratch& sc, const int8_t* q, const float* s_tok, int count,
                                 const void* const* wq, const float* const* s_ch, const int64_t* N, void* const* y,
                                 int64_t M, int64_t K, int32_t* acc, cudaStream_t stream) {
   if (count < 1 || count > kMaxGroup || (acc != nullptr && count != 1)) return PQ_ERR_SHAPE;
   const int64_t mb = (M + BM_PAIR - 1) / BM_PAIR;
   const int64_t kblocks = (K + BK - 1) / BK;
-  const int force_bn = [] { const char* e = getenv("PQ_W8A8_BN"); return e ? (e[0] == '1' ? 128 : (e[0] == '2' ? 256 : 0)) : 0; }();
-  const int force_splits = [] { const char* e = getenv("PQ_W8A8_SPLITS"); return e ? atoi(e) : 0; }();
+  // ablation knobs, read once per process
+  static const int force_bn = [] { const char* e = getenv("PQ_W8A8_BN"); return e ? (e[0] == '1' ? 128 : (e[0] == '2' ? 256 : 0)) : 0; }();
+  static const int force_splits = [] { const char* e = getenv("PQ_W8A8_SPLITS"); return e ? atoi(e) : 0; }();
   int best_bn = 256, best_splits = 1;
   const int64_t best_cost =
       plan_w8a8_pair_group(M, N, count, K, sm_count(), acc == nullptr && sc.partials != nullptr ? sc.partial_bytes : 0,
@@ -537,27 +581,21 @@ int launch_gemm_w8a8_pair_group(const Scratch& sc, const int8_t* q, const float*
   a.n_blocks = static_cast<int>(nb_total);
   a.k_blocks = static_cast<int>(kblocks);
   a.splits = best_splits;
+  a.wait_limit = wait_limit();
   a.ws = best_splits > 1 ? sc.partials : nullptr;
   a.counters = best_splits > 1 ? sc.counters : nullptr;
   if (acc != nullptr) {
     return use128 ? launch_pair_cfg<128, 7, 2, 2, 8, 1, true>(tq, maps, a, stream)
                   : launch_pair_cfg<256, 5, 2, 2, 8, 1, true>(tq, maps, a, stream);
   }
-  static const int variant = [] { const char* e = getenv("PQ_W8A8_PAIR_CFG"); return e ? atoi(e) : 0; }();
   if (use128) return launch_pair_cfg<128, 7, 2, 2, 8, 1, false>(tq, maps, a, stream);
-  if (variant == 1) return launch_pair_cfg<256, 6, 1, 2, 8, 1, false>(tq, maps, a, stream);
   return launch_pair_cfg<256, 5, 2, 2, 8, 1, false>(tq, maps, a, stream);
 }
 
-int launch_gemm_w8a8_pair_with(const Scratch& sc, const int8_t* q, const float* s_tok, const void* wq,
-                               const float* s_ch, int64_t M, int64_t N, int64_t K, void* y, int32_t* acc,
-                               cudaStream_t stream) {
+int launch_gemm_w8a8_pair(const Scratch& sc, const int8_t* q, const float* s_tok, const void* wq,
+                          const float* s_ch, int64_t M, int64_t N, int64_t K, void* y, int32_t* acc,
+                          cudaStream_t stream) {
   return launch_gemm_w8a8_pair_group(sc, q, s_tok, 1, &wq, &s_ch, &N, &y, M, K, acc, stream);
-}
-
-int launch_gemm_w8a8_pair(const int8_t* q, const float* s_tok, const void* wq, const float* s_ch, int64_t M,
-                          int64_t N, int64_t K, void* y, int32_t* acc, cudaStream_t stream) {
-  return launch_gemm_w8a8_pair_with(scratch(), q, s_tok, wq, s_ch, M, N, K, y, acc, stream);
 }
 
 }  // namespace pq

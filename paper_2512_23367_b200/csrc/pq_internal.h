@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "../../include/pq.h"
 
 namespace pq {
@@ -14,8 +16,9 @@ int* device_status_ptr();  // device address of the status word of the current d
 // Number of SMs of the current device (cached per device).
 int sm_count();
 
-// Caller-provided scratch of the current device (pq_set_workspace): arrival counters first, then
-// room for split-K partial accumulators.  All null/zero when none is registered.
+// Split-K scratch of one GEMM call (the caller's `workspace` argument, or the built-in array of
+// pq_gemm_w8a8_noalloc): arrival counters first, then room for the partial accumulators.  All
+// null/zero when the call has none.
 struct Scratch {
   unsigned int* counters = nullptr;   // kScratchCounters words, zero between calls
   int32_t* partials = nullptr;
@@ -23,7 +26,43 @@ struct Scratch {
 };
 constexpr int kScratchCounters = 16384;                       // 64 KB
 constexpr size_t kScratchHeaderBytes = kScratchCounters * 4;
-Scratch scratch();
+// The view of a caller's workspace: empty when the pointer is null or the room is below the header.
+inline Scratch scratch_from(void* workspace, size_t bytes) {
+  Scratch sc;
+  if (workspace != nullptr && bytes > kScratchHeaderBytes) {
+    sc.counters = static_cast<unsigned int*>(workspace);
+    sc.partials = reinterpret_cast<int32_t*>(static_cast<uint8_t*>(workspace) + kScratchHeaderBytes);
+    sc.partial_bytes = bytes - kScratchHeaderBytes;
+  }
+  return sc;
+}
+
+// Poll bound handed to every kernel (pq_set_wait_limit; default kWaitPollLimit of pq_ptx.cuh).
+uint32_t wait_limit();
+
+// Clears the counter header of the built-in scratch array of pq_gemm_w8a8_noalloc on the current
+// device, if that array has been used on it (after a wait ran out its counters may be non-zero).
+int reset_static_scratch();
+
+// Raises a kernel's dynamic shared-memory limit once per device (the attribute is per device and
+// per kernel; `once` is a function-local static of the launcher of that kernel).  Safe to race:
+// setting the attribute twice is harmless.
+struct PerDeviceOnce {
+  std::atomic<uint64_t> done{0};   // bit d: set on device d
+};
+template <typename Kernel>
+int set_dynamic_smem_once(PerDeviceOnce& once, Kernel kern, int bytes) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return PQ_ERR_CUDA;
+  const uint64_t bit = uint64_t(1) << dev;
+  if (once.done.load(std::memory_order_acquire) & bit) return PQ_OK;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) {
+    cudaGetLastError();
+    return PQ_ERR_CUDA;
+  }
+  once.done.fetch_or(bit, std::memory_order_release);
+  return PQ_OK;
+}
 
 // Whether kernels are launched with the programmatic-stream-serialization attribute (default
 // yes; PQ_PDL=0 in the environment turns it off, for ablations).
@@ -54,18 +93,17 @@ int launch_smooth_scales(const float* xa, const float* wa, int64_t K, float* s, 
 int launch_unpack_w4(const void* wp, int64_t N, int64_t K, int8_t* codes, cudaStream_t stream);
 
 // Prefill-shaped W8A8 GEMM (tcgen05 kind::i8) on CTA pairs (cta_group::2, 256-row tiles), for M > 128.
-// Exactly one of y / acc is non-null.
-int launch_gemm_w8a8_pair(const int8_t* q, const float* s_tok, const void* wq, const float* s_ch, int64_t M,
-                          int64_t N, int64_t K, void* y, int32_t* acc, cudaStream_t stream);
+// Exactly one of y / acc is non-null.  `sc`: split-K scratch of this call (may be empty).
+int launch_gemm_w8a8_pair(const Scratch& sc, const int8_t* q, const float* s_tok, const void* wq,
+                          const float* s_ch, int64_t M, int64_t N, int64_t K, void* y, int32_t* acc,
+                          cudaStream_t stream);
 // Linears that share the token codes and run as one launch of the pair GEMM: at most this many.
 constexpr int kMaxGroup = 4;
 // Host-only: the pair GEMM's choice of tile width and number of K parts (see the definition).
 int64_t plan_w8a8_pair(int64_t M, int64_t N, int64_t K, int sms, size_t scratch_bytes, int force_bn,
                        int force_splits, int* bn_out, int* splits_out);
-// The same with the split-K scratch given explicitly instead of taken from the device's registry.
-int launch_gemm_w8a8_pair_with(const Scratch& sc, const int8_t* q, const float* s_tok, const void* wq,
-                               const float* s_ch, int64_t M, int64_t N, int64_t K, void* y, int32_t* acc,
-                               cudaStream_t stream);
+// Bytes of split-K partial sums the plan (bn, splits) needs for these members; 0 when K is not split.
+size_t w8a8_pair_partial_bytes(int64_t M, const int64_t* N, int count, int bn, int splits);
 // `count` (1..kMaxGroup) linears over the same codes in one launch; arrays are host arrays of
 // device pointers / column counts.  acc (accumulator export) only with count == 1.
 int64_t plan_w8a8_pair_group(int64_t M, const int64_t* N, int count, int64_t K, int sms, size_t scratch_bytes,

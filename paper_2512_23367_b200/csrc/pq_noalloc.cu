@@ -1,8 +1,8 @@
 // pq_gemm_w8a8_noalloc: the W8A8 linear for callers that cannot allocate device memory.
 //
 // The W8A8 GEMM gets its split-K fast path (few output tiles, long K) only when it has scratch
-// memory for the parts' INT32 partial sums.  pq_gemm_w8a8 takes that scratch from a buffer the
-// caller registered with pq_set_workspace, which the caller had to allocate.  Some callers have
+// memory for the parts' INT32 partial sums.  pq_gemm_w8a8 takes that scratch from the workspace
+// argument of the call, a buffer which the caller had to allocate.  Some callers have
 // no allocator to ask: code that runs inside a stream capture or a latency-critical serving loop
 // where cudaMalloc (a synchronizing call) is forbidden, plug-ins whose host hands them only input
 // and output buffers, and programs that pre-size every byte of device memory at start-up.  For
@@ -18,8 +18,13 @@
 //   - it keeps the last call's contents.  The partial sums need no clearing (each is overwritten
 //     before it is read); the arrival counters must be zero when a call starts, which holds at load
 //     (static storage is zero-initialized) and is re-established by the kernel itself at the end of
-//     every call that completes.
+//     every call that completes.  A call whose bounded waits ran out (PQ_ERR_TIMEOUT) may leave them
+//     non-zero: pq_device_status(), which reports that condition, clears them again with a memset on
+//     the array's device address (no allocation).
 #include <cuda_runtime.h>
+
+#include <atomic>
+#include <mutex>
 
 #include "pq_internal.h"
 
@@ -37,10 +42,11 @@ static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBy
 
 constexpr int kMaxDevices = 64;
 struct PerDevice {
-  bool ready = false;
+  std::atomic<bool> ready{false};   // published last; the fill happens under g_mutex
   Scratch scratch;
 };
 PerDevice g_per_device[kMaxDevices];
+std::mutex g_mutex;
 
 // Once per device, with that device current: resolve the array's device address.
 int static_scratch(Scratch* out) {
@@ -50,16 +56,19 @@ int static_scratch(Scratch* out) {
     return PQ_ERR_CUDA;
   }
   PerDevice& d = g_per_device[dev];
-  if (!d.ready) {
-    unsigned char* ptr = nullptr;
-    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_static_scratch) != cudaSuccess || ptr == nullptr) {
-      cudaGetLastError();
-      return PQ_ERR_CUDA;
+  if (!d.ready.load(std::memory_order_acquire)) {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (!d.ready.load(std::memory_order_relaxed)) {
+      unsigned char* ptr = nullptr;
+      if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_static_scratch) != cudaSuccess || ptr == nullptr) {
+        cudaGetLastError();
+        return PQ_ERR_CUDA;
+      }
+      d.scratch.counters = reinterpret_cast<unsigned int*>(ptr);
+      d.scratch.partials = reinterpret_cast<int32_t*>(ptr + kScratchHeaderBytes);
+      d.scratch.partial_bytes = kStaticPartialBytes;
+      d.ready.store(true, std::memory_order_release);
     }
-    d.scratch.counters = reinterpret_cast<unsigned int*>(ptr);
-    d.scratch.partials = reinterpret_cast<int32_t*>(ptr + kScratchHeaderBytes);
-    d.scratch.partial_bytes = kStaticPartialBytes;
-    d.ready = true;
   }
   *out = d.scratch;
   return PQ_OK;
@@ -68,6 +77,24 @@ int static_scratch(Scratch* out) {
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 }  // namespace
+
+// After a wait ran out: put the array's arrival counters back to zero on the current device, if the
+// array was ever used there.  Called by pq_device_status (which has synchronized the device).
+int reset_static_scratch() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+    cudaGetLastError();
+    return PQ_ERR_CUDA;
+  }
+  PerDevice& d = g_per_device[dev];
+  if (!d.ready.load(std::memory_order_acquire)) return PQ_OK;
+  if (cudaMemset(d.scratch.counters, 0, kScratchHeaderBytes) != cudaSuccess) {
+    cudaGetLastError();
+    return PQ_ERR_CUDA;
+  }
+  return PQ_OK;
+}
+
 }  // namespace pq
 
 using namespace pq;
@@ -78,13 +105,14 @@ extern "C" int pq_gemm_w8a8_noalloc(const int8_t* q, const float* s_tok, const v
   if (M < 1 || M > 0x7fffffff || N < 8 || N % 8 != 0 || N > 0x7fffffff) return PQ_ERR_SHAPE;
   if (K < 16 || K % 16 != 0 || K >= 131072) return PQ_ERR_SHAPE;
   if (!aligned16(q) || !aligned16(wq) || !aligned16(y_f16)) return PQ_ERR_ALIGN;
+  if (M <= 128) {
+    // These token counts run on a schedule that reduces inside the SMs and uses no scratch at all:
+    // no limit applies.
+    return pq_gemm_w8a8(q, s_tok, wq, s_ch, M, N, K, y_f16, nullptr, 0, stream);
+  }
   const int64_t padded = ((M + 255) / 256) * 256 * (((N + 255) / 256) * 256);
   if (padded > kMaxPaddedOutputs) return PQ_ERR_LIMIT;   // beyond what the fixed scratch array serves
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (M <= 128) {
-    // These token counts run on schedules that reduce inside the SMs and use no scratch at all.
-    return pq_gemm_w8a8(q, s_tok, wq, s_ch, M, N, K, y_f16, stream);
-  }
   int major = 0, minor = 0, dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess ||
       cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
@@ -96,5 +124,5 @@ extern "C" int pq_gemm_w8a8_noalloc(const int8_t* q, const float* s_tok, const v
   Scratch sc;
   const int rc = static_scratch(&sc);
   if (rc != PQ_OK) return rc;
-  return launch_gemm_w8a8_pair_with(sc, q, s_tok, wq, s_ch, M, N, K, y_f16, nullptr, st);
+  return launch_gemm_w8a8_pair(sc, q, s_tok, wq, s_ch, M, N, K, y_f16, nullptr, st);
 }

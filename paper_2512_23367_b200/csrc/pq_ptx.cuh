@@ -8,9 +8,17 @@
 
 namespace pq {
 
-// Upper bound on polls of one mbarrier wait.  Legitimate waits in these kernels last
-// microseconds; the bound only turns a protocol bug into an error code instead of a hang.
+// Default upper bound on polls of one mbarrier wait.  Legitimate waits in these kernels last
+// microseconds; the bound only turns a protocol bug into an error code instead of a hang.  The
+// bound in force travels to the kernels as an argument (pq_set_wait_limit), so that a test can
+// make a wait run out without anything being broken.
 constexpr uint32_t kWaitPollLimit = 1u << 24;
+
+// What a bounded wait needs: the CTA's "somebody gave up" flag in shared memory and the poll bound.
+struct WaitCtx {
+  volatile int* abort_flag;
+  uint32_t limit;
+};
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -62,18 +70,18 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 }
 // Bounded wait.  Returns false if the bound expired or another role already gave up
 // (`abort_flag` in shared memory); the caller then leaves its loop and drains.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t i = 0; i < kWaitPollLimit; ++i) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& wc) {
+  for (uint32_t i = 0; i < wc.limit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 255u) == 255u && *abort_flag) return false;
+    if ((i & 255u) == 255u && *wc.abort_flag) return false;
   }
-  *abort_flag = 1;
+  *wc.abort_flag = 1;
   return false;
 }
 
 // The same with cluster-scope acquire: for barriers that CTAs of the cluster arrive on remotely.
-__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t i = 0; i < kWaitPollLimit; ++i) {
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, const WaitCtx& wc) {
+  for (uint32_t i = 0; i < wc.limit; ++i) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred P;\n\t"
@@ -83,9 +91,9 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
         : "r"(bar), "r"(parity)
         : "memory");
     if (ok) return true;
-    if ((i & 255u) == 255u && *abort_flag) return false;
+    if ((i & 255u) == 255u && *wc.abort_flag) return false;
   }
-  *abort_flag = 1;
+  *wc.abort_flag = 1;
   return false;
 }
 
@@ -93,8 +101,8 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
 // few hundred cycles (it queues behind the operand traffic in shared memory), so waits that follow
 // each other are issued together: their round trips overlap instead of adding up.
 __device__ __forceinline__ bool mbar_wait2(uint32_t bar_a, uint32_t par_a, uint32_t bar_b, uint32_t par_b,
-                                           volatile int* abort_flag) {
-  for (uint32_t i = 0; i < kWaitPollLimit; ++i) {
+                                           const WaitCtx& wc) {
+  for (uint32_t i = 0; i < wc.limit; ++i) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred P, Q;\n\t"
@@ -106,14 +114,14 @@ __device__ __forceinline__ bool mbar_wait2(uint32_t bar_a, uint32_t par_a, uint3
         : "r"(bar_a), "r"(par_a), "r"(bar_b), "r"(par_b)
         : "memory");
     if (ok) return true;
-    if ((i & 255u) == 255u && *abort_flag) return false;
+    if ((i & 255u) == 255u && *wc.abort_flag) return false;
   }
-  *abort_flag = 1;
+  *wc.abort_flag = 1;
   return false;
 }
 __device__ __forceinline__ bool mbar_wait3(uint32_t bar_a, uint32_t par_a, uint32_t bar_b, uint32_t par_b,
-                                           uint32_t bar_c, uint32_t par_c, volatile int* abort_flag) {
-  for (uint32_t i = 0; i < kWaitPollLimit; ++i) {
+                                           uint32_t bar_c, uint32_t par_c, const WaitCtx& wc) {
+  for (uint32_t i = 0; i < wc.limit; ++i) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred P, Q, R;\n\t"
@@ -127,15 +135,15 @@ __device__ __forceinline__ bool mbar_wait3(uint32_t bar_a, uint32_t par_a, uint3
         : "r"(bar_a), "r"(par_a), "r"(bar_b), "r"(par_b), "r"(bar_c), "r"(par_c)
         : "memory");
     if (ok) return true;
-    if ((i & 255u) == 255u && *abort_flag) return false;
+    if ((i & 255u) == 255u && *wc.abort_flag) return false;
   }
-  *abort_flag = 1;
+  *wc.abort_flag = 1;
   return false;
 }
 // Two barriers that CTAs of the cluster arrive on remotely (cluster-scope acquire).
 __device__ __forceinline__ bool mbar_wait2_cluster(uint32_t bar_a, uint32_t par_a, uint32_t bar_b, uint32_t par_b,
-                                                   volatile int* abort_flag) {
-  for (uint32_t i = 0; i < kWaitPollLimit; ++i) {
+                                                   const WaitCtx& wc) {
+  for (uint32_t i = 0; i < wc.limit; ++i) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred P, Q;\n\t"
@@ -147,9 +155,9 @@ __device__ __forceinline__ bool mbar_wait2_cluster(uint32_t bar_a, uint32_t par_
         : "r"(bar_a), "r"(par_a), "r"(bar_b), "r"(par_b)
         : "memory");
     if (ok) return true;
-    if ((i & 255u) == 255u && *abort_flag) return false;
+    if ((i & 255u) == 255u && *wc.abort_flag) return false;
   }
-  *abort_flag = 1;
+  *wc.abort_flag = 1;
   return false;
 }
 // Non-blocking look at two barriers: nonzero if both phases have completed (acquire, CTA scope).
@@ -165,6 +173,36 @@ __device__ __forceinline__ uint32_t mbar_test2(uint32_t bar_a, uint32_t par_a, u
       : "r"(bar_a), "r"(par_a), "r"(bar_b), "r"(par_b)
       : "memory");
   return ok;   // not consumed here: the caller can let the round trip overlap with other work
+}
+
+// Give-up path only: a short bounded wait for a copy or an MMA that is already in flight (it needs
+// nothing from anybody and ends by itself within microseconds).  Does not touch the abort flag.
+constexpr uint32_t kDrainPollLimit = 1u << 16;
+__device__ __forceinline__ bool mbar_drain(uint32_t bar, uint32_t parity) {
+  for (uint32_t i = 0; i < kDrainPollLimit; ++i) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred P;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 P, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, P;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    if (ok) return true;
+    __nanosleep(64);
+  }
+  return false;
+}
+// Give-up path only: lets copies in flight towards this CTA land when their barrier lives in another
+// CTA and cannot be polled from here.  Bounded in time (and in iterations).
+__device__ __forceinline__ void drain_sleep_us(uint32_t us) {
+  uint64_t t0, t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+  for (uint32_t i = 0; i < (1u << 14); ++i) {
+    __nanosleep(1000);
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    if (t - t0 > static_cast<uint64_t>(us) * 1000u) break;
+  }
 }
 
 // ---------------------------------------------------------------- fences

@@ -129,27 +129,22 @@ def test_full_size_layers_touch_every_tile(M, K, N):
 
 @pytest.mark.parametrize("M,K,N", [(512, 11008, 1024), (300, 11008, 520), (140, 6144, 136), (257, 8192, 264)])
 def test_split_k_through_scratch_matches_the_unsplit_result_bit_for_bit(M, K, N):
-    """Few tiles and a long K: with registered scratch the GEMM cuts K into parts and sums the INT32
-    partials exactly, so the FP16 output must equal the one computed without scratch, twice in a row
-    (the arrival counters go back to zero), and must match the oracle."""
+    """Few tiles and a long K: given a workspace the GEMM cuts K into parts and sums the INT32 partials
+    exactly, so the FP16 output must equal the one computed without a workspace, twice in a row (the
+    arrival counters go back to zero), and must match the oracle."""
+    need = pq.pq_workspace_bytes(M, N, K)
+    assert need > 0 and pq.pq_plan_w8a8(M, N, K, 148, need)[1] > 1      # K really is split
     x = synth.activations(M, K, seed=77)
     w = synth.weights(N, K, seed=78)
     q, s_tok = pq.pq_quantize_act(torch.from_numpy(x).to(DEV))
     wq, s_ch = pq.pq_pack_w8(torch.from_numpy(w).to(DEV))
+    ws = pq.pq_workspace_init(torch.full((need,), 0xAB, dtype=torch.uint8, device=DEV))
     pad = 2048
     buf = torch.full((pad + M * N + pad,), 7.0, dtype=torch.float16, device=DEV)
     y_split = buf[pad:pad + M * N].view(M, N)
-    pq.pq_gemm_w8a8(q, s_tok, wq, s_ch, N, y=y_split)          # scratch registered by the binding
-    y_again = pq.pq_gemm_w8a8(q, s_tok, wq, s_ch, N)
-    torch.cuda.synchronize()
-    pq.pq_set_workspace(None)
-    try:
-        y_plain = pq.pq_gemm_w8a8(q, s_tok, wq, s_ch, N)
-        torch.cuda.synchronize()
-    finally:
-        ws = torch.empty((64 << 20,), dtype=torch.uint8, device=DEV)
-        pq.pq_set_workspace(ws)
-        pq.binding._workspaces[torch.device(DEV).index or 0] = ws
+    pq.pq_gemm_w8a8(q, s_tok, wq, s_ch, N, y=y_split, workspace=ws)
+    y_again = pq.pq_gemm_w8a8(q, s_tok, wq, s_ch, N, workspace=ws)
+    y_plain = pq.pq_gemm_w8a8(q, s_tok, wq, s_ch, N)                    # no workspace: no split
     assert pq.pq_device_status() == 0
     assert torch.equal(y_split, y_plain) and torch.equal(y_again, y_plain)
     assert (buf[:pad] == 7.0).all() and (buf[pad + M * N:] == 7.0).all()
@@ -158,3 +153,34 @@ def test_split_k_through_scratch_matches_the_unsplit_result_bit_for_bit(M, K, N)
     rows = np.unique(np.concatenate([[0, 127, 128, M - 1], np.arange(0, M, 37)]))
     _, y_ref = oracle.gemm_w8a8(q_ref[rows], st_ref[rows], wq_ref, sc_ref)
     assert_y_close(_np(y_split)[rows], y_ref)
+
+
+def test_two_streams_with_their_own_workspaces_run_split_k_concurrently():
+    """Calls that may overlap on the GPU get separate workspaces: two streams each issue a chain of
+    split-K GEMMs (different inputs) with nothing ordering one chain against the other; every result
+    must equal the one computed serially, bit for bit."""
+    M, K, N = 512, 11008, 1024
+    need = pq.pq_workspace_bytes(M, N, K)
+    assert pq.pq_plan_w8a8(M, N, K, 148, need)[1] > 1
+    cases = []
+    for i in range(2):
+        x = synth.activations(M, K, seed=300 + i)
+        w = synth.weights(N, K, seed=310 + i)
+        q, s_tok = pq.pq_quantize_act(torch.from_numpy(x).to(DEV))
+        wq, s_ch = pq.pq_pack_w8(torch.from_numpy(w).to(DEV))
+        ws = pq.pq_workspace_init(torch.empty((need,), dtype=torch.uint8, device=DEV))
+        serial = pq.pq_gemm_w8a8(q, s_tok, wq, s_ch, N)                 # unsplit, default stream
+        cases.append((q, s_tok, wq, s_ch, ws, serial))
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream(device=DEV) for _ in cases]
+    reps = 12
+    outs = [[torch.empty((M, N), dtype=torch.float16, device=DEV) for _ in range(reps)] for _ in cases]
+    for r in range(reps):                                              # interleaved issue: the chains overlap
+        for (q, s_tok, wq, s_ch, ws, _), st, ys in zip(cases, streams, outs):
+            with torch.cuda.stream(st):
+                pq.pq_gemm_w8a8(q, s_tok, wq, s_ch, N, y=ys[r], workspace=ws)
+    torch.cuda.synchronize()
+    assert pq.pq_device_status() == 0
+    for (_, _, _, _, _, serial), ys in zip(cases, outs):
+        for y in ys:
+            assert torch.equal(y, serial)

@@ -41,7 +41,9 @@ def test_group_equals_one_call_per_member_and_the_oracle(M, K, Ns):
     pad = 512
     bufs = [torch.full((pad + M * N + pad,), 5.0, dtype=torch.float16, device=DEV) for N in Ns]
     ys = [b[pad:pad + M * N].view(M, N) for b, N in zip(bufs, Ns)]
-    out = pq.pq_gemm_w8a8_group(q, s_tok, members, ys)
+    need = pq.pq_workspace_bytes(M, Ns, K)
+    scratch = pq.pq_workspace_init(torch.empty((need,), dtype=torch.uint8, device=DEV)) if need else None
+    out = pq.pq_gemm_w8a8_group(q, s_tok, members, ys, workspace=scratch)
     torch.cuda.synchronize()
     assert pq.pq_device_status() == 0
     qo, so = oracle.quantize_act(x)
@@ -73,8 +75,11 @@ def test_two_group_calls_in_a_row_leave_the_split_k_scratch_clean():
     x = synth.activations(M, K, 4500)
     _, members = _members(K, Ns, 4501)
     q, s_tok = pq.pq_quantize_act(torch.from_numpy(x).to(DEV))
-    first = [y.clone() for y in pq.pq_gemm_w8a8_group(q, s_tok, members)]
-    second = pq.pq_gemm_w8a8_group(q, s_tok, members)
+    need = pq.pq_workspace_bytes(M, Ns, K)
+    assert need > 0                                                     # this group splits K
+    scratch = pq.pq_workspace_init(torch.empty((need,), dtype=torch.uint8, device=DEV))
+    first = [y.clone() for y in pq.pq_gemm_w8a8_group(q, s_tok, members, workspace=scratch)]
+    second = pq.pq_gemm_w8a8_group(q, s_tok, members, workspace=scratch)
     for a, b, (wq, s_ch, N) in zip(first, second, members):
         assert torch.equal(a, b)
         assert torch.equal(a, pq.pq_gemm_w8a8(q, s_tok, wq, s_ch, N))
@@ -163,7 +168,9 @@ def test_benchmark_groups_at_full_size_touch_every_tile(bits, M, K, Ns):
     assert np.array_equal(q.cpu().numpy(), qo)
     if bits == 8:
         members = [(*pq.pq_pack_w8(torch.from_numpy(w).to(DEV)), N) for w, N in zip(ws, Ns)]
-        out = pq.pq_gemm_w8a8_group(q, s_tok, members)
+        need = pq.pq_workspace_bytes(M, Ns, K)
+        scratch = pq.pq_workspace_init(torch.empty((need,), dtype=torch.uint8, device=DEV)) if need else None
+        out = pq.pq_gemm_w8a8_group(q, s_tok, members, workspace=scratch)
     else:
         members = [(*pq.pq_pack_w4(torch.from_numpy(w).to(DEV)), N) for w, N in zip(ws, Ns)]
         out = pq.pq_gemm_w4a8_group(q, s_tok, members)

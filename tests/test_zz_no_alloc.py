@@ -29,12 +29,22 @@ def _inputs(M, K, N, seed):
     return q, s_tok, wq, s_ch
 
 
-# shapes on which the kernel really splits K (few tiles, long K), one that does not, one with M <= 128
-@pytest.mark.parametrize("M,K,N", [(512, 11008, 1024), (300, 11008, 520), (257, 8192, 264), (512, 2048, 1000),
-                                   (96, 4096, 512)])
-def test_matches_the_allocating_entry_point_on_two_calls_in_a_row(M, K, N):
+STATIC_SCRATCH_BYTES = (32 << 20) + (64 << 10)      # the array inside the library
+
+
+# shapes on which the kernel really splits K (few tiles, long K), one that does not, and decode-shaped
+# token counts (no scratch at all) whose padded output is beyond the array's limit
+@pytest.mark.parametrize("M,K,N,split", [(512, 11008, 1024, True), (300, 11008, 520, True), (257, 8192, 264, True),
+                                         (512, 2048, 1000, False), (96, 4096, 512, False),
+                                         (1, 4096, 11008, False), (128, 4096, 11008, False)])
+def test_matches_the_allocating_entry_point_on_two_calls_in_a_row(M, K, N, split):
+    # the comparison is only worth something where the scratch array is really used: K must be split
+    # (token counts up to 128 run on the schedule that reduces inside the SMs, whatever the plan would say)
+    assert (M > 128 and pq.pq_plan_w8a8(M, N, K, 148, STATIC_SCRATCH_BYTES)[1] > 1) == split
     q, s_tok, wq, s_ch = _inputs(M, K, N, seed=900 + M)
-    y_ref = pq.pq_gemm_w8a8(q, s_tok, wq, s_ch, N)            # existing entry point (registered workspace)
+    need = pq.pq_workspace_bytes(M, N, K)
+    ws = pq.pq_workspace_init(torch.empty((need,), dtype=torch.uint8, device=DEV)) if need else None
+    y_ref = pq.pq_gemm_w8a8(q, s_tok, wq, s_ch, N, workspace=ws)   # existing entry point (caller's workspace)
     pad = 1024
     for _ in range(2):
         buf = torch.full((pad + M * N + pad,), 7.0, dtype=torch.float16, device=DEV)
