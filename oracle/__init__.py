@@ -61,6 +61,7 @@ def _load():
         lib.pqo_pack_w8_hadamard.argtypes = [vp, i64, i64, vp, vp]
         lib.pqo_pack_w4_hadamard.argtypes = [vp, i64, i64, i64, vp, vp]
         lib.pqo_smooth_scales.argtypes = [vp, vp, i64, vp, vp]
+        lib.pqo_swiglu_quantize.argtypes = [vp, vp, i64, i64, vp, vp, vp]
         lib.pqo_nibble_pack.argtypes = [vp, i64, i64, vp]
         lib.pqo_nibble_unpack.argtypes = [vp, i64, i64, vp]
         lib.pqo_gemm_w8a8.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp, vp]
@@ -184,6 +185,20 @@ def pack_w4_hadamard(w: np.ndarray, group: int = 128):
     s = np.empty((N, K // group), np.float16)
     _check(_load().pqo_pack_w4_hadamard(_p(w), N, K, group, _p(codes), _p(s)), "pack_w4_hadamard")
     return codes, s
+
+
+def swiglu_quantize(gate: np.ndarray, up: np.ndarray, want_h: bool = False):
+    """gate, up f16 [M,I] -> (q int8 [M,I], s_tok f32 [M]) of h = silu(gate) * up (binary32), quantized per
+    token by Eq. 1-2; with want_h also h f32 [M,I] as a third result."""
+    gate, up = _c(gate, np.float16), _c(up, np.float16)
+    if gate.shape != up.shape or gate.ndim != 2:
+        raise OracleError("swiglu_quantize: gate and up must be [M,I]")
+    M, I = gate.shape
+    q = np.empty((M, I), np.int8)
+    s = np.empty((M,), np.float32)
+    h = np.empty((M, I), np.float32) if want_h else None
+    _check(_load().pqo_swiglu_quantize(_p(gate), _p(up), M, I, _p(h), _p(q), _p(s)), "swiglu_quantize")
+    return (q, s, h) if want_h else (q, s)
 
 
 def col_absmax(a: np.ndarray) -> np.ndarray:

@@ -45,6 +45,15 @@
  *     applied as the textbook in-place butterfly (distances 1, 2, 4, ..., B/2 in this order, each
  *     step a' = a + b, b' = a - b in binary32), then one binary32 product with
  *     1 / sqrtf(B); the rotated values stay in binary32.
+ *   - The decoder layer's MLP between the gate/up linears and the down linear (the paper quantizes
+ *     "all linear layers" of such a decoder and times whole prefill passes, Table 3, but does not
+ *     define the activation): the gated form SwiGLU, h = silu(gate) * up, silu(g) = g / (1 + e^-g).
+ *     Its result is the down projection's input and is quantized per token by Eq. 1-2 directly
+ *     (pqo_swiglu_quantize).  Because a binary32 value decides an integer code here, the
+ *     evaluation is FIXED as a sequence of single binary32 operations (swiglu_f32 below): e^t by
+ *     range reduction t = n ln2 + r with ln2 split in two parts, the degree-7 Taylor polynomial
+ *     of e^r in Horner form with fused multiply-adds, an exact scaling by 2^n; then 1 + e, the
+ *     IEEE quotient g / (1 + e), and one product with `up`.  h stays in binary32.
  *
  * Arithmetic notes: integer dot products accumulate in int64 and are checked to
  * fit int32.  All binary32 steps are single IEEE operations (compile with
@@ -185,6 +194,60 @@ static void quantize_row_f32(const float* t, int64_t K, int as_weight, int8_t* q
     float c = r < -128.0f ? -128.0f : (r > 127.0f ? 127.0f : r);
     q[k] = (int8_t)c;
   }
+}
+
+/* ---------------------------------------------------------------- SwiGLU + per-token quantization
+ * silu(g) * u in binary32, as the fixed operation sequence named in the header.  g and u are
+ * exact (FP16 values).  The argument of the exponential is clamped to [-87, 88], where e^t and
+ * 2^n are normal binary32 numbers; beyond it silu is 0 or g to within 1e-33. */
+static float exp_f32(float t) {
+  const float log2e = 0x1.715476p+0f;                       /* 1 / ln 2, rounded to binary32 */
+  const float ln2_hi = 0x1.62e4p-1f, ln2_lo = 0x1.7f7d1cp-20f;   /* ln 2 = hi + lo, hi with 9 trailing zero bits */
+  float n = nearbyintf(t * log2e);
+  float r = fmaf(n, -ln2_hi, t);
+  r = fmaf(n, -ln2_lo, r);
+  float p = 0x1.a01a02p-13f;                                /* 1/7! */
+  p = fmaf(p, r, 0x1.6c16c2p-10f);                          /* 1/6! */
+  p = fmaf(p, r, 0x1.111112p-7f);                           /* 1/5! */
+  p = fmaf(p, r, 0x1.555556p-5f);                           /* 1/4! */
+  p = fmaf(p, r, 0x1.555556p-3f);                           /* 1/3! */
+  p = fmaf(p, r, 0.5f);
+  p = fmaf(p, r, 1.0f);
+  p = fmaf(p, r, 1.0f);
+  union { uint32_t u; float f; } two_n;
+  two_n.u = (uint32_t)((int32_t)n + 127) << 23;             /* 2^n, n in [-126, 127] */
+  return p * two_n.f;
+}
+
+static float swiglu_f32(float g, float u) {
+  float t = -g;
+  t = t < -87.0f ? -87.0f : (t > 88.0f ? 88.0f : t);
+  float d = 1.0f + exp_f32(t);
+  float silu = g / d;
+  return silu * u;
+}
+
+/* h[m,i] = silu(gate[m,i]) * up[m,i] in binary32 (out may be NULL), then Eq. 1-2 per token on h. */
+int pqo_swiglu_quantize(const uint16_t* gate, const uint16_t* up, int64_t M, int64_t I, float* h_out, int8_t* q,
+                        float* s_tok) {
+  if (M < 0 || I <= 0) return PQO_ERR_ARG;
+  int bad = 0;
+#pragma omp parallel for schedule(static)
+  for (int64_t m = 0; m < M; ++m) {
+    float* h = (float*)malloc((size_t)I * sizeof(float));
+    if (!h) {
+      bad = 1;
+      continue;
+    }
+    for (int64_t i = 0; i < I; ++i)
+      h[i] = swiglu_f32(pqo_half_to_float(gate[m * I + i]), pqo_half_to_float(up[m * I + i]));
+    if (h_out) {
+      for (int64_t i = 0; i < I; ++i) h_out[m * I + i] = h[i];
+    }
+    if (q && s_tok) quantize_row_f32(h, I, 0, q + m * I, s_tok + m);
+    free(h);
+  }
+  return bad ? PQO_ERR_ARG : PQO_OK;
 }
 
 /* Eq. 4, activation side: per-token INT8 quantization of X H. */

@@ -574,3 +574,85 @@ def test_static_scale_error_bound_inside_the_calibrated_range():
     # one scale for all tokens: rows without an outlier lose resolution against the per-token rule of Eq. 2
     qd, sd = oracle.quantize_act(x)
     assert (sd <= s * (1 + 1e-6)).all()
+
+
+# ---------------------------------------------------------------------------- SwiGLU + per-token quantization
+
+def _silu64(g):
+    g = g.astype(np.float64)
+    with np.errstate(over="ignore"):
+        return g / (1.0 + np.exp(-g))
+
+
+def test_swiglu_follows_the_definition_on_every_fp16_gate():
+    """h = silu(gate) * up with silu(g) = g / (1 + e^-g): the fixed binary32 sequence stays within 2 ulp of
+    the definition evaluated in binary64 for every finite FP16 gate value (up = 1), is exactly 0 at 0, equals
+    g once e^-g no longer registers beside 1, and vanishes for large negative g."""
+    g = np.arange(65536, dtype=np.uint16).view(np.float16)
+    g = g[np.isfinite(g)].reshape(1, -1)
+    _, _, h = oracle.swiglu_quantize(g, np.ones_like(g), want_h=True)
+    true = _silu64(g)
+    ulp = np.spacing(np.abs(true).astype(np.float32)).astype(np.float64)
+    normal = np.abs(true) > 1e-30
+    assert (np.abs(h - true)[normal] <= 2.0 * ulp[normal]).all()
+    assert (np.abs(h - true)[~normal] <= 1e-33).all()
+    gf = g.astype(np.float32)
+    assert (h[gf == 0] == 0).all()
+    assert np.array_equal(h[gf >= 17], gf[gf >= 17])              # e^-17 < 2^-24: 1 + e^-g rounds to 1
+    assert (np.abs(h[gf <= -104]) <= 1e-33).all()
+    # negative side: the minimum of silu is about -0.2785 near g = -1.2785
+    assert abs(float(h.min()) + 0.27846) < 1e-4
+
+
+def test_swiglu_is_gated_by_the_first_operand_and_scaled_by_the_second():
+    g = np.array([[1.0, -1.0, 2.0, 0.5]], np.float16)
+    u = np.array([[3.0, 3.0, -0.5, 0.0]], np.float16)
+    _, _, h = oracle.swiglu_quantize(g, u, want_h=True)
+    want = _silu64(g) * u.astype(np.float64)
+    assert np.allclose(h, want, rtol=3e-7, atol=0)
+    _, _, h_swapped = oracle.swiglu_quantize(u, g, want_h=True)
+    assert not np.allclose(h_swapped, want, rtol=1e-3)             # silu(u) * g is a different function
+
+
+def test_swiglu_quantize_reduces_to_the_pinned_quantizer_when_the_gate_factor_is_a_power_of_two():
+    """With gate = 32 everywhere, silu(32) = 32 exactly, so h = 32 * up exactly (a power of two): the codes
+    must be those of the pinned per-token quantizer on `up` and the scales 32 times its scales."""
+    from paper_2512_23367_b200 import synth
+    up = synth.activations(24, 640, seed=71)
+    up[3] = 0                                                       # a zero row stays a zero row
+    gate = np.full_like(up, 32.0)
+    q, s = oracle.swiglu_quantize(gate, up)
+    q_ref, s_ref = oracle.quantize_act(up)
+    assert np.array_equal(q, q_ref)
+    assert np.array_equal(s, 32.0 * s_ref)
+    assert s[3] == 0 and (q[3] == 0).all()
+    # gate = 0 closes every channel: the whole row is zero
+    q0, s0 = oracle.swiglu_quantize(np.zeros_like(up), up)
+    assert (q0 == 0).all() and (s0 == 0).all()
+    # the operands are not interchangeable: gating by `up` and scaling by 32 gives other codes
+    q_sw, _ = oracle.swiglu_quantize(up, gate)
+    assert not np.array_equal(q_sw, q_ref)
+
+
+def test_swiglu_quantize_closed_form_codes():
+    # gate = 64 (silu = 64 exactly), up = multiples of 1/128 with maximum 127.5/128: h = up * 64, scale 0.5 * 64 / 64...
+    up = np.array([[127.5 / 128, 0.5 / 128, 1.5 / 128, 2.5 / 128, -0.5 / 128, -1.5 / 128, -127.5 / 128, 64.0 / 128]], np.float16)
+    gate = np.full_like(up, 64.0)
+    q, s = oracle.swiglu_quantize(gate, up)
+    # a = 127.5/128 * 64 = 63.75, s = a / 127.5 = 0.5, codes = rne(h / 0.5) = rne(up * 128): ties to even, +max clamps to 127
+    assert s.tolist() == [0.5]
+    assert q[0].tolist() == [127, 0, 2, 2, 0, -2, -128, 64]
+
+
+def test_swiglu_quantize_half_step_bound_against_the_definition():
+    from paper_2512_23367_b200 import synth
+    rng = np.random.default_rng(5)
+    gate = (rng.standard_normal((16, 1024)) * 3).astype(np.float16)
+    up = synth.activations(16, 1024, seed=72)
+    q, s, h = oracle.swiglu_quantize(gate, up, want_h=True)
+    true = _silu64(gate) * up.astype(np.float64)
+    assert np.allclose(h, true, rtol=4e-7, atol=1e-30)
+    err = np.abs(true - q.astype(np.float64) * s.astype(np.float64)[:, None])
+    assert (err <= s.astype(np.float64)[:, None] * (0.5 + 1e-4)).all()
+    assert (np.abs(q.astype(np.int32)).max(axis=1) >= 127).all()    # every row uses the full range
+    assert np.array_equal(s, (np.abs(h).max(axis=1) / np.float32(127.5)).astype(np.float32))
