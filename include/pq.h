@@ -140,6 +140,24 @@ PQ_API int pq_quantize_act_static(const void* x_f16, const float* scale, int64_t
                                   float* s_tok, void* stream);
 
 /*
+ * The MLP's gated activation fused with the down projection's activation quantizer.  The paper
+ * quantizes all linear layers of a decoder and reports whole prefill passes (its latency table), but
+ * does not define the activation between the gate/up linears and the down linear; the gated form
+ * SwiGLU is taken:  h[m,i] = silu(gate[m,i]) * up[m,i],  silu(g) = g / (1 + e^-g).
+ * h is evaluated in FP32 as a FIXED sequence of single correctly rounded operations (the argument of
+ * the exponential clamped to [-87, 88]; e^t by the reduction t = n ln2 + r, the degree-7 Taylor
+ * polynomial of e^r in Horner form with fused multiply-adds and an exact scaling by 2^n; then 1 + e^t,
+ * the IEEE quotient g / (1 + e^t) and one product with `up`), because its value decides integer codes;
+ * it is not rounded to FP16.  Then pq_quantize_act's rule (Eq. 1-2 per token) is applied to h.
+ * One pass: 4 bytes read and 1 written per element, instead of an FP16 round trip of h plus a
+ * separate quantizer pass.
+ *   gate_f16, up_f16 [M,I] FP16 in (the outputs of the gate and up linears);  q [M,I] INT8 out;
+ *   s_tok [M] FP32 out;  I as K of the quantizer, I <= 16384 (PQ_ERR_SHAPE beyond).
+ */
+PQ_API int pq_swiglu_quantize(const void* gate_f16, const void* up_f16, int64_t M, int64_t I, int8_t* q,
+                              float* s_tok, void* stream);
+
+/*
  * Hadamard variant (Eq. 4: Y = (X H)(H^T W), H a normalized Hadamard matrix).  With W stored [N,K]
  * both operands are rotated along K: (X H)(W H)^T = X W^T.  A Hadamard matrix of order K does not
  * exist for every layer width (11008 = 2^8 * 43), so H = I (x) H_B / sqrt(B) is block diagonal, H_B

@@ -31,6 +31,7 @@ from .binding import (  # noqa: F401
     pq_quantize_act_static,
     pq_set_wait_limit,
     pq_smooth_scales,
+    pq_swiglu_quantize,
     pq_unpack_w4,
     pq_unpack_w8,
     pq_workspace_bytes,

@@ -40,6 +40,7 @@ SIGNATURES = {
                                           ctypes.POINTER(_i64), ctypes.POINTER(_vp), _i64, _i64, _vp,
                                           ctypes.c_size_t, _vp]),
     "pq_quantize_act_static": (ctypes.c_int, [_vp, _vp, _i64, _i64, _vp, _vp, _vp]),
+    "pq_swiglu_quantize": (ctypes.c_int, [_vp, _vp, _i64, _i64, _vp, _vp, _vp]),
     "pq_hadamard_block": (_i32, [_i64]),
     "pq_quantize_act_hadamard": (ctypes.c_int, [_vp, _i64, _i64, _vp, _vp, _vp]),
     "pq_pack_w8_hadamard": (ctypes.c_int, [_vp, _i64, _i64, _vp, _vp, _vp]),
@@ -191,6 +192,18 @@ def pq_quantize_act_static(x: torch.Tensor, scale: torch.Tensor, q: torch.Tensor
     _together(x, scale)
     _check("pq_quantize_act_static", lib().pq_quantize_act_static(x.data_ptr(), scale.data_ptr(), M, K, q.data_ptr(),
                                                                   s_tok.data_ptr(), _stream()))
+    return q, s_tok
+
+
+def pq_swiglu_quantize(gate: torch.Tensor, up: torch.Tensor, q: torch.Tensor | None = None,
+                       s_tok: torch.Tensor | None = None):
+    """The MLP's gated activation fused with the down projection's quantizer: gate, up f16 [M,I] ->
+    (q int8 [M,I], s_tok f32 [M]) of h = silu(gate) * up."""
+    M, I, q, s_tok = _rows(gate, q, s_tok)
+    _sized(up, torch.float16, M * I, "up")
+    _together(gate, up)
+    _check("pq_swiglu_quantize", lib().pq_swiglu_quantize(gate.data_ptr(), up.data_ptr(), M, I, q.data_ptr(),
+                                                          s_tok.data_ptr(), _stream()))
     return q, s_tok
 
 

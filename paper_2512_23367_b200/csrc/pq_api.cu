@@ -243,6 +243,17 @@ int pq_quantize_act_static(const void* x_f16, const float* scale, int64_t M, int
   return launch_quantize_act_static(x_f16, scale, M, K, q, s_tok, static_cast<cudaStream_t>(stream));
 }
 
+int pq_swiglu_quantize(const void* gate_f16, const void* up_f16, int64_t M, int64_t I, int8_t* q, float* s_tok,
+                       void* stream) {
+  if (!gate_f16 || !up_f16 || !q || !s_tok) return PQ_ERR_NULL;
+  int rc = check_rows(M, I);
+  if (rc != PQ_OK) return rc;
+  if (I > 16384) return PQ_ERR_SHAPE;
+  if (!aligned16(gate_f16) || !aligned16(up_f16) || !aligned16(q)) return PQ_ERR_ALIGN;
+  if ((rc = check_arch()) != PQ_OK) return rc;
+  return launch_swiglu_quantize(gate_f16, up_f16, M, I, q, s_tok, static_cast<cudaStream_t>(stream));
+}
+
 int32_t pq_hadamard_block(int64_t K) { return (K >= 16 && K % 16 == 0) ? hadamard_block_order(K) : 0; }
 
 int pq_quantize_act_hadamard(const void* x_f16, int64_t M, int64_t K, int8_t* q, float* s_tok, void* stream) {

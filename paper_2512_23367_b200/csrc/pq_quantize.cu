@@ -565,6 +565,130 @@ int launch_pack_w4_hadamard(const void* w, int64_t N, int64_t K, void* wp, void*
   return cuda_status(cudaGetLastError());
 }
 
+// ---------------------------------------------------------------------------- SwiGLU + per-token quantization
+namespace {
+
+// e^t for t in [-87, 88] as a fixed sequence of binary32 operations (every step a single correctly
+// rounded operation, so that the INT8 codes decided by the result are reproducible anywhere):
+// t = n ln2 + r with ln2 split into a part with 9 trailing zero bits (n * hi is exact) and a remainder,
+// e^r by the degree-7 Taylor polynomial in Horner form with fused multiply-adds, times 2^n (built from
+// its exponent field; n is in [-126, 127]).
+__device__ __forceinline__ float exp_fixed(float t) {
+  const float n = rintf(__fmul_rn(t, 1.44269502162933349609375f));      // 1 / ln 2 rounded to binary32
+  float r = __fmaf_rn(n, -0.693145751953125f, t);                       // ln 2, upper part
+  r = __fmaf_rn(n, -1.42860676533018704503775e-06f, r);                 // ln 2, lower part
+  float p = 1.98412701138295233249664e-04f;                             // 1/7!
+  p = __fmaf_rn(p, r, 1.38888892251998186111450e-03f);                  // 1/6!
+  p = __fmaf_rn(p, r, 8.33333376795053482055664e-03f);                  // 1/5!
+  p = __fmaf_rn(p, r, 4.16666679084300994873047e-02f);                  // 1/4!
+  p = __fmaf_rn(p, r, 1.66666671633720397949219e-01f);                  // 1/3!
+  p = __fmaf_rn(p, r, 0.5f);
+  p = __fmaf_rn(p, r, 1.0f);
+  p = __fmaf_rn(p, r, 1.0f);
+  const float two_n = __int_as_float((__float2int_rn(n) + 127) << 23);
+  return __fmul_rn(p, two_n);
+}
+
+// silu(g) * u, silu(g) = g / (1 + e^-g): clamp of the exponent's argument, e^t as above, one addition,
+// one IEEE division, one product.  Not rounded back to FP16.
+__device__ __forceinline__ float swiglu_fixed(float g, float u) {
+  const float t = fminf(fmaxf(-g, -87.0f), 88.0f);
+  const float d = __fadd_rn(1.0f, exp_fixed(t));
+  return __fmul_rn(__fdiv_rn(g, d), u);
+}
+
+// h = silu(gate) * up for one token row, kept in FP32 registers (I <= 8 * C * T), then the per-token
+// quantizer of Eq. 1-2 on h: the MLP's gated activation and the down projection's activation quantizer
+// in one pass over the gate/up outputs (4 bytes read, 1 written per element; no FP16 round trip of h).
+template <int T, int C>
+__global__ void __launch_bounds__(kThreads) swiglu_quantize_kernel(const uint4* __restrict__ gate,
+                                                                   const uint4* __restrict__ up, int64_t M, int K8,
+                                                                   uint2* __restrict__ q, float* __restrict__ scale) {
+  constexpr int kRowsPerBlock = kThreads / T;
+  constexpr int kWarpsPerRow = T / 32;
+  __shared__ float red[kThreads / 32];
+  const int tid = threadIdx.x;
+  const int t = tid % T;
+  const int64_t row = static_cast<int64_t>(blockIdx.x) * kRowsPerBlock + tid / T;
+  const bool live = row < M;
+
+  grid_dep_launch();
+  grid_dep_wait();   // gate and up are the outputs of the preceding GEMM
+
+  float v[C][8];
+  float a = 0.0f;
+#pragma unroll
+  for (int i = 0; i < C; ++i) {
+    const int c = t + i * T;
+    if (live && c < K8) {
+      const uint4 gr = __ldg(gate + row * K8 + c), ur = __ldg(up + row * K8 + c);
+      const __half* gh = reinterpret_cast<const __half*>(&gr);
+      const __half* uh = reinterpret_cast<const __half*>(&ur);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        v[i][j] = swiglu_fixed(__half2float(gh[j]), __half2float(uh[j]));
+        a = fmaxf(a, fabsf(v[i][j]));
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) v[i][j] = 0.0f;
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
+  if constexpr (kWarpsPerRow > 1) {
+    if ((tid & 31) == 0) red[tid >> 5] = a;
+    __syncthreads();
+    const int w0 = (tid / T) * kWarpsPerRow;
+#pragma unroll
+    for (int w = 0; w < kWarpsPerRow; ++w) a = fmaxf(a, red[w0 + w]);
+  }
+  if (!live) return;
+  const float s = __fdiv_rn(a, 127.5f);
+  const float f = (a == 0.0f) ? 0.0f : __fdiv_rn(127.5f, a);
+  if (t == 0) scale[row] = s;
+  uint2* qr = q + row * K8;
+#pragma unroll
+  for (int i = 0; i < C; ++i) {
+    const int c = t + i * T;
+    if (c < K8) {
+      qr[c] = make_uint2(codes4<false>(v[i][0], v[i][1], v[i][2], v[i][3], f),
+                         codes4<false>(v[i][4], v[i][5], v[i][6], v[i][7], f));
+    }
+  }
+}
+
+template <int T, int C>
+int launch_swiglu_team(const void* gate, const void* up, int64_t M, int K8, int8_t* q, float* s, cudaStream_t stream) {
+  constexpr int kRowsPerBlock = kThreads / T;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>((M + kRowsPerBlock - 1) / kRowsPerBlock), 1, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl_enabled() ? 1 : 0;
+  return cuda_status(cudaLaunchKernelEx(&cfg, swiglu_quantize_kernel<T, C>, static_cast<const uint4*>(gate),
+                                        static_cast<const uint4*>(up), M, K8, reinterpret_cast<uint2*>(q), s));
+}
+
+}  // namespace
+
+int launch_swiglu_quantize(const void* gate, const void* up, int64_t M, int64_t I, int8_t* q, float* s_tok,
+                           cudaStream_t stream) {
+  const int K8 = static_cast<int>(I / 8);
+  if (K8 > 256 * kCached) return PQ_ERR_SHAPE;   // the row has to fit the team's registers
+  // the narrowest team that holds the row with four chunks per thread; eight only for the longest rows
+  if (K8 <= 32 * 4) return launch_swiglu_team<32, 4>(gate, up, M, K8, q, s_tok, stream);
+  if (K8 <= 64 * 4) return launch_swiglu_team<64, 4>(gate, up, M, K8, q, s_tok, stream);
+  if (K8 <= 128 * 4) return launch_swiglu_team<128, 4>(gate, up, M, K8, q, s_tok, stream);
+  if (K8 <= 256 * 4) return launch_swiglu_team<256, 4>(gate, up, M, K8, q, s_tok, stream);
+  if (K8 <= 256 * 6) return launch_swiglu_team<256, 6>(gate, up, M, K8, q, s_tok, stream);
+  return launch_swiglu_team<256, kCached>(gate, up, M, K8, q, s_tok, stream);
+}
+
 // ---------------------------------------------------------------------------- static activation scale
 namespace {
 
