@@ -145,9 +145,9 @@ PQ_API int pq_quantize_act_static(const void* x_f16, const float* scale, int64_t
  * does not define the activation between the gate/up linears and the down linear; the gated form
  * SwiGLU is taken:  h[m,i] = silu(gate[m,i]) * up[m,i],  silu(g) = g / (1 + e^-g).
  * h is evaluated in FP32 as a FIXED sequence of single correctly rounded operations (the argument of
- * the exponential clamped to [-87, 88]; e^t by the reduction t = n ln2 + r, the degree-7 Taylor
- * polynomial of e^r in Horner form with fused multiply-adds and an exact scaling by 2^n; then 1 + e^t,
- * the IEEE quotient g / (1 + e^t) and one product with `up`), because its value decides integer codes;
+ * the exponential clamped to [-87, 88]; the reduction t = n ln2 + r, the degree-7 Taylor polynomial p
+ * of e^r in Horner form with fused multiply-adds, d = fma(p, 2^n, 1) = 1 + e^t; then the IEEE reciprocal
+ * of d, the product g * (1 / d) and one product with `up`), because its value decides integer codes;
  * it is not rounded to FP16.  Then pq_quantize_act's rule (Eq. 1-2 per token) is applied to h.
  * One pass: 4 bytes read and 1 written per element, instead of an FP16 round trip of h plus a
  * separate quantizer pass.

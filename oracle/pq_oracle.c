@@ -52,8 +52,9 @@
  *     (pqo_swiglu_quantize).  Because a binary32 value decides an integer code here, the
  *     evaluation is FIXED as a sequence of single binary32 operations (swiglu_f32 below): e^t by
  *     range reduction t = n ln2 + r with ln2 split in two parts, the degree-7 Taylor polynomial
- *     of e^r in Horner form with fused multiply-adds, an exact scaling by 2^n; then 1 + e, the
- *     IEEE quotient g / (1 + e), and one product with `up`.  h stays in binary32.
+ *     p of e^r in Horner form with fused multiply-adds; then d = fma(p, 2^n, 1) = 1 + e^t, the
+ *     IEEE reciprocal 1 / d, the product g * (1 / d) and one product with `up`.  h stays in
+ *     binary32.
  *
  * Arithmetic notes: integer dot products accumulate in int64 and are checked to
  * fit int32.  All binary32 steps are single IEEE operations (compile with
@@ -200,7 +201,7 @@ static void quantize_row_f32(const float* t, int64_t K, int as_weight, int8_t* q
  * silu(g) * u in binary32, as the fixed operation sequence named in the header.  g and u are
  * exact (FP16 values).  The argument of the exponential is clamped to [-87, 88], where e^t and
  * 2^n are normal binary32 numbers; beyond it silu is 0 or g to within 1e-33. */
-static float exp_f32(float t) {
+static float one_plus_exp_f32(float t) {
   const float log2e = 0x1.715476p+0f;                       /* 1 / ln 2, rounded to binary32 */
   const float ln2_hi = 0x1.62e4p-1f, ln2_lo = 0x1.7f7d1cp-20f;   /* ln 2 = hi + lo, hi with 9 trailing zero bits */
   float n = nearbyintf(t * log2e);
@@ -216,14 +217,14 @@ static float exp_f32(float t) {
   p = fmaf(p, r, 1.0f);
   union { uint32_t u; float f; } two_n;
   two_n.u = (uint32_t)((int32_t)n + 127) << 23;             /* 2^n, n in [-126, 127] */
-  return p * two_n.f;
+  return fmaf(p, two_n.f, 1.0f);                            /* 1 + e^t, one rounding */
 }
 
 static float swiglu_f32(float g, float u) {
   float t = -g;
   t = t < -87.0f ? -87.0f : (t > 88.0f ? 88.0f : t);
-  float d = 1.0f + exp_f32(t);
-  float silu = g / d;
+  float rcp = 1.0f / one_plus_exp_f32(t);
+  float silu = g * rcp;
   return silu * u;
 }
 

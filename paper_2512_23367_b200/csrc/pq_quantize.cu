@@ -568,13 +568,16 @@ int launch_pack_w4_hadamard(const void* w, int64_t N, int64_t K, void* wp, void*
 // ---------------------------------------------------------------------------- SwiGLU + per-token quantization
 namespace {
 
-// e^t for t in [-87, 88] as a fixed sequence of binary32 operations (every step a single correctly
+// 1 + e^t for t in [-87, 88] as a fixed sequence of binary32 operations (every step a single correctly
 // rounded operation, so that the INT8 codes decided by the result are reproducible anywhere):
-// t = n ln2 + r with ln2 split into a part with 9 trailing zero bits (n * hi is exact) and a remainder,
-// e^r by the degree-7 Taylor polynomial in Horner form with fused multiply-adds, times 2^n (built from
-// its exponent field; n is in [-126, 127]).
-__device__ __forceinline__ float exp_fixed(float t) {
-  const float n = rintf(__fmul_rn(t, 1.44269502162933349609375f));      // 1 / ln 2 rounded to binary32
+// t = n ln2 + r with n = rne(t / ln2) and ln2 split into a part with 9 trailing zero bits (n * hi is
+// exact) and a remainder, p = e^r by the degree-7 Taylor polynomial in Horner form with fused
+// multiply-adds, result fma(p, 2^n, 1).  rne(x) for |x| < 2^22 is taken as (x + 1.5 * 2^23) - 1.5 * 2^23:
+// the sum's low mantissa bits are n itself, so 2^n (n in [-126, 127]) is built from them with one
+// shift-and-add and no conversion instruction.
+__device__ __forceinline__ float one_plus_exp_fixed(float t) {
+  const float big = __fadd_rn(__fmul_rn(t, 1.44269502162933349609375f), 12582912.0f);   // 1 / ln 2 rounded to binary32
+  const float n = __fadd_rn(big, -12582912.0f);
   float r = __fmaf_rn(n, -0.693145751953125f, t);                       // ln 2, upper part
   r = __fmaf_rn(n, -1.42860676533018704503775e-06f, r);                 // ln 2, lower part
   float p = 1.98412701138295233249664e-04f;                             // 1/7!
@@ -585,28 +588,33 @@ __device__ __forceinline__ float exp_fixed(float t) {
   p = __fmaf_rn(p, r, 0.5f);
   p = __fmaf_rn(p, r, 1.0f);
   p = __fmaf_rn(p, r, 1.0f);
-  const float two_n = __int_as_float((__float2int_rn(n) + 127) << 23);
-  return __fmul_rn(p, two_n);
+  // as_int(big) = 0x4B400000 + n and 0x4B400000 << 23 == 0 (mod 2^32): (n + 127) << 23
+  const float two_n = __int_as_float((__float_as_int(big) << 23) + 0x3F800000);
+  return __fmaf_rn(p, two_n, 1.0f);
 }
 
-// silu(g) * u, silu(g) = g / (1 + e^-g): clamp of the exponent's argument, e^t as above, one addition,
-// one IEEE division, one product.  Not rounded back to FP16.
+// silu(g) * u, silu(g) = g / (1 + e^-g): clamp of the exponent's argument, d = 1 + e^t as above, the
+// IEEE reciprocal of d, and two products.  Not rounded back to FP16.
 __device__ __forceinline__ float swiglu_fixed(float g, float u) {
   const float t = fminf(fmaxf(-g, -87.0f), 88.0f);
-  const float d = __fadd_rn(1.0f, exp_fixed(t));
-  return __fmul_rn(__fdiv_rn(g, d), u);
+  return __fmul_rn(__fmul_rn(g, __frcp_rn(one_plus_exp_fixed(t))), u);
 }
 
 // h = silu(gate) * up for one token row, kept in FP32 registers (I <= 8 * C * T), then the per-token
 // quantizer of Eq. 1-2 on h: the MLP's gated activation and the down projection's activation quantizer
 // in one pass over the gate/up outputs (4 bytes read, 1 written per element; no FP16 round trip of h).
-template <int T, int C>
-__global__ void __launch_bounds__(kThreads) swiglu_quantize_kernel(const uint4* __restrict__ gate,
-                                                                   const uint4* __restrict__ up, int64_t M, int K8,
-                                                                   uint2* __restrict__ q, float* __restrict__ scale) {
-  constexpr int kRowsPerBlock = kThreads / T;
+// About 40 instructions per element (the fixed exponential and the reciprocal) next to 5 bytes of
+// traffic: the kernel needs many resident warps, so long rows are spread over 512 threads with three or
+// four 16-byte chunks each (<= 64 registers, 32 warps per SM) and all of a thread's loads are issued
+// before its first use.
+template <int BLOCK, int T, int C>
+__global__ void __launch_bounds__(BLOCK, 2048 / BLOCK / 2) swiglu_quantize_kernel(const uint4* __restrict__ gate,
+                                                                                const uint4* __restrict__ up, int64_t M,
+                                                                                int K8, uint2* __restrict__ q,
+                                                                                float* __restrict__ scale) {
+  constexpr int kRowsPerBlock = BLOCK / T;
   constexpr int kWarpsPerRow = T / 32;
-  __shared__ float red[kThreads / 32];
+  __shared__ float red[BLOCK / 32];
   const int tid = threadIdx.x;
   const int t = tid % T;
   const int64_t row = static_cast<int64_t>(blockIdx.x) * kRowsPerBlock + tid / T;
@@ -615,23 +623,27 @@ __global__ void __launch_bounds__(kThreads) swiglu_quantize_kernel(const uint4* 
   grid_dep_launch();
   grid_dep_wait();   // gate and up are the outputs of the preceding GEMM
 
+  uint4 gr[C], ur[C];
+#pragma unroll
+  for (int i = 0; i < C; ++i) {
+    const int c = t + i * T;
+    gr[i] = make_uint4(0u, 0u, 0u, 0u);   // silu(0) * 0 = 0: a chunk past the row's end adds nothing to the maximum
+    ur[i] = make_uint4(0u, 0u, 0u, 0u);
+    if (live && c < K8) {
+      gr[i] = __ldg(gate + row * K8 + c);
+      ur[i] = __ldg(up + row * K8 + c);
+    }
+  }
   float v[C][8];
   float a = 0.0f;
 #pragma unroll
   for (int i = 0; i < C; ++i) {
-    const int c = t + i * T;
-    if (live && c < K8) {
-      const uint4 gr = __ldg(gate + row * K8 + c), ur = __ldg(up + row * K8 + c);
-      const __half* gh = reinterpret_cast<const __half*>(&gr);
-      const __half* uh = reinterpret_cast<const __half*>(&ur);
+    const __half* gh = reinterpret_cast<const __half*>(&gr[i]);
+    const __half* uh = reinterpret_cast<const __half*>(&ur[i]);
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        v[i][j] = swiglu_fixed(__half2float(gh[j]), __half2float(uh[j]));
-        a = fmaxf(a, fabsf(v[i][j]));
-      }
-    } else {
-#pragma unroll
-      for (int j = 0; j < 8; ++j) v[i][j] = 0.0f;
+    for (int j = 0; j < 8; ++j) {
+      v[i][j] = swiglu_fixed(__half2float(gh[j]), __half2float(uh[j]));
+      a = fmaxf(a, fabsf(v[i][j]));
     }
   }
 #pragma unroll
@@ -658,19 +670,19 @@ __global__ void __launch_bounds__(kThreads) swiglu_quantize_kernel(const uint4* 
   }
 }
 
-template <int T, int C>
+template <int BLOCK, int T, int C>
 int launch_swiglu_team(const void* gate, const void* up, int64_t M, int K8, int8_t* q, float* s, cudaStream_t stream) {
-  constexpr int kRowsPerBlock = kThreads / T;
+  constexpr int kRowsPerBlock = BLOCK / T;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(static_cast<unsigned>((M + kRowsPerBlock - 1) / kRowsPerBlock), 1, 1);
-  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.blockDim = dim3(BLOCK, 1, 1);
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = pdl_enabled() ? 1 : 0;
-  return cuda_status(cudaLaunchKernelEx(&cfg, swiglu_quantize_kernel<T, C>, static_cast<const uint4*>(gate),
+  return cuda_status(cudaLaunchKernelEx(&cfg, swiglu_quantize_kernel<BLOCK, T, C>, static_cast<const uint4*>(gate),
                                         static_cast<const uint4*>(up), M, K8, reinterpret_cast<uint2*>(q), s));
 }
 
@@ -679,14 +691,15 @@ int launch_swiglu_team(const void* gate, const void* up, int64_t M, int K8, int8
 int launch_swiglu_quantize(const void* gate, const void* up, int64_t M, int64_t I, int8_t* q, float* s_tok,
                            cudaStream_t stream) {
   const int K8 = static_cast<int>(I / 8);
-  if (K8 > 256 * kCached) return PQ_ERR_SHAPE;   // the row has to fit the team's registers
-  // the narrowest team that holds the row with four chunks per thread; eight only for the longest rows
-  if (K8 <= 32 * 4) return launch_swiglu_team<32, 4>(gate, up, M, K8, q, s_tok, stream);
-  if (K8 <= 64 * 4) return launch_swiglu_team<64, 4>(gate, up, M, K8, q, s_tok, stream);
-  if (K8 <= 128 * 4) return launch_swiglu_team<128, 4>(gate, up, M, K8, q, s_tok, stream);
-  if (K8 <= 256 * 4) return launch_swiglu_team<256, 4>(gate, up, M, K8, q, s_tok, stream);
-  if (K8 <= 256 * 6) return launch_swiglu_team<256, 6>(gate, up, M, K8, q, s_tok, stream);
-  return launch_swiglu_team<256, kCached>(gate, up, M, K8, q, s_tok, stream);
+  if (K8 > 512 * 4) return PQ_ERR_SHAPE;   // the row has to fit the team's registers
+  // the narrowest team that holds the row with at most four chunks per thread
+  if (K8 <= 32 * 4) return launch_swiglu_team<256, 32, 4>(gate, up, M, K8, q, s_tok, stream);
+  if (K8 <= 64 * 4) return launch_swiglu_team<256, 64, 4>(gate, up, M, K8, q, s_tok, stream);
+  if (K8 <= 128 * 4) return launch_swiglu_team<256, 128, 4>(gate, up, M, K8, q, s_tok, stream);
+  if (K8 <= 256 * 3) return launch_swiglu_team<256, 256, 3>(gate, up, M, K8, q, s_tok, stream);
+  if (K8 <= 256 * 4) return launch_swiglu_team<256, 256, 4>(gate, up, M, K8, q, s_tok, stream);
+  if (K8 <= 512 * 3) return launch_swiglu_team<512, 512, 3>(gate, up, M, K8, q, s_tok, stream);
+  return launch_swiglu_team<512, 512, 4>(gate, up, M, K8, q, s_tok, stream);
 }
 
 // ---------------------------------------------------------------------------- static activation scale

@@ -84,6 +84,7 @@ class Workload:
     Ms: tuple[int, ...]
     linears: tuple[Linear, ...]
     n_outlier: int | None = None  # None -> round(0.01*K)
+    chain: bool = False           # the down projection's input is SwiGLU(gate output, up output), not its own draw
 
     def seed(self, linear_index: int) -> int:
         return 1000 * self.config + linear_index if self.config else 0
@@ -100,6 +101,12 @@ WORKLOADS = {
     # grouped calls apply): the same seven linears as c3, the token counts of c5.
     "c5l_w8a8_7b_decode_layer": Workload(7, "c5l_w8a8_7b_decode_layer", 8, (1, 4, 16, 64), LAYER_7B),
     "c5l_w4a8_7b_decode_layer": Workload(8, "c5l_w4a8_7b_decode_layer", 4, (1, 4, 16, 64), LAYER_7B),
+    # The 7B-class layer as a chain: the MLP's down projection consumes SwiGLU(gate, up) of the step's own
+    # gate/up outputs, re-quantized in the same pass (token counts of the prefill sweep).
+    "c3l_w8a8_7b_layer_chain": Workload(9, "c3l_w8a8_7b_layer_chain", 8, (128, 256, 512, 1024, 2048, 4096), LAYER_7B,
+                                        chain=True),
+    "c4l_w4a8_7b_layer_chain": Workload(10, "c4l_w4a8_7b_layer_chain", 4, (128, 256, 512, 1024, 2048, 4096), LAYER_7B,
+                                        chain=True),
 }
 
 

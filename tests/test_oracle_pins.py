@@ -585,7 +585,8 @@ def _silu64(g):
 
 
 def test_swiglu_follows_the_definition_on_every_fp16_gate():
-    """h = silu(gate) * up with silu(g) = g / (1 + e^-g): the fixed binary32 sequence stays within 2 ulp of
+    """h = silu(gate) * up with silu(g) = g / (1 + e^-g): the fixed binary32 sequence (which multiplies by the
+    rounded reciprocal of 1 + e^-g: two roundings where a quotient has one) stays within 2.5 ulp of
     the definition evaluated in binary64 for every finite FP16 gate value (up = 1), is exactly 0 at 0, equals
     g once e^-g no longer registers beside 1, and vanishes for large negative g."""
     g = np.arange(65536, dtype=np.uint16).view(np.float16)
@@ -594,7 +595,7 @@ def test_swiglu_follows_the_definition_on_every_fp16_gate():
     true = _silu64(g)
     ulp = np.spacing(np.abs(true).astype(np.float32)).astype(np.float64)
     normal = np.abs(true) > 1e-30
-    assert (np.abs(h - true)[normal] <= 2.0 * ulp[normal]).all()
+    assert (np.abs(h - true)[normal] <= 2.5 * ulp[normal]).all()
     assert (np.abs(h - true)[~normal] <= 1e-33).all()
     gf = g.astype(np.float32)
     assert (h[gf == 0] == 0).all()
