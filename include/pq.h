@@ -65,6 +65,10 @@ typedef enum {
 /* Static string for a status code. */
 PQ_API const char* pq_status_str(int status);
 
+/* Name of the CUDA error (e.g. "cudaErrorIllegalAddress") behind the most recent PQ_ERR_CUDA returned
+ * to the calling host thread; "" if there was none.  Static string; diagnostic only. */
+PQ_API const char* pq_last_cuda_error(void);
+
 /* Shape rules shared by the calls below (else PQ_ERR_SHAPE):
  *   M >= 1, N >= 8 with N % 8 == 0, K >= 16 with K % 16 == 0, K < 131072 (so that
  *   K * 128 * 128 fits INT32); W4 additionally needs group == 128 and K % 128 == 0. */

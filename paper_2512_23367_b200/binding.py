@@ -19,6 +19,7 @@ _i64, _i32, _vp = ctypes.c_int64, ctypes.c_int32, ctypes.c_void_p
 # name -> (restype, argtypes); mirrors include/pq.h
 SIGNATURES = {
     "pq_status_str": (ctypes.c_char_p, [ctypes.c_int]),
+    "pq_last_cuda_error": (ctypes.c_char_p, []),
     "pq_packed_w8_bytes": (ctypes.c_size_t, [_i64, _i64]),
     "pq_packed_w4_bytes": (ctypes.c_size_t, [_i64, _i64]),
     "pq_quantize_act": (ctypes.c_int, [_vp, _i64, _i64, _vp, _vp, _vp]),
@@ -60,6 +61,8 @@ class PQError(RuntimeError):
     def __init__(self, call: str, status: int):
         self.status = status
         msg = lib().pq_status_str(status).decode() if _lib is not None else "?"
+        if status == 5 and _lib is not None:
+            msg += ": " + lib().pq_last_cuda_error().decode()
         super().__init__(f"{call} failed: status {status} ({msg})")
 
 

@@ -109,9 +109,25 @@ int* device_status_ptr() {
 
 uint32_t wait_limit() { return g_wait_limit.load(std::memory_order_relaxed); }
 
+// Name of the CUDA error behind the calling thread's most recent PQ_ERR_CUDA ("" if none was recorded).
+static thread_local const char* g_last_cuda_error = "";
+void note_cuda_error(cudaError_t e) {
+  if (e != cudaSuccess) g_last_cuda_error = cudaGetErrorName(e);
+}
+
 int sm_count() {
   DeviceInfo* d = current_device();
   return d ? d->sms : 1;
+}
+
+// Whether one to four tokens take the CUDA-core row kernel (default yes; PQ_GEMV=0 sends them to the
+// tensor-core weight-streaming kernel instead, for ablations).
+static bool gemv_enabled() {
+  static const bool on = [] {
+    const char* e = getenv("PQ_GEMV");
+    return !(e != nullptr && e[0] == '0');
+  }();
+  return on;
 }
 
 bool pdl_enabled() {
@@ -148,6 +164,8 @@ int make_tmap_2d(CUtensorMap* out, const void* base, uint64_t rows, uint64_t col
 using namespace pq;
 
 extern "C" {
+
+const char* pq_last_cuda_error(void) { return g_last_cuda_error; }
 
 const char* pq_status_str(int status) {
   switch (status) {
@@ -336,6 +354,7 @@ static int gemm_w8a8_common(const int8_t* q, const float* s_tok, const void* wq,
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   // Up to 128 tokens: the weight-streaming schedule (tokens are the narrow MMA dimension, K split over a
   // cluster); beyond that the second CTA of a pair no longer holds only padding rows.
+  if (gemv_enabled() && gemv_rows_serves(8, M, N, K, sm_count())) return launch_gemv_rows_w8a8(q, s_tok, wq, s_ch, M, N, K, y, acc, st);
   if (M <= kSmallM_W8) return launch_smallm_w8a8(q, s_tok, wq, s_ch, M, N, K, y, acc, st);
   return launch_gemm_w8a8_pair(scratch_from(workspace, workspace_bytes), q, s_tok, wq, s_ch, M, N, K, y, acc, st);
 }
@@ -381,6 +400,7 @@ static int gemm_w4a8_common(const int8_t* q, const float* s_tok, const void* wp,
   if (!aligned16(q) || !aligned16(wp) || !aligned16(s_grp) || !aligned16(y) || !aligned16(acc_g)) return PQ_ERR_ALIGN;
   if ((rc = check_arch()) != PQ_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (gemv_enabled() && gemv_rows_serves(4, M, N, K, sm_count())) return launch_gemv_rows_w4a8(q, s_tok, wp, s_grp, M, N, K, y, acc_g, st);
   if (M <= kSmallM) return launch_smallm_w4a8(q, s_tok, wp, s_grp, M, N, K, y, acc_g, st);
   return launch_gemm_w4a8(q, s_tok, wp, s_grp, M, N, K, y, acc_g, st);
 }
@@ -481,9 +501,16 @@ int pq_device_status(int* host_status) {
   if (rc != PQ_OK) return rc;
   int* p = device_status_ptr();
   if (!p) return PQ_ERR_CUDA;
-  if (cudaDeviceSynchronize() != cudaSuccess) return PQ_ERR_CUDA;
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) {
+    note_cuda_error(e);
+    return PQ_ERR_CUDA;
+  }
   int v = 0;
-  if (cudaMemcpy(&v, p, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return PQ_ERR_CUDA;
+  if ((e = cudaMemcpy(&v, p, sizeof(int), cudaMemcpyDeviceToHost)) != cudaSuccess) {
+    note_cuda_error(e);
+    return PQ_ERR_CUDA;
+  }
   if (v != 0) {
     if (cudaMemset(p, 0, sizeof(int)) != cudaSuccess) return PQ_ERR_CUDA;
     // A call that gave up may have left arrival counters of the built-in scratch array non-zero.

@@ -127,6 +127,14 @@ int launch_smallm_w8a8(const int8_t* q, const float* s_tok, const void* wq, cons
 int launch_smallm_w4a8(const int8_t* q, const float* s_tok, const void* wp, const void* s_grp, int64_t M,
                        int64_t N, int64_t K, void* y, int32_t* acc_g, cudaStream_t stream);
 
+// One to four tokens on the CUDA cores (whole weight rows per CTA, ring filled ahead of the wait on the
+// preceding kernel); same results as the calls above.  gemv_rows_serves: whether it is the schedule of choice.
+bool gemv_rows_serves(int w_bits, int64_t M, int64_t N, int64_t K, int sms);
+int launch_gemv_rows_w8a8(const int8_t* q, const float* s_tok, const void* wq, const float* s_ch, int64_t M, int64_t N,
+                          int64_t K, void* y, int32_t* acc, cudaStream_t stream);
+int launch_gemv_rows_w4a8(const int8_t* q, const float* s_tok, const void* wp, const void* s_grp, int64_t M, int64_t N,
+                          int64_t K, void* y, int32_t* acc_g, cudaStream_t stream);
+
 // `count` (1..kMaxGroup) small-M linears over the same tokens in one launch (host arrays, as above).
 int launch_smallm_w8a8_group(const int8_t* q, const float* s_tok, int count, const void* const* wq,
                              const float* const* s_ch, const int64_t* N, void* const* y, int64_t M, int64_t K,
@@ -135,6 +143,12 @@ int launch_smallm_w4a8_group(const int8_t* q, const float* s_tok, int count, con
                              const void* const* s_grp, const int64_t* N, void* const* y, int64_t M, int64_t K,
                              int32_t* acc_g, cudaStream_t stream);
 
-inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? PQ_OK : PQ_ERR_CUDA; }
+// Remembers the name of a failed CUDA call for pq_last_cuda_error (per host thread).
+void note_cuda_error(cudaError_t e);
+inline int cuda_status(cudaError_t e) {
+  if (e == cudaSuccess) return PQ_OK;
+  note_cuda_error(e);
+  return PQ_ERR_CUDA;
+}
 
 }  // namespace pq
