@@ -53,6 +53,7 @@ def _load():
         lib.pqo_pack_w8_smooth.argtypes = [vp, vp, i64, i64, vp, vp]
         lib.pqo_pack_w4_smooth.argtypes = [vp, vp, i64, i64, i64, vp, vp]
         lib.pqo_quantize_act_static.argtypes = [vp, ctypes.c_float, i64, i64, vp, vp]
+        lib.pqo_quantize_act_static_channel.argtypes = [vp, vp, i64, i64, vp, vp]
         lib.pqo_col_absmax.argtypes = [vp, i64, i64, vp]
         lib.pqo_hadamard_block.restype = i64
         lib.pqo_hadamard_block.argtypes = [i64]
@@ -138,6 +139,18 @@ def quantize_act_static(x: np.ndarray, scale: float):
     q = np.empty((M, K), np.int8)
     s = np.empty((M,), np.float32)
     _check(_load().pqo_quantize_act_static(_p(x), float(np.float32(scale)), M, K, _p(q), _p(s)), "quantize_act_static")
+    return q, s
+
+
+def quantize_act_static_channel(x: np.ndarray, inv_s: np.ndarray):
+    """INT8 codes of x against one calibrated scale PER FEATURE CHANNEL, given as reciprocals inv_s f32 [K]:
+    (q int8 [M,K], s_tok f32 [M] = 1; the channel scales are the caller's to fold into the weights)."""
+    x = _c(x, np.float16)
+    M, K = x.shape
+    inv_s = _col(inv_s, K)
+    q = np.empty((M, K), np.int8)
+    s = np.empty((M,), np.float32)
+    _check(_load().pqo_quantize_act_static_channel(_p(x), _p(inv_s), M, K, _p(q), _p(s)), "quantize_act_static_channel")
     return q, s
 
 

@@ -367,6 +367,28 @@ int pqo_quantize_act_static(const uint16_t* x, float s, int64_t M, int64_t K, in
   return PQO_OK;
 }
 
+/*
+ * Static activation scales with one scale per feature channel (the other granularity the paper's
+ * "Preliminary" section names for calibrated scales): code = clamp(rne(X[m,k] * inv_s[k])), one
+ * binary32 product with the reciprocal of channel k's calibrated scale (given by the caller; a
+ * reciprocal that is not positive gives code 0).  A scale that depends on k cannot be taken out of
+ * the sum over k, so it is the caller's to fold into the weights (W[n,k] * s[k], as Eq. 3 does):
+ * the token scales are set to 1.
+ */
+int pqo_quantize_act_static_channel(const uint16_t* x, const float* inv_s, int64_t M, int64_t K, int8_t* q,
+                                    float* s_tok) {
+  if (M < 0 || K <= 0 || !inv_s) return PQO_ERR_ARG;
+  for (int64_t m = 0; m < M; ++m) {
+    s_tok[m] = 1.0f;
+    for (int64_t k = 0; k < K; ++k) {
+      float f = inv_s[k] > 0.0f ? inv_s[k] : 0.0f;
+      float r = nearbyintf(pqo_half_to_float(x[m * K + k]) * f);
+      q[m * K + k] = (int8_t)clampf(r, -128.0f, 127.0f);
+    }
+  }
+  return PQO_OK;
+}
+
 /* Eq. 3, activation side: quantize X S^-1.  s_inv: [K] binary32. */
 int pqo_quantize_act_smooth(const uint16_t* x, const float* s_inv, int64_t M, int64_t K, int8_t* q,
                             float* s_tok) {

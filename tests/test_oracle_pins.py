@@ -657,3 +657,32 @@ def test_swiglu_quantize_half_step_bound_against_the_definition():
     assert (err <= s.astype(np.float64)[:, None] * (0.5 + 1e-4)).all()
     assert (np.abs(q.astype(np.int32)).max(axis=1) >= 127).all()    # every row uses the full range
     assert np.array_equal(s, (np.abs(h).max(axis=1) / np.float32(127.5)).astype(np.float32))
+
+
+# ---------------------------------------------------------------------------- static scale per feature channel
+
+def test_static_channel_scales_reduce_to_the_per_tensor_rule_and_follow_closed_forms():
+    from paper_2512_23367_b200 import synth
+    x = synth.activations(6, 256, seed=33)
+    # the same power-of-two scale in every channel: exactly the per-tensor static quantizer
+    q, s_tok = oracle.quantize_act_static_channel(x, np.full((256,), 8.0, np.float32))
+    q_ref, _ = oracle.quantize_act_static(x, 0.125)
+    assert np.array_equal(q, q_ref) and (s_tok == 1.0).all()
+    # channel k has its own scale: closed forms with ties and saturation
+    xs = np.array([[0.5, 0.5, 2.5, -2.5, 100.0, -100.0, 1.0, 1.0]], np.float16)
+    inv = np.array([1.0, 3.0, 1.0, 1.0, 2.0, 2.0, 0.0, -1.0], np.float32)
+    q2, _ = oracle.quantize_act_static_channel(np.tile(xs, (1, 2)), np.tile(inv, 2))
+    assert q2[0, :8].tolist() == [0, 2, 2, -2, 127, -128, 0, 0]      # 0.5 -> 0 (tie to even), 1.5 -> 2, 2.5 -> 2, saturation, dead channels
+    # the scale really is applied per COLUMN: scaling the factor of one channel changes that channel's codes only
+    inv2 = np.full((256,), 8.0, np.float32)
+    inv2[7] = 16.0
+    q3, _ = oracle.quantize_act_static_channel(x, inv2)
+    assert np.array_equal(np.delete(q3, 7, axis=1), np.delete(q_ref, 7, axis=1)) and not np.array_equal(q3[:, 7], q_ref[:, 7])
+    # folded into the weights, the product is that of the plain operands: x ~ q / inv_s, (q) . (w * s) ~ x . w
+    w = synth.weights(8, 256, seed=34).astype(np.float64)
+    a = np.abs(x.astype(np.float32)).max(axis=0)
+    inv_s = (np.float32(127.0) / np.maximum(a, np.float32(1e-6))).astype(np.float32)
+    q4, _ = oracle.quantize_act_static_channel(x, inv_s)
+    approx = (q4.astype(np.float64) / inv_s.astype(np.float64)) @ w.T
+    exact = x.astype(np.float64) @ w.T
+    assert np.abs(approx - exact).max() <= 0.02 * np.abs(exact).max()
