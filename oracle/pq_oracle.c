@@ -39,8 +39,9 @@
  *     a channel whose activation or weight maximum is 0 gets s = 1;
  *   - the smoothed value X[m,k] * s^-1[k] (or W[n,k] * s[k]) is one binary32 product of the
  *     exact FP16 value and the factor; it is NOT rounded back to FP16;
- *   - Eq. 4 needs a Hadamard matrix of order K, which does not exist for every K of the paper's
- *     layers (11008 = 2^8 * 43): H is taken block-diagonal, H = I (x) H_B / sqrt(B), with H_B the
+ *   - Eq. 4 needs a Hadamard matrix of order K.  Where K is a power of two (up to 16384) that is the
+ *     Sylvester matrix H_K itself.  For the other widths of the paper's layers (11008 = 2^8 * 43) no
+ *     construction is at hand: H is taken block-diagonal, H = I (x) H_B / sqrt(B), with H_B the
  *     Sylvester matrix of order B = the largest power of two that divides K, at most 256.  It is
  *     applied as the textbook in-place butterfly (distances 1, 2, 4, ..., B/2 in this order, each
  *     step a' = a + b, b' = a - b in binary32), then one binary32 product with
@@ -140,6 +141,7 @@ static float smoothed(uint16_t h, const float* col, int64_t k) {
 
 /* Eq. 4: order of the Hadamard blocks for a row of length K (see the readings above). */
 int64_t pqo_hadamard_block(int64_t K) {
+  if (K >= 1 && K <= 16384 && (K & (K - 1)) == 0) return K;   /* a power of two: H of the row's own order */
   int64_t B = 1;
   while (B < 256 && K % (2 * B) == 0) B *= 2;
   return B;

@@ -466,20 +466,21 @@ def test_eq3_equivalence_and_smoothing_helps_on_outlier_channels():
 # ---------------------------------------------------------------------------- Eq. 4 (Hadamard variant)
 
 def test_hadamard_block_order():
-    assert [oracle.hadamard_block(K) for K in (16, 48, 208, 256, 2048, 4096, 6144, 11008)] == \
-        [16, 16, 16, 256, 256, 256, 256, 256]
+    # a power of two: the row's own order; otherwise the largest power of two dividing K, at most 256
+    assert [oracle.hadamard_block(K) for K in (16, 48, 208, 256, 512, 2048, 4096, 16384, 6144, 11008, 768, 32768)] == \
+        [16, 16, 16, 256, 512, 2048, 4096, 16384, 256, 256, 256, 256]
 
 
 def test_rotation_of_unit_rows_is_the_library_hadamard_matrix():
     """Row e_k times H is row k of H: compare the whole matrix with scipy's Sylvester construction."""
     from scipy.linalg import hadamard
-    for K, B in ((16, 16), (64, 64), (256, 256), (48, 16), (512, 256)):
+    for K, B in ((16, 16), (64, 64), (256, 256), (48, 16), (768, 256), (512, 512), (1024, 1024)):
         eye = np.eye(K, dtype=np.float16)
         H = oracle.rotate_rows(eye).astype(np.float64)
         want = np.kron(np.eye(K // B), hadamard(B).astype(np.float64) / np.sqrt(B))
         assert np.allclose(H, want, rtol=0, atol=1e-7)
         assert np.allclose(H @ H.T, np.eye(K), atol=1e-6)                 # orthogonal
-        if B in (16, 64, 256):                                           # 1/sqrt(B) is a power of two: exact
+        if B in (16, 64, 256, 1024):                                     # 1/sqrt(B) is a power of two: exact
             assert np.array_equal(H, want)
 
 
@@ -493,10 +494,14 @@ def test_rotation_matches_the_dense_product_and_preserves_norms():
     assert np.allclose(got, want, rtol=0, atol=2e-5 * np.abs(want).max())
     assert np.allclose(np.linalg.norm(got, axis=1), np.linalg.norm(a.astype(np.float64), axis=1), rtol=1e-6)
     # a lone spike of height A in a block becomes +-A/16 across that block (exactly), nothing elsewhere
-    spike = np.zeros((1, 512), np.float16)
+    spike = np.zeros((1, 768), np.float16)
     spike[0, 300] = 48.0
     r = oracle.rotate_rows(spike)
-    assert (np.abs(r[0, 256:]) == 3.0).all() and (r[0, :256] == 0).all()
+    assert (np.abs(r[0, 256:512]) == 3.0).all() and (r[0, :256] == 0).all() and (r[0, 512:] == 0).all()
+    # a row whose length is a power of two is rotated as a whole: the spike spreads over all of it
+    spike = np.zeros((1, 1024), np.float16)
+    spike[0, 300] = 48.0
+    assert (np.abs(oracle.rotate_rows(spike)) == 1.5).all()
 
 
 def test_hadamard_quantizers_are_the_plain_rule_on_the_rotated_values():
@@ -504,8 +509,8 @@ def test_hadamard_quantizers_are_the_plain_rule_on_the_rotated_values():
     FP16), so quantizing X H must equal the pinned plain quantizer applied to the rotated matrix."""
     from scipy.linalg import hadamard
     rng = np.random.default_rng(22)
-    K = 512
-    H = np.kron(np.eye(2), hadamard(256))
+    K = 768
+    H = np.kron(np.eye(3), hadamard(256))
     x = rng.integers(-3, 4, (6, K)).astype(np.float16) * 16                 # x H / 16 is an integer below 2048
     xr = (x.astype(np.float64) @ H / 16.0)
     assert np.array_equal(xr, np.round(xr)) and np.abs(xr).max() < 2048
@@ -686,3 +691,28 @@ def test_static_channel_scales_reduce_to_the_per_tensor_rule_and_follow_closed_f
     approx = (q4.astype(np.float64) / inv_s.astype(np.float64)) @ w.T
     exact = x.astype(np.float64) @ w.T
     assert np.abs(approx - exact).max() <= 0.02 * np.abs(exact).max()
+
+
+def test_full_order_hadamard_quantizers_are_the_plain_rule_on_the_rotated_values():
+    """K a power of two: H is the Sylvester matrix of order K.  Integer rows scaled by sqrt(K) keep the
+    rotation exact, so the quantizers of X H and W H must equal the pinned plain ones on X H_K / sqrt(K)."""
+    from scipy.linalg import hadamard
+    rng = np.random.default_rng(23)
+    K = 1024
+    H = hadamard(K).astype(np.float64)
+    x = rng.integers(-2, 3, (5, K)).astype(np.float16) * 32                 # x H / 32 is an integer below 2048
+    xr = x.astype(np.float64) @ H / 32.0
+    assert np.array_equal(xr, np.round(xr)) and np.abs(xr).max() < 2048
+    assert np.array_equal(oracle.rotate_rows(x).astype(np.float64), xr)
+    q, s = oracle.quantize_act_hadamard(x)
+    q2, s2 = oracle.quantize_act(xr.astype(np.float16))
+    assert np.array_equal(q, q2) and np.array_equal(s, s2)
+    w = rng.integers(-2, 3, (6, K)).astype(np.float16) * 32
+    wr = (w.astype(np.float64) @ H / 32.0).astype(np.float16)
+    for got, want in ((oracle.pack_w8_hadamard(w), oracle.pack_w8(wr)),
+                      (oracle.pack_w4_hadamard(w, 128), oracle.pack_w4(wr, 128))):
+        assert np.array_equal(got[0], want[0])
+        assert np.array_equal(got[1].view(np.uint8), want[1].view(np.uint8))
+    # (X H)(W H)^T = X W^T with the full matrix too
+    xf, wf = oracle.rotate_rows(x).astype(np.float64), oracle.rotate_rows(w).astype(np.float64)
+    assert np.allclose(xf @ wf.T, x.astype(np.float64) @ w.astype(np.float64).T, rtol=1e-9)
