@@ -144,6 +144,18 @@ PQ_API int pq_quantize_act_static(const void* x_f16, const float* scale, int64_t
                                   float* s_tok, void* stream);
 
 /*
+ * The same with one calibrated scale per feature channel (the per-channel granularity the paper's
+ * "Preliminary" section names), given as reciprocals:
+ *   code = clamp(rne(X[m,k] * inv_s[k]), -128, 127)   (one FP32 product; inv_s[k] <= 0 gives code 0),
+ *   s_tok[m] = 1: a scale that depends on k cannot be taken out of the sum over k, so the caller folds
+ *   s[k] = 1 / inv_s[k] into the weights (pq_pack_w8_smooth / pq_pack_w4_smooth with that vector, as for
+ *   Eq. 3) and uses the GEMM calls unchanged.
+ * inv_s: [K] FP32 device vector, 16-byte aligned.
+ */
+PQ_API int pq_quantize_act_static_channel(const void* x_f16, const float* inv_s, int64_t M, int64_t K, int8_t* q,
+                                          float* s_tok, void* stream);
+
+/*
  * The MLP's gated activation fused with the down projection's activation quantizer.  The paper
  * quantizes all linear layers of a decoder and reports whole prefill passes (its latency table), but
  * does not define the activation between the gate/up linears and the down linear; the gated form
@@ -163,10 +175,11 @@ PQ_API int pq_swiglu_quantize(const void* gate_f16, const void* up_f16, int64_t 
 
 /*
  * Hadamard variant (Eq. 4: Y = (X H)(H^T W), H a normalized Hadamard matrix).  With W stored [N,K]
- * both operands are rotated along K: (X H)(W H)^T = X W^T.  A Hadamard matrix of order K does not
- * exist for every layer width (11008 = 2^8 * 43), so H = I (x) H_B / sqrt(B) is block diagonal, H_B
- * the Sylvester matrix of order B = pq_hadamard_block(K) = the largest power of two dividing K, at
- * most 256.  The rotation is the in-place butterfly (distances 1, 2, ..., B/2 in this order) in FP32
+ * both operands are rotated along K: (X H)(W H)^T = X W^T.  Where K is a power of two (up to 16384) H
+ * is the Sylvester matrix of order K itself.  For other layer widths (11008 = 2^8 * 43) no construction
+ * is at hand, and H = I (x) H_B / sqrt(B) is block diagonal, H_B the Sylvester matrix of order
+ * B = the largest power of two dividing K, at most 256.  pq_hadamard_block(K) returns the order used
+ * (K or B).  The rotation is the in-place butterfly (distances 1, 2, ..., B/2 in this order) in FP32
  * on the exact FP16 inputs, times 1/sqrt(B); the rotated values are quantized from FP32.
  *   pq_quantize_act_hadamard: pq_quantize_act of X H (on line, fused into the quantizer kernel);
  *   pq_pack_w8_hadamard / pq_pack_w4_hadamard: pq_pack_w8 / pq_pack_w4 of W H (off line).

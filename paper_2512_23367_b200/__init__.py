@@ -29,6 +29,7 @@ from .binding import (  # noqa: F401
     pq_quantize_act_hadamard,
     pq_quantize_act_smooth,
     pq_quantize_act_static,
+    pq_quantize_act_static_channel,
     pq_set_wait_limit,
     pq_smooth_scales,
     pq_swiglu_quantize,

@@ -42,6 +42,7 @@ SIGNATURES = {
                                           ctypes.c_size_t, _vp]),
     "pq_quantize_act_static": (ctypes.c_int, [_vp, _vp, _i64, _i64, _vp, _vp, _vp]),
     "pq_swiglu_quantize": (ctypes.c_int, [_vp, _vp, _i64, _i64, _vp, _vp, _vp]),
+    "pq_quantize_act_static_channel": (ctypes.c_int, [_vp, _vp, _i64, _i64, _vp, _vp, _vp]),
     "pq_hadamard_block": (_i32, [_i64]),
     "pq_quantize_act_hadamard": (ctypes.c_int, [_vp, _i64, _i64, _vp, _vp, _vp]),
     "pq_pack_w8_hadamard": (ctypes.c_int, [_vp, _i64, _i64, _vp, _vp, _vp]),
@@ -195,6 +196,18 @@ def pq_quantize_act_static(x: torch.Tensor, scale: torch.Tensor, q: torch.Tensor
     _together(x, scale)
     _check("pq_quantize_act_static", lib().pq_quantize_act_static(x.data_ptr(), scale.data_ptr(), M, K, q.data_ptr(),
                                                                   s_tok.data_ptr(), _stream()))
+    return q, s_tok
+
+
+def pq_quantize_act_static_channel(x: torch.Tensor, inv_s: torch.Tensor, q: torch.Tensor | None = None,
+                                   s_tok: torch.Tensor | None = None):
+    """INT8 codes against one calibrated scale per feature channel: x f16 [M,K], inv_s f32 [K] (reciprocal
+    scales) -> (q int8 [M,K], s_tok f32 [M] = 1; fold the channel scales into the weights)."""
+    M, K, q, s_tok = _rows(x, q, s_tok)
+    inv_s = _factors(inv_s, K, "inv_s")
+    _together(x, inv_s)
+    _check("pq_quantize_act_static_channel", lib().pq_quantize_act_static_channel(x.data_ptr(), inv_s.data_ptr(), M, K,
+                                                                                  q.data_ptr(), s_tok.data_ptr(), _stream()))
     return q, s_tok
 
 

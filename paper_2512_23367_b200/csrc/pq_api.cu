@@ -261,6 +261,16 @@ int pq_quantize_act_static(const void* x_f16, const float* scale, int64_t M, int
   return launch_quantize_act_static(x_f16, scale, M, K, q, s_tok, static_cast<cudaStream_t>(stream));
 }
 
+int pq_quantize_act_static_channel(const void* x_f16, const float* inv_s, int64_t M, int64_t K, int8_t* q, float* s_tok,
+                                   void* stream) {
+  if (!x_f16 || !inv_s || !q || !s_tok) return PQ_ERR_NULL;
+  int rc = check_rows(M, K);
+  if (rc != PQ_OK) return rc;
+  if (!aligned16(x_f16) || !aligned16(q) || !aligned16(inv_s)) return PQ_ERR_ALIGN;
+  if ((rc = check_arch()) != PQ_OK) return rc;
+  return launch_quantize_act_static_channel(x_f16, inv_s, M, K, q, s_tok, static_cast<cudaStream_t>(stream));
+}
+
 int pq_swiglu_quantize(const void* gate_f16, const void* up_f16, int64_t M, int64_t I, int8_t* q, float* s_tok,
                        void* stream) {
   if (!gate_f16 || !up_f16 || !q || !s_tok) return PQ_ERR_NULL;

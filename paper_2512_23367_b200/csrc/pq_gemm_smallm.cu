@@ -19,6 +19,8 @@
 //               cross-CTA reduction, dequantization, FP16 store
 #include <cuda_fp16.h>
 
+#include <cstdlib>
+
 #include "pq_internal.h"
 #include "pq_ptx.cuh"
 
@@ -549,6 +551,9 @@ int launch_smallm(const int8_t* q, const float* s_tok, int count, const void* co
   const int ctas_per_sm = mpad >= 64 ? 2 : (kW4 ? 2 : 4);
   while (splits > 1 && n_tiles * splits * 10 > static_cast<int64_t>(ctas_per_sm) * sm_count() * 9) --splits;
   if (splits == 5 || splits == 7) --splits;
+  // ablation knob, read once: force the number of K parts (cluster size)
+  static const int force_splits = [] { const char* e = getenv("PQ_SMALLM_SPLITS"); return e ? atoi(e) : 0; }();
+  if (force_splits >= 1 && force_splits <= kMaxSplit) splits = force_splits;
   if (splits > k_blocks) splits = k_blocks;
 
   a.count = count;

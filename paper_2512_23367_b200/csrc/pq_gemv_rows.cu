@@ -44,8 +44,9 @@ namespace {
 
 constexpr int kConsumerWarps = 8;
 constexpr int kThreads = 32 * kConsumerWarps;
-constexpr int kMaxSlots = 16;
+constexpr int kMaxSlots = 32;
 constexpr int kCtaBytesMax = 112 * 1024;   // ring + token codes: a CTA stays below half an SM's shared memory
+constexpr int kSoloBytesMax = 216 * 1024;  // ... or takes the SM alone, when that lets the ring hold its whole share
 constexpr int kCodeBytesMax = 44 * 1024;
 constexpr int kFillBatch = 12;             // 16-byte chunks of codes a thread has in flight at once
 
@@ -409,7 +410,7 @@ template <bool kW4, int MT, int RQ, bool kExportAcc>
 int launch_rows_cfg(const RowArgs& a, int smem_bytes, int grid, cudaStream_t stream) {
   auto kern = gemv_rows_kernel<kW4, MT, RQ, kExportAcc>;
   static PerDeviceOnce once;
-  if (const int rc = set_dynamic_smem_once(once, kern, kCtaBytesMax + 1024); rc != PQ_OK) return rc;
+  if (const int rc = set_dynamic_smem_once(once, kern, kSoloBytesMax + 1024); rc != PQ_OK) return rc;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(static_cast<unsigned>(grid), 1, 1);
   cfg.blockDim = dim3(kThreads, 1, 1);
@@ -435,16 +436,32 @@ struct RowPlan {
   int rq, slots, grid, mt, code_bytes, smem_bytes;
   bool fits;
 };
+bool plan_rows_within(int cta_bytes_max, int w_bits, int64_t M, int64_t N, int64_t K, int sms, RowPlan* out);
+
+// Two CTAs of consecutive launches per SM where a CTA's whole share fits half an SM.  Otherwise, for one
+// token and a share of a few large row sets, one CTA per SM with a ring of up to 216 KB if THAT holds the
+// whole share (the next launch's CTAs then start when this one's leave, and their loads run under the dead
+// time between the launches: 11008 -> 4096 W4, 10.2 -> 8.1 us; with many small sets the half-SM ring with
+// refills is the better one: 4096 -> 11008 W4, 8.5 against 9.2 us).  Else the half-SM ring with refills.
 bool plan_rows(int w_bits, int64_t M, int64_t N, int64_t K, int sms, RowPlan* out) {
+  RowPlan half, solo;
+  if (!plan_rows_within(kCtaBytesMax, w_bits, M, N, K, sms, &half)) return false;
+  if (!half.fits && M == 1 && plan_rows_within(kSoloBytesMax, w_bits, M, N, K, sms, &solo) && solo.fits && solo.slots <= 8)
+    half = solo;
+  *out = half;
+  return true;
+}
+
+bool plan_rows_within(int cta_bytes_max, int w_bits, int64_t M, int64_t N, int64_t K, int sms, RowPlan* out) {
   if (M < 1 || M > 4 || N < 4 || N % 4 != 0 || sms < 1) return false;
   const int64_t row_bytes = w_bits == 4 ? K / 2 : K;
-  if (row_bytes % 16 != 0 || row_bytes > kCtaBytesMax) return false;
+  if (row_bytes % 16 != 0 || row_bytes > cta_bytes_max) return false;
   RowPlan pl;
   pl.mt = M <= 1 ? 1 : (M <= 2 ? 2 : 4);
   const int64_t code_bytes = pl.mt * ((K + 127) / 128) * 128;
   if (code_bytes > kCodeBytesMax) return false;
   pl.code_bytes = static_cast<int>(code_bytes);
-  const int ring_max = kCtaBytesMax - pl.code_bytes;
+  const int ring_max = cta_bytes_max - pl.code_bytes;
   if (2 * 2 * row_bytes > ring_max) return false;                            // at least two slots of two rows
   // Row sets of four rows where three of them fit the ring, else of two.
   pl.rq = (3 * 4 * row_bytes <= ring_max) ? 4 : 2;
@@ -496,15 +513,17 @@ int launch_rows(const int8_t* q, const float* s_tok, const void* w, const float*
 
 }  // namespace
 
-// Whether the row kernel is the schedule for this shape.  It wins where a CTA's whole share of the weights
-// fits its ring (everything is in flight before the call may look at its tokens) and, for W4 with one or
-// two tokens, always (measured against the tensor-core weight-streaming kernel on the 7B-class shapes: W4,
-// one token, 4.3 / 8.5 / 10.2 us against 7.6 / 11.5 / 12.0 us; with a share that does not fit, W8 and the
-// four-token cases lose: the refills and the dp4a work land on the critical path behind the wait).
+// Whether the row kernel is the schedule for this shape: where a CTA's whole share of the weights fits its
+// ring (everything is in flight before the call may look at its tokens), and for W4 with one token always.
+// Measured against the tensor-core weight-streaming kernel on the 7B-class shapes (4096^2, 4096 -> 11008,
+// 11008 -> 4096), one token: W4 4.4 / 8.5 / 8.1 us against 7.5 / 11.5 / 11.9 us, W8 (4096^2) 5.7 against
+// 6.2 us; W4 with four tokens at 4096^2 6.5 against 7.8 us.  With a share that does not fit, W8 and the
+// multi-token cases lose (the refills and the dp4a work land on the critical path behind the wait) and stay
+// on the tensor cores.
 bool gemv_rows_serves(int w_bits, int64_t M, int64_t N, int64_t K, int sms) {
   RowPlan pl;
   if (!plan_rows(w_bits, M, N, K, sms, &pl)) return false;
-  return pl.fits || (w_bits == 4 && M <= 2);
+  return pl.fits || (w_bits == 4 && M == 1);
 }
 
 int launch_gemv_rows_w8a8(const int8_t* q, const float* s_tok, const void* wq, const float* s_ch, int64_t M, int64_t N,

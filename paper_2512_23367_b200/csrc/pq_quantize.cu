@@ -12,8 +12,10 @@
 
 namespace pq {
 
-// Order of the Hadamard blocks for rows of length K (Eq. 4): the largest power of two dividing K, at most 256.
+// Order of the Hadamard blocks for rows of length K (Eq. 4): K itself where K is a power of two (up to
+// 16384: the Sylvester matrix of the row's own order), else the largest power of two dividing K, at most 256.
 int hadamard_block_order(int64_t K) {
+  if (K >= 1 && K <= 16384 && (K & (K - 1)) == 0) return static_cast<int>(K);
   int B = 1;
   while (B < 256 && K % (2 * B) == 0) B *= 2;
   return B;
@@ -186,7 +188,7 @@ __device__ __forceinline__ void hadamard_chunk(float (&v)[8], int lane, int chun
 // the block = j + 8 l' + 64 (i mod 4): distances 1-4 stay inside a chunk, 8-32 are lane exchanges at XOR
 // distance 1-4, 64 and 128 pair chunks of the same thread -- three exchanges per element instead of five.
 template <int C>
-__device__ __forceinline__ void hadamard_rows(float (&v)[C][8], int lane, int chunks_per_block, float norm) {
+__device__ __forceinline__ void hadamard_rows(float (&v)[C][8], int lane, int chunks_per_block, float norm, float* xch) {
 #pragma unroll
   for (int i = 0; i < C; ++i) {
 #pragma unroll
@@ -216,7 +218,7 @@ __device__ __forceinline__ void hadamard_rows(float (&v)[C][8], int lane, int ch
     }
   }
 #pragma unroll
-  for (int di = 1; di < 4; di <<= 1) {
+  for (int di = 1; di < C; di <<= 1) {
     if (8 * di < chunks_per_block) {
 #pragma unroll
       for (int i = 0; i < C; ++i) {
@@ -228,6 +230,43 @@ __device__ __forceinline__ void hadamard_rows(float (&v)[C][8], int lane, int ch
             v[i + di][j] = __fsub_rn(a, b);
           }
         }
+      }
+    }
+  }
+  // Blocks longer than 8 C chunks (only rows rotated as a whole): the four 8-lane groups of the warp hold
+  // consecutive runs of 8 C chunks -- two more lane exchanges, at chunk distances 8 C and 16 C.
+#pragma unroll
+  for (int dl = 8; dl < 32; dl <<= 1) {
+    if (dl * C < chunks_per_block) {
+      const float sign = (lane & dl) != 0 ? -1.0f : 1.0f;
+#pragma unroll
+      for (int i = 0; i < C; ++i) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const float other = __shfl_xor_sync(0xffffffffu, v[i][j], dl);
+          v[i][j] = __fmaf_rn(sign, v[i][j], other);
+        }
+      }
+    }
+  }
+  // ... and the warps of the row team hold consecutive runs of 32 C chunks: one exchange through shared
+  // memory per remaining level (chunk distances 32 C, 64 C, ...), `xch` = this block's exchange buffer
+  // (8 C floats per thread, or null when no level needs it).  Every thread of the block takes part.
+  if (xch != nullptr) {
+    for (int dw = 1; dw * 32 * C < chunks_per_block; dw <<= 1) {
+      __syncthreads();                      // the previous level's reads are done
+#pragma unroll
+      for (int i = 0; i < C; ++i) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) xch[(i * 8 + j) * kThreads + threadIdx.x] = v[i][j];
+      }
+      __syncthreads();
+      const int partner = static_cast<int>(threadIdx.x) ^ (32 * dw);
+      const float sign = (threadIdx.x & (32 * dw)) != 0 ? -1.0f : 1.0f;
+#pragma unroll
+      for (int i = 0; i < C; ++i) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) v[i][j] = __fmaf_rn(sign, v[i][j], xch[(i * 8 + j) * kThreads + partner]);
       }
     }
   }
@@ -286,7 +325,11 @@ __global__ void __launch_bounds__(kThreads) quantize_rows_rot_kernel(const uint4
       }
     }
   }
-  if constexpr (kRotate) hadamard_rows<C>(v, lane, chunks_per_block, norm);   // all lanes take part in the exchanges
+  if constexpr (kRotate) {
+    // all lanes (and, for rows rotated as a whole by more than one warp, all threads) take part in the exchanges
+    extern __shared__ float xch_raw[];
+    hadamard_rows<C>(v, lane, chunks_per_block, norm, chunks_per_block > 32 * C ? xch_raw : nullptr);
+  }
 #pragma unroll
   for (int i = 0; i < C; ++i) {
 #pragma unroll
@@ -327,18 +370,24 @@ template <int T, int C, bool kDivide, bool kRotate>
 int launch_rows_rot_team(const uint4* xp, int64_t M, int K8, uint2* qp, float* s, int chunks_per_block, float norm,
                          const float4* col, cudaStream_t stream) {
   constexpr int kRowsPerBlock = kThreads / T;
+  auto kern = quantize_rows_rot_kernel<T, C, kDivide, kRotate>;
+  // rows rotated as a whole by more than one warp exchange through shared memory: 8 C floats per thread
+  const int xch_bytes = (kRotate && chunks_per_block > 32 * C) ? kThreads * C * 8 * static_cast<int>(sizeof(float)) : 0;
+  if (xch_bytes > 48 * 1024) {
+    static PerDeviceOnce once;
+    if (const int rc = set_dynamic_smem_once(once, kern, xch_bytes); rc != PQ_OK) return rc;
+  }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(static_cast<unsigned>((M + kRowsPerBlock - 1) / kRowsPerBlock), 1, 1);
   cfg.blockDim = dim3(kThreads, 1, 1);
-  cfg.dynamicSmemBytes = 0;
+  cfg.dynamicSmemBytes = static_cast<size_t>(xch_bytes);
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = (!kDivide && pdl_enabled()) ? 1 : 0;
-  return cuda_status(cudaLaunchKernelEx(&cfg, quantize_rows_rot_kernel<T, C, kDivide, kRotate>, xp, M, K8, qp, s,
-                                        chunks_per_block, norm, col));
+  return cuda_status(cudaLaunchKernelEx(&cfg, kern, xp, M, K8, qp, s, chunks_per_block, norm, col));
 }
 
 // col == nullptr: Eq. 4 rotation; otherwise Eq. 3 column factors.
@@ -381,10 +430,15 @@ int launch_rows(const void* x, int64_t M, int64_t K, int8_t* q, float* s, const 
   const uint4* xp = static_cast<const uint4*>(x);
   uint2* qp = reinterpret_cast<uint2*>(q);
   const float4* cp = reinterpret_cast<const float4*>(col);
-  // Pick the narrowest row team that still keeps the whole row in registers.
-  if (K8 <= 32 * kCached) return launch_rows_team<32, kDivide, kSmooth>(xp, M, K8, qp, s, cp, stream);
-  if (K8 <= 64 * kCached) return launch_rows_team<64, kDivide, kSmooth>(xp, M, K8, qp, s, cp, stream);
-  if (K8 <= 128 * kCached) return launch_rows_team<128, kDivide, kSmooth>(xp, M, K8, qp, s, cp, stream);
+  // The narrowest row team that still keeps the whole row in registers -- widened while the launch would
+  // leave the SMs short of warps (few or short rows: the kernel is then bound by the latency of its loads,
+  // and more threads per row means more loads in flight), as long as every thread still has a chunk.
+  int T = K8 <= 32 * kCached ? 32 : (K8 <= 64 * kCached ? 64 : (K8 <= 128 * kCached ? 128 : 256));
+  const int64_t want_threads = static_cast<int64_t>(sm_count()) * 1536;
+  while (T < 256 && M * T < want_threads && 2 * T <= K8) T *= 2;
+  if (T == 32) return launch_rows_team<32, kDivide, kSmooth>(xp, M, K8, qp, s, cp, stream);
+  if (T == 64) return launch_rows_team<64, kDivide, kSmooth>(xp, M, K8, qp, s, cp, stream);
+  if (T == 128) return launch_rows_team<128, kDivide, kSmooth>(xp, M, K8, qp, s, cp, stream);
   return launch_rows_team<256, kDivide, kSmooth>(xp, M, K8, qp, s, cp, stream);
 }
 
@@ -512,6 +566,52 @@ __global__ void __launch_bounds__(kThreads) pack_w4_rot_kernel(const __half* __r
   (void)G;
 }
 
+// Group-wise INT4 packing of W H for rows rotated as a whole (K a power of two above 256).  One block per
+// output channel: the row is rotated in shared memory in FP32 by the in-place butterfly (distances 1, 2, ...,
+// K/2 in this order, each step one rounded sum and one rounded difference), scaled by 1/sqrt(K), and warp w
+// quantizes the groups w, w + 8, ... exactly as pack_w4_kernel does.
+__global__ void __launch_bounds__(kThreads) pack_w4_rotfull_kernel(const __half* __restrict__ w, int64_t N, int K,
+                                                                   uint8_t* __restrict__ wp,
+                                                                   __half* __restrict__ s_grp, float norm) {
+  extern __shared__ float rot_row[];
+  const int64_t n = blockIdx.x;
+  const int tid = threadIdx.x;
+  for (int k = tid; k < K; k += kThreads) rot_row[k] = __half2float(w[n * K + k]);
+  __syncthreads();
+  for (int h = 1; h < K; h <<= 1) {
+    for (int p = tid; p < K / 2; p += kThreads) {
+      const int idx = (p / h) * 2 * h + (p % h);
+      const float a = rot_row[idx], b = rot_row[idx + h];
+      rot_row[idx] = __fadd_rn(a, b);
+      rot_row[idx + h] = __fsub_rn(a, b);
+    }
+    __syncthreads();
+  }
+  for (int k = tid; k < K; k += kThreads) rot_row[k] = __fmul_rn(rot_row[k], norm);
+  __syncthreads();
+  const int lane = tid & 31;
+  for (int g = tid >> 5; g < K / 128; g += kThreads / 32) {
+    const int k0 = g * 128 + (lane >> 3) * 32;
+    const int b = (lane & 7) * 2;
+    const float v0 = rot_row[k0 + b], v1 = rot_row[k0 + b + 1], v2 = rot_row[k0 + 16 + b], v3 = rot_row[k0 + 16 + b + 1];
+    float a = fmaxf(fmaxf(fabsf(v0), fabsf(v1)), fmaxf(fabsf(v2), fabsf(v3)));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
+    const __half s16 = __float2half_rn(__fdiv_rn(a, 7.5f));
+    const float sf = __half2float(s16);
+    if (lane == 0) s_grp[static_cast<int64_t>(g) * N + n] = s16;
+    auto code4 = [sf](float x) -> uint32_t {
+      if (sf == 0.0f) return 0u;
+      const int r = __float2int_rn(__fdiv_rn(x, sf));
+      return static_cast<uint32_t>(max(-8, min(7, r))) & 0xfu;
+    };
+    const uint32_t byte0 = code4(v0) | (code4(v2) << 4);
+    const uint32_t byte1 = code4(v1) | (code4(v3) << 4);
+    uint8_t* out = wp + n * (K / 2) + k0 / 2 + b;
+    *reinterpret_cast<uint16_t*>(out) = static_cast<uint16_t>(byte0 | (byte1 << 8));
+  }
+}
+
 // Launched (plainly, stream-ordered) behind the offline weight kernels.  A GEMM that follows in
 // the stream may request weight tiles before its own wait on its predecessor; with this kernel
 // in between, that predecessor starts only after the packed weights are complete and visible.
@@ -557,6 +657,17 @@ int launch_quantize_act_hadamard(const void* x, int64_t M, int64_t K, int8_t* q,
 int launch_pack_w4_hadamard(const void* w, int64_t N, int64_t K, void* wp, void* s_grp, cudaStream_t stream) {
   const int B = hadamard_block_order(K);
   const float norm = 1.0f / sqrtf(static_cast<float>(B));
+  if (B > 256) {
+    // the row is rotated as a whole
+    const int smem = static_cast<int>(K) * static_cast<int>(sizeof(float));
+    if (smem > 48 * 1024) {
+      static PerDeviceOnce once;
+      if (const int rc = set_dynamic_smem_once(once, pack_w4_rotfull_kernel, smem > 64 * 1024 ? smem : 64 * 1024); rc != PQ_OK) return rc;
+    }
+    pack_w4_rotfull_kernel<<<static_cast<unsigned>(N), kThreads, smem, stream>>>(
+        static_cast<const __half*>(w), N, static_cast<int>(K), static_cast<uint8_t*>(wp), static_cast<__half*>(s_grp), norm);
+    return cuda_status(cudaGetLastError());
+  }
   const int64_t warps = N * ((K + 255) / 256);
   const unsigned blocks = static_cast<unsigned>((warps + kThreads / 32 - 1) / (kThreads / 32));
   pack_w4_rot_kernel<<<blocks, kThreads, 0, stream>>>(static_cast<const __half*>(w), N, static_cast<int>(K),
@@ -723,7 +834,54 @@ __global__ void __launch_bounds__(kThreads) quantize_static_kernel(const uint4* 
   }
 }
 
+// The same with one calibrated scale per feature channel, given as reciprocals inv_s[k]: one product per
+// element; a reciprocal that is not positive gives code 0.  Token scales are 1 (the channel scales belong
+// into the weights).
+__global__ void __launch_bounds__(kThreads) quantize_static_channel_kernel(const uint4* __restrict__ x, int64_t M, int K8,
+                                                                           uint2* __restrict__ q,
+                                                                           float* __restrict__ s_tok,
+                                                                           const float4* __restrict__ inv_s) {
+  grid_dep_launch();
+  grid_dep_wait();
+  const int64_t total = M * K8;
+  for (int64_t i = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x; i < total;
+       i += static_cast<int64_t>(gridDim.x) * kThreads) {
+    const int c = static_cast<int>(i % K8);
+    float4 f0 = __ldg(inv_s + 2 * c), f1 = __ldg(inv_s + 2 * c + 1);
+    f0.x = fmaxf(f0.x, 0.0f); f0.y = fmaxf(f0.y, 0.0f); f0.z = fmaxf(f0.z, 0.0f); f0.w = fmaxf(f0.w, 0.0f);
+    f1.x = fmaxf(f1.x, 0.0f); f1.y = fmaxf(f1.y, 0.0f); f1.z = fmaxf(f1.z, 0.0f); f1.w = fmaxf(f1.w, 0.0f);
+    const uint4 v = __ldg(x + i);
+    const __half* h = reinterpret_cast<const __half*>(&v);
+    q[i] = make_uint2(
+        codes4<false>(__fmul_rn(__half2float(h[0]), f0.x), __fmul_rn(__half2float(h[1]), f0.y),
+                      __fmul_rn(__half2float(h[2]), f0.z), __fmul_rn(__half2float(h[3]), f0.w), 1.0f),
+        codes4<false>(__fmul_rn(__half2float(h[4]), f1.x), __fmul_rn(__half2float(h[5]), f1.y),
+                      __fmul_rn(__half2float(h[6]), f1.z), __fmul_rn(__half2float(h[7]), f1.w), 1.0f));
+    if (c == 0) s_tok[i / K8] = 1.0f;
+  }
+}
+
 }  // namespace
+
+int launch_quantize_act_static_channel(const void* x, const float* inv_s, int64_t M, int64_t K, int8_t* q, float* s_tok,
+                                       cudaStream_t stream) {
+  const int K8 = static_cast<int>(K / 8);
+  const int64_t total = M * K8;
+  int64_t blocks = (total + kThreads - 1) / kThreads;
+  const int64_t cap = static_cast<int64_t>(sm_count()) * 16;
+  if (blocks > cap) blocks = cap;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(blocks), 1, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl_enabled() ? 1 : 0;
+  return cuda_status(cudaLaunchKernelEx(&cfg, quantize_static_channel_kernel, static_cast<const uint4*>(x), M, K8,
+                                        reinterpret_cast<uint2*>(q), s_tok, reinterpret_cast<const float4*>(inv_s)));
+}
 
 int launch_quantize_act_static(const void* x, const float* s_ptr, int64_t M, int64_t K, int8_t* q, float* s_tok,
                                cudaStream_t stream) {

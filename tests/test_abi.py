@@ -61,7 +61,7 @@ def test_argument_errors_come_back_as_status_codes_without_a_device():
     assert L.pq_smooth_scales(16, 16, 0, 16, 16, None) == PQ_ERR_SHAPE
     assert L.pq_quantize_act_hadamard(16, 4, 16400, 16, 16, None) == PQ_ERR_SHAPE   # row does not fit the registers
     assert L.pq_pack_w4_hadamard(16, 16, 192, 128, 16, 16, None) == PQ_ERR_SHAPE     # K % 128
-    assert [L.pq_hadamard_block(K) for K in (16, 48, 208, 2048, 4096, 11008, 20)] == [16, 16, 16, 256, 256, 256, 0]
+    assert [L.pq_hadamard_block(K) for K in (16, 48, 208, 2048, 4096, 11008, 20)] == [16, 16, 16, 2048, 4096, 256, 0]
     assert L.pq_quantize_act_static(16, None, 4, 64, 16, 16, None) == PQ_ERR_NULL
     assert L.pq_quantize_act_static(16, 16, 4, 60, 16, 16, None) == PQ_ERR_SHAPE
     assert L.pq_packed_w8_bytes(8, 256) == 2048 and L.pq_packed_w4_bytes(8, 256) == 1024

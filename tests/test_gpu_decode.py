@@ -59,8 +59,8 @@ def run_w4(M, N, K, seed):
 
 SMALL = [(1, 256, 256), (4, 136, 384), (16, 520, 1024), (17, 128, 128), (33, 264, 2048), (64, 1024, 1152),
          (3, 8, 128), (48, 4096, 256),
-         # M <= 4 takes the register-streaming CUDA-core kernels: rows not a multiple of the grid,
-         # rows longer and shorter than one ring pass, every token count
+         # one to four tokens may take the CUDA-core row kernel: row sets not a multiple of the grid, shares
+         # that fit the ring and shares that need refills, K with a short last 128-block, every token count
          (2, 1000, 640), (3, 2376, 4224), (4, 152, 11008), (1, 4744, 128), (2, 8, 8192)]
 
 

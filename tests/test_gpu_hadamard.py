@@ -22,10 +22,11 @@ def _np(t):
     return t.cpu().numpy()
 
 
-# block orders 16 / 32 / 64 / 128 / 256; row teams of 32 / 64 / 128 / 256 threads; ragged last row blocks;
-# the benchmark widths 2048, 4096, 6144, 11008
+# block orders 16 / 32 / 64 / 128 / 256 and whole rows of 512 ... 16384 (K a power of two); row teams of
+# 32 / 64 / 128 / 256 threads; ragged last row blocks; the benchmark widths 2048, 4096, 6144, 11008
 @pytest.mark.parametrize("M,K", [(1, 16), (3, 48), (5, 96), (7, 192), (9, 384), (16, 256), (33, 2048), (130, 4096),
-                                 (20, 6144), (70, 11008), (4, 16384)])
+                                 (20, 6144), (70, 11008), (4, 16384), (6, 512), (11, 1024), (3, 8192), (5, 768),
+                                 (2, 12288), (300, 128), (9, 64), (5, 32)])
 def test_quantize_act_hadamard_bit_exact(M, K):
     assert pq.pq_hadamard_block(K) == oracle.hadamard_block(K)
     x = synth.activations(M, K, 7000 + M)
@@ -36,16 +37,17 @@ def test_quantize_act_hadamard_bit_exact(M, K):
 
 
 def test_spike_and_zero_rows():
-    x = np.zeros((3, 512), np.float16)
+    x = np.zeros((3, 768), np.float16)
     x[0, 300] = 48.0                      # -> +-3 over the second block of 256, token scale 3 / 127.5
     q, s_tok = pq.pq_quantize_act_hadamard(_t(x))
     q, s_tok = _np(q), _np(s_tok)
-    assert (q[0, :256] == 0).all() and (np.abs(q[0, 256:].astype(np.int16)) >= 127).all()
+    assert (q[0, :256] == 0).all() and (q[0, 512:] == 0).all() and (np.abs(q[0, 256:512].astype(np.int16)) >= 127).all()
     assert s_tok[0] == np.float32(3.0) / np.float32(127.5)
     assert (q[1:] == 0).all() and (s_tok[1:] == 0).all()
 
 
-@pytest.mark.parametrize("N,K", [(8, 128), (24, 384), (264, 640), (96, 4096), (16, 11008)])
+@pytest.mark.parametrize("N,K", [(8, 128), (24, 384), (264, 640), (96, 4096), (16, 11008), (40, 512), (24, 2048), (8, 16384),
+                                 (16, 256), (16, 768)])
 def test_weight_packers_of_WH_bit_exact(N, K):
     w = synth.weights(N, K, 7100 + N)
     wq, s_ch = pq.pq_pack_w8_hadamard(_t(w))
