@@ -184,3 +184,46 @@ def test_two_streams_with_their_own_workspaces_run_split_k_concurrently():
     for (_, _, _, _, _, serial), ys in zip(cases, outs):
         for y in ys:
             assert torch.equal(y, serial)
+
+
+def test_host_threads_call_concurrently_on_their_own_streams():
+    """The library keeps no per-call host state: four host threads, each with its own stream, inputs and
+    workspace, issue split-K and unsplit GEMMs at the same time (ctypes drops the GIL inside the calls); every
+    result equals the one computed serially."""
+    import threading
+    shapes = [(512, 11008, 1024), (300, 1024, 520), (512, 11008, 1024), (140, 6144, 136)]
+    cases = []
+    for i, (M, K, N) in enumerate(shapes):
+        x, w = synth.activations(M, K, seed=500 + i), synth.weights(N, K, seed=510 + i)
+        q, s_tok = pq.pq_quantize_act(torch.from_numpy(x).to(DEV))
+        wq, s_ch = pq.pq_pack_w8(torch.from_numpy(w).to(DEV))
+        need = pq.pq_workspace_bytes(M, N, K)
+        ws = pq.pq_workspace_init(torch.empty((need,), dtype=torch.uint8, device=DEV)) if need else None
+        serial = pq.pq_gemm_w8a8(q, s_tok, wq, s_ch, N)
+        cases.append((q, s_tok, wq, s_ch, N, ws, serial))
+    torch.cuda.synchronize()
+    results, errors = [None] * len(cases), []
+
+    def work(i):
+        try:
+            q, s_tok, wq, s_ch, N, ws, _ = cases[i]
+            st = torch.cuda.Stream(device=DEV)
+            outs = []
+            with torch.cuda.stream(st):
+                for _ in range(20):
+                    outs.append(pq.pq_gemm_w8a8(q, s_tok, wq, s_ch, N, workspace=ws))
+            st.synchronize()
+            results[i] = outs
+        except Exception as e:      # surfaced below: an exception in a thread must fail the test
+            errors.append(e)
+
+    threads = [threading.Thread(target=work, args=(i,)) for i in range(len(cases))]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    assert pq.pq_device_status() == 0
+    for (_, _, _, _, _, _, serial), outs in zip(cases, results):
+        for y in outs:
+            assert torch.equal(y, serial)
