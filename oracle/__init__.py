@@ -62,6 +62,7 @@ def _load():
         lib.pqo_pack_w8_hadamard.argtypes = [vp, i64, i64, vp, vp]
         lib.pqo_pack_w4_hadamard.argtypes = [vp, i64, i64, i64, vp, vp]
         lib.pqo_smooth_scales.argtypes = [vp, vp, i64, vp, vp]
+        lib.pqo_smooth_scales_alpha.argtypes = [vp, vp, i64, ctypes.c_int, vp, vp]
         lib.pqo_swiglu_quantize.argtypes = [vp, vp, i64, i64, vp, vp, vp]
         lib.pqo_nibble_pack.argtypes = [vp, i64, i64, vp]
         lib.pqo_nibble_unpack.argtypes = [vp, i64, i64, vp]
@@ -230,6 +231,17 @@ def smooth_scales(x_absmax: np.ndarray, w_absmax: np.ndarray):
         raise OracleError("smooth_scales: two vectors of the same length")
     s, s_inv = np.empty_like(xa), np.empty_like(xa)
     _check(_load().pqo_smooth_scales(_p(xa), _p(wa), xa.shape[0], _p(s), _p(s_inv)), "smooth_scales")
+    return s, s_inv
+
+
+def smooth_scales_alpha(x_absmax: np.ndarray, w_absmax: np.ndarray, alpha_quarters: int):
+    """Eq. 3 with alpha = alpha_quarters / 4 (0 ... 4): (s, s_inv) f32 [K]."""
+    xa, wa = _c(x_absmax, np.float32), _c(w_absmax, np.float32)
+    if xa.shape != wa.shape or xa.ndim != 1:
+        raise OracleError("smooth_scales_alpha: two vectors of the same length")
+    s, s_inv = np.empty_like(xa), np.empty_like(xa)
+    _check(_load().pqo_smooth_scales_alpha(_p(xa), _p(wa), xa.shape[0], int(alpha_quarters), _p(s), _p(s_inv)),
+           "smooth_scales_alpha")
     return s, s_inv
 
 

@@ -516,6 +516,38 @@ int pqo_smooth_scales(const float* x_absmax, const float* w_absmax, int64_t K, f
   return PQO_OK;
 }
 
+/* Eq. 3 with the migration strength alpha a multiple of 1/4 (alpha = a / 4, a = 0 ... 4):
+ *   s_j = max|X_j|^alpha / max|W_j|^(1 - alpha),
+ * with the quarter powers written as square roots so that every step is a correctly rounded binary32
+ * operation: x^(1/4) = sqrtf(sqrtf(x)), x^(1/2) = sqrtf(x), x^(3/4) = sqrtf(x) * sqrtf(sqrtf(x)) (one
+ * rounded product), x^0 = 1, x^1 = x; then one division, and s_inv = 1 / s.  a = 2 is pqo_smooth_scales. */
+static float quarter_power(float x, int a) {
+  switch (a) {
+    case 0: return 1.0f;
+    case 1: return sqrtf(sqrtf(x));
+    case 2: return sqrtf(x);
+    case 3: return sqrtf(x) * sqrtf(sqrtf(x));
+    default: return x;
+  }
+}
+
+int pqo_smooth_scales_alpha(const float* x_absmax, const float* w_absmax, int64_t K, int alpha_quarters, float* s,
+                            float* s_inv) {
+  if (K <= 0 || alpha_quarters < 0 || alpha_quarters > 4) return PQO_ERR_ARG;
+  for (int64_t k = 0; k < K; ++k) {
+    if (!(x_absmax[k] > 0.0f) || !(w_absmax[k] > 0.0f)) {
+      s[k] = 1.0f;
+      s_inv[k] = 1.0f;
+      continue;
+    }
+    float num = quarter_power(x_absmax[k], alpha_quarters);
+    float den = quarter_power(w_absmax[k], 4 - alpha_quarters);
+    s[k] = num / den;
+    s_inv[k] = 1.0f / s[k];
+  }
+  return PQO_OK;
+}
+
 /* Interchange form of INT4 codes: byte j of a row holds k = 2j in bits 0-3 and
  * k = 2j+1 in bits 4-7, two's complement. */
 int pqo_nibble_pack(const int8_t* codes, int64_t N, int64_t K, uint8_t* bytes) {

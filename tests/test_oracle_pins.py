@@ -716,3 +716,38 @@ def test_full_order_hadamard_quantizers_are_the_plain_rule_on_the_rotated_values
     # (X H)(W H)^T = X W^T with the full matrix too
     xf, wf = oracle.rotate_rows(x).astype(np.float64), oracle.rotate_rows(w).astype(np.float64)
     assert np.allclose(xf @ wf.T, x.astype(np.float64) @ w.astype(np.float64).T, rtol=1e-9)
+
+
+# ---------------------------------------------------------------------------- Eq. 3 with alpha a multiple of 1/4
+
+def test_smooth_scales_for_quarter_alphas():
+    """s_j = max|X_j|^alpha / max|W_j|^(1-alpha): closed forms on fourth powers, the alpha = 1/2 case is the
+    pinned pqo_smooth_scales bit for bit, the extremes put all of the range on one side, and the binary64
+    power agrees to rounding."""
+    xa = np.array([16.0, 81.0, 256.0, 1.0, 0.0, 625.0], np.float32)
+    wa = np.array([1.0, 16.0, 81.0, 16.0, 4.0, 0.0], np.float32)
+    want = {0: [1 / 1.0, 1 / 16.0, 1 / 81.0, 1 / 16.0, 1, 1],          # 1 / max|W|
+            1: [2 / 1.0, 3 / 8.0, 4 / 27.0, 1 / 8.0, 1, 1],            # x^(1/4) / w^(3/4)
+            2: [4 / 1.0, 9 / 4.0, 16 / 9.0, 1 / 4.0, 1, 1],
+            3: [8 / 1.0, 27 / 2.0, 64 / 3.0, 1 / 2.0, 1, 1],           # x^(3/4) / w^(1/4)
+            4: [16.0, 81.0, 256.0, 1.0, 1, 1]}                          # max|X|
+    for a, vals in want.items():
+        s, s_inv = oracle.smooth_scales_alpha(xa, wa, a)
+        assert np.array_equal(s, np.array(vals, np.float64).astype(np.float32)), a
+        assert np.array_equal(s_inv, (np.float32(1.0) / s).astype(np.float32))
+    rng = np.random.default_rng(9)
+    xr = (rng.random(512) * 50 + 0.01).astype(np.float32)
+    wr = (rng.random(512) * 0.3 + 0.001).astype(np.float32)
+    s2, i2 = oracle.smooth_scales_alpha(xr, wr, 2)
+    s_ref, i_ref = oracle.smooth_scales(xr, wr)
+    assert np.array_equal(s2, s_ref) and np.array_equal(i2, i_ref)
+    for a in range(5):
+        s, _ = oracle.smooth_scales_alpha(xr, wr, a)
+        true = xr.astype(np.float64) ** (a / 4) / wr.astype(np.float64) ** (1 - a / 4)
+        assert np.allclose(s, true, rtol=4e-7)
+    # what alpha does: the smoothed maxima are (x w)^(1-alpha) on the activation side and (x w)^alpha on the
+    # weight side -- their product stays x w, and they meet at alpha = 1/2
+    for a in range(5):
+        s, _ = oracle.smooth_scales_alpha(xr, wr, a)
+        xw = xr.astype(np.float64) * wr.astype(np.float64)
+        assert np.allclose(xr / s, xw ** (1 - a / 4), rtol=1e-6) and np.allclose(wr * s, xw ** (a / 4), rtol=1e-6)
