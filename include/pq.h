@@ -124,6 +124,13 @@ PQ_API int pq_pack_w4(const void* w_f16, int64_t N, int64_t K, int32_t group, vo
 PQ_API int pq_col_absmax(const void* a_f16, int64_t R, int64_t K, float* out, void* stream);
 PQ_API int pq_smooth_scales(const float* x_absmax, const float* w_absmax, int64_t K, float* s, float* s_inv,
                             void* stream);
+/* The same for a migration strength alpha = alpha_quarters / 4 (0 ... 4, else PQ_ERR_SHAPE):
+ * s[k] = x_absmax[k]^alpha / w_absmax[k]^(1 - alpha), the quarter powers taken as square roots
+ * (x^(1/4) = sqrt(sqrt(x)), x^(3/4) = sqrt(x) * sqrt(sqrt(x))) so that every step is a correctly rounded FP32
+ * operation; alpha_quarters = 2 is pq_smooth_scales.  Any other factor vector a caller computes itself goes
+ * into the quantizer and pack calls just the same. */
+PQ_API int pq_smooth_scales_alpha(const float* x_absmax, const float* w_absmax, int64_t K, int32_t alpha_quarters,
+                                  float* s, float* s_inv, void* stream);
 PQ_API int pq_quantize_act_smooth(const void* x_f16, const float* s_inv, int64_t M, int64_t K, int8_t* q,
                                   float* s_tok, void* stream);
 PQ_API int pq_pack_w8_smooth(const void* w_f16, const float* s, int64_t N, int64_t K, void* wq, float* s_ch,

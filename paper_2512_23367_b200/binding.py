@@ -49,6 +49,7 @@ SIGNATURES = {
     "pq_pack_w4_hadamard": (ctypes.c_int, [_vp, _i64, _i64, _i32, _vp, _vp, _vp]),
     "pq_col_absmax": (ctypes.c_int, [_vp, _i64, _i64, _vp, _vp]),
     "pq_smooth_scales": (ctypes.c_int, [_vp, _vp, _i64, _vp, _vp, _vp]),
+    "pq_smooth_scales_alpha": (ctypes.c_int, [_vp, _vp, _i64, _i32, _vp, _vp, _vp]),
     "pq_quantize_act_smooth": (ctypes.c_int, [_vp, _vp, _i64, _i64, _vp, _vp, _vp]),
     "pq_pack_w8_smooth": (ctypes.c_int, [_vp, _vp, _i64, _i64, _vp, _vp, _vp]),
     "pq_pack_w4_smooth": (ctypes.c_int, [_vp, _vp, _i64, _i64, _i32, _vp, _vp, _vp]),
@@ -266,13 +267,14 @@ def pq_col_absmax(a: torch.Tensor) -> torch.Tensor:
     return out
 
 
-def pq_smooth_scales(x_absmax: torch.Tensor, w_absmax: torch.Tensor):
-    """Eq. 3 with alpha = 0.5: (s, s_inv) f32 [K] from the column maxima of X and of W."""
+def pq_smooth_scales(x_absmax: torch.Tensor, w_absmax: torch.Tensor, alpha_quarters: int = 2):
+    """Eq. 3: (s, s_inv) f32 [K] from the column maxima of X and of W, alpha = alpha_quarters / 4 (default 1/2)."""
     xa = _dev(x_absmax, torch.float32, "x_absmax")
     wa = _factors(w_absmax, xa.shape[0], "w_absmax")
     s, s_inv = torch.empty_like(xa), torch.empty_like(xa)
-    _check("pq_smooth_scales", lib().pq_smooth_scales(xa.data_ptr(), wa.data_ptr(), xa.shape[0], s.data_ptr(),
-                                                      s_inv.data_ptr(), _stream()))
+    _check("pq_smooth_scales_alpha", lib().pq_smooth_scales_alpha(xa.data_ptr(), wa.data_ptr(), xa.shape[0],
+                                                                  int(alpha_quarters), s.data_ptr(), s_inv.data_ptr(),
+                                                                  _stream()))
     return s, s_inv
 
 

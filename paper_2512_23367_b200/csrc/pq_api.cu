@@ -326,12 +326,17 @@ int pq_col_absmax(const void* a_f16, int64_t R, int64_t K, float* out, void* str
   return launch_col_absmax(a_f16, R, K, out, static_cast<cudaStream_t>(stream));
 }
 
-int pq_smooth_scales(const float* x_absmax, const float* w_absmax, int64_t K, float* s, float* s_inv, void* stream) {
+int pq_smooth_scales_alpha(const float* x_absmax, const float* w_absmax, int64_t K, int32_t alpha_quarters, float* s,
+                           float* s_inv, void* stream) {
   if (!x_absmax || !w_absmax || !s || !s_inv) return PQ_ERR_NULL;
-  if (K < 1 || K >= 131072) return PQ_ERR_SHAPE;
+  if (K < 1 || K >= 131072 || alpha_quarters < 0 || alpha_quarters > 4) return PQ_ERR_SHAPE;
   const int rc = check_arch();
   if (rc != PQ_OK) return rc;
-  return launch_smooth_scales(x_absmax, w_absmax, K, s, s_inv, static_cast<cudaStream_t>(stream));
+  return launch_smooth_scales(x_absmax, w_absmax, K, alpha_quarters, s, s_inv, static_cast<cudaStream_t>(stream));
+}
+
+int pq_smooth_scales(const float* x_absmax, const float* w_absmax, int64_t K, float* s, float* s_inv, void* stream) {
+  return pq_smooth_scales_alpha(x_absmax, w_absmax, K, 2, s, s_inv, stream);
 }
 
 int pq_unpack_w8(const void* wq, int64_t N, int64_t K, int8_t* codes, void* stream) {

@@ -94,7 +94,8 @@ int launch_swiglu_quantize(const void* gate, const void* up, int64_t M, int64_t 
 int launch_quantize_act_static_channel(const void* x, const float* inv_s, int64_t M, int64_t K, int8_t* q, float* s_tok,
                                        cudaStream_t stream);
 int launch_col_absmax(const void* a, int64_t R, int64_t K, float* out, cudaStream_t stream);
-int launch_smooth_scales(const float* xa, const float* wa, int64_t K, float* s, float* s_inv, cudaStream_t stream);
+int launch_smooth_scales(const float* xa, const float* wa, int64_t K, int alpha_quarters, float* s, float* s_inv,
+                         cudaStream_t stream);
 int launch_unpack_w4(const void* wp, int64_t N, int64_t K, int8_t* codes, cudaStream_t stream);
 
 // Prefill-shaped W8A8 GEMM (tcgen05 kind::i8) on CTA pairs (cta_group::2, 256-row tiles), for M > 128.

@@ -934,15 +934,28 @@ __global__ void __launch_bounds__(kThreads) col_absmax_kernel(const uint4* __res
 
 // Eq. 3 with alpha = 1/2, literally: sqrt(max|X_j|) / sqrt(max|W_j|), and its reciprocal; three and
 // one correctly rounded FP32 operations.  A channel with a zero maximum keeps s = 1.
+// x^(a/4) for a = 0 ... 4 out of correctly rounded square roots and at most one rounded product.
+__device__ __forceinline__ float quarter_power(float x, int a) {
+  const float r2 = __fsqrt_rn(x);
+  switch (a) {
+    case 0: return 1.0f;
+    case 1: return __fsqrt_rn(r2);
+    case 2: return r2;
+    case 3: return __fmul_rn(r2, __fsqrt_rn(r2));
+    default: return x;
+  }
+}
+
+// alpha = a / 4: s = x^alpha / w^(1 - alpha); a = 2 is Eq. 3 as the paper sets it.
 __global__ void __launch_bounds__(kThreads) smooth_scales_kernel(const float* __restrict__ xa,
-                                                                 const float* __restrict__ wa, int64_t K,
+                                                                 const float* __restrict__ wa, int64_t K, int a,
                                                                  float* __restrict__ s, float* __restrict__ s_inv) {
   const int64_t k = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x;
   if (k >= K) return;
   const float x = xa[k], w = wa[k];
   float sv = 1.0f, si = 1.0f;
   if (x > 0.0f && w > 0.0f) {
-    sv = __fdiv_rn(__fsqrt_rn(x), __fsqrt_rn(w));
+    sv = __fdiv_rn(quarter_power(x, a), quarter_power(w, 4 - a));
     si = __fdiv_rn(1.0f, sv);
   }
   s[k] = sv;
@@ -961,9 +974,10 @@ int launch_col_absmax(const void* a, int64_t R, int64_t K, float* out, cudaStrea
   return cuda_status(cudaGetLastError());
 }
 
-int launch_smooth_scales(const float* xa, const float* wa, int64_t K, float* s, float* s_inv, cudaStream_t stream) {
+int launch_smooth_scales(const float* xa, const float* wa, int64_t K, int alpha_quarters, float* s, float* s_inv,
+                         cudaStream_t stream) {
   const unsigned blocks = static_cast<unsigned>((K + kThreads - 1) / kThreads);
-  smooth_scales_kernel<<<blocks, kThreads, 0, stream>>>(xa, wa, K, s, s_inv);
+  smooth_scales_kernel<<<blocks, kThreads, 0, stream>>>(xa, wa, K, alpha_quarters, s, s_inv);
   return cuda_status(cudaGetLastError());
 }
 

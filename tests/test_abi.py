@@ -59,6 +59,7 @@ def test_argument_errors_come_back_as_status_codes_without_a_device():
     assert L.pq_pack_w4_smooth(16, 16, 16, 256, 64, 16, 16, None) == PQ_ERR_SHAPE   # group != 128
     assert L.pq_col_absmax(16, 0, 64, 16, None) == PQ_ERR_SHAPE
     assert L.pq_smooth_scales(16, 16, 0, 16, 16, None) == PQ_ERR_SHAPE
+    assert L.pq_smooth_scales_alpha(16, 16, 64, 5, 16, 16, None) == PQ_ERR_SHAPE      # alpha beyond 4/4
     assert L.pq_quantize_act_hadamard(16, 4, 16400, 16, 16, None) == PQ_ERR_SHAPE   # row does not fit the registers
     assert L.pq_pack_w4_hadamard(16, 16, 192, 128, 16, 16, None) == PQ_ERR_SHAPE     # K % 128
     assert [L.pq_hadamard_block(K) for K in (16, 48, 208, 2048, 4096, 11008, 20)] == [16, 16, 16, 2048, 4096, 256, 0]

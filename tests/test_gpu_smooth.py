@@ -41,6 +41,25 @@ def test_smooth_scales_bit_exact_including_dead_channels():
     assert _np(s)[5] == 1.0 and _np(s)[9] == 1.0
 
 
+@pytest.mark.parametrize("alpha_quarters", [0, 1, 2, 3, 4])
+def test_smooth_scales_for_quarter_alphas_bit_exact(alpha_quarters):
+    rng = np.random.default_rng(63)
+    xa = rng.uniform(0.01, 80.0, 11008).astype(np.float32)
+    wa = rng.uniform(0.001, 0.3, 11008).astype(np.float32)
+    xa[5], wa[9] = 0.0, 0.0
+    s, s_inv = pq.pq_smooth_scales(_t(xa), _t(wa), alpha_quarters)
+    so, sio = oracle.smooth_scales_alpha(xa, wa, alpha_quarters)
+    assert np.array_equal(_np(s).view(np.uint32), so.view(np.uint32))
+    assert np.array_equal(_np(s_inv).view(np.uint32), sio.view(np.uint32))
+
+
+def test_alpha_outside_the_quarters_is_refused():
+    v = _t(np.ones(64, np.float32))
+    with pytest.raises(pq.PQError) as err:
+        pq.pq_smooth_scales(v, v, 5)
+    assert err.value.status == 2
+
+
 # row teams of 32 / 64 / 128 / 256 threads, ragged row blocks, K beyond the register-cached part
 @pytest.mark.parametrize("M,K", [(1, 16), (16, 256), (9, 2048), (130, 4096), (33, 6144), (70, 11008), (5, 20480)])
 def test_quantize_act_smooth_bit_exact(M, K):
