@@ -227,3 +227,22 @@ def test_host_threads_call_concurrently_on_their_own_streams():
     for (_, _, _, _, _, _, serial), outs in zip(cases, results):
         for y in outs:
             assert torch.equal(y, serial)
+
+
+@pytest.mark.parametrize("M", [1, 16, 130])
+def test_longest_k_the_int32_accumulator_allows(M):
+    """K = 131056 is the largest K the shape rule admits (K * 128 * 128 < 2^31): with every code at -128 the
+    accumulator reaches 131056 * 16384 = 2 147 221 504, 262 144 below the INT32 limit, on every schedule."""
+    K, N = 131056, 264
+    q = torch.full((M, K), -128, dtype=torch.int8, device=DEV)
+    wq = torch.full((N * K,), 0x80, dtype=torch.uint8, device=DEV)
+    acc = pq.pq_acc_w8a8(q, wq, N)
+    assert pq.pq_device_status() == 0
+    assert (acc == K * 16384).all() and K * 16384 < 2 ** 31
+    q[:, 1::2] = 127                                   # alternate signs: the sum stays small, every product is extreme
+    acc = _np(pq.pq_acc_w8a8(q, wq, N))
+    assert (acc == (K // 2) * (16384 - 127 * 128)).all()
+    with pytest.raises(pq.PQError) as err:             # one step further is refused before anything runs
+        pq.pq_acc_w8a8(torch.zeros((M, 131072), dtype=torch.int8, device=DEV),
+                       torch.zeros((N * 131072,), dtype=torch.uint8, device=DEV), N)
+    assert err.value.status == 2
