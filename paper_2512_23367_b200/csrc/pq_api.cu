@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 
 #include <atomic>
+#include <cstdio>
 #include <cstdlib>
 #include <mutex>
 
@@ -128,6 +129,18 @@ static bool gemv_enabled() {
     return !(e != nullptr && e[0] == '0');
   }();
   return on;
+}
+
+// PQ_LOG=1 in the environment: one line on stderr per GEMM call saying which schedule it was given.
+static bool log_enabled() {
+  static const bool on = [] {
+    const char* e = getenv("PQ_LOG");
+    return e != nullptr && e[0] == '1';
+  }();
+  return on;
+}
+static void log_dispatch(const char* call, const char* schedule, int64_t M, int64_t N, int64_t K) {
+  if (log_enabled()) fprintf(stderr, "[pq] %s M=%lld N=%lld K=%lld -> %s\n", call, (long long)M, (long long)N, (long long)K, schedule);
 }
 
 bool pdl_enabled() {
@@ -369,8 +382,15 @@ static int gemm_w8a8_common(const int8_t* q, const float* s_tok, const void* wq,
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   // Up to 128 tokens: the weight-streaming schedule (tokens are the narrow MMA dimension, K split over a
   // cluster); beyond that the second CTA of a pair no longer holds only padding rows.
-  if (gemv_enabled() && gemv_rows_serves(8, M, N, K, sm_count())) return launch_gemv_rows_w8a8(q, s_tok, wq, s_ch, M, N, K, y, acc, st);
-  if (M <= kSmallM_W8) return launch_smallm_w8a8(q, s_tok, wq, s_ch, M, N, K, y, acc, st);
+  if (gemv_enabled() && gemv_rows_serves(8, M, N, K, sm_count())) {
+    log_dispatch("w8a8", "CUDA-core row kernel", M, N, K);
+    return launch_gemv_rows_w8a8(q, s_tok, wq, s_ch, M, N, K, y, acc, st);
+  }
+  if (M <= kSmallM_W8) {
+    log_dispatch("w8a8", "tensor-core weight streaming", M, N, K);
+    return launch_smallm_w8a8(q, s_tok, wq, s_ch, M, N, K, y, acc, st);
+  }
+  log_dispatch("w8a8", "pair GEMM", M, N, K);
   return launch_gemm_w8a8_pair(scratch_from(workspace, workspace_bytes), q, s_tok, wq, s_ch, M, N, K, y, acc, st);
 }
 
@@ -415,8 +435,15 @@ static int gemm_w4a8_common(const int8_t* q, const float* s_tok, const void* wp,
   if (!aligned16(q) || !aligned16(wp) || !aligned16(s_grp) || !aligned16(y) || !aligned16(acc_g)) return PQ_ERR_ALIGN;
   if ((rc = check_arch()) != PQ_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (gemv_enabled() && gemv_rows_serves(4, M, N, K, sm_count())) return launch_gemv_rows_w4a8(q, s_tok, wp, s_grp, M, N, K, y, acc_g, st);
-  if (M <= kSmallM) return launch_smallm_w4a8(q, s_tok, wp, s_grp, M, N, K, y, acc_g, st);
+  if (gemv_enabled() && gemv_rows_serves(4, M, N, K, sm_count())) {
+    log_dispatch("w4a8", "CUDA-core row kernel", M, N, K);
+    return launch_gemv_rows_w4a8(q, s_tok, wp, s_grp, M, N, K, y, acc_g, st);
+  }
+  if (M <= kSmallM) {
+    log_dispatch("w4a8", "tensor-core weight streaming", M, N, K);
+    return launch_smallm_w4a8(q, s_tok, wp, s_grp, M, N, K, y, acc_g, st);
+  }
+  log_dispatch("w4a8", "pair GEMM", M, N, K);
   return launch_gemm_w4a8(q, s_tok, wp, s_grp, M, N, K, y, acc_g, st);
 }
 
