@@ -430,12 +430,10 @@ int launch_rows(const void* x, int64_t M, int64_t K, int8_t* q, float* s, const 
   const uint4* xp = static_cast<const uint4*>(x);
   uint2* qp = reinterpret_cast<uint2*>(q);
   const float4* cp = reinterpret_cast<const float4*>(col);
-  // The narrowest row team that still keeps the whole row in registers -- widened while the launch would
-  // leave the SMs short of warps (few or short rows: the kernel is then bound by the latency of its loads,
-  // and more threads per row means more loads in flight), as long as every thread still has a chunk.
-  int T = K8 <= 32 * kCached ? 32 : (K8 <= 64 * kCached ? 64 : (K8 <= 128 * kCached ? 128 : 256));
-  const int64_t want_threads = static_cast<int64_t>(sm_count()) * 1536;
-  while (T < 256 && M * T < want_threads && 2 * T <= K8) T *= 2;
+  // The narrowest row team that still keeps the whole row in registers.  (Wider teams for short launches --
+  // more loads in flight per row -- were measured and lose: the maximum then crosses warps through shared
+  // memory and a block barrier; 2048 x 2048: 4.4 us with 32 threads per row, 5.2 with 128, 7.1 with 256.)
+  const int T = K8 <= 32 * kCached ? 32 : (K8 <= 64 * kCached ? 64 : (K8 <= 128 * kCached ? 128 : 256));
   if (T == 32) return launch_rows_team<32, kDivide, kSmooth>(xp, M, K8, qp, s, cp, stream);
   if (T == 64) return launch_rows_team<64, kDivide, kSmooth>(xp, M, K8, qp, s, cp, stream);
   if (T == 128) return launch_rows_team<128, kDivide, kSmooth>(xp, M, K8, qp, s, cp, stream);
