@@ -18,7 +18,7 @@ __device__ int g_status_word = 0;
 namespace {
 
 constexpr int kMaxDevices = 64;
-constexpr int64_t kSmallM = 64;      // W4A8: M at or below this takes the weight-streaming schedule
+constexpr int64_t kSmallM = 128;     // W4A8: M at or below this takes the weight-streaming schedule
 constexpr int64_t kSmallM_W8 = 128;  // W8A8
 
 // Facts about a device, filled in by the first call on it.  Host threads may make that first call

@@ -1,4 +1,4 @@
-// Small-M (decode-shaped; W8A8: M <= 128, W4A8: M <= 64) linear for sm_100a: a weight-streaming schedule
+// Small-M (decode-shaped; M <= 128) linear for sm_100a: a weight-streaming schedule
 // that computes the same result as the prefill kernels.
 //
 // The roles of the two operands are swapped: a tile of 128 WEIGHT rows is the 128-lane operand
@@ -30,8 +30,6 @@ namespace {
 constexpr int BW = 128;   // weight rows per tile (TMEM lanes)
 constexpr int BK = 128;   // K per block = one W4 group
 constexpr int UMMA_K = 32;
-constexpr int kNumThreads = 256;      // W8 and 64-token W4; the other W4 variants add two widening warps
-constexpr int kNumThreadsW4 = 320;
 constexpr int kUnpackThreads = 64;    // per K block (one pair of warps)
 constexpr int kMaxSplit = 8;  // portable cluster size
 
@@ -44,14 +42,20 @@ struct Cfg {
   static constexpr int kTxBytes = kWBytes + kQBytes + kSBytes;
   // Short rings and small footprints: three or four CTAs fit on an SM, so the CTAs of the NEXT
   // launch become resident (and stream their weights) while this launch reduces and stores.
-  static constexpr int STAGES = MPAD == 64 ? 4 : 3;
-  static_assert(!(kW4 && MPAD > 64), "the W4 variant keeps MPAD partial results per thread in registers");
-  // W4 with up to 32 tokens: two pairs of widening warps (the 64-token variant needs its registers
-  // for the per-thread partial results and keeps one pair and two co-resident CTAs)
-  static constexpr int kUnpackPairs = (kW4 && MPAD < 64) ? 2 : 1;
-  static constexpr int kThreads = kUnpackPairs == 2 ? kNumThreadsW4 : kNumThreads;
-  static constexpr int kMinCtasPerSm = MPAD >= 64 ? 2 : (kW4 ? 2 : 4);
-  static constexpr int A8_SLOTS = kW4 ? 2 : 0;                   // widened weight tiles: one per pair of widening warps
+  static constexpr int STAGES = (kW4 && MPAD > 64) ? 6 : (MPAD == 64 ? 4 : 3);
+  // W4: two pairs of widening warps, except at 64 tokens (that variant needs its registers for the 64
+  // per-thread partial results and keeps one pair and two co-resident CTAs).  At 128 tokens one CTA
+  // owns the SM: a six-deep ring, four widened slots, eight epilogue warps.
+  static constexpr int kUnpackPairs = (kW4 && MPAD != 64) ? 2 : 1;
+  // Warps: 0 producer, 1 MMA issuer, 2-3 first widening pair, then the epilogue warps (W4 at 128 tokens:
+  // two per TMEM lane quadrant, 64 token columns each, so that a thread keeps 64 partial results), then
+  // the second widening pair.
+  static constexpr int kEpiWarps = (kW4 && MPAD > 64) ? 8 : 4;
+  static constexpr int kEpiEnd = 4 + kEpiWarps;                  // first warp after the epilogue warps
+  static constexpr int kEpiCols = MPAD / (kEpiWarps / 4);        // token columns per epilogue warp
+  static constexpr int kThreads = 32 * (kEpiEnd + (kUnpackPairs == 2 ? 2 : 0));
+  static constexpr int kMinCtasPerSm = (kW4 && MPAD > 64) ? 1 : (MPAD >= 64 ? 2 : (kW4 ? 2 : 4));
+  static constexpr int A8_SLOTS = kW4 ? (MPAD > 64 ? 4 : 2) : 0;                   // widened weight tiles: one per pair of widening warps
   static constexpr int kA8Bytes = BW * BK;
   static constexpr int SC_SLOTS = kW4 ? 6 : 0;                   // FP32 scale rows (128 floats)
   static constexpr int ACC_SLOTS = kW4 ? 4 : 1;
@@ -62,7 +66,10 @@ struct Cfg {
   static constexpr int kBarOff = (kRingEnd > kRedBytes ? kRingEnd : kRedBytes);
   static constexpr int kNumBars = 2 * STAGES + 2 * A8_SLOTS + 2 * SC_SLOTS + 2 * ACC_SLOTS + 1;   // + the MMA issuer's drain barrier
   static constexpr int kMiscOff = kBarOff + kNumBars * 8;
-  static constexpr int kDynamic = kMiscOff + 16 + 1024;
+  // A CTA that takes all 512 TMEM columns must be alone on its SM (a second one would block in
+  // tcgen05.alloc): its shared-memory request is raised past half an SM's so that it always is.
+  static constexpr int kNeeded = kMiscOff + 16 + 1024;
+  static constexpr int kDynamic = (ACC_SLOTS * MPAD > 256 && kNeeded < 117 * 1024) ? 117 * 1024 : kNeeded;
   static constexpr uint32_t kTmemCols = (ACC_SLOTS * MPAD) < 32 ? 32 : (ACC_SLOTS * MPAD);
 };
 
@@ -187,11 +194,11 @@ smallm_kernel(const __grid_constant__ SmallMaps maps, const __grid_constant__ CU
     }
     for (int s = 0; s < C::SC_SLOTS; ++s) {
       mbar_init(bar_sc_full + s * 8, kUnpackThreads / 32);
-      mbar_init(bar_sc_empty + s * 8, 4);
+      mbar_init(bar_sc_empty + s * 8, C::kEpiWarps);
     }
     for (int s = 0; s < C::ACC_SLOTS; ++s) {
       mbar_init(bar_acc_full + s * 8, 1);
-      mbar_init(bar_acc_empty + s * 8, 4);
+      mbar_init(bar_acc_empty + s * 8, C::kEpiWarps);
     }
     fence_mbar_init();
     // Start the weight stream at once: the first ring pass needs no wait, neither on a stage
@@ -211,7 +218,7 @@ smallm_kernel(const __grid_constant__ SmallMaps maps, const __grid_constant__ CU
 
   // W4: per-thread partial results of the epilogue warps, P[m] for weight row n0 + 32*quad + lane.
   // (W8 copies its one accumulator from tensor memory straight into the reduction tile.)
-  constexpr int kPartials = kW4 ? MPAD : 1;
+  constexpr int kPartials = kW4 ? C::kEpiCols : 1;
   uint32_t P[kPartials];
 #pragma unroll
   for (int m = 0; m < kPartials; ++m) P[m] = 0u;
@@ -272,11 +279,11 @@ smallm_kernel(const __grid_constant__ SmallMaps maps, const __grid_constant__ CU
         if (ok) umma_commit(bar_acc_full);
       }
     }
-  } else if (warp < 4 || warp >= 8) {
+  } else if (warp < 4 || warp >= C::kEpiEnd) {
     // ------------------------------------------------------------ W4: widen nibbles to INT8
     if constexpr (kW4) {
-      const int pair = warp >= 8 ? 1 : 0;                      // warps 2-3: even K blocks, warps 8-9: odd ones
-      const int ut = threadIdx.x - (pair ? 256 : 64);
+      const int pair = warp >= C::kEpiEnd ? 1 : 0;             // warps 2-3: even K blocks, the last two warps: odd ones
+      const int ut = threadIdx.x - (pair ? C::kEpiEnd * 32 : 64);
       for (int j = pair; j < nkb; j += C::kUnpackPairs) {
         const uint32_t it = static_cast<uint32_t>(j);
         const uint32_t s = it % C::STAGES, ph = (it / C::STAGES) & 1u;
@@ -323,6 +330,7 @@ smallm_kernel(const __grid_constant__ SmallMaps maps, const __grid_constant__ CU
     const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
     const int n_local = quad * 32 + lane;
     if constexpr (kW4) {
+      const int col0 = ((warp - 4) >> 2) * C::kEpiCols;   // this warp's first token column
       constexpr int CH = MPAD < 32 ? MPAD : 32;  // columns promoted per tcgen05.ld
       for (int j = 0; j < nkb; ++j) {
         const uint32_t it = static_cast<uint32_t>(j);
@@ -334,16 +342,16 @@ smallm_kernel(const __grid_constant__ SmallMaps maps, const __grid_constant__ CU
         tc_fence_after_sync();
         const float sg = (reinterpret_cast<const float*>(smem + C::kScOff) + v * BW)[n_local];
 #pragma unroll
-        for (int c0 = 0; c0 < MPAD; c0 += CH) {
+        for (int c0 = 0; c0 < C::kEpiCols; c0 += CH) {
           uint32_t r[CH];
-          tmem_ld_cols<CH>(lane_addr + a * MPAD + c0, r);
+          tmem_ld_cols<CH>(lane_addr + a * MPAD + col0 + c0, r);
           tmem_ld_wait();
           if constexpr (kExportAcc) {
             const int n = n0 + n_local;
 #pragma unroll
             for (int m = 0; m < CH; ++m) {
-              if (c0 + m < p.M && n < N_mem)
-                p.acc[(static_cast<int64_t>(kb0 + j) * p.M + c0 + m) * N_mem + n] = static_cast<int32_t>(r[m]) >> 4;
+              if (col0 + c0 + m < p.M && n < N_mem)
+                p.acc[(static_cast<int64_t>(kb0 + j) * p.M + col0 + c0 + m) * N_mem + n] = static_cast<int32_t>(r[m]) >> 4;
             }
           } else {
 #pragma unroll
@@ -387,10 +395,11 @@ smallm_kernel(const __grid_constant__ SmallMaps maps, const __grid_constant__ CU
   // stage ring is free and holds this CTA's partial tile as red[m][n] (32-bit words).
   uint32_t* red = reinterpret_cast<uint32_t*>(smem);
   const bool do_reduce = !(kW4 && kExportAcc);
-  if (do_reduce && kW4 && warp >= 4 && warp < 8) {
+  if (do_reduce && kW4 && warp >= 4 && warp < C::kEpiEnd) {
     const int n_local = (warp & 3) * 32 + lane;
+    const int col0 = ((warp - 4) >> 2) * C::kEpiCols;
 #pragma unroll
-    for (int m = 0; m < kPartials; ++m) red[m * BW + n_local] = P[m];
+    for (int m = 0; m < kPartials; ++m) red[(col0 + m) * BW + n_local] = P[m];
   }
   tc_fence_before_sync();
   __syncwarp();
@@ -409,9 +418,9 @@ smallm_kernel(const __grid_constant__ SmallMaps maps, const __grid_constant__ CU
       mbar_drain(bar_drain, 0u);
     }
   }
-  if (do_reduce && warp >= 4 && warp < 8) {
+  if (do_reduce && warp >= 4 && warp < C::kEpiEnd) {
     // Thread t owns four consecutive output channels (one 16-byte word of every part's partial
-    // tile) for the rows m = rank + splits * (t / 32 + 4 i): the remote loads of all parts of a row
+    // tile) for the rows m = rank + splits * (t / 32 + kEpiWarps i): the remote loads of all parts of a row
     // are issued together, so a row costs one distributed-shared-memory round trip, not `splits`.
     const int t = threadIdx.x - 128;
     const int nq = t & 31, msub = t >> 5;
@@ -422,7 +431,7 @@ smallm_kernel(const __grid_constant__ SmallMaps maps, const __grid_constant__ CU
 #pragma unroll
       for (int j = 0; j < 4; ++j) sc[j] = __ldg(s_ch_mem + n + j);   // N is a multiple of 8: n < N covers n + 3
     }
-    for (int m = static_cast<int>(my_rank) + p.splits * msub; m < p.M; m += 4 * p.splits) {
+    for (int m = static_cast<int>(my_rank) + p.splits * msub; m < p.M; m += C::kEpiWarps * p.splits) {
       const uint32_t addr = smem_base + static_cast<uint32_t>(m * BW + 4 * nq) * 4u;
       uint4 part[kMaxSplit];
 #pragma unroll
@@ -507,7 +516,6 @@ int launch_smallm(const int8_t* q, const float* s_tok, int count, const void* co
                   cudaStream_t stream) {
   if (count < 1 || count > kMaxGroup || (acc != nullptr && count != 1)) return PQ_ERR_SHAPE;
   const int mpad = M <= 16 ? 16 : (M <= 32 ? 32 : (M <= 64 ? 64 : 128));
-  if (kW4 && mpad > 64) return PQ_ERR_SHAPE;   // (the W4A8 dispatch sends M > 64 to the pair kernel)
   const int k_blocks = static_cast<int>((K + BK - 1) / BK);
 
   CUtensorMap tq;
@@ -548,7 +556,7 @@ int launch_smallm(const int8_t* q, const float* s_tok, int count, const void* co
   // nearly fills the device leaves clusters for a second wave (2048 -> 6144 at M = 64: 12.8 us with
   // clusters of 6, 7.4 us with clusters of 4).  Stay below 90 % of the resident capacity, and off the
   // cluster sizes 5 and 7.
-  const int ctas_per_sm = mpad >= 64 ? 2 : (kW4 ? 2 : 4);
+  const int ctas_per_sm = (kW4 && mpad > 64) ? 1 : (mpad >= 64 ? 2 : (kW4 ? 2 : 4));
   while (splits > 1 && n_tiles * splits * 10 > static_cast<int64_t>(ctas_per_sm) * sm_count() * 9) --splits;
   if (splits == 5 || splits == 7) --splits;
   // ablation knob, read once: force the number of K parts (cluster size)
@@ -572,12 +580,7 @@ int launch_smallm(const int8_t* q, const float* s_tok, int count, const void* co
     case 16: return ex ? launch_cfg<16, kW4, true>(maps, tq, a, nt, stream) : launch_cfg<16, kW4, false>(maps, tq, a, nt, stream);
     case 32: return ex ? launch_cfg<32, kW4, true>(maps, tq, a, nt, stream) : launch_cfg<32, kW4, false>(maps, tq, a, nt, stream);
     case 64: return ex ? launch_cfg<64, kW4, true>(maps, tq, a, nt, stream) : launch_cfg<64, kW4, false>(maps, tq, a, nt, stream);
-    default:
-      if constexpr (kW4) {
-        return PQ_ERR_SHAPE;
-      } else {
-        return ex ? launch_cfg<128, false, true>(maps, tq, a, nt, stream) : launch_cfg<128, false, false>(maps, tq, a, nt, stream);
-      }
+    default: return ex ? launch_cfg<128, kW4, true>(maps, tq, a, nt, stream) : launch_cfg<128, kW4, false>(maps, tq, a, nt, stream);
   }
 }
 

@@ -100,7 +100,7 @@ def _members_w4(K, Ns, seed):
     (257, 384, (1000, 136, 8)),
     (2048, 512, (2048, 2048, 2048)),
     (600, 1024, (256, 768, 264, 128)),
-    (65, 128, (16, 24)),
+    (129, 128, (16, 24)),
 ])
 def test_w4a8_group_equals_one_call_per_member_and_the_oracle(M, K, Ns):
     x = synth.activations(M, K, 5000 + M)
@@ -124,7 +124,8 @@ def test_w4a8_group_equals_one_call_per_member_and_the_oracle(M, K, Ns):
 
 @pytest.mark.parametrize("M,K,Ns", [(1, 512, (256, 520)), (16, 512, (256, 520)), (64, 512, (256, 520)),
                                     (3, 4224, (2376, 136, 8)), (33, 1024, (128, 128, 128, 264)),
-                                    (7, 4096, (4096, 4096, 4096))])
+                                    (7, 4096, (4096, 4096, 4096)), (65, 128, (16, 24)), (100, 1024, (1408, 520)),
+                                    (128, 4096, (4096, 4096, 4096))])
 def test_w4a8_small_token_counts_group_on_the_weight_streaming_kernel(M, K, Ns):
     """Decode-shaped W4A8 sums its K parts in FP32 in a fixed order, but the number of parts depends on
     how many tiles the launch holds: the grouped result may differ from the per-member call in the last
