@@ -24,12 +24,15 @@
 // sums in registers.
 //
 // Warp roles (512 threads; register budgets moved with setmaxnreg):
-//   warp 0        TMA producer: codes, packed weights and scales of a group on one local barrier
-//                 (weights and scales requested before the wait on the preceding kernel)
+//   warp 0        TMA producer of the token codes: a ring of four 16 KB stages, freed by the MMAs
+//   warp 2        TMA producer of packed weights + scales: a ring of its own (six slots of 8.25 KB), freed
+//                 by the widening, so that it runs ahead of the MMAs and -- these being constants of the
+//                 model -- ahead of the wait on the preceding kernel.  (With one ring for everything the
+//                 loop load -> widen -> MMA -> free bounded the kernel: 64.2 against 59.6 us.)
 //   warp 1        MMA issuer (leader CTA only; owns TMEM allocation in both CTAs).  It shares its
 //                 scheduler with busy warps, so it is kept to two waits, four MMAs and two commits
-//                 per group: "widened" (which implies "codes landed": the widening warp saw the
-//                 stage's barrier first) and "accumulator free"
+//                 per group: "widened" (which implies "codes landed": the widening warp waits for the
+//                 stage's barrier before it signals) and "accumulator free"
 //   warps 4-7     widen nibbles -> INT8 (16 x code: the nibble sits in the high half of the byte,
 //                 which keeps two's complement; 1/16 is folded exactly into the FP32 scale).
 //                 Warp w takes every fourth K-group whole, so that the proxy fence that ends a
@@ -47,7 +50,8 @@ namespace {
 constexpr int BT_CTA = 128, BT_PAIR = 256;   // tokens per CTA / per tile (MMA N, TMEM columns)
 constexpr int BC_CTA = 128, BC_PAIR = 256;   // output channels per CTA (TMEM lanes) / per tile (MMA M)
 constexpr int BK = 128, UMMA_K = 32;
-constexpr int STAGES = 4;       // codes + packed weights + scales; also the widened-weight slots
+constexpr int STAGES = 4;       // token-code stages; also the widened-weight slots
+constexpr int P_SLOTS = 6;      // packed weights + FP16 scales of a group: a ring of its own, freed by the widening
 constexpr int SC_SLOTS = 8;     // FP32 scale rows (this CTA's 128 channels)
 constexpr int ACC_SLOTS = 2;    // TMEM accumulators of BT_PAIR columns
 constexpr int kNumThreads = 512;
@@ -59,15 +63,16 @@ constexpr int kRegsCtl = 64, kRegsUnpack = 64, kRegsPromote = 192;   // x128, x1
 constexpr int kQBytes = BT_CTA * BK;            // 16 KB of token codes
 constexpr int kPBytes = BC_CTA * BK / 2;        // 8 KB packed weights
 constexpr int kSBytes = BC_CTA * 2;             // FP16 scales of one group
-constexpr int kStageBytes = kQBytes + kPBytes + 1024;  // scales padded to keep 1024-B alignment
-constexpr int kTxBytes = kQBytes + kPBytes + kSBytes;
+constexpr int kStageBytes = kQBytes;            // a stage of the code ring
+constexpr int kPSlotBytes = kPBytes + kSBytes;  // a slot of the packed ring
 constexpr int kW8Bytes = BC_CTA * BK;           // 16 KB widened weights
 constexpr int kOutBoxBytes = 32 * 32 * 2;
 constexpr int kW8Off = STAGES * kStageBytes;
-constexpr int kScOff = kW8Off + STAGES * kW8Bytes;
+constexpr int kPOff = kW8Off + STAGES * kW8Bytes;
+constexpr int kScOff = kPOff + P_SLOTS * kPSlotBytes;
 constexpr int kOutOff = kScOff + SC_SLOTS * BC_CTA * 4;
 constexpr int kBarOff = kOutOff + kPromoteWarps * kOutBufs * kOutBoxBytes;
-constexpr int kNumBars = 3 * STAGES + 2 * SC_SLOTS + 2 * ACC_SLOTS + 1;   // + the MMA issuer's drain barrier
+constexpr int kNumBars = 3 * STAGES + 2 * P_SLOTS + 2 * SC_SLOTS + 2 * ACC_SLOTS + 1;   // + the MMA issuer's drain barrier
 constexpr int kMiscOff = kBarOff + kNumBars * 8;
 constexpr int kDynamicSmem = kMiscOff + 16 + 1024;
 static_assert(kDynamicSmem <= 232448, "exceeds the shared memory of one CTA");
@@ -129,10 +134,12 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t smem_base = smem_u32(smem);
-  const uint32_t bar_full = smem_base + kBarOff;              // local: codes, packed weights, scales landed
+  const uint32_t bar_full = smem_base + kBarOff;              // local: token codes landed
   const uint32_t bar_empty = bar_full + STAGES * 8;           // local: the pair's MMAs of the group completed
   const uint32_t bar_w8_full = bar_empty + STAGES * 8;        // LEADER: both CTAs' widened weights written
-  const uint32_t bar_sc_full = bar_w8_full + STAGES * 8;      // local: FP32 scales written
+  const uint32_t bar_p_full = bar_w8_full + STAGES * 8;       // local: packed weights and scales landed
+  const uint32_t bar_p_empty = bar_p_full + P_SLOTS * 8;      // local: the widening warp has read them
+  const uint32_t bar_sc_full = bar_p_empty + P_SLOTS * 8;     // local: FP32 scales written
   const uint32_t bar_sc_empty = bar_sc_full + SC_SLOTS * 8;   // local: promotion warps read them
   const uint32_t bar_acc_full = bar_sc_empty + SC_SLOTS * 8;  // local: group accumulator complete
   const uint32_t bar_acc_empty = bar_acc_full + ACC_SLOTS * 8;  // LEADER: both CTAs' promotion drained it
@@ -156,6 +163,10 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       mbar_init(bar_full + s * 8, 1);
       mbar_init(bar_empty + s * 8, 1);    // the MMAs' commit: by then the widening has read the stage too
       mbar_init(bar_w8_full + s * 8, 2);  // one widening warp in each CTA
+    }
+    for (int s = 0; s < P_SLOTS; ++s) {
+      mbar_init(bar_p_full + s * 8, 1);
+      mbar_init(bar_p_empty + s * 8, 1);
     }
     for (int s = 0; s < SC_SLOTS; ++s) {
       mbar_init(bar_sc_full + s * 8, 1);
@@ -186,50 +197,44 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const uint32_t tmem_base = *tmem_slot;
 
   grid_dep_launch();   // nothing above touched global data; the successor may begin its set-up
-  uint32_t issued = 0;   // producer thread: ring passes it has requested (for the give-up path)
+  uint32_t issued = 0;   // producer threads: loads each has requested on its ring (for the give-up path)
 
   if (warp < 4) {
     setmaxnreg_dec<kRegsCtl>();
     if (warp == 0 && lane == 0) {
-      // ---------------------------------------------------------- TMA producer (both CTAs)
-      auto load_weights = [&](uint32_t s, int g, int member, int c0) {
-        const uint32_t dst = smem_base + s * kStageBytes;
-        mbar_arrive_expect_tx(bar_full + s * 8, kTxBytes);   // the whole stage, codes included
-        tma_load_2d(dst + kQBytes, &maps.w[member], bar_full + s * 8, g * (BK / 2), c0);
-        tma_load_2d(dst + kQBytes + kPBytes, &maps.s[member], bar_full + s * 8, c0, g);
-      };
-      auto load_codes = [&](uint32_t s, int g, int t0) {
-        tma_load_2d(smem_base + s * kStageBytes, &tm_q, bar_full + s * 8, g * BK, t0);
-      };
-      auto tok0 = [&](const W4Tile& t) { return t.m_blk * BT_PAIR + static_cast<int>(rank) * BT_CTA; };
-      // First ring pass of the first tile: weights and scales (constants) before the wait on the
-      // preceding kernel, the codes it may have produced after it.
-      int pre = 0;
-      if (pair_id < num_tiles) {
-        pre = p.k_blocks < STAGES ? p.k_blocks : STAGES;
-        const W4Tile t = locate_tile(p, pair_id);
-        for (int g = 0; g < pre; ++g)
-          load_weights(static_cast<uint32_t>(g), g, t.g, t.c0 + static_cast<int>(rank) * BC_CTA);
-      }
-      grid_dep_wait();
-      if (pair_id < num_tiles) {
-        const W4Tile t = locate_tile(p, pair_id);
-        for (int g = 0; g < pre; ++g) load_codes(static_cast<uint32_t>(g), g, tok0(t));
-      }
-      uint32_t it = static_cast<uint32_t>(pre);
+      // ---------------------------------------------------------- TMA producer of the token codes (both CTAs)
+      grid_dep_wait();   // the codes may come from the preceding kernel
+      uint32_t it = 0;
       bool ok = true;
       for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs) {
         const W4Tile t = locate_tile(p, tile);
-        const int t0 = tok0(t), c0 = t.c0 + static_cast<int>(rank) * BC_CTA;
-        for (int g = (tile == pair_id ? pre : 0); g < p.k_blocks; ++g, ++it) {
+        const int t0 = t.m_blk * BT_PAIR + static_cast<int>(rank) * BT_CTA;
+        for (int g = 0; g < p.k_blocks; ++g, ++it) {
           const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
-          if (!mbar_wait(bar_empty + s * 8, ph ^ 1u, wc)) { ok = false; break; }
-          load_weights(s, g, t.g, c0);
-          load_codes(s, g, t0);
+          if (it >= STAGES && !mbar_wait(bar_empty + s * 8, ph ^ 1u, wc)) { ok = false; break; }
+          mbar_arrive_expect_tx(bar_full + s * 8, kQBytes);
+          tma_load_2d(smem_base + s * kStageBytes, &tm_q, bar_full + s * 8, g * BK, t0);
         }
       }
       issued = it;
-      (void)ok;
+    } else if (warp == 2 && lane == 0) {
+      // ---------------------------------------------------------- TMA producer of packed weights + scales
+      // (constants of the model: this stream does not wait for the preceding kernel)
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs) {
+        const W4Tile t = locate_tile(p, tile);
+        const int c0 = t.c0 + static_cast<int>(rank) * BC_CTA;
+        for (int g = 0; g < p.k_blocks; ++g, ++it) {
+          const uint32_t ps = it % P_SLOTS, pph = (it / P_SLOTS) & 1u;
+          if (it >= P_SLOTS && !mbar_wait(bar_p_empty + ps * 8, pph ^ 1u, wc)) { ok = false; break; }
+          const uint32_t dst = smem_base + kPOff + ps * kPSlotBytes;
+          mbar_arrive_expect_tx(bar_p_full + ps * 8, kPSlotBytes);
+          tma_load_2d(dst, &maps.w[t.g], bar_p_full + ps * 8, g * (BK / 2), c0);
+          tma_load_2d(dst + kPBytes, &maps.s[t.g], bar_p_full + ps * 8, c0, g);
+        }
+      }
+      issued = it;
     } else if (warp == 1 && lane == 0 && rank == 0) {
       // ---------------------------------------------------------- MMA issuer (leader only)
       constexpr uint32_t idesc = umma_idesc_s8(BC_PAIR, BT_PAIR);
@@ -258,17 +263,18 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     setmaxnreg_dec<kRegsUnpack>();
     const uint32_t s = static_cast<uint32_t>(warp - 4);     // this warp's stage and widened slot
     const uint32_t w8_full0 = mapa_u32(bar_w8_full, 0);
-    const uint8_t* stage = smem + s * kStageBytes;
-    const uint4* packed = reinterpret_cast<const uint4*>(stage + kQBytes);
     uint8_t* w8 = smem + kW8Off + s * kW8Bytes;
     const int total = pair_id < num_tiles ? ((num_tiles - pair_id + num_pairs - 1) / num_pairs) * p.k_blocks : 0;
     for (uint32_t it = s; it < static_cast<uint32_t>(total); it += kUnpackWarps) {
       const uint32_t ph = (it / STAGES) & 1u;
       const uint32_t v = it % SC_SLOTS, vph = (it / SC_SLOTS) & 1u;
-      // stage landed; the slot's previous MMAs are done; the scale row has been read
-      const bool w = mbar_wait3(bar_full + s * 8, ph, bar_empty + s * 8, ph ^ 1u, bar_sc_empty + v * 8, vph ^ 1u,
+      const uint32_t ps = it % P_SLOTS, pph = (it / P_SLOTS) & 1u;
+      // packed weights landed; the widened slot's previous MMAs are done; the scale row has been read
+      const bool w = mbar_wait3(bar_p_full + ps * 8, pph, bar_empty + s * 8, ph ^ 1u, bar_sc_empty + v * 8, vph ^ 1u,
                                 wc);
       if (!__all_sync(0xffffffffu, w)) break;
+      const uint8_t* pslot = smem + kPOff + ps * kPSlotBytes;
+      const uint4* packed = reinterpret_cast<const uint4*>(pslot);
 #pragma unroll 4
       for (int i = 0; i < (BC_CTA * 4) / 32; ++i) {
         const int idx = lane + i * 32;
@@ -284,7 +290,7 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         *reinterpret_cast<uint4*>(row + (((2 * j) ^ sw) << 4)) = lo;       // k = 32j .. 32j+15
         *reinterpret_cast<uint4*>(row + (((2 * j + 1) ^ sw) << 4)) = hi;   // k = 32j+16 .. 32j+31
       }
-      const __half2* sh = reinterpret_cast<const __half2*>(stage + kQBytes + kPBytes);
+      const __half2* sh = reinterpret_cast<const __half2*>(pslot + kPBytes);
       float2* sc = reinterpret_cast<float2*>(smem + kScOff + v * BC_CTA * 4);
 #pragma unroll
       for (int i = 0; i < BC_CTA / 64; ++i) {
@@ -292,10 +298,12 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         sc[lane + 32 * i] = make_float2(f.x * 0.0625f, f.y * 0.0625f);
       }
       fence_proxy_async_smem();  // generic-proxy writes -> visible to the tensor-core (async) proxy
-      __syncwarp();
+      // "widened" tells the MMA issuer that the group's codes are there too
+      if (!__all_sync(0xffffffffu, mbar_wait(bar_full + s * 8, ph, wc))) break;
       if (lane == 0) {
         mbar_arrive_cluster_addr(w8_full0 + s * 8);
         mbar_arrive(bar_sc_full + v * 8);
+        mbar_arrive(bar_p_empty + ps * 8);
       }
     }
   } else {
@@ -433,6 +441,9 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     if (threadIdx.x == 0) {
       const uint32_t first = issued > static_cast<uint32_t>(STAGES) ? issued - STAGES : 0u;
       for (uint32_t i = first; i < issued; ++i) mbar_drain(bar_full + (i % STAGES) * 8, (i / STAGES) & 1u);
+    } else if (threadIdx.x == 64) {
+      const uint32_t first = issued > static_cast<uint32_t>(P_SLOTS) ? issued - P_SLOTS : 0u;
+      for (uint32_t i = first; i < issued; ++i) mbar_drain(bar_p_full + (i % P_SLOTS) * 8, (i / P_SLOTS) & 1u);
     } else if (threadIdx.x == 32 && rank == 0) {
       umma_commit_pair_mcast(bar_drain, 0x1);
       mbar_drain(bar_drain, 0u);
