@@ -47,18 +47,27 @@
 namespace pq {
 namespace {
 
-constexpr int BT_CTA = 128, BT_PAIR = 256;   // tokens per CTA / per tile (MMA N, TMEM columns)
+// Tokens per tile (MMA N, TMEM columns) / per CTA.  Narrower tiles give a deeper accumulator ring (512
+// columns / BT_PAIR slots) but measured slower: 2048 x 4096 x 4096 takes 57 us at 256, 68 us at 160 and
+// 77 us at 128 tokens, with four or eight widening warps alike.
+constexpr int BT_PAIR = 256, BT_CTA = BT_PAIR / 2;
 constexpr int BC_CTA = 128, BC_PAIR = 256;   // output channels per CTA (TMEM lanes) / per tile (MMA M)
 constexpr int BK = 128, UMMA_K = 32;
 constexpr int STAGES = 4;       // token-code stages; also the widened-weight slots
 constexpr int P_SLOTS = 6;      // packed weights + FP16 scales of a group: a ring of its own, freed by the widening
 constexpr int SC_SLOTS = 8;     // FP32 scale rows (this CTA's 128 channels)
-constexpr int ACC_SLOTS = 2;    // TMEM accumulators of BT_PAIR columns
-constexpr int kNumThreads = 512;
-constexpr int kUnpackWarps = 4;
+constexpr int ACC_SLOTS = 512 / BT_PAIR;    // TMEM accumulators of BT_PAIR columns
+constexpr int kUnpackWarps = 4;                     // widening warps: kUnpackPerSlot share a group's 128 rows
+constexpr int kUnpackPerSlot = 1;                   // warps that share one group's rows (a warp per group measured
+                                                    // best: 57.3 us against 61.8 us with two, 2048 x 4096 x 4096)
+constexpr int kUnpackTeams = kUnpackWarps / kUnpackPerSlot;   // team t takes the groups t, t + kUnpackTeams, ...
 constexpr int kPromoteWarps = 8;
+constexpr int kFirstPromote = 4 + kUnpackWarps;
+constexpr int kNumThreads = 32 * (kFirstPromote + kPromoteWarps);
+constexpr int kWidenBatch = 4;  // 16-byte loads of a widening thread in flight
 constexpr int kOutBufs = 2;     // staging boxes per promotion warp
-constexpr int kRegsCtl = 64, kRegsUnpack = 64, kRegsPromote = 192;   // x128, x128, x256 threads = 64 Ki
+constexpr int kRegsCtl = 56, kRegsUnpack = 72, kRegsPromote = 192;
+constexpr int kRegsTotal = 128 * kRegsCtl + 32 * kUnpackWarps * kRegsUnpack + 32 * kPromoteWarps * kRegsPromote;
 
 constexpr int kQBytes = BT_CTA * BK;            // 16 KB of token codes
 constexpr int kPBytes = BC_CTA * BK / 2;        // 8 KB packed weights
@@ -66,7 +75,8 @@ constexpr int kSBytes = BC_CTA * 2;             // FP16 scales of one group
 constexpr int kStageBytes = kQBytes;            // a stage of the code ring
 constexpr int kPSlotBytes = kPBytes + kSBytes;  // a slot of the packed ring
 constexpr int kW8Bytes = BC_CTA * BK;           // 16 KB widened weights
-constexpr int kOutBoxBytes = 32 * 32 * 2;
+constexpr int kOutTok = BT_CTA % 32 == 0 ? 32 : 16;   // tokens per stored box
+constexpr int kOutBoxBytes = kOutTok * 32 * 2;
 constexpr int kW8Off = STAGES * kStageBytes;
 constexpr int kPOff = kW8Off + STAGES * kW8Bytes;
 constexpr int kScOff = kPOff + P_SLOTS * kPSlotBytes;
@@ -77,8 +87,9 @@ constexpr int kMiscOff = kBarOff + kNumBars * 8;
 constexpr int kDynamicSmem = kMiscOff + 16 + 1024;
 static_assert(kDynamicSmem <= 232448, "exceeds the shared memory of one CTA");
 static_assert(BK / UMMA_K == 4, "the MMA issuer is unrolled for four steps per group");
-static_assert(kUnpackWarps == STAGES, "a widening warp always works on the same stage and slot");
-static_assert(128 * kRegsCtl + 128 * kRegsUnpack + 256 * kRegsPromote <= 65536, "register budget");
+static_assert(kUnpackWarps % 4 == 0 && kUnpackWarps % kUnpackPerSlot == 0 && STAGES % kUnpackTeams == 0 &&
+              BC_CTA / kUnpackPerSlot >= 64, "widening teams");
+static_assert(kRegsTotal <= 65536, "register budget");
 
 struct W4Args {
   const float* s_tok;
@@ -154,7 +165,8 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const int pair_id = blockIdx.x >> 1;
   const int num_pairs = gridDim.x >> 1;
   const int num_tiles = p.m_blocks * p.n_blocks;
-  constexpr uint32_t kTmemCols = ACC_SLOTS * BT_PAIR;  // 512
+  constexpr uint32_t kTmemCols = 512;
+  static_assert(ACC_SLOTS * BT_PAIR <= 512 && BT_PAIR % 32 == 0, "accumulator slots");
 
   if (threadIdx.x == 0) {
     *abort_flag = 0;
@@ -162,14 +174,14 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(bar_full + s * 8, 1);
       mbar_init(bar_empty + s * 8, 1);    // the MMAs' commit: by then the widening has read the stage too
-      mbar_init(bar_w8_full + s * 8, 2);  // one widening warp in each CTA
+      mbar_init(bar_w8_full + s * 8, 2 * kUnpackPerSlot);  // the slot's widening warps in each CTA
     }
     for (int s = 0; s < P_SLOTS; ++s) {
       mbar_init(bar_p_full + s * 8, 1);
-      mbar_init(bar_p_empty + s * 8, 1);
+      mbar_init(bar_p_empty + s * 8, kUnpackPerSlot);
     }
     for (int s = 0; s < SC_SLOTS; ++s) {
-      mbar_init(bar_sc_full + s * 8, 1);
+      mbar_init(bar_sc_full + s * 8, kUnpackPerSlot);
       mbar_init(bar_sc_empty + s * 8, kPromoteWarps);
     }
     for (int s = 0; s < ACC_SLOTS; ++s) {
@@ -258,15 +270,17 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       }
       (void)ok;
     }
-  } else if (warp < 8) {
-    // ------------------------------------------------------------ widen nibbles (warps 4..7)
+  } else if (warp < kFirstPromote) {
+    // ------------------------------------------------------------ widen nibbles
     setmaxnreg_dec<kRegsUnpack>();
-    const uint32_t s = static_cast<uint32_t>(warp - 4);     // this warp's stage and widened slot
+    const uint32_t team = static_cast<uint32_t>(warp - 4) / kUnpackPerSlot;
+    const int sub = (warp - 4) % kUnpackPerSlot;                               // its share of the slot's 128 rows
+    constexpr int kRows = BC_CTA / kUnpackPerSlot;
     const uint32_t w8_full0 = mapa_u32(bar_w8_full, 0);
-    uint8_t* w8 = smem + kW8Off + s * kW8Bytes;
     const int total = pair_id < num_tiles ? ((num_tiles - pair_id + num_pairs - 1) / num_pairs) * p.k_blocks : 0;
-    for (uint32_t it = s; it < static_cast<uint32_t>(total); it += kUnpackWarps) {
-      const uint32_t ph = (it / STAGES) & 1u;
+    for (uint32_t it = team; it < static_cast<uint32_t>(total); it += kUnpackTeams) {
+      const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;   // the group's code stage and widened slot
+      uint8_t* w8 = smem + kW8Off + s * kW8Bytes;
       const uint32_t v = it % SC_SLOTS, vph = (it / SC_SLOTS) & 1u;
       const uint32_t ps = it % P_SLOTS, pph = (it / P_SLOTS) & 1u;
       // packed weights landed; the widened slot's previous MMAs are done; the scale row has been read
@@ -274,26 +288,33 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                                 wc);
       if (!__all_sync(0xffffffffu, w)) break;
       const uint8_t* pslot = smem + kPOff + ps * kPSlotBytes;
-      const uint4* packed = reinterpret_cast<const uint4*>(pslot);
-#pragma unroll 4
-      for (int i = 0; i < (BC_CTA * 4) / 32; ++i) {
-        const int idx = lane + i * 32;
-        const int r = idx >> 2, j = idx & 3;  // channel row of this CTA, 32-k run of the group
-        const uint4 w4 = packed[idx];
-        uint4 lo, hi;
-        lo.x = (w4.x << 4) & 0xF0F0F0F0u; hi.x = w4.x & 0xF0F0F0F0u;
-        lo.y = (w4.y << 4) & 0xF0F0F0F0u; hi.y = w4.y & 0xF0F0F0F0u;
-        lo.z = (w4.z << 4) & 0xF0F0F0F0u; hi.z = w4.z & 0xF0F0F0F0u;
-        lo.w = (w4.w << 4) & 0xF0F0F0F0u; hi.w = w4.w & 0xF0F0F0F0u;
-        uint8_t* row = w8 + r * 128;
-        const int sw = r & 7;  // 128-byte swizzle: 16-byte chunk index XOR (row mod 8)
-        *reinterpret_cast<uint4*>(row + (((2 * j) ^ sw) << 4)) = lo;       // k = 32j .. 32j+15
-        *reinterpret_cast<uint4*>(row + (((2 * j + 1) ^ sw) << 4)) = hi;   // k = 32j+16 .. 32j+31
-      }
-      const __half2* sh = reinterpret_cast<const __half2*>(pslot + kPBytes);
-      float2* sc = reinterpret_cast<float2*>(smem + kScOff + v * BC_CTA * 4);
+      const uint4* packed = reinterpret_cast<const uint4*>(pslot) + sub * kRows * 4;
+      // Lane l owns the 32-k run (l & 3) of the channel rows (l >> 2) + 8 i, i = 0..15: its row's swizzle
+      // term is one constant.  kWidenBatch loads are in flight before the first result is stored.
+      const int j = lane & 3, sw = (lane >> 2) & 7;
+      uint8_t* row0 = w8 + (sub * kRows + (lane >> 2)) * 128;
+      const int off_lo = ((2 * j) ^ sw) << 4, off_hi = ((2 * j + 1) ^ sw) << 4;
+#pragma unroll 1
+      for (int b = 0; b < (kRows * 4) / 32; b += kWidenBatch) {
+        uint4 w4[kWidenBatch];
 #pragma unroll
-      for (int i = 0; i < BC_CTA / 64; ++i) {
+        for (int i = 0; i < kWidenBatch; ++i) w4[i] = packed[lane + (b + i) * 32];
+#pragma unroll
+        for (int i = 0; i < kWidenBatch; ++i) {
+          uint4 lo, hi;
+          lo.x = (w4[i].x << 4) & 0xF0F0F0F0u; hi.x = w4[i].x & 0xF0F0F0F0u;
+          lo.y = (w4[i].y << 4) & 0xF0F0F0F0u; hi.y = w4[i].y & 0xF0F0F0F0u;
+          lo.z = (w4[i].z << 4) & 0xF0F0F0F0u; hi.z = w4[i].z & 0xF0F0F0F0u;
+          lo.w = (w4[i].w << 4) & 0xF0F0F0F0u; hi.w = w4[i].w & 0xF0F0F0F0u;
+          uint8_t* row = row0 + (b + i) * (8 * 128);   // 128-byte swizzle: 16-byte chunk index XOR (row mod 8)
+          *reinterpret_cast<uint4*>(row + off_lo) = lo;   // k = 32j .. 32j+15
+          *reinterpret_cast<uint4*>(row + off_hi) = hi;   // k = 32j+16 .. 32j+31
+        }
+      }
+      const __half2* sh = reinterpret_cast<const __half2*>(pslot + kPBytes) + sub * (kRows / 2);
+      float2* sc = reinterpret_cast<float2*>(smem + kScOff + v * BC_CTA * 4) + sub * (kRows / 2);
+#pragma unroll
+      for (int i = 0; i < kRows / 64; ++i) {
         const float2 f = __half22float2(sh[lane + 32 * i]);
         sc[lane + 32 * i] = make_float2(f.x * 0.0625f, f.y * 0.0625f);
       }
@@ -312,8 +333,8 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     grid_dep_wait();                    // token scales come from the preceding kernel; Y is overwritten
     constexpr int HT = BT_PAIR / 2;     // token columns per promotion warp
     constexpr int LC = 16;              // token columns per tcgen05.ld (the next one is in flight during the arithmetic)
-    constexpr int CH = 32, NLD = HT / CH;   // tokens per stored box
-    const int pw = warp - 8;
+    constexpr int CH = kOutTok, NLD = HT / CH;   // tokens per stored box
+    const int pw = warp - kFirstPromote;
     const int quad = warp & 3;          // TMEM lanes 32*quad .. are this warp's: 32 output channels
     const int half = pw >> 2;           // which 128 of the tile's 256 tokens
     const int c_local = quad * 32 + lane;
@@ -468,7 +489,7 @@ int launch_w4(const CUtensorMap& tq, const W4Maps& maps, const W4Args& a, cudaSt
   static const int regs_ok = [kern] {
     cudaFuncAttributes fa;
     if (cudaFuncGetAttributes(&fa, kern) != cudaSuccess) return -1;
-    return fa.numRegs * kNumThreads >= 128 * kRegsCtl + 128 * kRegsUnpack + 256 * kRegsPromote ? 1 : 0;
+    return fa.numRegs * kNumThreads >= kRegsTotal ? 1 : 0;
   }();
   if (regs_ok <= 0) {
     cudaGetLastError();
@@ -516,7 +537,7 @@ int launch_gemm_w4a8_group(const int8_t* q, const float* s_tok, int count, const
     if (acc_g == nullptr) {
       rc = make_tmap_2d(&maps.s[g], s_grp[src], static_cast<uint64_t>(K / 128), static_cast<uint64_t>(N[src]), 1, BC_CTA, 2, 0);
       if (rc != PQ_OK) return rc;
-      rc = make_tmap_2d(&maps.y[g], y[src], static_cast<uint64_t>(M), static_cast<uint64_t>(N[src]), 32, 32, 2, 64);
+      rc = make_tmap_2d(&maps.y[g], y[src], static_cast<uint64_t>(M), static_cast<uint64_t>(N[src]), kOutTok, 32, 2, 64);
     } else {
       rc = make_tmap_2d(&maps.s[g], q, static_cast<uint64_t>(M), static_cast<uint64_t>(K / 2), 1, BC_CTA, 2, 0);
       maps.y[g] = tq;  // not used by the accumulator export
