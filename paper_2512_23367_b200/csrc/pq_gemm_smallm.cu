@@ -42,7 +42,7 @@ struct Cfg {
   static constexpr int kTxBytes = kWBytes + kQBytes + kSBytes;
   // Short rings and small footprints: three or four CTAs fit on an SM, so the CTAs of the NEXT
   // launch become resident (and stream their weights) while this launch reduces and stores.
-  static constexpr int STAGES = (kW4 && MPAD > 64) ? 6 : (MPAD == 64 ? 4 : 3);
+  static constexpr int STAGES = (kW4 && MPAD > 64) ? 6 : ((kW4 || MPAD == 64) ? 4 : 3);
   // W4: two pairs of widening warps, except at 64 tokens (that variant needs its registers for the 64
   // per-thread partial results and keeps one pair and two co-resident CTAs).  At 128 tokens one CTA
   // owns the SM: a six-deep ring, four widened slots, eight epilogue warps.
@@ -64,6 +64,10 @@ struct Cfg {
   static constexpr int kRingEnd = kScOff + SC_SLOTS * BW * 4;
   static constexpr int kRedBytes = MPAD * BW * 4;                // aliases the stage ring
   static constexpr int kBarOff = (kRingEnd > kRedBytes ? kRingEnd : kRedBytes);
+  // A barrier's phases are told apart by one parity bit, so a warp may only wait on barriers whose every
+  // phase it sees in turn: with two widening pairs alternating over the K blocks, each ring's length is even.
+  static_assert(!kW4 || (STAGES % kUnpackPairs == 0 && A8_SLOTS % kUnpackPairs == 0 && SC_SLOTS % kUnpackPairs == 0),
+                "ring lengths and widening pairs");
   static constexpr int kNumBars = 2 * STAGES + 2 * A8_SLOTS + 2 * SC_SLOTS + 2 * ACC_SLOTS + 1;   // + the MMA issuer's drain barrier
   static constexpr int kMiscOff = kBarOff + kNumBars * 8;
   // A CTA that takes all 512 TMEM columns must be alone on its SM (a second one would block in

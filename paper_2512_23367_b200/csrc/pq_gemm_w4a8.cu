@@ -25,12 +25,12 @@
 //
 // Warp roles (512 threads; register budgets moved with setmaxnreg):
 //   warp 0        TMA producer of the token codes: a ring of four 16 KB stages, freed by the MMAs
-//   warp 2        TMA producer of packed weights + scales: a ring of its own (six slots of 8.25 KB), freed
+//   warp 2        TMA producer of packed weights + scales: a ring of its own (four slots of 8.25 KB), freed
 //                 by the widening, so that it runs ahead of the MMAs and -- these being constants of the
 //                 model -- ahead of the wait on the preceding kernel.  (With one ring for everything the
 //                 loop load -> widen -> MMA -> free bounded the kernel: 64.2 against 59.6 us.)
 //   warp 1        MMA issuer (leader CTA only; owns TMEM allocation in both CTAs).  It shares its
-//                 scheduler with busy warps, so it is kept to two waits, four MMAs and two commits
+//                 scheduler with busy warps, so it is kept to two waits, four MMAs and three commits
 //                 per group: "widened" (which implies "codes landed": the widening warp waits for the
 //                 stage's barrier before it signals) and "accumulator free"
 //   warps 4-7     widen nibbles -> INT8 (16 x code: the nibble sits in the high half of the byte,
@@ -49,12 +49,13 @@ namespace {
 
 // Tokens per tile (MMA N, TMEM columns) / per CTA.  Narrower tiles give a deeper accumulator ring (512
 // columns / BT_PAIR slots) but measured slower: 2048 x 4096 x 4096 takes 57 us at 256, 68 us at 160 and
-// 77 us at 128 tokens, with four or eight widening warps alike.
+// 77 us at 128 tokens, with four or eight widening warps and with deeper code and weight rings alike.
 constexpr int BT_PAIR = 256, BT_CTA = BT_PAIR / 2;
 constexpr int BC_CTA = 128, BC_PAIR = 256;   // output channels per CTA (TMEM lanes) / per tile (MMA M)
 constexpr int BK = 128, UMMA_K = 32;
-constexpr int STAGES = 4;       // token-code stages; also the widened-weight slots
-constexpr int P_SLOTS = 6;      // packed weights + FP16 scales of a group: a ring of its own, freed by the widening
+constexpr int Q_STAGES = 4;     // token-code stages, freed by the MMAs
+constexpr int W8_SLOTS = 4;     // widened-weight slots, freed by the MMAs
+constexpr int P_SLOTS = 4;      // packed weights + FP16 scales of a group: a ring of its own, freed by the widening
 constexpr int SC_SLOTS = 8;     // FP32 scale rows (this CTA's 128 channels)
 constexpr int ACC_SLOTS = 512 / BT_PAIR;    // TMEM accumulators of BT_PAIR columns
 constexpr int kUnpackWarps = 4;                     // widening warps: kUnpackPerSlot share a group's 128 rows
@@ -77,17 +78,22 @@ constexpr int kPSlotBytes = kPBytes + kSBytes;  // a slot of the packed ring
 constexpr int kW8Bytes = BC_CTA * BK;           // 16 KB widened weights
 constexpr int kOutTok = BT_CTA % 32 == 0 ? 32 : 16;   // tokens per stored box
 constexpr int kOutBoxBytes = kOutTok * 32 * 2;
-constexpr int kW8Off = STAGES * kStageBytes;
-constexpr int kPOff = kW8Off + STAGES * kW8Bytes;
+constexpr int kW8Off = Q_STAGES * kStageBytes;
+constexpr int kPOff = kW8Off + W8_SLOTS * kW8Bytes;
 constexpr int kScOff = kPOff + P_SLOTS * kPSlotBytes;
 constexpr int kOutOff = kScOff + SC_SLOTS * BC_CTA * 4;
 constexpr int kBarOff = kOutOff + kPromoteWarps * kOutBufs * kOutBoxBytes;
-constexpr int kNumBars = 3 * STAGES + 2 * P_SLOTS + 2 * SC_SLOTS + 2 * ACC_SLOTS + 1;   // + the MMA issuer's drain barrier
+constexpr int kNumBars = 2 * Q_STAGES + 2 * W8_SLOTS + 2 * P_SLOTS + 2 * SC_SLOTS + 2 * ACC_SLOTS + 1;   // + the MMA issuer's drain barrier
 constexpr int kMiscOff = kBarOff + kNumBars * 8;
 constexpr int kDynamicSmem = kMiscOff + 16 + 1024;
 static_assert(kDynamicSmem <= 232448, "exceeds the shared memory of one CTA");
 static_assert(BK / UMMA_K == 4, "the MMA issuer is unrolled for four steps per group");
-static_assert(kUnpackWarps % 4 == 0 && kUnpackWarps % kUnpackPerSlot == 0 && STAGES % kUnpackTeams == 0 &&
+// A barrier's phases are told apart by one parity bit, so a warp may only wait on barriers whose every phase it
+// sees in turn: each ring's length is a multiple of the number of widening teams (team t then always meets the
+// same stages and slots).
+static_assert(Q_STAGES % kUnpackTeams == 0 && W8_SLOTS % kUnpackTeams == 0 && P_SLOTS % kUnpackTeams == 0 &&
+              SC_SLOTS % kUnpackTeams == 0, "ring lengths and widening teams");
+static_assert(kUnpackWarps % 4 == 0 && kUnpackWarps % kUnpackPerSlot == 0 &&
               BC_CTA / kUnpackPerSlot >= 64, "widening teams");
 static_assert(kRegsTotal <= 65536, "register budget");
 
@@ -146,9 +152,10 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t smem_base = smem_u32(smem);
   const uint32_t bar_full = smem_base + kBarOff;              // local: token codes landed
-  const uint32_t bar_empty = bar_full + STAGES * 8;           // local: the pair's MMAs of the group completed
-  const uint32_t bar_w8_full = bar_empty + STAGES * 8;        // LEADER: both CTAs' widened weights written
-  const uint32_t bar_p_full = bar_w8_full + STAGES * 8;       // local: packed weights and scales landed
+  const uint32_t bar_empty = bar_full + Q_STAGES * 8;         // local: the MMAs that read the code stage completed
+  const uint32_t bar_w8_full = bar_empty + Q_STAGES * 8;      // LEADER: both CTAs' widened weights written
+  const uint32_t bar_w8_empty = bar_w8_full + W8_SLOTS * 8;   // local: the MMAs that read the widened slot completed
+  const uint32_t bar_p_full = bar_w8_empty + W8_SLOTS * 8;    // local: packed weights and scales landed
   const uint32_t bar_p_empty = bar_p_full + P_SLOTS * 8;      // local: the widening warp has read them
   const uint32_t bar_sc_full = bar_p_empty + P_SLOTS * 8;     // local: FP32 scales written
   const uint32_t bar_sc_empty = bar_sc_full + SC_SLOTS * 8;   // local: promotion warps read them
@@ -171,10 +178,13 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   if (threadIdx.x == 0) {
     *abort_flag = 0;
     mbar_init(bar_drain, 1);
-    for (int s = 0; s < STAGES; ++s) {
+    for (int s = 0; s < Q_STAGES; ++s) {
       mbar_init(bar_full + s * 8, 1);
-      mbar_init(bar_empty + s * 8, 1);    // the MMAs' commit: by then the widening has read the stage too
+      mbar_init(bar_empty + s * 8, 1);    // the MMAs' commit
+    }
+    for (int s = 0; s < W8_SLOTS; ++s) {
       mbar_init(bar_w8_full + s * 8, 2 * kUnpackPerSlot);  // the slot's widening warps in each CTA
+      mbar_init(bar_w8_empty + s * 8, 1);                  // the MMAs' commit
     }
     for (int s = 0; s < P_SLOTS; ++s) {
       mbar_init(bar_p_full + s * 8, 1);
@@ -222,8 +232,8 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         const W4Tile t = locate_tile(p, tile);
         const int t0 = t.m_blk * BT_PAIR + static_cast<int>(rank) * BT_CTA;
         for (int g = 0; g < p.k_blocks; ++g, ++it) {
-          const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
-          if (it >= STAGES && !mbar_wait(bar_empty + s * 8, ph ^ 1u, wc)) { ok = false; break; }
+          const uint32_t s = it % Q_STAGES, ph = (it / Q_STAGES) & 1u;
+          if (it >= Q_STAGES && !mbar_wait(bar_empty + s * 8, ph ^ 1u, wc)) { ok = false; break; }
           mbar_arrive_expect_tx(bar_full + s * 8, kQBytes);
           tma_load_2d(smem_base + s * kStageBytes, &tm_q, bar_full + s * 8, g * BK, t0);
         }
@@ -253,20 +263,22 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       const int total = pair_id < num_tiles ? ((num_tiles - pair_id + num_pairs - 1) / num_pairs) * p.k_blocks : 0;   // groups of this pair
       bool ok = true;
       for (uint32_t it = 0; it < static_cast<uint32_t>(total); ++it) {
-        const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
+        const uint32_t sq = it % Q_STAGES;
+        const uint32_t sw = it % W8_SLOTS, wph = (it / W8_SLOTS) & 1u;
         const uint32_t a = it % ACC_SLOTS, aph = (it / ACC_SLOTS) & 1u;
         // Operands are prepared before the waits, and the wait most likely to open last comes last.
-        const uint64_t w_desc = umma_desc_k_sw128(smem_base + kW8Off + s * kW8Bytes);   // 256 channel rows (both CTAs)
-        const uint64_t q_desc = umma_desc_k_sw128(smem_base + s * kStageBytes);         // 256 token rows (both CTAs)
+        const uint64_t w_desc = umma_desc_k_sw128(smem_base + kW8Off + sw * kW8Bytes);   // 256 channel rows (both CTAs)
+        const uint64_t q_desc = umma_desc_k_sw128(smem_base + sq * kStageBytes);         // token rows of both CTAs
         const uint32_t d_tmem = tmem_base + a * BT_PAIR;
-        if (!mbar_wait2_cluster(bar_w8_full + s * 8, ph, bar_acc_empty + a * 8, aph ^ 1u, wc)) { ok = false; break; }
+        if (!mbar_wait2_cluster(bar_w8_full + sw * 8, wph, bar_acc_empty + a * 8, aph ^ 1u, wc)) { ok = false; break; }
         tc_fence_after_sync();
         umma_i8_pair_imm<0>(d_tmem, w_desc, q_desc, idesc);
         umma_i8_pair_imm<1>(d_tmem, w_desc + 2, q_desc + 2, idesc);
         umma_i8_pair_imm<1>(d_tmem, w_desc + 4, q_desc + 4, idesc);
         umma_i8_pair_imm<1>(d_tmem, w_desc + 6, q_desc + 6, idesc);
         umma_commit_pair_mcast(bar_acc_full + a * 8, 0x3);
-        umma_commit_pair_mcast(bar_empty + s * 8, 0x3);   // frees the stage and the widened slot in both CTAs
+        umma_commit_pair_mcast(bar_empty + sq * 8, 0x3);      // frees the code stage in both CTAs
+        umma_commit_pair_mcast(bar_w8_empty + sw * 8, 0x3);   // and the widened slot
       }
       (void)ok;
     }
@@ -279,12 +291,13 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     const uint32_t w8_full0 = mapa_u32(bar_w8_full, 0);
     const int total = pair_id < num_tiles ? ((num_tiles - pair_id + num_pairs - 1) / num_pairs) * p.k_blocks : 0;
     for (uint32_t it = team; it < static_cast<uint32_t>(total); it += kUnpackTeams) {
-      const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;   // the group's code stage and widened slot
+      const uint32_t sq = it % Q_STAGES, qph = (it / Q_STAGES) & 1u;   // the group's code stage
+      const uint32_t s = it % W8_SLOTS, ph = (it / W8_SLOTS) & 1u;     // and widened slot
       uint8_t* w8 = smem + kW8Off + s * kW8Bytes;
       const uint32_t v = it % SC_SLOTS, vph = (it / SC_SLOTS) & 1u;
       const uint32_t ps = it % P_SLOTS, pph = (it / P_SLOTS) & 1u;
       // packed weights landed; the widened slot's previous MMAs are done; the scale row has been read
-      const bool w = mbar_wait3(bar_p_full + ps * 8, pph, bar_empty + s * 8, ph ^ 1u, bar_sc_empty + v * 8, vph ^ 1u,
+      const bool w = mbar_wait3(bar_p_full + ps * 8, pph, bar_w8_empty + s * 8, ph ^ 1u, bar_sc_empty + v * 8, vph ^ 1u,
                                 wc);
       if (!__all_sync(0xffffffffu, w)) break;
       const uint8_t* pslot = smem + kPOff + ps * kPSlotBytes;
@@ -320,7 +333,7 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       }
       fence_proxy_async_smem();  // generic-proxy writes -> visible to the tensor-core (async) proxy
       // "widened" tells the MMA issuer that the group's codes are there too
-      if (!__all_sync(0xffffffffu, mbar_wait(bar_full + s * 8, ph, wc))) break;
+      if (!__all_sync(0xffffffffu, mbar_wait(bar_full + sq * 8, qph, wc))) break;
       if (lane == 0) {
         mbar_arrive_cluster_addr(w8_full0 + s * 8);
         mbar_arrive(bar_sc_full + v * 8);
@@ -460,8 +473,8 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     // done so before this CTA's shared and tensor memory go away: the producer's loads (their barriers
     // are local) and the leader's MMAs (they read both CTAs' shared memory and write both tensor memories).
     if (threadIdx.x == 0) {
-      const uint32_t first = issued > static_cast<uint32_t>(STAGES) ? issued - STAGES : 0u;
-      for (uint32_t i = first; i < issued; ++i) mbar_drain(bar_full + (i % STAGES) * 8, (i / STAGES) & 1u);
+      const uint32_t first = issued > static_cast<uint32_t>(Q_STAGES) ? issued - Q_STAGES : 0u;
+      for (uint32_t i = first; i < issued; ++i) mbar_drain(bar_full + (i % Q_STAGES) * 8, (i / Q_STAGES) & 1u);
     } else if (threadIdx.x == 64) {
       const uint32_t first = issued > static_cast<uint32_t>(P_SLOTS) ? issued - P_SLOTS : 0u;
       for (uint32_t i = first; i < issued; ++i) mbar_drain(bar_p_full + (i % P_SLOTS) * 8, (i / P_SLOTS) & 1u);
