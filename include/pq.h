@@ -276,7 +276,8 @@ PQ_API int pq_gemm_w8a8_group(const int8_t* q, const float* s_tok, int32_t count
                               int64_t K, void* workspace, size_t workspace_bytes, void* stream);
 
 /* The same for W4A8 linears (pq_gemm_w4a8 per member; one launch for all of them, except at M <= 128 when
- * the members together hold more 128-channel tiles than the device has SMs).  For M <= 128 the FP32
+ * the members together hold more 128-channel tiles than the device has SMs).  For M <= 128, and for M <= 256
+ * when the members' 128-channel tiles x 2 token blocks do not exceed the number of SMs, the FP32
  * group sums of the K parts are added in a fixed order, but the number of parts depends on how many tiles
  * the launch holds, so the grouped result may differ from the per-member call in the last FP32 bit. */
 PQ_API int pq_gemm_w4a8_group(const int8_t* q, const float* s_tok, int32_t count, const void* const* wp,

@@ -20,6 +20,8 @@ namespace {
 constexpr int kMaxDevices = 64;
 constexpr int64_t kSmallM = 128;     // W4A8: M at or below this takes the weight-streaming schedule
 constexpr int64_t kSmallM_W8 = 128;  // W8A8
+constexpr int64_t kStreamM_W4 = 256; // W4A8 above kSmallM: the weight-streaming schedule in blocks of 128 tokens, where every
+                                     // (128-channel tile, token block) pair gets an SM of its own (few, long tiles)
 
 // Facts about a device, filled in by the first call on it.  Host threads may make that first call
 // concurrently: the fill happens under a mutex and `probed` is published last.
@@ -427,6 +429,13 @@ int pq_acc_w8a8(const int8_t* q, const void* wq, int64_t M, int64_t N, int64_t K
   return gemm_w8a8_common(q, nullptr, wq, nullptr, M, N, K, nullptr, acc, nullptr, 0, stream);
 }
 
+// W4A8 between kSmallM and kStreamM_W4 tokens: the pair kernel's 256 x 256 tiles leave most SM pairs idle when
+// the linear is narrow (256 x 4096 -> 4096: 16 tiles, 30.9 us); the weight-streaming kernel splits K over
+// clusters instead.  `tiles` = 128-channel tiles of all members of the launch.
+static bool w4a8_streams_in_blocks(int64_t M, int64_t tiles) {
+  return M > kSmallM && M <= kStreamM_W4 && tiles * ((M + 127) / 128) <= sm_count();
+}
+
 static int gemm_w4a8_common(const int8_t* q, const float* s_tok, const void* wp, const void* s_grp, int32_t group,
                             int64_t M, int64_t N, int64_t K, void* y, int32_t* acc_g, void* stream) {
   int rc = check_gemm(M, N, K);
@@ -439,7 +448,7 @@ static int gemm_w4a8_common(const int8_t* q, const float* s_tok, const void* wp,
     log_dispatch("w4a8", "CUDA-core row kernel", M, N, K);
     return launch_gemv_rows_w4a8(q, s_tok, wp, s_grp, M, N, K, y, acc_g, st);
   }
-  if (M <= kSmallM) {
+  if (M <= kSmallM || w4a8_streams_in_blocks(M, (N + 127) / 128)) {
     log_dispatch("w4a8", "tensor-core weight streaming", M, N, K);
     return launch_smallm_w4a8(q, s_tok, wp, s_grp, M, N, K, y, acc_g, st);
   }
@@ -483,6 +492,13 @@ int pq_gemm_w4a8_group(const int8_t* q, const float* s_tok, int32_t count, const
     }
     return launch_smallm_w4a8_group(q, s_tok, count, wp, s_grp_f16, N, y_f16, M, K, nullptr,
                                     static_cast<cudaStream_t>(stream));
+  }
+  {
+    int64_t tiles = 0;
+    for (int g = 0; g < count; ++g) tiles += (N[g] + 127) / 128;
+    if (w4a8_streams_in_blocks(M, tiles))
+      return launch_smallm_w4a8_group(q, s_tok, count, wp, s_grp_f16, N, y_f16, M, K, nullptr,
+                                      static_cast<cudaStream_t>(stream));
   }
   return launch_gemm_w4a8_group(q, s_tok, count, wp, s_grp_f16, N, y_f16, M, K, nullptr,
                                 static_cast<cudaStream_t>(stream));

@@ -160,6 +160,8 @@ smallm_kernel(const __grid_constant__ SmallMaps maps, const __grid_constant__ CU
   const CUtensorMap* tm_w = &maps.w[member];
   const CUtensorMap* tm_s = &maps.s[member];
   const int split = blockIdx.y;                       // == rank in the cluster (cluster = all of grid.y)
+  const int m0 = static_cast<int>(blockIdx.z) * MPAD;  // first token of this CTA (grid.z runs over blocks of MPAD tokens)
+  const int m_live = p.M - m0 < MPAD ? p.M - m0 : MPAD;
   const int kb0 = static_cast<int>(static_cast<int64_t>(p.k_blocks) * split / p.splits);
   const int kb1 = static_cast<int>(static_cast<int64_t>(p.k_blocks) * (split + 1) / p.splits);
   const int nkb = kb1 - kb0;
@@ -177,7 +179,7 @@ smallm_kernel(const __grid_constant__ SmallMaps maps, const __grid_constant__ CU
   };
   auto issue_codes = [&](int j) {
     const uint32_t s = static_cast<uint32_t>(j) % C::STAGES;
-    tma_load_2d(smem_base + s * C::kStageBytes + C::kWBytes, &tm_q, bar_full + s * 8, (kb0 + j) * BK, 0);
+    tma_load_2d(smem_base + s * C::kStageBytes + C::kWBytes, &tm_q, bar_full + s * 8, (kb0 + j) * BK, m0);
   };
 
   if (threadIdx.x == 64) {
@@ -354,8 +356,8 @@ smallm_kernel(const __grid_constant__ SmallMaps maps, const __grid_constant__ CU
             const int n = n0 + n_local;
 #pragma unroll
             for (int m = 0; m < CH; ++m) {
-              if (col0 + c0 + m < p.M && n < N_mem)
-                p.acc[(static_cast<int64_t>(kb0 + j) * p.M + col0 + c0 + m) * N_mem + n] = static_cast<int32_t>(r[m]) >> 4;
+              if (col0 + c0 + m < m_live && n < N_mem)
+                p.acc[(static_cast<int64_t>(kb0 + j) * p.M + m0 + col0 + c0 + m) * N_mem + n] = static_cast<int32_t>(r[m]) >> 4;
             }
           } else {
 #pragma unroll
@@ -435,7 +437,7 @@ smallm_kernel(const __grid_constant__ SmallMaps maps, const __grid_constant__ CU
 #pragma unroll
       for (int j = 0; j < 4; ++j) sc[j] = __ldg(s_ch_mem + n + j);   // N is a multiple of 8: n < N covers n + 3
     }
-    for (int m = static_cast<int>(my_rank) + p.splits * msub; m < p.M; m += C::kEpiWarps * p.splits) {
+    for (int m = static_cast<int>(my_rank) + p.splits * msub; m < m_live; m += C::kEpiWarps * p.splits) {
       const uint32_t addr = smem_base + static_cast<uint32_t>(m * BW + 4 * nq) * 4u;
       uint4 part[kMaxSplit];
 #pragma unroll
@@ -452,9 +454,9 @@ smallm_kernel(const __grid_constant__ SmallMaps maps, const __grid_constant__ CU
             tot[2] += __uint_as_float(part[r].z); tot[3] += __uint_as_float(part[r].w);
           }
         }
-        const float st = __ldg(p.s_tok + m);
+        const float st = __ldg(p.s_tok + m0 + m);
         const __half2 h01 = __floats2half2_rn(tot[0] * st, tot[1] * st), h23 = __floats2half2_rn(tot[2] * st, tot[3] * st);
-        *reinterpret_cast<uint2*>(y_mem + static_cast<int64_t>(m) * N_mem + n) =
+        *reinterpret_cast<uint2*>(y_mem + static_cast<int64_t>(m0 + m) * N_mem + n) =
             make_uint2(*reinterpret_cast<const uint32_t*>(&h01), *reinterpret_cast<const uint32_t*>(&h23));
       } else {
         int32_t tot[4] = {0, 0, 0, 0};
@@ -466,14 +468,14 @@ smallm_kernel(const __grid_constant__ SmallMaps maps, const __grid_constant__ CU
           }
         }
         if constexpr (kExportAcc) {
-          *reinterpret_cast<int4*>(p.acc + static_cast<int64_t>(m) * N_mem + n) = make_int4(tot[0], tot[1], tot[2], tot[3]);
+          *reinterpret_cast<int4*>(p.acc + static_cast<int64_t>(m0 + m) * N_mem + n) = make_int4(tot[0], tot[1], tot[2], tot[3]);
         } else {
-          const float st = __ldg(p.s_tok + m);
+          const float st = __ldg(p.s_tok + m0 + m);
           float v[4];
 #pragma unroll
           for (int j = 0; j < 4; ++j) v[j] = __fmul_rn(__fmul_rn(__int2float_rn(tot[j]), st), sc[j]);
           const __half2 h01 = __floats2half2_rn(v[0], v[1]), h23 = __floats2half2_rn(v[2], v[3]);
-          *reinterpret_cast<uint2*>(y_mem + static_cast<int64_t>(m) * N_mem + n) =
+          *reinterpret_cast<uint2*>(y_mem + static_cast<int64_t>(m0 + m) * N_mem + n) =
               make_uint2(*reinterpret_cast<const uint32_t*>(&h01), *reinterpret_cast<const uint32_t*>(&h23));
         }
       }
@@ -490,13 +492,14 @@ smallm_kernel(const __grid_constant__ SmallMaps maps, const __grid_constant__ CU
 }
 
 template <int MPAD, bool kW4, bool kExportAcc>
-int launch_cfg(const SmallMaps& maps, const CUtensorMap& tq, const SmallArgs& a, int n_tiles, cudaStream_t stream) {
+int launch_cfg(const SmallMaps& maps, const CUtensorMap& tq, const SmallArgs& a, int n_tiles, int m_blocks,
+               cudaStream_t stream) {
   using C = Cfg<MPAD, kW4>;
   auto kern = smallm_kernel<MPAD, kW4, kExportAcc>;
   static PerDeviceOnce once;   // one per kernel variant
   if (const int rc = set_dynamic_smem_once(once, kern, C::kDynamic); rc != PQ_OK) return rc;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(static_cast<unsigned>(n_tiles), static_cast<unsigned>(a.splits), 1);
+  cfg.gridDim = dim3(static_cast<unsigned>(n_tiles), static_cast<unsigned>(a.splits), static_cast<unsigned>(m_blocks));
   cfg.blockDim = dim3(C::kThreads, 1, 1);
   cfg.dynamicSmemBytes = C::kDynamic;
   cfg.stream = stream;
@@ -520,6 +523,7 @@ int launch_smallm(const int8_t* q, const float* s_tok, int count, const void* co
                   cudaStream_t stream) {
   if (count < 1 || count > kMaxGroup || (acc != nullptr && count != 1)) return PQ_ERR_SHAPE;
   const int mpad = M <= 16 ? 16 : (M <= 32 ? 32 : (M <= 64 ? 64 : 128));
+  const int m_blocks = static_cast<int>((M + mpad - 1) / mpad);   // > 1 only beyond 128 tokens
   const int k_blocks = static_cast<int>((K + BK - 1) / BK);
 
   CUtensorMap tq;
@@ -554,14 +558,15 @@ int launch_smallm(const int8_t* q, const float* s_tok, int count, const void* co
   if (n_tiles > 0x3fffffff) return PQ_ERR_SHAPE;
 
   // Aim at two resident CTAs per SM; the split is the cluster size (<= 8) and <= K blocks.
-  int splits = static_cast<int>((2 * sm_count()) / n_tiles);
+  const int64_t units = n_tiles * m_blocks;   // (channel tile, token block) pairs, each split over a cluster
+  int splits = static_cast<int>((2 * sm_count()) / units);
   splits = splits < 1 ? 1 : (splits > kMaxSplit ? kMaxSplit : splits);
   // Variants with two CTAs per SM have no room to spare: a cluster has to fit one GPC, so a grid that
   // nearly fills the device leaves clusters for a second wave (2048 -> 6144 at M = 64: 12.8 us with
   // clusters of 6, 7.4 us with clusters of 4).  Stay below 90 % of the resident capacity, and off the
   // cluster sizes 5 and 7.
   const int ctas_per_sm = (kW4 && mpad > 64) ? 1 : (mpad >= 64 ? 2 : (kW4 ? 2 : 4));
-  while (splits > 1 && n_tiles * splits * 10 > static_cast<int64_t>(ctas_per_sm) * sm_count() * 9) --splits;
+  while (splits > 1 && units * splits * 10 > static_cast<int64_t>(ctas_per_sm) * sm_count() * 9) --splits;
   if (splits == 5 || splits == 7) --splits;
   // ablation knob, read once: force the number of K parts (cluster size)
   static const int force_splits = [] { const char* e = getenv("PQ_SMALLM_SPLITS"); return e ? atoi(e) : 0; }();
@@ -581,10 +586,10 @@ int launch_smallm(const int8_t* q, const float* s_tok, int count, const void* co
   const bool ex = acc != nullptr;
   const int nt = static_cast<int>(n_tiles);
   switch (mpad) {
-    case 16: return ex ? launch_cfg<16, kW4, true>(maps, tq, a, nt, stream) : launch_cfg<16, kW4, false>(maps, tq, a, nt, stream);
-    case 32: return ex ? launch_cfg<32, kW4, true>(maps, tq, a, nt, stream) : launch_cfg<32, kW4, false>(maps, tq, a, nt, stream);
-    case 64: return ex ? launch_cfg<64, kW4, true>(maps, tq, a, nt, stream) : launch_cfg<64, kW4, false>(maps, tq, a, nt, stream);
-    default: return ex ? launch_cfg<128, kW4, true>(maps, tq, a, nt, stream) : launch_cfg<128, kW4, false>(maps, tq, a, nt, stream);
+    case 16: return ex ? launch_cfg<16, kW4, true>(maps, tq, a, nt, m_blocks, stream) : launch_cfg<16, kW4, false>(maps, tq, a, nt, m_blocks, stream);
+    case 32: return ex ? launch_cfg<32, kW4, true>(maps, tq, a, nt, m_blocks, stream) : launch_cfg<32, kW4, false>(maps, tq, a, nt, m_blocks, stream);
+    case 64: return ex ? launch_cfg<64, kW4, true>(maps, tq, a, nt, m_blocks, stream) : launch_cfg<64, kW4, false>(maps, tq, a, nt, m_blocks, stream);
+    default: return ex ? launch_cfg<128, kW4, true>(maps, tq, a, nt, m_blocks, stream) : launch_cfg<128, kW4, false>(maps, tq, a, nt, m_blocks, stream);
   }
 }
 

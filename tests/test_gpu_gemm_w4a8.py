@@ -69,6 +69,8 @@ def test_tiny_linear_every_element(M):
     (128, 128, 128), (130, 264, 256), (257, 520, 1024), (65, 8, 128), (300, 1024, 4096),
     (129, 136, 11008), (512, 256, 384), (96, 4096, 512), (1, 256, 512), (64, 384, 1280),
     (128, 4096, 4096), (100, 11008, 1024), (65, 1000, 11008), (113, 4096, 11008),
+    # 129..256 tokens: narrow linears stream their weights in two token blocks, wide ones stay on the pair kernel
+    (200, 4096, 1024), (256, 1152, 4224), (129, 4096, 384), (130, 9608, 256), (200, 9736, 384),
 ])
 def test_shapes_spanning_tiles_and_ragged_tails(M, N, K):
     run_case(M, N, K, seed=M + N + K)

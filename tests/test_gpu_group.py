@@ -125,7 +125,7 @@ def test_w4a8_group_equals_one_call_per_member_and_the_oracle(M, K, Ns):
 @pytest.mark.parametrize("M,K,Ns", [(1, 512, (256, 520)), (16, 512, (256, 520)), (64, 512, (256, 520)),
                                     (3, 4224, (2376, 136, 8)), (33, 1024, (128, 128, 128, 264)),
                                     (7, 4096, (4096, 4096, 4096)), (65, 128, (16, 24)), (100, 1024, (1408, 520)),
-                                    (128, 4096, (4096, 4096, 4096))])
+                                    (128, 4096, (4096, 4096, 4096)), (200, 1024, (1408, 520)), (256, 4096, (4096, 4096))])
 def test_w4a8_small_token_counts_group_on_the_weight_streaming_kernel(M, K, Ns):
     """Decode-shaped W4A8 sums its K parts in FP32 in a fixed order, but the number of parts depends on
     how many tiles the launch holds: the grouped result may differ from the per-member call in the last
