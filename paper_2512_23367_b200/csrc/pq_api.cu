@@ -20,7 +20,7 @@ namespace {
 constexpr int kMaxDevices = 64;
 constexpr int64_t kSmallM = 128;     // W4A8: M at or below this takes the weight-streaming schedule
 constexpr int64_t kSmallM_W8 = 128;  // W8A8
-constexpr int64_t kStreamM_W4 = 256; // W4A8 above kSmallM: the weight-streaming schedule in blocks of 128 tokens, where every
+constexpr int64_t kStreamM = 256;    // above the limits above: the weight-streaming schedule in blocks of 128 tokens, where every
                                      // (128-channel tile, token block) pair gets an SM of its own (few, long tiles)
 
 // Facts about a device, filled in by the first call on it.  Host threads may make that first call
@@ -374,6 +374,13 @@ int pq_unpack_w4(const void* wp, int64_t N, int64_t K, int8_t* codes, void* stre
 
 static bool aligned256(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
 
+// 129..256 tokens: a narrow linear gives the pair kernel few 256 x 256 tiles (256 x 4096 -> 4096: 16 on 74 SM
+// pairs); the weight-streaming kernel takes it in two token blocks and splits K over clusters instead.
+// `tiles` = 128-channel tiles of all members of the launch.
+static bool w8a8_streams_in_blocks(int64_t M, int64_t tiles) {
+  return M > kSmallM_W8 && M <= kStreamM && tiles * ((M + 127) / 128) <= sm_count();
+}
+
 static int gemm_w8a8_common(const int8_t* q, const float* s_tok, const void* wq, const float* s_ch, int64_t M,
                             int64_t N, int64_t K, void* y, int32_t* acc, void* workspace, size_t workspace_bytes,
                             void* stream) {
@@ -388,7 +395,7 @@ static int gemm_w8a8_common(const int8_t* q, const float* s_tok, const void* wq,
     log_dispatch("w8a8", "CUDA-core row kernel", M, N, K);
     return launch_gemv_rows_w8a8(q, s_tok, wq, s_ch, M, N, K, y, acc, st);
   }
-  if (M <= kSmallM_W8) {
+  if (M <= kSmallM_W8 || w8a8_streams_in_blocks(M, (N + 127) / 128)) {
     log_dispatch("w8a8", "tensor-core weight streaming", M, N, K);
     return launch_smallm_w8a8(q, s_tok, wq, s_ch, M, N, K, y, acc, st);
   }
@@ -416,7 +423,9 @@ int pq_gemm_w8a8_group(const int8_t* q, const float* s_tok, int32_t count, const
   if (!aligned16(q) || !aligned256(workspace)) return PQ_ERR_ALIGN;
   int rc = check_arch();
   if (rc != PQ_OK) return rc;
-  if (M <= kSmallM_W8) {
+  int64_t tiles = 0;
+  for (int g = 0; g < count; ++g) tiles += (N[g] + 127) / 128;
+  if (M <= kSmallM_W8 || w8a8_streams_in_blocks(M, tiles)) {
     return launch_smallm_w8a8_group(q, s_tok, count, wq, s_ch, N, y_f16, M, K, nullptr,
                                     static_cast<cudaStream_t>(stream));
   }
@@ -429,11 +438,11 @@ int pq_acc_w8a8(const int8_t* q, const void* wq, int64_t M, int64_t N, int64_t K
   return gemm_w8a8_common(q, nullptr, wq, nullptr, M, N, K, nullptr, acc, nullptr, 0, stream);
 }
 
-// W4A8 between kSmallM and kStreamM_W4 tokens: the pair kernel's 256 x 256 tiles leave most SM pairs idle when
+// W4A8 between kSmallM and kStreamM tokens: the pair kernel's 256 x 256 tiles leave most SM pairs idle when
 // the linear is narrow (256 x 4096 -> 4096: 16 tiles, 30.9 us); the weight-streaming kernel splits K over
 // clusters instead.  `tiles` = 128-channel tiles of all members of the launch.
 static bool w4a8_streams_in_blocks(int64_t M, int64_t tiles) {
-  return M > kSmallM && M <= kStreamM_W4 && tiles * ((M + 127) / 128) <= sm_count();
+  return M > kSmallM && M <= kStreamM && tiles * ((M + 127) / 128) <= sm_count();
 }
 
 static int gemm_w4a8_common(const int8_t* q, const float* s_tok, const void* wp, const void* s_grp, int32_t group,
@@ -530,6 +539,11 @@ size_t pq_workspace_bytes(int64_t M, const int64_t* N, int32_t count, int64_t K,
     if (check_gemm(M, N[g], K) != PQ_OK) return 0;
   }
   if (M <= kSmallM_W8) return 0;   // the weight-streaming schedule reduces inside the SMs
+  if (M <= kStreamM) {             // ... and so it does in two token blocks, for narrow linears
+    int64_t tiles = 0;
+    for (int g = 0; g < count; ++g) tiles += (N[g] + 127) / 128;
+    if (tiles * ((M + 127) / 128) <= sms) return 0;
+  }
   int bn = 256, sp = 1;
   // the schedule chosen when room is no constraint
   if (plan_w8a8_pair_group(M, N, count, K, sms, ~size_t(0), 0, 0, &bn, &sp) < 0 || sp <= 1) return 0;

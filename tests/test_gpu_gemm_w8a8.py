@@ -67,6 +67,8 @@ def test_config1_tiny_linear_every_element():
 @pytest.mark.parametrize("M,N,K", [
     (128, 256, 128), (130, 264, 144), (257, 520, 1040), (200, 384, 2048), (65, 8, 16),
     (300, 1024, 4096), (129, 136, 11008), (512, 256, 256), (96, 4096, 512),
+    # 129..256 tokens: narrow linears stream their weights in two token blocks, wide ones stay on the pair kernel
+    (256, 4096, 1024), (200, 1152, 4224), (130, 9608, 256), (200, 9736, 384),
 ])
 def test_shapes_spanning_tiles_and_ragged_tails(M, N, K):
     run_case(M, N, K, seed=M + N + K)
@@ -127,7 +129,7 @@ def test_full_size_layers_touch_every_tile(M, K, N):
     run_case(M, N, K, seed=2000 + N % 97, rows=rows, cols=cols)
 
 
-@pytest.mark.parametrize("M,K,N", [(512, 11008, 1024), (300, 11008, 520), (140, 6144, 136), (257, 8192, 264)])
+@pytest.mark.parametrize("M,K,N", [(512, 11008, 1024), (300, 11008, 520), (260, 6144, 136), (257, 8192, 264)])
 def test_split_k_through_scratch_matches_the_unsplit_result_bit_for_bit(M, K, N):
     """Few tiles and a long K: given a workspace the GEMM cuts K into parts and sums the INT32 partials
     exactly, so the FP16 output must equal the one computed without a workspace, twice in a row (the

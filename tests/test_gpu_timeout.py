@@ -23,7 +23,7 @@ def _case(kind):
     """-> (call() -> y, reinit(), check(y)) on one small shape per kernel; check compares a few token rows
     with the oracle."""
     M, K, N = {"w8a8_pair": (300, 1024, 520), "w8a8_pair_split_k": (512, 11008, 1024), "w8a8_noalloc": (512, 11008, 1024),
-               "w8a8_small_m": (16, 2048, 1024), "w4a8_pair": (300, 1024, 520), "w4a8_small_m": (16, 2048, 1024), "w4a8_small_m_128": (100, 2048, 1024), "w4a8_small_m_blocks": (200, 2048, 1024),
+               "w8a8_small_m": (16, 2048, 1024), "w8a8_small_m_blocks": (200, 2048, 1024), "w4a8_pair": (300, 1024, 520), "w4a8_small_m": (16, 2048, 1024), "w4a8_small_m_128": (100, 2048, 1024), "w4a8_small_m_blocks": (200, 2048, 1024),
                "w8a8_rows": (3, 2048, 1024), "w4a8_rows": (2, 2048, 1024)}[kind]
     x, w = synth.activations(M, K, 31), synth.weights(N, K, 32)
     q, s_tok = pq.pq_quantize_act(torch.from_numpy(x).to(DEV))
@@ -54,7 +54,7 @@ def _case(kind):
             (lambda: ws is not None and pq.pq_workspace_init(ws)), check)
 
 
-@pytest.mark.parametrize("kind", ["w8a8_pair", "w8a8_pair_split_k", "w8a8_noalloc", "w8a8_small_m", "w4a8_pair", "w4a8_small_m", "w4a8_small_m_128", "w4a8_small_m_blocks",
+@pytest.mark.parametrize("kind", ["w8a8_pair", "w8a8_pair_split_k", "w8a8_noalloc", "w8a8_small_m", "w8a8_small_m_blocks", "w4a8_pair", "w4a8_small_m", "w4a8_small_m_128", "w4a8_small_m_blocks",
                                   "w8a8_rows", "w4a8_rows"])
 def test_a_wait_that_runs_out_is_reported_and_leaves_everything_usable(kind):
     call, reinit, check = _case(kind)
