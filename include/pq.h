@@ -262,8 +262,9 @@ PQ_API int pq_acc_w4a8(const int8_t* q, const void* wp, int32_t group, int64_t M
  * Several W8A8 linears over the SAME quantized tokens (the q/k/v projections, or gate and up, of
  * the layers the paper quantizes) as one call.  Result: exactly what `count` calls of pq_gemm_w8a8
  * with (wq[g], s_ch[g], N[g], y_f16[g]) give, bit for bit.  The members' output tiles are scheduled
- * together in a single kernel launch (of the prefill kernel for M > 128, of the weight-streaming
- * kernel below), which fills the SMs' waves across the members and pays the per-launch fixed cost
+ * together in a single kernel launch (of the weight-streaming kernel up to 128 tokens, and up to 256
+ * where the members' 128-channel tiles x 2 token blocks do not exceed the number of SMs; of the
+ * prefill kernel otherwise), which fills the SMs' waves across the members and pays the per-launch fixed cost
  * once -- at decode-shaped token counts that fixed cost is most of a call.
  *   count: 1..PQ_MAX_GROUP.  wq, s_ch, N, y_f16: HOST arrays of `count` entries (device pointers
  *   and column counts; read during the call, not retained).  q, s_tok, M, K as in pq_gemm_w8a8.
@@ -291,7 +292,8 @@ PQ_API int pq_gemm_w4a8_group(const int8_t* q, const float* s_tok, int32_t count
  *     and K runs the schedule it would pick with unlimited room, on a GPU with `sms`
  *     multiprocessors (148 on a B200); 0 when that schedule does not split K (then no workspace is
  *     of any use) or when an argument is invalid.  The maximum over the shapes a caller issues
- *     serves all of them.  pq_gemm_w4a8 and every decode-shaped call (M <= 128) need none.
+ *     serves all of them.  pq_gemm_w4a8 and every call that the weight-streaming kernel serves (M <= 128, narrow
+ *     linears up to M = 256) need none.
  *   pq_workspace_init: zeroes the first 64 KB of `workspace` on `stream` (bytes >= 65536, 256-byte
  *     aligned).  GEMM calls enqueued afterwards on that stream (or after a synchronization) may
  *     use the workspace.  A buffer the caller has zero-filled by other means is equally good.
@@ -300,7 +302,8 @@ PQ_API size_t pq_workspace_bytes(int64_t M, const int64_t* N, int32_t count, int
 PQ_API int pq_workspace_init(void* workspace, size_t bytes, void* stream);
 
 /*
- * Host-only query (touches no device): the schedule pq_gemm_w8a8 picks for M > 128 on a GPU with
+ * Host-only query (touches no device): the schedule of the prefill kernel (the one pq_gemm_w8a8 uses
+ * beyond the token counts of the weight-streaming kernel) on a GPU with
  * `sms` multiprocessors and a workspace of `scratch_bytes` (0 = none): the output tile
  * width (*tile_n = 256 or 128 columns) and the number of parts K is cut into (*k_parts, 1 = no
  * split).  For capacity planning and tests; the result has no effect on later calls.
