@@ -212,7 +212,6 @@ smallm_kernel(const __grid_constant__ SmallMaps maps, const __grid_constant__ CU
     const int first = nkb < C::STAGES ? nkb : C::STAGES;
     for (int j = 0; j < first; ++j) issue_weights(j);
   }
-  grid_dep_launch();   // the successor may start streaming its own weights
   if (warp == 1) {
     tmem_alloc(smem_u32(tmem_slot), C::kTmemCols);
     tmem_relinquish();
@@ -221,6 +220,11 @@ smallm_kernel(const __grid_constant__ SmallMaps maps, const __grid_constant__ CU
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
+  // The successor may now become resident and start streaming its own weights.  Only now: every CTA of this
+  // launch holds its tensor memory before a later launch's CTA can ask for any (a CTA that took all columns
+  // of an SM and then waited for this launch, while a CTA of this launch still waited for columns, would never
+  // be released).
+  grid_dep_launch();
 
   // W4: per-thread partial results of the epilogue warps, P[m] for weight row n0 + 32*quad + lane.
   // (W8 copies its one accumulator from tensor memory straight into the reduction tile.)
