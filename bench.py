@@ -351,6 +351,16 @@ class GpuWorkload:
     def run_layer(self, L: LayerBuffers, only: str | None = None):
         pq, wl = self.pq, self.wl
         for gi, (K, idxs) in enumerate(L.groups):
+            if only == "linear":
+                # every linear as ONE call (quantizer + GEMM; one launch where the row kernel serves)
+                for i in idxs:
+                    a, b = L.packed[i]
+                    if wl.w_bits == 8:
+                        pq.pq_linear_w8a8(L.xs[gi], a, b, wl.linears[i].N, y=L.ys[i], q_tmp=L.qs[gi], s_tok_tmp=L.s_toks[gi],
+                                          workspace=self.workspace)
+                    else:
+                        pq.pq_linear_w4a8(L.xs[gi], a, b, wl.linears[i].N, y=L.ys[i], q_tmp=L.qs[gi], s_tok_tmp=L.s_toks[gi])
+                continue
             if only == "quantize_smooth":
                 pq.pq_quantize_act_smooth(L.xs[gi], L.s_invs[gi], L.qs[gi], L.s_toks[gi])
                 continue
@@ -467,10 +477,16 @@ def side_workload(pq, torch, name: str, M: int, dev, stream, grouped: bool, peak
     _, unit, value = w.value_of(step_ms)
     roof = w.roofline(gemm_ms, n, peaks, peak_kind)
     quant_gbs = step_bytes(wl, M)["quantize"] / (quant_ms * len(w.groups) * 1e-3) / 1e9
-    return {"workload": name, "M": M, "w_bits": wl.w_bits, "value": value, "unit": unit, "ms_per_step": step_ms,
-            "launches_per_step": w.launches_per_step, "frac": roof["frac"], "avg_launch_us": roof["avg_launch_us"],
-            "roofline": roof, "quantize_frac_of_hbm": quant_gbs / float(peaks["hbm_gbs"]),
-            "rotation_layers": w.n_layers}
+    out = {"workload": name, "M": M, "w_bits": wl.w_bits, "value": value, "unit": unit, "ms_per_step": step_ms,
+           "launches_per_step": w.launches_per_step, "frac": roof["frac"], "avg_launch_us": roof["avg_launch_us"],
+           "roofline": roof, "quantize_frac_of_hbm": quant_gbs / float(peaks["hbm_gbs"]),
+           "rotation_layers": w.n_layers}
+    if M <= 4:
+        # the same step with every linear as one call (pq_linear_*: the row kernel quantizes its own tokens)
+        lin_ms, _ = w.time_replays(w.kind_graphs("linear"), 1, min_ms)
+        out["one_call_linear"] = {"ms_per_step": lin_ms, "value": w.value_of(lin_ms)[2], "unit": unit,
+                                  "calls_per_step": sum(len(idxs) for _, idxs in w.groups)}
+    return out
 
 
 def run_ours(args, wl: synth.Workload, M: int):
@@ -772,7 +788,10 @@ def run_ours(args, wl: synth.Workload, M: int):
 # --------------------------------------------------------------------------- one operation (profilers, per-shape timing)
 
 QUANT_OPS = ("quantize", "quantize_smooth", "quantize_hadamard", "quantize_static", "swiglu_quantize")
-ONE_OPS = QUANT_OPS + ("gemm_w8a8", "gemm_w4a8")
+# linear_*: the one-call linear (quantizer + GEMM; one launch where the row kernel serves); quant_gemm_*: the
+# same work as two calls (the time per PAIR of launches), for comparison
+LINEAR_OPS = ("linear_w8a8", "linear_w4a8", "quant_gemm_w8a8", "quant_gemm_w4a8")
+ONE_OPS = QUANT_OPS + ("gemm_w8a8", "gemm_w4a8") + LINEAR_OPS
 
 
 def run_one_op(args):
@@ -797,9 +816,9 @@ def run_one_op(args):
     packed = []
     for g in range(G if op not in QUANT_OPS else 0):
         w = torch.from_numpy(synth.weights(N, K, 9001 + g)).to(dev)
-        packed.append(pq.pq_pack_w8(w) if op == "gemm_w8a8" else pq.pq_pack_w4(w))
+        packed.append(pq.pq_pack_w8(w) if op.endswith("w8a8") else pq.pq_pack_w4(w))
         del w
-    need = pq.pq_workspace_bytes(M, [N] * G, K) if op == "gemm_w8a8" else 0
+    need = pq.pq_workspace_bytes(M, [N] * G, K) if op.endswith("w8a8") else 0
     ws = pq.pq_workspace_init(torch.empty((need,), dtype=torch.uint8, device=dev)) if need else None
     bufs = []
     for _ in range(sets):
@@ -823,6 +842,16 @@ def run_one_op(args):
             pq.pq_quantize_act_static(b["x"], b["scale"], b["q"], b["s_tok"])
         elif op == "swiglu_quantize":
             pq.pq_swiglu_quantize(b["x"], b["up"], b["q"], b["s_tok"])
+        elif op == "linear_w8a8":
+            pq.pq_linear_w8a8(b["x"], b["w"][0][0], b["w"][0][1], N, y=b["y"][0], q_tmp=b["q"], s_tok_tmp=b["s_tok"], workspace=ws)
+        elif op == "linear_w4a8":
+            pq.pq_linear_w4a8(b["x"], b["w"][0][0], b["w"][0][1], N, y=b["y"][0], q_tmp=b["q"], s_tok_tmp=b["s_tok"])
+        elif op == "quant_gemm_w8a8":
+            pq.pq_quantize_act(b["x"], b["q"], b["s_tok"])
+            pq.pq_gemm_w8a8(b["q"], b["s_tok"], b["w"][0][0], b["w"][0][1], N, y=b["y"][0], workspace=ws)
+        elif op == "quant_gemm_w4a8":
+            pq.pq_quantize_act(b["x"], b["q"], b["s_tok"])
+            pq.pq_gemm_w4a8(b["q"], b["s_tok"], b["w"][0][0], b["w"][0][1], N, y=b["y"][0])
         elif G > 1 and op == "gemm_w8a8":
             pq.pq_gemm_w8a8_group(b["q"], b["s_tok"], [(w[0], w[1], N) for w in b["w"]], b["y"], workspace=ws)
         elif G > 1:
@@ -867,7 +896,7 @@ def run_one_op(args):
         out["GBps"] = ((5 if op == "swiglu_quantize" else 3) * M * K + 4 * M + (4 * K if op == "quantize_smooth" else 0)) / med / 1e3
     else:
         out["TOPS"] = 2 * M * G * N * K / med / 1e6
-        wbytes = N * K + 4 * N if op == "gemm_w8a8" else N * K // 2 + (K // 128) * N * 2
+        wbytes = N * K + 4 * N if op.endswith("w8a8") else N * K // 2 + (K // 128) * N * 2
         out["GBps"] = (G * wbytes + M * K + 4 * M + 2 * M * G * N) / med / 1e3
     print(json.dumps(out))
 

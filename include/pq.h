@@ -238,6 +238,23 @@ PQ_API int pq_gemm_w8a8(const int8_t* q, const float* s_tok, const void* wq, con
                  void* stream);
 
 /*
+ * The whole path of one linear in one call: per-token quantization of the FP16 activations (Eq. 1-2,
+ * exactly pq_quantize_act) followed by pq_gemm_w8a8 / pq_gemm_w4a8 on the result.  Y is bit for bit what
+ * the two calls give.  For the smallest decode shapes (one to four tokens, where the CUDA-core row
+ * kernel is the schedule) the GEMM kernel quantizes its tokens itself and nothing else is launched: a
+ * decode step is a chain of dependent launches, and each launch costs microseconds whatever it does.
+ *   x_f16 [M,K] device; q_tmp int8 [M,K] and s_tok_tmp float [M]: device buffers of the caller for the
+ *   codes and scales (written when two kernels run; their contents are unspecified afterwards);
+ *   everything else as in pq_gemm_w8a8 / pq_gemm_w4a8.  On an argument error nothing is launched.
+ */
+PQ_API int pq_linear_w8a8(const void* x_f16, const void* wq, const float* s_ch, int64_t M, int64_t N,
+                          int64_t K, void* y_f16, int8_t* q_tmp, float* s_tok_tmp, void* workspace,
+                          size_t workspace_bytes, void* stream);
+PQ_API int pq_linear_w4a8(const void* x_f16, const void* wp, const void* s_grp_f16, int32_t group,
+                          int64_t M, int64_t N, int64_t K, void* y_f16, int8_t* q_tmp, float* s_tok_tmp,
+                          void* stream);
+
+/*
  * W4A8 linear: INT4 codes are widened to INT8 inside the kernel, multiplied in
  * integers per K-group and dequantized per group into an FP32 running sum:
  *   ACC_g[m,n] = sum_{k in group g} Q[m,k] * C[n,k]        exact, INT32

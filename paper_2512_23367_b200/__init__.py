@@ -22,6 +22,8 @@ from .binding import (  # noqa: F401
     pq_hadamard_block,
     pq_pack_w4,
     pq_pack_w4_hadamard,
+    pq_linear_w4a8,
+    pq_linear_w8a8,
     pq_pack_w8,
     pq_pack_w8_hadamard,
     pq_plan_w8a8,

@@ -42,6 +42,8 @@ SIGNATURES = {
                                           ctypes.c_size_t, _vp]),
     "pq_quantize_act_static": (ctypes.c_int, [_vp, _vp, _i64, _i64, _vp, _vp, _vp]),
     "pq_swiglu_quantize": (ctypes.c_int, [_vp, _vp, _i64, _i64, _vp, _vp, _vp]),
+    "pq_linear_w8a8": (ctypes.c_int, [_vp, _vp, _vp, _i64, _i64, _i64, _vp, _vp, _vp, _vp, ctypes.c_size_t, _vp]),
+    "pq_linear_w4a8": (ctypes.c_int, [_vp, _vp, _vp, _i32, _i64, _i64, _i64, _vp, _vp, _vp, _vp]),
     "pq_quantize_act_static_channel": (ctypes.c_int, [_vp, _vp, _i64, _i64, _vp, _vp, _vp]),
     "pq_hadamard_block": (_i32, [_i64]),
     "pq_quantize_act_hadamard": (ctypes.c_int, [_vp, _i64, _i64, _vp, _vp, _vp]),
@@ -440,6 +442,46 @@ def pq_gemm_w4a8(q, s_tok, wp, s_grp, N: int, group: int = GROUP, y: torch.Tenso
     y = _out(y, M, N, q)
     _check("pq_gemm_w4a8", lib().pq_gemm_w4a8(q.data_ptr(), s_tok.data_ptr(), wp.data_ptr(), s_grp.data_ptr(),
                                               group, M, N, K, y.data_ptr(), _stream()))
+    return y
+
+
+def _linear_args(x, y, q_tmp, s_tok_tmp, N):
+    if x.dim() != 2:
+        raise ValueError("x: expected a 2-D tensor [M,K]")
+    M, K = x.shape
+    _sized(x, torch.float16, M * K, "x")
+    if q_tmp is None:
+        q_tmp = torch.empty((M, K), dtype=torch.int8, device=x.device)
+    if s_tok_tmp is None:
+        s_tok_tmp = torch.empty((M,), dtype=torch.float32, device=x.device)
+    _sized(q_tmp, torch.int8, M * K, "q_tmp"), _sized(s_tok_tmp, torch.float32, M, "s_tok_tmp")
+    if y is not None:
+        _sized(y, torch.float16, M * N, "y")
+    return M, K, _out(y, M, N, x), q_tmp, s_tok_tmp
+
+
+def pq_linear_w8a8(x, wq, s_ch, N: int, y: torch.Tensor | None = None, q_tmp: torch.Tensor | None = None,
+                   s_tok_tmp: torch.Tensor | None = None, workspace: torch.Tensor | None = None) -> torch.Tensor:
+    """x f16 [M,K] -> y f16 [M,N]: pq_quantize_act + pq_gemm_w8a8 in one call (one launch for one to four tokens
+    where the row kernel serves).  q_tmp / s_tok_tmp: the caller's buffers for codes and scales (allocated here
+    when not given)."""
+    M, K, y, q_tmp, s_tok_tmp = _linear_args(x, y, q_tmp, s_tok_tmp, N)
+    _sized(wq, torch.uint8, N * K, "wq"), _sized(s_ch, torch.float32, N, "s_ch")
+    ws, ws_bytes = _ws(workspace)
+    _together(x, wq, s_ch, y, q_tmp, s_tok_tmp, workspace)
+    _check("pq_linear_w8a8", lib().pq_linear_w8a8(x.data_ptr(), wq.data_ptr(), s_ch.data_ptr(), M, N, K, y.data_ptr(),
+                                                  q_tmp.data_ptr(), s_tok_tmp.data_ptr(), ws, ws_bytes, _stream()))
+    return y
+
+
+def pq_linear_w4a8(x, wp, s_grp, N: int, group: int = GROUP, y: torch.Tensor | None = None,
+                   q_tmp: torch.Tensor | None = None, s_tok_tmp: torch.Tensor | None = None) -> torch.Tensor:
+    """x f16 [M,K] -> y f16 [M,N]: pq_quantize_act + pq_gemm_w4a8 in one call (see pq_linear_w8a8)."""
+    M, K, y, q_tmp, s_tok_tmp = _linear_args(x, y, q_tmp, s_tok_tmp, N)
+    _sized(wp, torch.uint8, N * K // 2, "wp"), _sized(s_grp, torch.float16, (K // max(group, 1)) * N, "s_grp")
+    _together(x, wp, s_grp, y, q_tmp, s_tok_tmp)
+    _check("pq_linear_w4a8", lib().pq_linear_w4a8(x.data_ptr(), wp.data_ptr(), s_grp.data_ptr(), group, M, N, K,
+                                                  y.data_ptr(), q_tmp.data_ptr(), s_tok_tmp.data_ptr(), _stream()))
     return y
 
 

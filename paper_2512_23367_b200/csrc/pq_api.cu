@@ -471,6 +471,41 @@ int pq_gemm_w4a8(const int8_t* q, const float* s_tok, const void* wp, const void
   return gemm_w4a8_common(q, s_tok, wp, s_grp_f16, group, M, N, K, y_f16, nullptr, stream);
 }
 
+// S1-S4 in one call.  Where the CUDA-core row kernel serves the shape it quantizes its own tokens (one launch);
+// otherwise the quantizer and the GEMM run one after the other through the caller's q / s_tok buffers.
+int pq_linear_w8a8(const void* x_f16, const void* wq, const float* s_ch, int64_t M, int64_t N, int64_t K, void* y_f16,
+                   int8_t* q_tmp, float* s_tok_tmp, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!x_f16 || !wq || !s_ch || !y_f16 || !q_tmp || !s_tok_tmp) return PQ_ERR_NULL;
+  int rc = check_gemm(M, N, K);
+  if (rc != PQ_OK) return rc;
+  if (!aligned16(x_f16) || !aligned16(wq) || !aligned16(y_f16) || !aligned16(q_tmp) || !aligned256(workspace)) return PQ_ERR_ALIGN;
+  if ((rc = check_arch()) != PQ_OK) return rc;
+  if (gemv_enabled() && gemv_rows_serves(8, M, N, K, sm_count())) {
+    log_dispatch("w8a8", "CUDA-core row kernel, tokens quantized in the kernel", M, N, K);
+    return launch_gemv_rows_w8a8_x(x_f16, wq, s_ch, M, N, K, y_f16, static_cast<cudaStream_t>(stream));
+  }
+  rc = pq_quantize_act(x_f16, M, K, q_tmp, s_tok_tmp, stream);
+  if (rc != PQ_OK) return rc;
+  return pq_gemm_w8a8(q_tmp, s_tok_tmp, wq, s_ch, M, N, K, y_f16, workspace, workspace_bytes, stream);
+}
+
+int pq_linear_w4a8(const void* x_f16, const void* wp, const void* s_grp_f16, int32_t group, int64_t M, int64_t N,
+                   int64_t K, void* y_f16, int8_t* q_tmp, float* s_tok_tmp, void* stream) {
+  if (!x_f16 || !wp || !s_grp_f16 || !y_f16 || !q_tmp || !s_tok_tmp) return PQ_ERR_NULL;
+  int rc = check_gemm(M, N, K);
+  if (rc != PQ_OK) return rc;
+  if (group != 128 || K % 128 != 0) return PQ_ERR_SHAPE;
+  if (!aligned16(x_f16) || !aligned16(wp) || !aligned16(s_grp_f16) || !aligned16(y_f16) || !aligned16(q_tmp)) return PQ_ERR_ALIGN;
+  if ((rc = check_arch()) != PQ_OK) return rc;
+  if (gemv_enabled() && gemv_rows_serves(4, M, N, K, sm_count())) {
+    log_dispatch("w4a8", "CUDA-core row kernel, tokens quantized in the kernel", M, N, K);
+    return launch_gemv_rows_w4a8_x(x_f16, wp, s_grp_f16, M, N, K, y_f16, static_cast<cudaStream_t>(stream));
+  }
+  rc = pq_quantize_act(x_f16, M, K, q_tmp, s_tok_tmp, stream);
+  if (rc != PQ_OK) return rc;
+  return pq_gemm_w4a8(q_tmp, s_tok_tmp, wp, s_grp_f16, group, M, N, K, y_f16, stream);
+}
+
 int pq_gemm_w4a8_group(const int8_t* q, const float* s_tok, int32_t count, const void* const* wp,
                        const void* const* s_grp_f16, int32_t group, const int64_t* N, void* const* y_f16, int64_t M,
                        int64_t K, void* stream) {

@@ -38,6 +38,7 @@
 
 #include "pq_internal.h"
 #include "pq_ptx.cuh"
+#include "pq_quant_math.cuh"
 
 namespace pq {
 namespace {
@@ -49,10 +50,12 @@ constexpr int kCtaBytesMax = 112 * 1024;   // ring + token codes: a CTA stays be
 constexpr int kSoloBytesMax = 216 * 1024;  // ... or takes the SM alone, when that lets the ring hold its whole share
 constexpr int kCodeBytesMax = 44 * 1024;
 constexpr int kFillBatch = 12;             // 16-byte chunks of codes a thread has in flight at once
+constexpr int kXBatch = 6;                 // ... of FP16 activations, where the kernel quantizes them itself
 
 struct RowArgs {
   const uint8_t* w;        // W8: [N, K] codes; W4: [N, K/2] packed
   const int8_t* q;         // [M, K]
+  const __half* x;         // kFuseX: [M, K] FP16 activations instead of q and s_tok
   const float* s_tok;      // [M]
   const float* s_ch;       // W8: [N]
   const __half* s_grp;     // W4: [K/128, N]
@@ -124,7 +127,9 @@ __device__ __forceinline__ int lane_reduce_scatter(T (&v)[V], int lane) {
   return which;
 }
 
-template <bool kW4, int MT, int RQ, bool kExportAcc>
+// kFuseX: the kernel quantizes its own tokens (Eq. 1-2, the arithmetic of the quantizer kernels) instead of
+// reading codes and token scales: one launch less on the critical path of a decode step.
+template <bool kW4, int MT, int RQ, bool kExportAcc, bool kFuseX = false>
 __global__ void __launch_bounds__(kThreads, 2) gemv_rows_kernel(const RowArgs p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
@@ -188,6 +193,70 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_rows_kernel(const RowArgs p)
     // 16-byte chunk c sits at position code_pos(c, b & 7).  Tokens >= M and bytes >= K read as zero.
     // This copy sits on the critical path of the call (nothing else can start before it), and a load
     // takes a round trip to the L2: a thread issues all its loads of a batch before it stores any.
+    float st[MT];
+    if constexpr (kFuseX) {
+      // Pass 1: every token's largest magnitude (all of the CTA's threads over all of x; a CTA reads the
+      // few KB of x by itself, from the L2).  Pass 2 reads x again (now from the L1) and writes the codes.
+      __shared__ float red[kConsumerWarps][MT];
+      const int x_chunks = p.K >> 3;                      // 16-byte chunks (8 values) of one token
+      float amax[MT];
+#pragma unroll
+      for (int m = 0; m < MT; ++m) amax[m] = 0.0f;
+#pragma unroll
+      for (int m = 0; m < MT; ++m) {
+        if (m < p.M) {
+          const uint4* xr = reinterpret_cast<const uint4*>(p.x + static_cast<int64_t>(m) * p.K);
+          for (int c0 = threadIdx.x; c0 < x_chunks; c0 += kXBatch * kThreads) {
+            uint4 v[kXBatch];
+#pragma unroll
+            for (int u = 0; u < kXBatch; ++u) {
+              const int c = c0 + u * kThreads;
+              v[u] = c < x_chunks ? xr[c] : make_uint4(0u, 0u, 0u, 0u);
+            }
+#pragma unroll
+            for (int u = 0; u < kXBatch; ++u) amax[m] = fmaxf(amax[m], absmax8(v[u]));
+          }
+        }
+      }
+#pragma unroll
+      for (int m = 0; m < MT; ++m) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) amax[m] = fmaxf(amax[m], __shfl_xor_sync(0xffffffffu, amax[m], o));
+        if (lane == 0) red[warp][m] = amax[m];
+      }
+      __syncthreads();
+      float fm[MT];
+#pragma unroll
+      for (int m = 0; m < MT; ++m) {
+        float a = 0.0f;
+#pragma unroll
+        for (int w = 0; w < kConsumerWarps; ++w) a = fmaxf(a, red[w][m]);
+        act_scale(a, &st[m], &fm[m]);
+        if (kExportAcc || m >= p.M) st[m] = 0.0f;
+      }
+      const int chunks_per_row = p.kblocks * 8;
+      const int k_chunks = p.K >> 4;
+      const int total = MT * chunks_per_row;
+      for (int i = threadIdx.x; i < total; i += kThreads) {
+        const int m = i / chunks_per_row, c = i - m * chunks_per_row;
+        uint4 out = make_uint4(0u, 0u, 0u, 0u);
+        if (m < p.M && c < k_chunks) {
+          const uint4* xr = reinterpret_cast<const uint4*>(p.x + static_cast<int64_t>(m) * p.K) + 2 * c;
+          const uint4 lo = xr[0], hi = xr[1];
+          const __half* hl = reinterpret_cast<const __half*>(&lo);
+          const __half* hh = reinterpret_cast<const __half*>(&hi);
+          float f = fm[0];
+#pragma unroll
+          for (int j = 1; j < MT; ++j) f = (m == j) ? fm[j] : f;
+          out.x = codes4<false>(__half2float(hl[0]), __half2float(hl[1]), __half2float(hl[2]), __half2float(hl[3]), f);
+          out.y = codes4<false>(__half2float(hl[4]), __half2float(hl[5]), __half2float(hl[6]), __half2float(hl[7]), f);
+          out.z = codes4<false>(__half2float(hh[0]), __half2float(hh[1]), __half2float(hh[2]), __half2float(hh[3]), f);
+          out.w = codes4<false>(__half2float(hh[4]), __half2float(hh[5]), __half2float(hh[6]), __half2float(hh[7]), f);
+        }
+        const int b = c >> 3, cc = c & 7;
+        *reinterpret_cast<uint4*>(smem + (codes - smem_base) + m * code_row + b * 128 + (code_pos<kW4>(cc, b & 7) << 4)) = out;
+      }
+    } else
     {
       const int chunks_per_row = p.kblocks * 8;
       const int k_chunks = p.K >> 4;
@@ -214,9 +283,10 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_rows_kernel(const RowArgs p)
       }
     }
     __syncthreads();   // the codes are in place (and the barriers exist) before anybody goes on
-    float st[MT];
+    if constexpr (!kFuseX) {
 #pragma unroll
-    for (int m = 0; m < MT; ++m) st[m] = (!kExportAcc && m < p.M) ? __ldg(p.s_tok + m) : 0.0f;
+      for (int m = 0; m < MT; ++m) st[m] = (!kExportAcc && m < p.M) ? __ldg(p.s_tok + m) : 0.0f;
+    }
     const int sw = lane & 7;                 // this lane's blocks are l, l + 32, ...: (b & 7) == (l & 7)
 
     for (int j = warp; j < my_sets; j += kConsumerWarps) {
@@ -406,9 +476,9 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_rows_kernel(const RowArgs p)
   }
 }
 
-template <bool kW4, int MT, int RQ, bool kExportAcc>
+template <bool kW4, int MT, int RQ, bool kExportAcc, bool kFuseX = false>
 int launch_rows_cfg(const RowArgs& a, int smem_bytes, int grid, cudaStream_t stream) {
-  auto kern = gemv_rows_kernel<kW4, MT, RQ, kExportAcc>;
+  auto kern = gemv_rows_kernel<kW4, MT, RQ, kExportAcc, kFuseX>;
   static PerDeviceOnce once;
   if (const int rc = set_dynamic_smem_once(once, kern, kSoloBytesMax + 1024); rc != PQ_OK) return rc;
   cudaLaunchConfig_t cfg = {};
@@ -424,10 +494,10 @@ int launch_rows_cfg(const RowArgs& a, int smem_bytes, int grid, cudaStream_t str
   return cuda_status(cudaLaunchKernelEx(&cfg, kern, a));
 }
 
-template <bool kW4, int MT, bool kExportAcc>
+template <bool kW4, int MT, bool kExportAcc, bool kFuseX = false>
 int launch_rows_rq(int rq, const RowArgs& a, int smem_bytes, int grid, cudaStream_t stream) {
-  return rq == 4 ? launch_rows_cfg<kW4, MT, 4, kExportAcc>(a, smem_bytes, grid, stream)
-                 : launch_rows_cfg<kW4, MT, 2, kExportAcc>(a, smem_bytes, grid, stream);
+  return rq == 4 ? launch_rows_cfg<kW4, MT, 4, kExportAcc, kFuseX>(a, smem_bytes, grid, stream)
+                 : launch_rows_cfg<kW4, MT, 2, kExportAcc, kFuseX>(a, smem_bytes, grid, stream);
 }
 
 // Shape of a launch: rows per row set, ring depth, grid, shared memory.  `fits`: the ring holds a CTA's
@@ -481,13 +551,14 @@ bool plan_rows_within(int cta_bytes_max, int w_bits, int64_t M, int64_t N, int64
 
 template <bool kW4>
 int launch_rows(const int8_t* q, const float* s_tok, const void* w, const float* s_ch, const void* s_grp, int64_t M,
-                int64_t N, int64_t K, void* y, int32_t* acc, cudaStream_t stream) {
+                int64_t N, int64_t K, void* y, int32_t* acc, cudaStream_t stream, const void* x = nullptr) {
   RowPlan pl;
   if (!plan_rows(kW4 ? 4 : 8, M, N, K, sm_count(), &pl)) return PQ_ERR_SHAPE;
   RowArgs a;
   a.row_bytes = static_cast<int>(kW4 ? K / 2 : K);
   a.w = static_cast<const uint8_t*>(w);
   a.q = q;
+  a.x = static_cast<const __half*>(x);
   a.s_tok = s_tok;
   a.s_ch = s_ch;
   a.s_grp = static_cast<const __half*>(s_grp);
@@ -504,6 +575,14 @@ int launch_rows(const int8_t* q, const float* s_tok, const void* w, const float*
   a.slots = pl.slots;
   const int rq = pl.rq, grid = pl.grid, smem_bytes = pl.smem_bytes;
   const bool ex = acc != nullptr;
+  if (x != nullptr) {   // the kernel quantizes its own tokens
+    if (ex) return PQ_ERR_SHAPE;
+    switch (pl.mt) {
+      case 1: return launch_rows_rq<kW4, 1, false, true>(rq, a, smem_bytes, grid, stream);
+      case 2: return launch_rows_rq<kW4, 2, false, true>(rq, a, smem_bytes, grid, stream);
+      default: return launch_rows_rq<kW4, 4, false, true>(rq, a, smem_bytes, grid, stream);
+    }
+  }
   switch (pl.mt) {
     case 1: return ex ? launch_rows_rq<kW4, 1, true>(rq, a, smem_bytes, grid, stream) : launch_rows_rq<kW4, 1, false>(rq, a, smem_bytes, grid, stream);
     case 2: return ex ? launch_rows_rq<kW4, 2, true>(rq, a, smem_bytes, grid, stream) : launch_rows_rq<kW4, 2, false>(rq, a, smem_bytes, grid, stream);
@@ -534,6 +613,16 @@ int launch_gemv_rows_w8a8(const int8_t* q, const float* s_tok, const void* wq, c
 int launch_gemv_rows_w4a8(const int8_t* q, const float* s_tok, const void* wp, const void* s_grp, int64_t M, int64_t N,
                           int64_t K, void* y, int32_t* acc_g, cudaStream_t stream) {
   return launch_rows<true>(q, s_tok, wp, nullptr, s_grp, M, N, K, y, acc_g, stream);
+}
+
+// The same from FP16 activations: the kernel quantizes them itself.
+int launch_gemv_rows_w8a8_x(const void* x, const void* wq, const float* s_ch, int64_t M, int64_t N, int64_t K, void* y,
+                            cudaStream_t stream) {
+  return launch_rows<false>(nullptr, nullptr, wq, s_ch, nullptr, M, N, K, y, nullptr, stream, x);
+}
+int launch_gemv_rows_w4a8_x(const void* x, const void* wp, const void* s_grp, int64_t M, int64_t N, int64_t K, void* y,
+                            cudaStream_t stream) {
+  return launch_rows<true>(nullptr, nullptr, wp, nullptr, s_grp, M, N, K, y, nullptr, stream, x);
 }
 
 }  // namespace pq

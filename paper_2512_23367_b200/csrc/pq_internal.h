@@ -133,6 +133,11 @@ int launch_smallm_w4a8(const int8_t* q, const float* s_tok, const void* wp, cons
 // One to four tokens on the CUDA cores (whole weight rows per CTA, ring filled ahead of the wait on the
 // preceding kernel); same results as the calls above.  gemv_rows_serves: whether it is the schedule of choice.
 bool gemv_rows_serves(int w_bits, int64_t M, int64_t N, int64_t K, int sms);
+// The same from FP16 activations [M, K]: the kernel quantizes its tokens itself (Eq. 1-2).
+int launch_gemv_rows_w8a8_x(const void* x, const void* wq, const float* s_ch, int64_t M, int64_t N, int64_t K, void* y,
+                            cudaStream_t stream);
+int launch_gemv_rows_w4a8_x(const void* x, const void* wp, const void* s_grp, int64_t M, int64_t N, int64_t K, void* y,
+                            cudaStream_t stream);
 int launch_gemv_rows_w8a8(const int8_t* q, const float* s_tok, const void* wq, const float* s_ch, int64_t M, int64_t N,
                           int64_t K, void* y, int32_t* acc, cudaStream_t stream);
 int launch_gemv_rows_w4a8(const int8_t* q, const float* s_tok, const void* wp, const void* s_grp, int64_t M, int64_t N,

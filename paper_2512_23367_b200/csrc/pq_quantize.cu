@@ -9,6 +9,7 @@
 
 #include "pq_internal.h"
 #include "pq_ptx.cuh"
+#include "pq_quant_math.cuh"
 
 namespace pq {
 
@@ -25,27 +26,6 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kCached = 8;  // 16-byte chunks of a row that one thread keeps in registers
-
-__device__ __forceinline__ float absmax8(const uint4& v) {
-  const __half2* h = reinterpret_cast<const __half2*>(&v);
-  __half2 m = __hmax2(__hmax2(__habs2(h[0]), __habs2(h[1])), __hmax2(__habs2(h[2]), __habs2(h[3])));
-  return fmaxf(__low2float(m), __high2float(m));
-}
-
-// Eq. 1 for four values at a time.
-// Four scaled values -> four INT8 codes in one word (code i in byte i): round to nearest even, then two
-// packing conversions that saturate to [-128, 127].
-template <bool kDivide>
-__device__ __forceinline__ uint32_t codes4(float x0, float x1, float x2, float x3, float f) {
-  const int a0 = __float2int_rn(kDivide ? __fdiv_rn(x0, f) : __fmul_rn(x0, f));
-  const int a1 = __float2int_rn(kDivide ? __fdiv_rn(x1, f) : __fmul_rn(x1, f));
-  const int a2 = __float2int_rn(kDivide ? __fdiv_rn(x2, f) : __fmul_rn(x2, f));
-  const int a3 = __float2int_rn(kDivide ? __fdiv_rn(x3, f) : __fmul_rn(x3, f));
-  uint32_t hi, out;
-  asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(a3), "r"(a2), "r"(0));
-  asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(out) : "r"(a1), "r"(a0), "r"(hi));
-  return out;
-}
 
 // The eight values of a 16-byte chunk as the quantizer sees them: the FP16 elements, times the
 // column factors of Eq. 3 (one FP32 product each, not rounded back to FP16) when kSmooth.
