@@ -24,7 +24,7 @@ def _case(kind):
     with the oracle."""
     M, K, N = {"w8a8_pair": (300, 1024, 520), "w8a8_pair_split_k": (512, 11008, 1024), "w8a8_noalloc": (512, 11008, 1024),
                "w8a8_small_m": (16, 2048, 1024), "w8a8_small_m_blocks": (200, 2048, 1024), "w4a8_pair": (300, 1024, 520), "w4a8_small_m": (16, 2048, 1024), "w4a8_small_m_128": (100, 2048, 1024), "w4a8_small_m_blocks": (200, 2048, 1024),
-               "w8a8_rows": (3, 2048, 1024), "w4a8_rows": (2, 2048, 1024)}[kind]
+               "w8a8_rows": (3, 2048, 1024), "w4a8_rows": (2, 2048, 1024), "w4a8_linear_rows": (2, 2048, 1024)}[kind]
     x, w = synth.activations(M, K, 31), synth.weights(N, K, 32)
     q, s_tok = pq.pq_quantize_act(torch.from_numpy(x).to(DEV))
     y = torch.empty((M, N), dtype=torch.float16, device=DEV)
@@ -39,6 +39,10 @@ def _case(kind):
         g, ref = y_gpu.cpu().numpy()[rows].astype(np.float64), ref.astype(np.float64)
         assert np.all(np.abs(g - ref) <= 2.0 ** -10 * np.abs(ref) + 1e-3)
 
+    if kind == "w4a8_linear_rows":     # the row kernel quantizing its own tokens
+        wp, sg = pq.pq_pack_w4(torch.from_numpy(w).to(DEV))
+        xd = torch.from_numpy(x).to(DEV)
+        return (lambda: pq.pq_linear_w4a8(xd, wp, sg, N, y=y, q_tmp=q, s_tok_tmp=s_tok)), (lambda: None), check
     if kind.startswith("w4a8"):
         wp, sg = pq.pq_pack_w4(torch.from_numpy(w).to(DEV))
         return (lambda: pq.pq_gemm_w4a8(q, s_tok, wp, sg, N, y=y)), (lambda: None), check
@@ -55,7 +59,7 @@ def _case(kind):
 
 
 @pytest.mark.parametrize("kind", ["w8a8_pair", "w8a8_pair_split_k", "w8a8_noalloc", "w8a8_small_m", "w8a8_small_m_blocks", "w4a8_pair", "w4a8_small_m", "w4a8_small_m_128", "w4a8_small_m_blocks",
-                                  "w8a8_rows", "w4a8_rows"])
+                                  "w8a8_rows", "w4a8_rows", "w4a8_linear_rows"])
 def test_a_wait_that_runs_out_is_reported_and_leaves_everything_usable(kind):
     call, reinit, check = _case(kind)
     reinit()
