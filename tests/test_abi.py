@@ -40,6 +40,13 @@ def test_argument_errors_come_back_as_status_codes_without_a_device():
     assert L.pq_gemm_w4a8(16, 16, 16, 16, 64, 4, 16, 256, 16, None) == PQ_ERR_SHAPE   # group != 128
     assert L.pq_gemm_w4a8(16, 16, 16, 16, 128, 4, 16, 192, 16, None) == PQ_ERR_SHAPE  # K % 128
     assert L.pq_pack_w4(16, 16, 256, 128, None, 16, None) == PQ_ERR_NULL
+    # x, wq, s_ch, M, N, K, y, q_tmp, s_tok_tmp, workspace, bytes, stream
+    assert L.pq_linear_w8a8(16, 16, 16, 4, 16, 64, 16, None, 16, None, 0, None) == PQ_ERR_NULL        # no q_tmp
+    assert L.pq_linear_w8a8(16, 16, 16, 4, 12, 64, 16, 16, 16, None, 0, None) == PQ_ERR_SHAPE         # N % 8
+    assert L.pq_linear_w8a8(8, 16, 16, 4, 16, 64, 16, 16, 16, None, 0, None) == PQ_ERR_ALIGN
+    # x, wp, s_grp, group, M, N, K, y, q_tmp, s_tok_tmp, stream
+    assert L.pq_linear_w4a8(16, 16, 16, 64, 4, 16, 256, 16, 16, 16, None) == PQ_ERR_SHAPE             # group != 128
+    assert L.pq_linear_w4a8(16, 16, 16, 128, 4, 16, 256, 16, 16, None, None) == PQ_ERR_NULL           # no s_tok_tmp
     import ctypes
     ptrs = (ctypes.c_void_p * 2)(16, 16)
     holes = (ctypes.c_void_p * 2)(16, None)
@@ -147,6 +154,17 @@ def test_binding_measures_every_operand_before_the_call():
         pq.pq_gemm_w4a8_group(q2, st2, [(wp, sg[:-1], N)])
     with pytest.raises(ValueError, match="q: expected"):
         pq.pq_quantize_act(torch.zeros((M, K), dtype=torch.float16), q=torch.zeros((M, K - 1), dtype=torch.int8))
+    x, x2 = torch.zeros((M, K), dtype=torch.float16), torch.zeros((M, 128), dtype=torch.float16)
+    with pytest.raises(ValueError, match="wq: expected"):
+        pq.pq_linear_w8a8(x, wq[:-1], sc, N)
+    with pytest.raises(ValueError, match="q_tmp: expected"):
+        pq.pq_linear_w8a8(x, wq, sc, N, q_tmp=torch.zeros((M, K - 1), dtype=torch.int8))
+    with pytest.raises(ValueError, match="y: expected"):
+        pq.pq_linear_w8a8(x, wq, sc, N, y=y[:-1])
+    with pytest.raises(ValueError, match="s_grp: expected"):
+        pq.pq_linear_w4a8(x2, wp, sg[:-1], N)
+    with pytest.raises(ValueError, match="s_tok_tmp: expected"):
+        pq.pq_linear_w4a8(x2, wp, sg, N, s_tok_tmp=torch.ones(M - 1))
     with pytest.raises(TypeError):
         pq.pq_gemm_w8a8(q, st, wq.to(torch.int8), sc, N, y)
     with pytest.raises(ValueError, match="CUDA"):          # right sizes, wrong memory: there is no CPU path
